@@ -1,0 +1,121 @@
+"""CPU oracle for scaled-dot-product attention -- TEST INFRASTRUCTURE, NOT THE PRODUCT.
+
+Only the test-suite, the smoke check and the benchmark's ``cpu_baseline`` / ``--impl reference``
+legs may import this package.  It shares no code with the CUDA library and never imports it.
+
+``forward`` is the paper's definition (Eq. 3 with the softmax split of Eq. 4) evaluated in
+IEEE double by ``sd_attn_oracle.c``; this module only builds that C file with gcc, marshals
+numpy arrays into it and hands the results back.  No arithmetic of the method lives here.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+import subprocess
+import threading
+
+import numpy as np
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_SRC = os.path.join(_HERE, "sd_attn_oracle.c")
+_LIB = os.path.join(_HERE, "libsd_attn_oracle.so")
+_lock = threading.Lock()
+_lib = None
+
+F16, F32 = 0, 1
+
+
+def build(force: bool = False) -> str:
+    """Compile the C oracle with gcc (plain -O2, OpenMP, no fast-math, no FP contraction)."""
+    stale = (not os.path.exists(_LIB)) or os.path.getmtime(_LIB) < os.path.getmtime(_SRC)
+    if force or stale:
+        tmp = _LIB + ".tmp.%d" % os.getpid()
+        cmd = ["gcc", "-O2", "-std=c11", "-fopenmp", "-ffp-contract=off", "-fPIC", "-shared",
+               "-o", tmp, _SRC, "-lm"]
+        subprocess.run(cmd, check=True, capture_output=True)
+        os.replace(tmp, _LIB)
+    return _LIB
+
+
+def _load():
+    global _lib
+    with _lock:
+        if _lib is None:
+            lib = ctypes.CDLL(build())
+            lib.sd_attn_oracle_forward.restype = ctypes.c_int
+            lib.sd_attn_oracle_forward.argtypes = [
+                ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p,      # q k v
+                ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p,      # out L S
+                ctypes.c_void_p,                                        # probs
+                ctypes.c_int, ctypes.c_int, ctypes.c_int, ctypes.c_int, ctypes.c_int,
+                ctypes.c_float, ctypes.c_int,
+                ctypes.c_void_p, ctypes.c_int64]
+            lib.sd_attn_oracle_max_threads.restype = ctypes.c_int
+            lib.sd_attn_oracle_set_threads.argtypes = [ctypes.c_int]
+            lib.sd_attn_oracle_half_to_double.argtypes = [ctypes.c_void_p, ctypes.c_void_p,
+                                                          ctypes.c_int64]
+            _lib = lib
+    return _lib
+
+
+def max_threads() -> int:
+    return int(_load().sd_attn_oracle_max_threads())
+
+
+def set_threads(n: int) -> None:
+    _load().sd_attn_oracle_set_threads(int(n))
+
+
+def half_to_double(bits: np.ndarray) -> np.ndarray:
+    """Widen raw binary16 bit patterns (uint16) with the oracle's own decoder."""
+    bits = np.ascontiguousarray(bits, dtype=np.uint16)
+    out = np.empty(bits.shape, dtype=np.float64)
+    _load().sd_attn_oracle_half_to_double(bits.ctypes.data, out.ctypes.data, bits.size)
+    return out
+
+
+def forward(q: np.ndarray, k: np.ndarray, v: np.ndarray, scale, rows=None, want_probs=False):
+    """Attention of Eq. 3 in double precision.
+
+    q: [B,H,Nq,d], k and v: [B,H,Nk,d]; all float16 or all float32 numpy arrays.
+    scale: rounded to binary32 first (the value the C-ABI of the GPU library receives).
+    rows: optional 1-D int64 array of flattened row ids ``(b*H+h)*Nq+i``; then only those
+          rows are evaluated and the leading axes of the results are ``[len(rows)]``.
+    Returns ``(out, L, S)`` or ``(out, L, S, P)``: out float64 ``[B,H,Nq,d]`` (or [n,d]),
+    L and S float64 ``[B,H,Nq]`` (or [n]) as in Eq. 4, P float64 ``[..., Nk]``.
+    """
+    if q.dtype != k.dtype or q.dtype != v.dtype:
+        raise TypeError("q, k, v must share one dtype")
+    if q.dtype == np.float16:
+        dtype = F16
+    elif q.dtype == np.float32:
+        dtype = F32
+    else:
+        raise TypeError("dtype must be float16 or float32")
+    if q.ndim != 4 or k.ndim != 4 or v.ndim != 4:
+        raise ValueError("expected [B,H,N,d] arrays")
+    B, H, Nq, d = q.shape
+    if k.shape[:2] != (B, H) or k.shape[3] != d or v.shape != k.shape:
+        raise ValueError("shape mismatch between q, k, v")
+    Nk = k.shape[2]
+    q = np.ascontiguousarray(q)
+    k = np.ascontiguousarray(k)
+    v = np.ascontiguousarray(v)
+    if rows is None:
+        lead = (B, H, Nq)
+        rows_ptr, n_rows = None, 0
+    else:
+        rows = np.ascontiguousarray(rows, dtype=np.int64).ravel()
+        lead = (rows.size,)
+        rows_ptr, n_rows = rows.ctypes.data, rows.size
+    out = np.zeros(lead + (d,), dtype=np.float64)
+    L = np.zeros(lead, dtype=np.float64)
+    S = np.zeros(lead, dtype=np.float64)
+    P = np.zeros(lead + (Nk,), dtype=np.float64) if want_probs else None
+    rc = _load().sd_attn_oracle_forward(
+        q.ctypes.data, k.ctypes.data, v.ctypes.data, out.ctypes.data, L.ctypes.data,
+        S.ctypes.data, P.ctypes.data if want_probs else None,
+        B, H, Nq, Nk, d, ctypes.c_float(float(np.float32(scale))), dtype, rows_ptr, n_rows)
+    if rc != 0:
+        raise RuntimeError("sd_attn_oracle_forward failed with code %d" % rc)
+    return (out, L, S, P) if want_probs else (out, L, S)
