@@ -1,0 +1,144 @@
+/*
+ * sd_attn.h -- C ABI of the B200 (sm_100a) attention library.
+ *
+ * One operation:  out = softmax(Q K^T * scale) V  per (batch, head)      (paper Eq. 3),
+ * the scaled-dot-product attention inside every transformer block of the Stable Diffusion
+ * 1.4 UNet: self-attention (Nk == Nq = 4096/1024/256/64 latent tokens, head dim 40/80/160)
+ * and cross-attention against Nk = 77 text tokens.  Sec. 3.2 of the paper describes two ways
+ * to evaluate it -- a partially fused softmax over a materialised score matrix (Sec. 3.2.1,
+ * Eq. 4) and FlashAttention (Sec. 3.2.2); both are exact, so every mode below returns the
+ * same result up to rounding.
+ *
+ * Conventions that hold for every entry point
+ *   - Pointers named q, k, v, out, workspace are DEVICE pointers owned by the caller; the
+ *     library never allocates, frees or keeps them.  `stream` is a cudaStream_t passed as
+ *     void* (NULL = the legacy default stream).  Handles and status words are HOST objects.
+ *   - Layout: q and out are dense [B][H][Nq][d], k and v dense [B][H][Nk][d], d innermost,
+ *     no strides; `d` is the true head dim (padding to tensor-core widths is internal).
+ *     `out` must not overlap any input.
+ *   - Every function returns an sd_attn_status.  Validation happens before any launch: a
+ *     non-OK return means nothing was enqueued.  No function throws, aborts or exits.
+ *   - sd_attn_forward is asynchronous and stream-ordered: it does not synchronise, allocate
+ *     or read back.  One handle serves one host thread at a time.
+ */
+#ifndef SD_ATTN_H_
+#define SD_ATTN_H_
+
+#include <stddef.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct sd_attn_handle sd_attn_handle; /* opaque; created and destroyed by the library */
+
+typedef enum {
+    SD_ATTN_OK = 0,
+    SD_ATTN_ERR_INVALID_VALUE = 1,  /* null pointer, non-positive size, non-finite scale, bad mode */
+    SD_ATTN_ERR_UNSUPPORTED = 2,    /* dtype/d/Nk outside what the requested mode implements   */
+    SD_ATTN_ERR_ALIGNMENT = 3,      /* a tensor pointer is not 16-byte aligned                  */
+    SD_ATTN_ERR_WORKSPACE = 4,      /* two-pass mode without enough caller-provided scratch     */
+    SD_ATTN_ERR_ARCH = 5,           /* the current device is not compute capability 10.x        */
+    SD_ATTN_ERR_CUDA = 6,           /* a CUDA runtime/driver call failed                        */
+    SD_ATTN_ERR_DEVICE_TIMEOUT = 7  /* a bounded wait inside a kernel expired (see query_status) */
+} sd_attn_status;
+
+typedef enum {
+    SD_ATTN_F16 = 0, /* IEEE binary16 q/k/v/out, binary32 accumulation            */
+    SD_ATTN_F32 = 1  /* binary32 throughout (plain FMA arithmetic, no TF32)        */
+} sd_attn_dtype;
+
+typedef enum {
+    SD_ATTN_MODE_AUTO = 0,    /* F16: CROSS when Nk fits one key tile, else FUSED.  F32: SIMT */
+    SD_ATTN_MODE_FUSED = 1,   /* single-pass online softmax (FlashAttention, Sec. 3.2.2)      */
+    SD_ATTN_MODE_CROSS = 2,   /* all keys in one shared-memory tile, plain softmax            */
+    SD_ATTN_MODE_TWOPASS = 3, /* partially fused softmax of Sec. 3.2.1: scores and [L,S] in HBM */
+    SD_ATTN_MODE_SIMT = 4     /* CUDA-core kernel, F16 or F32 storage, fp32 arithmetic        */
+} sd_attn_mode;
+
+/* Largest Nk the CROSS mode accepts (one key tile). */
+#define SD_ATTN_CROSS_MAX_NK 128
+/* Largest head dim any mode accepts; F16 tensor-core modes need d to be a multiple of 8. */
+#define SD_ATTN_MAX_D 160
+
+/*
+ * Create a handle on the CURRENT CUDA device.  Checks the architecture (ERR_ARCH unless
+ * compute capability 10.x), resolves the driver's tensor-map encoder, raises the kernels'
+ * dynamic shared-memory limits and allocates one 64-byte device status block.  No stream
+ * work.  *out receives the handle (NULL on failure).
+ */
+int sd_attn_create(sd_attn_handle **out);
+
+/*
+ * out = softmax(q k^T * scale) v, Eq. 3, for every (b, h); see the conventions above.
+ *   B, H, Nq, Nk, d : sizes; all > 0 except Nq == 0, which is an OK no-op.  Nk == 0 is
+ *                     INVALID_VALUE (a softmax over no keys is undefined).
+ *   scale           : the multiplier applied to q.k (1/sqrt(d) in the paper); any finite
+ *                     value, used as given.
+ *   dtype           : sd_attn_dtype of all four tensors.
+ * Errors: INVALID_VALUE, UNSUPPORTED (d > SD_ATTN_MAX_D; F16 tensor-core modes with d % 8 != 0;
+ * CROSS with Nk > SD_ATTN_CROSS_MAX_NK; F32 in a tensor-core mode), ALIGNMENT, WORKSPACE
+ * (TWOPASS only), CUDA.
+ */
+int sd_attn_forward(sd_attn_handle *h, const void *q, const void *k, const void *v, void *out,
+                    int B, int H, int Nq, int Nk, int d, float scale, int dtype, void *stream);
+
+/*
+ * The same operation (Eq. 3) for callers whose tensors live in HOST memory: q, k, v, out are HOST
+ * pointers (pinned memory makes the copies asynchronous; pageable memory works but serialises).
+ * `staging` is caller-owned DEVICE scratch of at least sd_attn_host_staging_bytes(...) bytes,
+ * 256-byte aligned.  Enqueues on `stream`: three host-to-device copies, sd_attn_forward on the
+ * staged tensors, one device-to-host copy of the result.  Does not synchronise: `out` is valid
+ * once the stream has drained.  Errors as sd_attn_forward, plus WORKSPACE if `staging` is NULL,
+ * misaligned or too small.
+ */
+int sd_attn_forward_host(sd_attn_handle *h, const void *q, const void *k, const void *v, void *out,
+                         void *staging, size_t staging_bytes, int B, int H, int Nq, int Nk, int d,
+                         float scale, int dtype, void *stream);
+
+/* Device scratch sd_attn_forward_host needs: q, k, v and out, each rounded up to 256 bytes. */
+size_t sd_attn_host_staging_bytes(int B, int H, int Nq, int Nk, int d, int dtype);
+
+/* Destroy a handle and its status block.  NULL is an OK no-op. */
+int sd_attn_destroy(sd_attn_handle *h);
+
+/* Choose the kernel family for later forwards (default AUTO). */
+int sd_attn_set_mode(sd_attn_handle *h, int mode);
+
+/*
+ * Scratch the TWOPASS mode needs for a call of this shape: the score matrix
+ * A = q k^T * scale as binary32 [B][H][Nq][Nk] (Sec. 3.2.1) followed by the row statistics
+ * [L, S] of Eq. 4 as binary32 [B][H][Nq][2].  Zero for every other mode.
+ */
+size_t sd_attn_workspace_bytes(int mode, int B, int H, int Nq, int Nk, int d, int dtype);
+
+/* Lend caller-owned device scratch (256-byte aligned) to the handle; (NULL, 0) withdraws it. */
+int sd_attn_set_workspace(sd_attn_handle *h, void *workspace, size_t bytes);
+
+/*
+ * After a TWOPASS forward: device pointers into the workspace of that call's score matrix and
+ * [L,S] tensor (valid until the workspace is reused).  Either output pointer may be NULL.
+ */
+int sd_attn_twopass_buffers(sd_attn_handle *h, const float **scores, const float **row_stats);
+
+/*
+ * Synchronise `stream`, then read and clear the device status block.  Returns OK,
+ * ERR_DEVICE_TIMEOUT (a kernel gave up a bounded wait and returned early: the outputs of the
+ * calls since the last query are not valid) or ERR_CUDA.  If `detail` is non-NULL it receives
+ * four host ints: {code, block index, wait site, tile index} of the first failure.
+ */
+int sd_attn_query_status(sd_attn_handle *h, void *stream, int *detail);
+
+/* Which kernel family the last successful forward used (an sd_attn_mode, never AUTO). */
+int sd_attn_last_mode(const sd_attn_handle *h);
+
+/* How many kernels of this library the handle has launched since it was created. */
+long long sd_attn_launch_count(const sd_attn_handle *h);
+
+/* Static, NUL-terminated description of a status code. */
+const char *sd_attn_status_string(int status);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* SD_ATTN_H_ */

@@ -1,0 +1,227 @@
+"""ctypes binding of the C-ABI attention library (argument marshalling only).
+
+Function names mirror ``include/sd_attn.h``.  Tensors are passed as raw device addresses
+(``tensor.data_ptr()``); PyTorch only owns the memory and the streams.  There is no fallback:
+if ``libsd_attn.so`` is missing or fails to load, every call raises.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from typing import Optional
+
+_PKG = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_PKG, "libsd_attn.so")
+
+# status codes, dtypes and modes of include/sd_attn.h
+OK, ERR_INVALID_VALUE, ERR_UNSUPPORTED, ERR_ALIGNMENT, ERR_WORKSPACE, ERR_ARCH, ERR_CUDA, ERR_DEVICE_TIMEOUT = range(8)
+F16, F32 = 0, 1
+MODE_AUTO, MODE_FUSED, MODE_CROSS, MODE_TWOPASS, MODE_SIMT = range(5)
+MODE_NAMES = {MODE_AUTO: "auto", MODE_FUSED: "fused", MODE_CROSS: "cross", MODE_TWOPASS: "twopass",
+              MODE_SIMT: "simt"}
+CROSS_MAX_NK = 128
+MAX_D = 160
+
+EXPORTS = ["sd_attn_create", "sd_attn_forward", "sd_attn_destroy", "sd_attn_set_mode",
+           "sd_attn_workspace_bytes", "sd_attn_set_workspace", "sd_attn_twopass_buffers",
+           "sd_attn_query_status", "sd_attn_last_mode", "sd_attn_launch_count", "sd_attn_status_string",
+           "sd_attn_forward_host", "sd_attn_host_staging_bytes", "sd_attn_debug_dump_cross_scores"]
+
+_lib = None
+
+
+class SdAttnError(RuntimeError):
+    def __init__(self, status: int, where: str):
+        self.status = status
+        super().__init__("%s failed: status %d (%s)" % (where, status, status_string(status)))
+
+
+def load() -> ctypes.CDLL:
+    """Load libsd_attn.so (built in-tree by ``build.py``).  Raises if it is absent."""
+    global _lib
+    if _lib is not None:
+        return _lib
+    if not os.path.exists(LIB_PATH):
+        raise FileNotFoundError(
+            "%s not found: build it with `python -m paper_2304_11267_b200.build` "
+            "(there is no CPU fallback)" % LIB_PATH)
+    lib = ctypes.CDLL(LIB_PATH)
+    vp, ci, cf, sz = ctypes.c_void_p, ctypes.c_int, ctypes.c_float, ctypes.c_size_t
+    lib.sd_attn_create.restype = ci
+    lib.sd_attn_create.argtypes = [ctypes.POINTER(vp)]
+    lib.sd_attn_forward.restype = ci
+    lib.sd_attn_forward.argtypes = [vp, vp, vp, vp, vp, ci, ci, ci, ci, ci, cf, ci, vp]
+    lib.sd_attn_forward_host.restype = ci
+    lib.sd_attn_forward_host.argtypes = [vp, vp, vp, vp, vp, vp, sz, ci, ci, ci, ci, ci, cf, ci, vp]
+    lib.sd_attn_host_staging_bytes.restype = sz
+    lib.sd_attn_host_staging_bytes.argtypes = [ci, ci, ci, ci, ci, ci]
+    lib.sd_attn_destroy.restype = ci
+    lib.sd_attn_destroy.argtypes = [vp]
+    lib.sd_attn_set_mode.restype = ci
+    lib.sd_attn_set_mode.argtypes = [vp, ci]
+    lib.sd_attn_workspace_bytes.restype = sz
+    lib.sd_attn_workspace_bytes.argtypes = [ci, ci, ci, ci, ci, ci, ci]
+    lib.sd_attn_set_workspace.restype = ci
+    lib.sd_attn_set_workspace.argtypes = [vp, vp, sz]
+    lib.sd_attn_twopass_buffers.restype = ci
+    lib.sd_attn_twopass_buffers.argtypes = [vp, ctypes.POINTER(vp), ctypes.POINTER(vp)]
+    lib.sd_attn_query_status.restype = ci
+    lib.sd_attn_query_status.argtypes = [vp, vp, ctypes.POINTER(ci)]
+    lib.sd_attn_last_mode.restype = ci
+    lib.sd_attn_last_mode.argtypes = [vp]
+    lib.sd_attn_launch_count.restype = ctypes.c_longlong
+    lib.sd_attn_launch_count.argtypes = [vp]
+    lib.sd_attn_status_string.restype = ctypes.c_char_p
+    lib.sd_attn_status_string.argtypes = [ci]
+    lib.sd_attn_debug_dump_cross_scores.restype = ci
+    lib.sd_attn_debug_dump_cross_scores.argtypes = [vp, vp]
+    _lib = lib
+    return lib
+
+
+def status_string(status: int) -> str:
+    return load().sd_attn_status_string(int(status)).decode()
+
+
+# ------------------------------------------------------------------ one-to-one wrappers
+
+def sd_attn_create() -> int:
+    h = ctypes.c_void_p()
+    rc = load().sd_attn_create(ctypes.byref(h))
+    if rc != OK:
+        raise SdAttnError(rc, "sd_attn_create")
+    return h.value
+
+
+def sd_attn_destroy(handle: Optional[int]) -> int:
+    return load().sd_attn_destroy(handle)
+
+
+def sd_attn_forward(handle, q, k, v, out, B, H, Nq, Nk, d, scale, dtype, stream=0) -> int:
+    """Raw call: q, k, v, out are device addresses (ints).  Returns the status code."""
+    return load().sd_attn_forward(handle, q, k, v, out, B, H, Nq, Nk, d, ctypes.c_float(scale), dtype,
+                                  stream or None)
+
+
+def sd_attn_forward_host(handle, q, k, v, out, staging, staging_bytes, B, H, Nq, Nk, d, scale, dtype,
+                         stream=0) -> int:
+    """Raw call with HOST addresses for q, k, v, out and a device staging buffer."""
+    return load().sd_attn_forward_host(handle, q, k, v, out, staging, staging_bytes, B, H, Nq, Nk, d,
+                                       ctypes.c_float(scale), dtype, stream or None)
+
+
+def sd_attn_host_staging_bytes(B, H, Nq, Nk, d, dtype) -> int:
+    return int(load().sd_attn_host_staging_bytes(B, H, Nq, Nk, d, dtype))
+
+
+def sd_attn_set_mode(handle, mode: int) -> int:
+    return load().sd_attn_set_mode(handle, mode)
+
+
+def sd_attn_workspace_bytes(mode, B, H, Nq, Nk, d, dtype) -> int:
+    return int(load().sd_attn_workspace_bytes(mode, B, H, Nq, Nk, d, dtype))
+
+
+def sd_attn_set_workspace(handle, ptr, nbytes) -> int:
+    return load().sd_attn_set_workspace(handle, ptr or None, nbytes)
+
+
+def sd_attn_twopass_buffers(handle):
+    a, s = ctypes.c_void_p(), ctypes.c_void_p()
+    rc = load().sd_attn_twopass_buffers(handle, ctypes.byref(a), ctypes.byref(s))
+    if rc != OK:
+        raise SdAttnError(rc, "sd_attn_twopass_buffers")
+    return a.value, s.value
+
+
+def sd_attn_query_status(handle, stream=0):
+    detail = (ctypes.c_int * 4)()
+    rc = load().sd_attn_query_status(handle, stream or None, detail)
+    return rc, list(detail)
+
+
+def sd_attn_last_mode(handle) -> int:
+    return load().sd_attn_last_mode(handle)
+
+
+def sd_attn_launch_count(handle) -> int:
+    return int(load().sd_attn_launch_count(handle))
+
+
+def sd_attn_debug_dump_cross_scores(handle, ptr) -> int:
+    return load().sd_attn_debug_dump_cross_scores(handle, ptr or None)
+
+
+# ------------------------------------------------------------------ convenience for torch tensors
+
+class Attention:
+    """A handle plus torch-tensor marshalling: ``Attention().forward(q, k, v)``."""
+
+    def __init__(self, mode: int = MODE_AUTO):
+        self.handle = sd_attn_create()
+        self._workspace = None
+        if mode != MODE_AUTO:
+            self.set_mode(mode)
+
+    def set_mode(self, mode: int) -> None:
+        rc = sd_attn_set_mode(self.handle, mode)
+        if rc != OK:
+            raise SdAttnError(rc, "sd_attn_set_mode")
+
+    def forward(self, q, k, v, scale: Optional[float] = None, out=None, stream: Optional[int] = None):
+        import torch
+        if not (q.is_cuda and k.is_cuda and v.is_cuda):
+            raise ValueError("q, k, v must be CUDA tensors")
+        if not (q.is_contiguous() and k.is_contiguous() and v.is_contiguous()):
+            raise ValueError("q, k, v must be contiguous [B,H,N,d] tensors")
+        if q.dtype == torch.float16:
+            dtype = F16
+        elif q.dtype == torch.float32:
+            dtype = F32
+        else:
+            raise TypeError("float16 or float32 only")
+        B, H, Nq, d = q.shape
+        Nk = k.shape[2]
+        if out is None:
+            out = torch.empty_like(q)
+        if scale is None:
+            scale = float(d) ** -0.5
+        if stream is None:
+            stream = torch.cuda.current_stream(q.device).cuda_stream
+        rc = sd_attn_forward(self.handle, q.data_ptr(), k.data_ptr(), v.data_ptr(), out.data_ptr(),
+                             B, H, Nq, Nk, d, scale, dtype, stream)
+        if rc == ERR_WORKSPACE:
+            need = sd_attn_workspace_bytes(MODE_TWOPASS, B, H, Nq, Nk, d, dtype)
+            self._workspace = torch.empty(need, dtype=torch.uint8, device=q.device)
+            rc = sd_attn_set_workspace(self.handle, self._workspace.data_ptr(), need)
+            if rc == OK:
+                rc = sd_attn_forward(self.handle, q.data_ptr(), k.data_ptr(), v.data_ptr(), out.data_ptr(),
+                                     B, H, Nq, Nk, d, scale, dtype, stream)
+        if rc != OK:
+            raise SdAttnError(rc, "sd_attn_forward")
+        return out
+
+    def check(self, stream: int = 0) -> None:
+        """Synchronise and raise if a kernel reported an expired wait."""
+        rc, detail = sd_attn_query_status(self.handle, stream)
+        if rc != OK:
+            raise SdAttnError(rc, "device status %s" % detail)
+
+    @property
+    def last_mode(self) -> int:
+        return sd_attn_last_mode(self.handle)
+
+    @property
+    def launch_count(self) -> int:
+        return sd_attn_launch_count(self.handle)
+
+    def close(self) -> None:
+        if self.handle:
+            sd_attn_destroy(self.handle)
+            self.handle = None
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass

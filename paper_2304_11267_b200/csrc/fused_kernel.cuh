@@ -1,0 +1,327 @@
+// Fused single-pass attention (the FlashAttention evaluation of Eq. 3, Sec. 3.2.2) for sm_100a.
+//
+// The score matrix never leaves the chip: keys and values stream through shared memory in tiles of
+// BN keys, S = Q K^T lands in tensor memory, the softmax reductions of Eq. 4 are kept as running
+// per-row (max, sum), and O accumulates in tensor memory.  The paper keeps this kernel to d = 40
+// because its accumulators live in registers on mobile GPUs; here they live in the 512-column
+// tensor memory, so every head dim up to 160 takes the same path.
+//
+// One CTA owns TWO tiles of 128 query rows and ping-pongs between them so that the tensor pipe
+// works on one tile while the other is in its softmax:
+//   warps 0-3  softmax of tile 0 (thread = query row = TMEM lane)      warp 8  TMA producer
+//   warps 4-7  softmax of tile 1                                        warp 9  MMA issuer, TMEM owner
+// Per key tile j and query tile t:
+//   S_t = Q_t K_j^T          tcgen05.mma, both operands from swizzled shared memory
+//   softmax warps            row max; O_t is rescaled only when the running max grew by more than
+//                            2^8 (so p <= 256 fits fp16); p = exp2(s*c - m*c); P_t as packed fp16 over
+//                            the columns of S_t
+//   O_t += P_t V_j           tcgen05.mma, P from tensor memory, V as an N-major shared-memory operand
+// All waits are bounded; an expired wait raises a block-wide abort flag and the kernel returns.
+#pragma once
+#include <cuda.h>
+
+#include "cross_kernel.cuh"  // TILE_M, CHUNK_COLS, CHUNK_ROW_BYTES
+#include "tc_common.cuh"
+
+namespace sd_attn {
+
+constexpr int FUSED_THREADS = 320;
+constexpr int FUSED_MAX_STAGES = 4;
+constexpr int FUSED_SMEM_BUDGET = 220 * 1024;
+constexpr float FUSED_RESCALE_LOG2 = 8.0f;  // rescale O only when the max grew by more than 2^8
+
+struct FusedArgs {
+    __half* out;  // [BH][Nq][d]
+    int Nq, Nk, d;
+    int dpad;     // d rounded up to 16
+    int nch;      // 64-column chunks per row
+    int stages;   // K/V ring depth
+    float scale_log2e;
+    int negate;
+    int* status;
+};
+
+__host__ inline int fused_block_n(int d) { return ((d + 15) / 16 * 16) <= 128 ? 128 : 64; }
+
+__host__ inline void fused_fill_args(FusedArgs* a, __half* out, int Nq, int Nk, int d, float scale_log2e, bool negate,
+                                     int* status) {
+    a->out = out;
+    a->Nq = Nq; a->Nk = Nk; a->d = d;
+    a->dpad = (d + 15) / 16 * 16;
+    a->nch = (d + CHUNK_COLS - 1) / CHUNK_COLS;
+    const int bn = fused_block_n(d);
+    const int q_bytes = 2 * a->nch * TILE_M * CHUNK_ROW_BYTES;
+    const int stage_bytes = 2 * a->nch * bn * CHUNK_ROW_BYTES;
+    int stages = (FUSED_SMEM_BUDGET - q_bytes) / stage_bytes;
+    if (stages > FUSED_MAX_STAGES) stages = FUSED_MAX_STAGES;
+    a->stages = stages;
+    a->scale_log2e = scale_log2e;
+    a->negate = negate ? 1 : 0;
+    a->status = status;
+}
+
+__host__ inline size_t fused_smem_bytes(const FusedArgs& a) {
+    const int bn = fused_block_n(a.d);
+    return (size_t)2 * a.nch * TILE_M * CHUNK_ROW_BYTES + (size_t)a.stages * 2 * a.nch * bn * CHUNK_ROW_BYTES + 1024;
+}
+__host__ inline size_t fused_smem_bytes_max() { return FUSED_SMEM_BUDGET + 1024; }
+
+enum {
+    SITE_F_Q = 10, SITE_F_K = 11, SITE_F_V = 12, SITE_F_EMPTY = 13, SITE_F_S = 14, SITE_F_P = 15, SITE_F_O = 16
+};
+
+template <int BN>
+__global__ void __launch_bounds__(FUSED_THREADS, 1)
+fused_attention_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__ CUtensorMap tmap_k,
+                       const __grid_constant__ CUtensorMap tmap_v, const FusedArgs args) {
+    extern __shared__ uint8_t fused_smem_raw[];
+    __shared__ __align__(8) uint64_t bar_q_full[2], bar_s_full[2], bar_p_full[2], bar_o_full[2];
+    __shared__ __align__(8) uint64_t bar_k_full[FUSED_MAX_STAGES], bar_v_full[FUSED_MAX_STAGES],
+        bar_kv_empty[FUSED_MAX_STAGES];
+    __shared__ uint32_t tmem_base_slot;
+    __shared__ int abort_flag;
+
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int bh = blockIdx.y;
+    const int row_base = blockIdx.x * 2 * TILE_M;
+    const int n_qtiles = (row_base + TILE_M < args.Nq) ? 2 : 1;
+    const int n_kv = (args.Nk + BN - 1) / BN;
+    const int nch = args.nch, dpad = args.dpad, stages = args.stages;
+
+    const uint32_t smem_base = (smem_u32(fused_smem_raw) + 1023u) & ~1023u;
+    const uint32_t q_tile_bytes = nch * TILE_M * CHUNK_ROW_BYTES;
+    const uint32_t kv_tile_bytes = nch * BN * CHUNK_ROW_BYTES;
+    const uint32_t q_smem = smem_base;                       // [2][nch][128 rows][128 B]
+    const uint32_t kv_smem = q_smem + 2 * q_tile_bytes;      // [stages][K | V][nch][BN rows][128 B]
+    volatile int* abort_p = &abort_flag;
+
+    if (tid == 0) {
+        abort_flag = 0;
+        for (int t = 0; t < 2; ++t) {
+            mbar_init(smem_u32(&bar_q_full[t]), 1);
+            mbar_init(smem_u32(&bar_s_full[t]), 1);
+            mbar_init(smem_u32(&bar_p_full[t]), TILE_M);
+            mbar_init(smem_u32(&bar_o_full[t]), 1);
+        }
+        for (int s = 0; s < FUSED_MAX_STAGES; ++s) {
+            mbar_init(smem_u32(&bar_k_full[s]), 1);
+            mbar_init(smem_u32(&bar_v_full[s]), 1);
+            mbar_init(smem_u32(&bar_kv_empty[s]), 1);
+        }
+        mbar_init_fence();
+    }
+    if (warp == 9) {
+        tmem_alloc(smem_u32(&tmem_base_slot), 512);
+        tmem_relinquish();
+    }
+    tc_fence_before_sync();
+    __syncthreads();
+    tc_fence_after_sync();
+    const uint32_t tmem_base = tmem_base_slot;
+    // columns: S_0 | S_1 | O_0 | O_1 ; P_t reuses the first BN/2 columns of S_t
+    const uint32_t tmem_o0 = tmem_base + 2 * BN;
+
+    if (warp == 8) {
+        // ------------------------------------------------------------ TMA producer
+        if (lane == 0) {
+            tma_prefetch_desc(&tmap_q);
+            tma_prefetch_desc(&tmap_k);
+            tma_prefetch_desc(&tmap_v);
+            for (int t = 0; t < n_qtiles; ++t) {
+                const uint32_t bar = smem_u32(&bar_q_full[t]);
+                mbar_arrive_expect_tx(bar, q_tile_bytes);
+                for (int ch = 0; ch < nch; ++ch)
+                    tma_load_3d(q_smem + t * q_tile_bytes + ch * TILE_M * CHUNK_ROW_BYTES, &tmap_q, bar,
+                                ch * CHUNK_COLS, row_base + t * TILE_M, bh);
+            }
+            for (int j = 0; j < n_kv; ++j) {
+                const int s = j % stages;
+                if (j >= stages &&
+                    !mbar_wait(smem_u32(&bar_kv_empty[s]), ((j / stages) - 1) & 1, abort_p, args.status, SITE_F_EMPTY, j))
+                    break;
+                const uint32_t k_dst = kv_smem + s * 2 * kv_tile_bytes, v_dst = k_dst + kv_tile_bytes;
+                const uint32_t bk = smem_u32(&bar_k_full[s]), bv = smem_u32(&bar_v_full[s]);
+                mbar_arrive_expect_tx(bk, kv_tile_bytes);
+                for (int ch = 0; ch < nch; ++ch)
+                    tma_load_3d(k_dst + ch * BN * CHUNK_ROW_BYTES, &tmap_k, bk, ch * CHUNK_COLS, j * BN, bh);
+                mbar_arrive_expect_tx(bv, kv_tile_bytes);
+                for (int ch = 0; ch < nch; ++ch)
+                    tma_load_3d(v_dst + ch * BN * CHUNK_ROW_BYTES, &tmap_v, bv, ch * CHUNK_COLS, j * BN, bh);
+            }
+        }
+    } else if (warp == 9) {
+        // ------------------------------------------------------------ MMA issuer
+        if (lane == 0) {
+            const uint32_t idesc_s = idesc_f16(TILE_M, BN, false, false, args.negate != 0);
+            const uint32_t idesc_o = idesc_f16(TILE_M, dpad, false, true, false);
+            const int ksteps_s = (args.d + 15) / 16;
+            auto issue_s = [&](int t, int s) {   // S_t = Q_t K_s^T
+                const uint32_t qa = q_smem + t * q_tile_bytes, kb = kv_smem + s * 2 * kv_tile_bytes;
+                for (int kk = 0; kk < ksteps_s; ++kk) {
+                    const int ch = kk >> 2, within = (kk & 3) * 32;
+                    mma_f16_ss(tmem_base + t * BN,
+                               smem_desc_sw128(qa + ch * TILE_M * CHUNK_ROW_BYTES + within, 16, 1024),
+                               smem_desc_sw128(kb + ch * BN * CHUNK_ROW_BYTES + within, 16, 1024), idesc_s, kk > 0);
+                }
+                tc_commit(smem_u32(&bar_s_full[t]));
+            };
+            auto issue_o = [&](int t, int s, bool accumulate) {   // O_t (+)= P_t V_s
+                const uint32_t vb = kv_smem + s * 2 * kv_tile_bytes + kv_tile_bytes;
+#pragma unroll
+                for (int kk = 0; kk < BN / 16; ++kk)
+                    mma_f16_ts(tmem_o0 + t * dpad, tmem_base + t * BN + kk * 8,
+                               smem_desc_sw128(vb + kk * 16 * CHUNK_ROW_BYTES, BN * CHUNK_ROW_BYTES, 1024), idesc_o,
+                               accumulate || kk > 0);
+            };
+            bool ok = true;
+            for (int t = 0; t < n_qtiles && ok; ++t)
+                ok = mbar_wait(smem_u32(&bar_q_full[t]), 0, abort_p, args.status, SITE_F_Q, t);
+            if (ok) ok = mbar_wait(smem_u32(&bar_k_full[0]), 0, abort_p, args.status, SITE_F_K, 0);
+            if (ok) {
+                tc_fence_after_sync();
+                for (int t = 0; t < n_qtiles; ++t) issue_s(t, 0);
+            }
+            for (int j = 0; j < n_kv && ok; ++j) {
+                const int s = j % stages;
+                ok = mbar_wait(smem_u32(&bar_v_full[s]), (j / stages) & 1, abort_p, args.status, SITE_F_V, j);
+                for (int t = 0; t < n_qtiles && ok; ++t) {
+                    ok = mbar_wait(smem_u32(&bar_p_full[t]), j & 1, abort_p, args.status, SITE_F_P, j);
+                    if (!ok) break;
+                    tc_fence_after_sync();
+                    issue_o(t, s, j > 0);
+                    if (t == n_qtiles - 1) tc_commit(smem_u32(&bar_kv_empty[s]));  // K_j and V_j fully consumed
+                    if (j + 1 < n_kv) {
+                        const int s1 = (j + 1) % stages;
+                        ok = mbar_wait(smem_u32(&bar_k_full[s1]), ((j + 1) / stages) & 1, abort_p, args.status,
+                                       SITE_F_K, j + 1);
+                        if (!ok) break;
+                        tc_fence_after_sync();
+                        issue_s(t, s1);
+                    } else {
+                        tc_commit(smem_u32(&bar_o_full[t]));
+                    }
+                }
+            }
+        }
+    } else {
+        // ------------------------------------------------------------ softmax warps
+        const int t = warp >> 2;                 // query tile of this warpgroup
+        if (t < n_qtiles) {
+            const int r = tid & (TILE_M - 1);    // row inside the tile = TMEM lane
+            const uint32_t lane_off = (uint32_t)((warp & 3) * 32) << 16;
+            const uint32_t tmem_s = tmem_base + t * BN + lane_off;
+            const uint32_t tmem_o = tmem_o0 + t * dpad + lane_off;
+            const float c2 = args.scale_log2e;
+            float m_run = -INFINITY;  // running max, in raw score units
+            float l_run = 0.f;        // running sum of p (relative to m_run)
+            bool ok = true;
+            for (int j = 0; j < n_kv; ++j) {
+                ok = mbar_wait(smem_u32(&bar_s_full[t]), j & 1, abort_p, args.status, SITE_F_S, j);
+                ok = __all_sync(0xffffffffu, ok);
+                if (!ok) break;
+                tc_fence_after_sync();
+                const int valid = args.Nk - j * BN;   // columns >= valid are zero-filled keys
+                float row_max = -INFINITY;
+#pragma unroll
+                for (int g = 0; g < BN / 16; ++g) {
+                    uint32_t x[16];
+                    tmem_ld16(tmem_s + g * 16, x);
+                    tmem_wait_ld();
+                    if (valid >= BN) {
+#pragma unroll
+                        for (int c = 0; c < 16; ++c) row_max = fmaxf(row_max, __uint_as_float(x[c]));
+                    } else {
+#pragma unroll
+                        for (int c = 0; c < 16; ++c)
+                            if (g * 16 + c < valid) row_max = fmaxf(row_max, __uint_as_float(x[c]));
+                    }
+                }
+                if (j == 0) {
+                    m_run = row_max;
+                } else {
+                    const bool grow = (row_max - m_run) * c2 > FUSED_RESCALE_LOG2;
+                    if (__any_sync(0xffffffffu, grow)) {
+                        const float alpha = grow ? ex2_approx((m_run - row_max) * c2) : 1.f;
+                        if (grow) m_run = row_max;
+                        l_run *= alpha;
+                        for (int g = 0; g < (dpad >> 4); ++g) {
+                            uint32_t x[16];
+                            tmem_ld16(tmem_o + g * 16, x);
+                            tmem_wait_ld();
+#pragma unroll
+                            for (int c = 0; c < 16; ++c) x[c] = __float_as_uint(__uint_as_float(x[c]) * alpha);
+                            tmem_st16(tmem_o + g * 16, x);
+                        }
+                    }
+                }
+                const float neg_mc = -m_run * c2;
+#pragma unroll
+                for (int g = 0; g < BN / 16; ++g) {
+                    uint32_t x[16], packed[8];
+                    tmem_ld16(tmem_s + g * 16, x);
+                    tmem_wait_ld();
+                    float p[16];
+#pragma unroll
+                    for (int c = 0; c < 16; ++c) p[c] = ex2_approx(fmaf(__uint_as_float(x[c]), c2, neg_mc));
+                    if (valid < BN) {
+#pragma unroll
+                        for (int c = 0; c < 16; ++c)
+                            if (g * 16 + c >= valid) p[c] = 0.f;
+                    }
+#pragma unroll
+                    for (int c = 0; c < 16; ++c) l_run += p[c];
+#pragma unroll
+                    for (int c = 0; c < 8; ++c) packed[c] = pack_half2(p[2 * c], p[2 * c + 1]);
+                    tmem_st8(tmem_s + g * 8, packed);
+                }
+                tmem_wait_st();
+                tc_fence_before_sync();
+                mbar_arrive(smem_u32(&bar_p_full[t]));
+            }
+            if (ok) ok = mbar_wait(smem_u32(&bar_o_full[t]), 0, abort_p, args.status, SITE_F_O, t);
+            ok = __all_sync(0xffffffffu, ok);
+            if (ok) {
+                tc_fence_after_sync();
+                const float inv = 1.f / l_run;
+                const int row = row_base + t * TILE_M + r;
+                __half* orow = args.out + ((size_t)bh * args.Nq + row) * args.d;
+                for (int g = 0; g < (dpad >> 4); ++g) {
+                    uint32_t x[16];
+                    tmem_ld16(tmem_o + g * 16, x);
+                    tmem_wait_ld();
+                    uint4 lo, hi;
+                    lo.x = pack_half2(__uint_as_float(x[0]) * inv, __uint_as_float(x[1]) * inv);
+                    lo.y = pack_half2(__uint_as_float(x[2]) * inv, __uint_as_float(x[3]) * inv);
+                    lo.z = pack_half2(__uint_as_float(x[4]) * inv, __uint_as_float(x[5]) * inv);
+                    lo.w = pack_half2(__uint_as_float(x[6]) * inv, __uint_as_float(x[7]) * inv);
+                    hi.x = pack_half2(__uint_as_float(x[8]) * inv, __uint_as_float(x[9]) * inv);
+                    hi.y = pack_half2(__uint_as_float(x[10]) * inv, __uint_as_float(x[11]) * inv);
+                    hi.z = pack_half2(__uint_as_float(x[12]) * inv, __uint_as_float(x[13]) * inv);
+                    hi.w = pack_half2(__uint_as_float(x[14]) * inv, __uint_as_float(x[15]) * inv);
+                    if (row < args.Nq) {
+                        if (g * 16 + 8 <= args.d) *reinterpret_cast<uint4*>(orow + g * 16) = lo;
+                        if (g * 16 + 16 <= args.d) *reinterpret_cast<uint4*>(orow + g * 16 + 8) = hi;
+                    }
+                }
+            }
+        }
+    }
+
+    // ------------------------------------------------------------ teardown (every thread arrives)
+    tc_fence_before_sync();
+    __syncthreads();
+    if (warp == 8 && lane == 0 && abort_flag) {
+        // gave up somewhere: give copies still in flight a bounded chance to land
+        for (int s = 0; s < stages; ++s) {
+            mbar_drain(smem_u32(&bar_k_full[s]), 0);
+            mbar_drain(smem_u32(&bar_v_full[s]), 0);
+        }
+    }
+    __syncthreads();
+    if (warp == 9) {
+        __syncwarp();
+        tmem_dealloc(tmem_base, 512);
+    }
+}
+
+}  // namespace sd_attn

@@ -1,0 +1,378 @@
+// Host side of the C ABI declared in include/sd_attn.h: handle management, argument validation,
+// kernel selection, TMA tensor-map construction and launches.  No entry point here synchronises
+// (except query_status, whose job it is), allocates in forward, or touches caller tensors on the host.
+#include <cuda.h>
+#include <cuda_fp16.h>
+#include <cuda_runtime.h>
+#include <math.h>
+#include <stdint.h>
+#include <stdio.h>
+#include <stdlib.h>
+#include <string.h>
+
+#include "../../include/sd_attn.h"
+#include "../../include/sd_attn_debug.h"
+#include "cross_kernel.cuh"
+#include "fused_kernel.cuh"
+#include "simt_kernel.cuh"
+#include "twopass_kernel.cuh"
+
+using namespace sd_attn;
+
+typedef CUresult (*encode_tiled_fn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                    const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                    CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+struct sd_attn_handle {
+    int device;
+    int mode;
+    int last_mode;
+    long long launches;
+    int* dev_status;          // DEV_STATUS_INTS ints on the device
+    void* workspace;          // caller-owned
+    size_t workspace_bytes;
+    const float* tp_scores;   // where the last TWOPASS call put A and [L,S]
+    const float* tp_stats;
+    float* dump_scores;       // bring-up hook of the cross kernel (see sd_attn_debug.h)
+    encode_tiled_fn encode_tiled;
+    cudaError_t last_cuda_error;
+    int sm_count;
+};
+
+static const float LOG2E = 1.4426950408889634f;
+
+extern "C" const char* sd_attn_status_string(int status) {
+    switch (status) {
+        case SD_ATTN_OK: return "ok";
+        case SD_ATTN_ERR_INVALID_VALUE: return "invalid value";
+        case SD_ATTN_ERR_UNSUPPORTED: return "unsupported dtype, head dim or size for the requested mode";
+        case SD_ATTN_ERR_ALIGNMENT: return "pointer not 16-byte aligned";
+        case SD_ATTN_ERR_WORKSPACE: return "two-pass workspace missing or too small";
+        case SD_ATTN_ERR_ARCH: return "device is not compute capability 10.x (sm_100)";
+        case SD_ATTN_ERR_CUDA: return "a CUDA call failed";
+        case SD_ATTN_ERR_DEVICE_TIMEOUT: return "a bounded wait inside a kernel expired";
+        default: return "unknown status";
+    }
+}
+
+static int cuda_fail(sd_attn_handle* h, cudaError_t e) {
+    if (h) h->last_cuda_error = e;
+    if (getenv("SD_ATTN_LOG")) fprintf(stderr, "[sd_attn] CUDA error: %s\n", cudaGetErrorString(e));
+    return SD_ATTN_ERR_CUDA;
+}
+
+template <typename K>
+static cudaError_t raise_smem_limit(K kernel, size_t bytes) {
+    return cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bytes);
+}
+
+extern "C" int sd_attn_create(sd_attn_handle** out) {
+    if (!out) return SD_ATTN_ERR_INVALID_VALUE;
+    *out = nullptr;
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return cuda_fail(nullptr, e);
+    int major = 0, sms = 0;
+    e = cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev);
+    if (e != cudaSuccess) return cuda_fail(nullptr, e);
+    if (major != 10) return SD_ATTN_ERR_ARCH;
+    cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+
+    sd_attn_handle* h = (sd_attn_handle*)calloc(1, sizeof(sd_attn_handle));
+    if (!h) return SD_ATTN_ERR_INVALID_VALUE;
+    h->device = dev;
+    h->mode = SD_ATTN_MODE_AUTO;
+    h->last_mode = SD_ATTN_MODE_AUTO;
+    h->sm_count = sms;
+
+    void* fn = nullptr;
+    cudaDriverEntryPointQueryResult qres;
+    e = cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres);
+    if (e != cudaSuccess || qres != cudaDriverEntryPointSuccess || !fn) {
+        free(h);
+        return cuda_fail(nullptr, e != cudaSuccess ? e : cudaErrorUnknown);
+    }
+    h->encode_tiled = (encode_tiled_fn)fn;
+
+    // dynamic shared memory ceilings of every kernel, once
+    e = raise_smem_limit(cross_attention_kernel, cross_smem_bytes(3, 128));
+    if (e == cudaSuccess) e = raise_smem_limit(fused_attention_kernel<128>, fused_smem_bytes_max());
+    if (e == cudaSuccess) e = raise_smem_limit(fused_attention_kernel<64>, fused_smem_bytes_max());
+    if (e == cudaSuccess) e = raise_smem_limit(twopass_scores_kernel, twopass_scores_smem_bytes(3));
+    if (e == cudaSuccess) e = raise_smem_limit(twopass_pv_kernel, twopass_pv_smem_bytes(3));
+    if (e == cudaSuccess) e = raise_smem_limit(simt_attention_kernel<float, 5>, simt_smem_bytes(160));
+    if (e == cudaSuccess) e = raise_smem_limit(simt_attention_kernel<__half, 5>, simt_smem_bytes(160));
+    if (e == cudaSuccess) e = raise_smem_limit(simt_attention_kernel<float, 4>, simt_smem_bytes(128));
+    if (e == cudaSuccess) e = raise_smem_limit(simt_attention_kernel<__half, 4>, simt_smem_bytes(128));
+    if (e == cudaSuccess) e = cudaMalloc((void**)&h->dev_status, sizeof(int) * DEV_STATUS_INTS);
+    if (e == cudaSuccess) e = cudaMemset(h->dev_status, 0, sizeof(int) * DEV_STATUS_INTS);
+    if (e != cudaSuccess) {
+        if (h->dev_status) cudaFree(h->dev_status);
+        free(h);
+        return cuda_fail(nullptr, e);
+    }
+    *out = h;
+    return SD_ATTN_OK;
+}
+
+extern "C" int sd_attn_destroy(sd_attn_handle* h) {
+    if (!h) return SD_ATTN_OK;
+    cudaError_t e = cudaSuccess;
+    if (h->dev_status) e = cudaFree(h->dev_status);
+    free(h);
+    return e == cudaSuccess ? SD_ATTN_OK : SD_ATTN_ERR_CUDA;
+}
+
+extern "C" int sd_attn_set_mode(sd_attn_handle* h, int mode) {
+    if (!h || mode < SD_ATTN_MODE_AUTO || mode > SD_ATTN_MODE_SIMT) return SD_ATTN_ERR_INVALID_VALUE;
+    h->mode = mode;
+    return SD_ATTN_OK;
+}
+
+extern "C" size_t sd_attn_workspace_bytes(int mode, int B, int H, int Nq, int Nk, int d, int dtype) {
+    (void)d;
+    (void)dtype;
+    if (mode != SD_ATTN_MODE_TWOPASS || B <= 0 || H <= 0 || Nq <= 0 || Nk <= 0) return 0;
+    const size_t rows = (size_t)B * H * Nq;
+    const size_t scores = (rows * (size_t)Nk * sizeof(float) + 255) & ~(size_t)255;
+    return scores + rows * 2 * sizeof(float);
+}
+
+extern "C" int sd_attn_set_workspace(sd_attn_handle* h, void* workspace, size_t bytes) {
+    if (!h) return SD_ATTN_ERR_INVALID_VALUE;
+    if ((workspace == nullptr) != (bytes == 0)) return SD_ATTN_ERR_INVALID_VALUE;
+    if (((uintptr_t)workspace & 255u) != 0) return SD_ATTN_ERR_ALIGNMENT;
+    h->workspace = workspace;
+    h->workspace_bytes = bytes;
+    return SD_ATTN_OK;
+}
+
+extern "C" int sd_attn_twopass_buffers(sd_attn_handle* h, const float** scores, const float** row_stats) {
+    if (!h || !h->tp_scores) return SD_ATTN_ERR_INVALID_VALUE;
+    if (scores) *scores = h->tp_scores;
+    if (row_stats) *row_stats = h->tp_stats;
+    return SD_ATTN_OK;
+}
+
+extern "C" int sd_attn_last_mode(const sd_attn_handle* h) { return h ? h->last_mode : SD_ATTN_MODE_AUTO; }
+extern "C" long long sd_attn_launch_count(const sd_attn_handle* h) { return h ? h->launches : 0; }
+
+extern "C" int sd_attn_debug_dump_cross_scores(sd_attn_handle* h, float* device_buffer) {
+    if (!h) return SD_ATTN_ERR_INVALID_VALUE;
+    h->dump_scores = device_buffer;
+    return SD_ATTN_OK;
+}
+
+extern "C" int sd_attn_query_status(sd_attn_handle* h, void* stream, int* detail) {
+    if (!h) return SD_ATTN_ERR_INVALID_VALUE;
+    int host[DEV_STATUS_INTS];
+    cudaStream_t s = (cudaStream_t)stream;
+    cudaError_t e = cudaStreamSynchronize(s);
+    if (e == cudaSuccess) e = cudaMemcpy(host, h->dev_status, sizeof(host), cudaMemcpyDeviceToHost);
+    if (e != cudaSuccess) return cuda_fail(h, e);
+    if (detail) memcpy(detail, host, 4 * sizeof(int));
+    if (host[0] != 0) {
+        e = cudaMemset(h->dev_status, 0, sizeof(host));
+        if (e != cudaSuccess) return cuda_fail(h, e);
+        return SD_ATTN_ERR_DEVICE_TIMEOUT;
+    }
+    return SD_ATTN_OK;
+}
+
+// A [BH][N][d] fp16 tensor seen by the TMA as (x = d, y = N, z = BH); tiles are 64 columns wide
+// (one 128-byte swizzled row) by `box_rows` rows.  Columns >= d and rows >= N read as zero.
+static int make_tmap(sd_attn_handle* h, CUtensorMap* map, const void* base, int BH, int N, int d, int box_rows) {
+    cuuint64_t dims[3] = {(cuuint64_t)d, (cuuint64_t)N, (cuuint64_t)BH};
+    cuuint64_t strides[2] = {(cuuint64_t)d * 2, (cuuint64_t)N * d * 2};
+    cuuint32_t box[3] = {(cuuint32_t)CHUNK_COLS, (cuuint32_t)box_rows, 1};
+    cuuint32_t estr[3] = {1, 1, 1};
+    CUresult r = h->encode_tiled(map, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 3, const_cast<void*>(base), dims, strides, box,
+                                 estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                                 CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (r != CUDA_SUCCESS) {
+        if (getenv("SD_ATTN_LOG")) fprintf(stderr, "[sd_attn] cuTensorMapEncodeTiled failed: %d\n", (int)r);
+        h->last_cuda_error = cudaErrorInvalidValue;
+        return SD_ATTN_ERR_CUDA;
+    }
+    return SD_ATTN_OK;
+}
+
+static int next_pow2_cols(int cols) {
+    int p = 32;
+    while (p < cols) p <<= 1;
+    return p;
+}
+
+struct Problem {
+    const void *q, *k, *v;
+    void* out;
+    int BH, Nq, Nk, d;
+    float scale;
+    cudaStream_t stream;
+};
+
+template <typename T>
+static int launch_simt(sd_attn_handle* h, const Problem& p) {
+    dim3 grid((p.Nq + SIMT_BLOCK_ROWS - 1) / SIMT_BLOCK_ROWS, p.BH), block(SIMT_WARPS * 32);
+    const size_t smem = simt_smem_bytes(p.d);
+    const T *q = (const T*)p.q, *k = (const T*)p.k, *v = (const T*)p.v;
+    T* o = (T*)p.out;
+    switch ((p.d + 31) / 32) {
+        case 1: simt_attention_kernel<T, 1><<<grid, block, smem, p.stream>>>(q, k, v, o, p.Nq, p.Nk, p.d, p.scale); break;
+        case 2: simt_attention_kernel<T, 2><<<grid, block, smem, p.stream>>>(q, k, v, o, p.Nq, p.Nk, p.d, p.scale); break;
+        case 3: simt_attention_kernel<T, 3><<<grid, block, smem, p.stream>>>(q, k, v, o, p.Nq, p.Nk, p.d, p.scale); break;
+        case 4: simt_attention_kernel<T, 4><<<grid, block, smem, p.stream>>>(q, k, v, o, p.Nq, p.Nk, p.d, p.scale); break;
+        default: simt_attention_kernel<T, 5><<<grid, block, smem, p.stream>>>(q, k, v, o, p.Nq, p.Nk, p.d, p.scale); break;
+    }
+    cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess) return cuda_fail(h, e);
+    h->launches += 1;
+    return SD_ATTN_OK;
+}
+
+static int launch_cross(sd_attn_handle* h, const Problem& p) {
+    CrossArgs a;
+    a.out = (__half*)p.out;
+    a.Nq = p.Nq; a.Nk = p.Nk; a.d = p.d;
+    a.kn = (p.Nk + 15) / 16 * 16;
+    a.dpad = (p.d + 15) / 16 * 16;
+    a.nch = (p.d + CHUNK_COLS - 1) / CHUNK_COLS;
+    a.tmem_cols = next_pow2_cols(a.kn + a.dpad);
+    a.scale_log2e = fabsf(p.scale) * LOG2E;
+    a.negate = p.scale < 0.f;
+    a.status = h->dev_status;
+    a.dump_scores = h->dump_scores;
+    CUtensorMap tq, tk, tv;
+    int rc = make_tmap(h, &tq, p.q, p.BH, p.Nq, p.d, TILE_M);
+    if (rc == SD_ATTN_OK) rc = make_tmap(h, &tk, p.k, p.BH, p.Nk, p.d, a.kn);
+    if (rc == SD_ATTN_OK) rc = make_tmap(h, &tv, p.v, p.BH, p.Nk, p.d, a.kn);
+    if (rc != SD_ATTN_OK) return rc;
+    dim3 grid((p.Nq + TILE_M - 1) / TILE_M, p.BH), block(CROSS_THREADS);
+    cross_attention_kernel<<<grid, block, cross_smem_bytes(a.nch, a.kn), p.stream>>>(tq, tk, tv, a);
+    cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess) return cuda_fail(h, e);
+    h->launches += 1;
+    return SD_ATTN_OK;
+}
+
+static int launch_fused(sd_attn_handle* h, const Problem& p) {
+    FusedArgs a;
+    const int bn = fused_block_n(p.d);
+    fused_fill_args(&a, (__half*)p.out, p.Nq, p.Nk, p.d, fabsf(p.scale) * LOG2E, p.scale < 0.f, h->dev_status);
+    CUtensorMap tq, tk, tv;
+    int rc = make_tmap(h, &tq, p.q, p.BH, p.Nq, p.d, TILE_M);
+    if (rc == SD_ATTN_OK) rc = make_tmap(h, &tk, p.k, p.BH, p.Nk, p.d, bn);
+    if (rc == SD_ATTN_OK) rc = make_tmap(h, &tv, p.v, p.BH, p.Nk, p.d, bn);
+    if (rc != SD_ATTN_OK) return rc;
+    dim3 grid((p.Nq + 2 * TILE_M - 1) / (2 * TILE_M), p.BH), block(FUSED_THREADS);
+    if (bn == 128)
+        fused_attention_kernel<128><<<grid, block, fused_smem_bytes(a), p.stream>>>(tq, tk, tv, a);
+    else
+        fused_attention_kernel<64><<<grid, block, fused_smem_bytes(a), p.stream>>>(tq, tk, tv, a);
+    cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess) return cuda_fail(h, e);
+    h->launches += 1;
+    return SD_ATTN_OK;
+}
+
+static int launch_twopass(sd_attn_handle* h, const Problem& p) {
+    const size_t need = sd_attn_workspace_bytes(SD_ATTN_MODE_TWOPASS, p.BH, 1, p.Nq, p.Nk, p.d, SD_ATTN_F16);
+    if (!h->workspace || h->workspace_bytes < need) return SD_ATTN_ERR_WORKSPACE;
+    const size_t rows = (size_t)p.BH * p.Nq;
+    float* scores = (float*)h->workspace;
+    float* stats = (float*)((char*)h->workspace + ((rows * (size_t)p.Nk * sizeof(float) + 255) & ~(size_t)255));
+    TwoPassArgs a;
+    twopass_fill_args(&a, scores, stats, (__half*)p.out, p.Nq, p.Nk, p.d, p.scale, h->dev_status);
+    CUtensorMap tq, tk, tv;
+    int rc = make_tmap(h, &tq, p.q, p.BH, p.Nq, p.d, TILE_M);
+    if (rc == SD_ATTN_OK) rc = make_tmap(h, &tk, p.k, p.BH, p.Nk, p.d, TWOPASS_BN);
+    if (rc == SD_ATTN_OK) rc = make_tmap(h, &tv, p.v, p.BH, p.Nk, p.d, TWOPASS_BN);
+    if (rc != SD_ATTN_OK) return rc;
+    dim3 grid((p.Nq + TILE_M - 1) / TILE_M, p.BH);
+    // pass 1 (Sec. 3.2.1): A = q k^T * scale to HBM, per-block partial (max, sum), final [L, S]
+    twopass_scores_kernel<<<grid, TWOPASS_THREADS, twopass_scores_smem_bytes(a.nch), p.stream>>>(tq, tk, a);
+    cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess) return cuda_fail(h, e);
+    // pass 2: exp(a - L) / S applied while A is loaded as the left operand of the product with V
+    twopass_pv_kernel<<<grid, TWOPASS_THREADS, twopass_pv_smem_bytes(a.nch), p.stream>>>(tv, a);
+    e = cudaGetLastError();
+    if (e != cudaSuccess) return cuda_fail(h, e);
+    h->launches += 2;
+    h->tp_scores = scores;
+    h->tp_stats = stats;
+    return SD_ATTN_OK;
+}
+
+extern "C" int sd_attn_forward(sd_attn_handle* h, const void* q, const void* k, const void* v, void* out, int B, int H,
+                               int Nq, int Nk, int d, float scale, int dtype, void* stream) {
+    if (!h) return SD_ATTN_ERR_INVALID_VALUE;
+    if (B <= 0 || H <= 0 || Nq < 0 || Nk <= 0 || d <= 0) return SD_ATTN_ERR_INVALID_VALUE;
+    if (!isfinite(scale)) return SD_ATTN_ERR_INVALID_VALUE;
+    if (dtype != SD_ATTN_F16 && dtype != SD_ATTN_F32) return SD_ATTN_ERR_UNSUPPORTED;
+    if (d > SD_ATTN_MAX_D) return SD_ATTN_ERR_UNSUPPORTED;
+    if ((long long)B * H > 65535) return SD_ATTN_ERR_UNSUPPORTED;
+    if (Nq == 0) return SD_ATTN_OK;
+    if (!q || !k || !v || !out) return SD_ATTN_ERR_INVALID_VALUE;
+    if ((((uintptr_t)q | (uintptr_t)k | (uintptr_t)v | (uintptr_t)out) & 15u) != 0) return SD_ATTN_ERR_ALIGNMENT;
+
+    int mode = h->mode;
+    const bool tensor_ok = (dtype == SD_ATTN_F16) && (d % 8 == 0);
+    if (mode == SD_ATTN_MODE_AUTO) {
+        if (!tensor_ok) mode = SD_ATTN_MODE_SIMT;
+        else mode = (Nk <= SD_ATTN_CROSS_MAX_NK) ? SD_ATTN_MODE_CROSS : SD_ATTN_MODE_FUSED;
+    }
+    if (mode != SD_ATTN_MODE_SIMT && !tensor_ok) return SD_ATTN_ERR_UNSUPPORTED;
+    if (mode == SD_ATTN_MODE_CROSS && Nk > SD_ATTN_CROSS_MAX_NK) return SD_ATTN_ERR_UNSUPPORTED;
+
+    Problem p = {q, k, v, out, B * H, Nq, Nk, d, scale, (cudaStream_t)stream};
+    int rc;
+    switch (mode) {
+        case SD_ATTN_MODE_SIMT:
+            rc = (dtype == SD_ATTN_F16) ? launch_simt<__half>(h, p) : launch_simt<float>(h, p);
+            break;
+        case SD_ATTN_MODE_CROSS: rc = launch_cross(h, p); break;
+        case SD_ATTN_MODE_FUSED: rc = launch_fused(h, p); break;
+        case SD_ATTN_MODE_TWOPASS: rc = launch_twopass(h, p); break;
+        default: rc = SD_ATTN_ERR_INVALID_VALUE;
+    }
+    if (rc == SD_ATTN_OK) h->last_mode = mode;
+    if (rc == SD_ATTN_OK && getenv("SD_ATTN_LOG"))
+        fprintf(stderr, "[sd_attn] forward BH=%d Nq=%d Nk=%d d=%d dtype=%d -> mode %d\n", B * H, Nq, Nk, d, dtype, mode);
+    return rc;
+}
+
+static size_t round256(size_t x) { return (x + 255) & ~(size_t)255; }
+
+extern "C" size_t sd_attn_host_staging_bytes(int B, int H, int Nq, int Nk, int d, int dtype) {
+    if (B <= 0 || H <= 0 || Nq < 0 || Nk <= 0 || d <= 0) return 0;
+    const size_t es = dtype == SD_ATTN_F32 ? 4 : 2;
+    const size_t qb = round256((size_t)B * H * Nq * d * es), kb = round256((size_t)B * H * Nk * d * es);
+    return 2 * qb + 2 * kb;
+}
+
+extern "C" int sd_attn_forward_host(sd_attn_handle* h, const void* q, const void* k, const void* v, void* out,
+                                    void* staging, size_t staging_bytes, int B, int H, int Nq, int Nk, int d,
+                                    float scale, int dtype, void* stream) {
+    if (!h) return SD_ATTN_ERR_INVALID_VALUE;
+    if (B <= 0 || H <= 0 || Nq < 0 || Nk <= 0 || d <= 0) return SD_ATTN_ERR_INVALID_VALUE;
+    if (dtype != SD_ATTN_F16 && dtype != SD_ATTN_F32) return SD_ATTN_ERR_UNSUPPORTED;
+    if (Nq == 0) return SD_ATTN_OK;
+    if (!q || !k || !v || !out) return SD_ATTN_ERR_INVALID_VALUE;
+    const size_t need = sd_attn_host_staging_bytes(B, H, Nq, Nk, d, dtype);
+    if (!staging || staging_bytes < need || ((uintptr_t)staging & 255u)) return SD_ATTN_ERR_WORKSPACE;
+    const size_t es = dtype == SD_ATTN_F32 ? 4 : 2;
+    const size_t q_bytes = (size_t)B * H * Nq * d * es, k_bytes = (size_t)B * H * Nk * d * es;
+    char* dq = (char*)staging;
+    char* dk = dq + round256(q_bytes);
+    char* dv = dk + round256(k_bytes);
+    char* dout = dv + round256(k_bytes);
+    cudaStream_t s = (cudaStream_t)stream;
+    cudaError_t e = cudaMemcpyAsync(dq, q, q_bytes, cudaMemcpyHostToDevice, s);
+    if (e == cudaSuccess) e = cudaMemcpyAsync(dk, k, k_bytes, cudaMemcpyHostToDevice, s);
+    if (e == cudaSuccess) e = cudaMemcpyAsync(dv, v, k_bytes, cudaMemcpyHostToDevice, s);
+    if (e != cudaSuccess) return cuda_fail(h, e);
+    const int rc = sd_attn_forward(h, dq, dk, dv, dout, B, H, Nq, Nk, d, scale, dtype, stream);
+    if (rc != SD_ATTN_OK) return rc;
+    e = cudaMemcpyAsync(out, dout, q_bytes, cudaMemcpyDeviceToHost, s);
+    return e == cudaSuccess ? SD_ATTN_OK : cuda_fail(h, e);
+}
