@@ -1,0 +1,390 @@
+#!/usr/bin/env python
+"""Benchmark of the attention hot path on B200.
+
+  python bench.py --gpus N --steps K --warmup W            # the CUDA library (one rank per GPU)
+  python bench.py --impl reference --steps K --warmup W    # the CPU oracle, as it stands
+
+A step is one pass of the hot path over the full-resolution self-attention workload: B=2, H=8,
+Nq=Nk=4096, d=40, fp16, once on the plain N(0,1) inputs and once on the peaked (Q x 4) inputs --
+two launches of the fused kernel.  Rank 0 prints ONE JSON line.  Multi-GPU runs are weak scaling:
+every rank runs the same per-GPU work on its own inputs; attention has no exchange step, so there
+is no data-path collective, only a barrier and a max over ranks of the device time.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+from paper_2304_11267_b200 import distributed as D  # noqa: E402
+from paper_2304_11267_b200 import workloads  # noqa: E402
+
+METRIC = "attention TFLOP/s (4*B*H*Nq*Nk*d FLOPs per call), 4096-token self-attention"
+UNIT = "TFLOP/s"
+NOMINAL_FP16_TFLOPS = 2250.0
+ROTATING_SETS = 8   # 8 x 42 MB of q/k/v/out for the two variants = 336 MB, above the 126 MB L2
+# DRAM bytes per launch of the fused kernel on this workload (dram__bytes_read.sum + dram__bytes_write.sum
+# from one ncu capture; see profiles/fused_c2_self_4096_d40.md).  None until a capture has been read.
+FUSED_TRAFFIC_BYTES_PER_LAUNCH = None
+
+
+def measured_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            p = json.load(f)
+        return {"hbm_gbs": float(p["hbm_gbs"]), "tflops": float(p["bf16_tflops"]),
+                "tflops_sustained": float(p.get("bf16_tflops_sustained", p["bf16_tflops"])), "source": "measured"}
+    return {"hbm_gbs": 6650.0, "tflops": 1590.0, "tflops_sustained": 1400.0, "source": "fallback"}
+
+
+class ClockSampler(threading.Thread):
+    """Samples SM clock and throttle reasons through NVML while the timed region runs."""
+    REASONS = {0x4: "sw_power_cap", 0x8: "hw_slowdown", 0x20: "sw_thermal_slowdown",
+               0x40: "hw_thermal_slowdown", 0x80: "hw_power_brake_slowdown"}
+
+    def __init__(self, device_index: int):
+        super().__init__(daemon=True)
+        self.samples, self.reasons, self.power = [], set(), []
+        self.max_mhz = None
+        self._stop_evt = threading.Event()
+        self.nvml = None
+        try:
+            import pynvml
+            import torch
+            pynvml.nvmlInit()
+            self.nvml = pynvml
+            try:
+                uuid = "GPU-" + str(torch.cuda.get_device_properties(device_index).uuid)
+                self.h = pynvml.nvmlDeviceGetHandleByUUID(uuid)
+            except Exception:
+                self.h = pynvml.nvmlDeviceGetHandleByIndex(device_index)
+            self.max_mhz = int(pynvml.nvmlDeviceGetMaxClockInfo(self.h, pynvml.NVML_CLOCK_SM))
+        except Exception:
+            self.nvml = None
+
+    def sample_once(self):
+        if self.nvml is None:
+            return
+        n = self.nvml
+        try:
+            self.samples.append(int(n.nvmlDeviceGetClockInfo(self.h, n.NVML_CLOCK_SM)))
+            get = getattr(n, "nvmlDeviceGetCurrentClocksEventReasons", None) or \
+                getattr(n, "nvmlDeviceGetCurrentClocksThrottleReasons")
+            mask = int(get(self.h))
+            for bit, name in self.REASONS.items():
+                if mask & bit:
+                    self.reasons.add(name)
+            self.power.append(n.nvmlDeviceGetPowerUsage(self.h) / 1000.0)
+        except Exception:
+            pass
+
+    def run(self):
+        while not self._stop_evt.is_set():
+            self.sample_once()
+            time.sleep(0.002)
+
+    def stop(self):
+        self._stop_evt.set()
+        self.join(timeout=2)
+        return {"sm_mhz": float(np.median(self.samples)) if self.samples else None,
+                "sm_max_mhz": self.max_mhz, "reasons": sorted(self.reasons), "samples": len(self.samples),
+                "power_w_max": max(self.power) if self.power else None}
+
+
+# ------------------------------------------------------------------------------------------ oracle arm
+
+def oracle_sample_rows(call, every):
+    return np.arange(0, call.B * call.H * call.Nq, every, dtype=np.int64)
+
+
+def time_oracle(calls_inputs, every):
+    """Seconds the oracle needs for every `every`-th row of each call, and the FLOPs that covers."""
+    import oracle
+    t0 = time.perf_counter()
+    flops = 0
+    for call, (q, k, v) in calls_inputs:
+        rows = oracle_sample_rows(call, every)
+        oracle.forward(q, k, v, call.scale(), rows=rows)
+        flops += 4 * len(rows) * call.Nk * call.d
+    return time.perf_counter() - t0, flops
+
+
+def cpu_baseline(calls_inputs):
+    """The oracle as it stands on this machine's host cores, on a bounded sample (about 10-30 s of work)."""
+    import oracle
+    dt, flops = time_oracle(calls_inputs, 16)                 # calibration pass: 1/16 of the rows
+    every = 1
+    while every < 16 and dt * 16 / every > 30.0:              # full pass estimated above 30 s: thin it
+        every *= 2
+    if every < 16:
+        dt, flops = time_oracle(calls_inputs, every)
+    return {"value": flops / dt / 1e12, "unit": UNIT, "cores": oracle.max_threads(), "kind": "oracle",
+            "sample": "every %s row of both variants of the step (%d of %d rows), %.1f s" % (
+                "" if every == 1 else "%d-th" % every,
+                sum(len(oracle_sample_rows(c, every)) for c, _ in calls_inputs),
+                sum(c.B * c.H * c.Nq for c, _ in calls_inputs), dt),
+            "seconds": dt}
+
+
+def run_reference(args):
+    rank, _, world = D.env_world()
+    if rank != 0:
+        return 0
+    import oracle
+    calls = workloads.config2()
+    calls_inputs = [(c, workloads.make_inputs(c)) for c in calls]
+    every = 32   # each step: every 32nd row of both variants, about a third of a second on 8 cores
+    for _ in range(args.warmup):
+        time_oracle(calls_inputs, every)
+    t0 = time.perf_counter()
+    flops = 0
+    for _ in range(args.steps):
+        _, f = time_oracle(calls_inputs, every)
+        flops += f
+    dt = time.perf_counter() - t0
+    value = flops / dt / 1e12
+    sample = "each step: every 32nd row of both variants (%d rows of %d)" % (
+        sum(len(oracle_sample_rows(c, every)) for c in calls), sum(c.B * c.H * c.Nq for c in calls))
+    line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * dt / max(args.steps, 1),
+            "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+            "config": workload_config(),
+            "cpu_baseline": {"value": value, "unit": UNIT, "cores": oracle.max_threads(), "kind": "oracle",
+                             "sample": sample},
+            "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+            "gpu_launches": 0}
+    print(json.dumps(line))
+    return 0
+
+
+def workload_config():
+    return {"workload": "c2: self-attention B=2 H=8 Nq=Nk=4096 d=40 fp16, scale 1/sqrt(40); each step = plain N(0,1) "
+                        "call + peaked (Q x 4) call",
+            "l2": "inputs larger than L2: rotating through %d input/output sets (336 MB)" % ROTATING_SETS,
+            "per_gpu_units": "32 (batch, head) problems per step per GPU", "parallelism": "replicated per GPU, no collective"}
+
+
+# ------------------------------------------------------------------------------------------ CUDA arm
+
+def make_sets(calls, n_sets, device, rank):
+    import torch
+    sets = []
+    for r in range(n_sets):
+        entry = []
+        for c in calls:
+            shifted = workloads.Call(c.name, c.B, c.H, c.Nq, c.Nk, c.d, c.config_index,
+                                     call_index=c.call_index + 1000 * r + 100000 * rank, peaked=c.peaked,
+                                     padded_text=c.padded_text)
+            q, k, v = workloads.make_inputs(shifted)
+            tq, tk, tv = (torch.from_numpy(x).to(device) for x in (q, k, v))
+            entry.append((c, tq, tk, tv, torch.empty_like(tq)))
+        sets.append(entry)
+    return sets
+
+
+def run_ours(args):
+    import torch
+    from paper_2304_11267_b200 import binding as bd
+    rank, local_rank, world = D.init_process_group("nccl")
+    if not torch.cuda.is_available():
+        raise RuntimeError("bench.py needs a CUDA device: there is no CPU fallback (use --impl reference for the oracle)")
+    torch.cuda.set_device(local_rank)
+    device = torch.device("cuda", local_rank)
+    att = bd.Attention()
+    stream = torch.cuda.current_stream().cuda_stream
+    calls = workloads.config2()
+    sets = make_sets(calls, ROTATING_SETS, device, rank)
+    flops_per_step = sum(c.flops for c in calls)
+    launches_per_step = len(calls)
+
+    def step(i):
+        for c, tq, tk, tv, to in sets[i % ROTATING_SETS]:
+            rc = bd.sd_attn_forward(att.handle, tq.data_ptr(), tk.data_ptr(), tv.data_ptr(), to.data_ptr(),
+                                    c.B, c.H, c.Nq, c.Nk, c.d, float(c.scale()), bd.F16, stream)
+            if rc != bd.OK:
+                raise bd.SdAttnError(rc, "sd_attn_forward")
+
+    for i in range(max(args.warmup, 3)):
+        step(i)
+    att.check(stream)
+    assert att.last_mode == bd.MODE_FUSED
+
+    sampler = ClockSampler(local_rank)
+    start, end = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    launches0 = att.launch_count
+    D.barrier(world)
+    torch.cuda.synchronize()
+    sampler.start()
+    start.record()
+    for i in range(args.steps):
+        step(i)
+    end.record()
+    sampler.sample_once()
+    torch.cuda.synchronize()
+    clocks = sampler.stop()
+    D.barrier(world)
+    gpu_launches = att.launch_count - launches0
+    att.check(stream)
+    ms_total = D.max_over_ranks(start.elapsed_time(end), world, device)
+    ms_per_step = ms_total / args.steps
+    value = world * flops_per_step / (ms_per_step * 1e-3) / 1e12
+
+    # --- end to end through the C ABI with host buffers (pinned), copies inside the timed region
+    c0 = calls[0]
+    hsets = []
+    for c, tq, tk, tv, to in sets[0]:
+        hq, hk, hv = (t.cpu().pin_memory() for t in (tq, tk, tv))
+        hsets.append((c, hq, hk, hv, torch.empty_like(hq).pin_memory()))
+    need = bd.sd_attn_host_staging_bytes(c0.B, c0.H, c0.Nq, c0.Nk, c0.d, bd.F16)
+    staging = torch.empty(need, dtype=torch.uint8, device=device)
+    h2d = sum(hq.numel() * 2 + hk.numel() * 2 + hv.numel() * 2 for _, hq, hk, hv, _ in hsets)
+    d2h = sum(ho.numel() * 2 for *_, ho in hsets)
+
+    def e2e_step():
+        for c, hq, hk, hv, ho in hsets:
+            rc = bd.sd_attn_forward_host(att.handle, hq.data_ptr(), hk.data_ptr(), hv.data_ptr(), ho.data_ptr(),
+                                         staging.data_ptr(), need, c.B, c.H, c.Nq, c.Nk, c.d, float(c.scale()),
+                                         bd.F16, stream)
+            if rc != bd.OK:
+                raise bd.SdAttnError(rc, "sd_attn_forward_host")
+
+    e2e_steps = max(3, min(args.steps, 30))
+    for _ in range(3):
+        e2e_step()
+    D.barrier(world)
+    torch.cuda.synchronize()
+    start.record()
+    for _ in range(e2e_steps):
+        e2e_step()
+    end.record()
+    torch.cuda.synchronize()
+    D.barrier(world)
+    e2e_ms = D.max_over_ranks(start.elapsed_time(end), world, device) / e2e_steps
+    e2e = {"value": world * flops_per_step / (e2e_ms * 1e-3) / 1e12, "unit": UNIT, "ms_per_step": e2e_ms,
+           "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "steps": e2e_steps,
+           "api": "sd_attn_forward_host, pinned host buffers"}
+    # the step's result as a user would read it: finite and inside the hull of V
+    res = hsets[0][4]
+    assert torch.isfinite(res.float()).all()
+
+    if rank != 0:
+        return 0
+
+    peaks = measured_peaks()
+    per_launch_s = ms_per_step * 1e-3 / launches_per_step
+    achieved = calls[0].flops / per_launch_s / 1e12
+    roofline = {"bound": "tensor", "kernel": "fused_attention_kernel<128>", "achieved": achieved,
+                "peak": peaks["tflops"], "unit": "TFLOP/s", "frac": achieved / peaks["tflops"],
+                "peak_source": "%s cuBLAS bf16 burst (fp16 peak = bf16 peak, nominal ratio 1.0)" % peaks["source"],
+                "frac_of_nominal_2250": achieved / NOMINAL_FP16_TFLOPS,
+                "traffic": FUSED_TRAFFIC_BYTES_PER_LAUNCH, "algorithmic_bytes": calls[0].io_bytes(),
+                "us_per_launch": per_launch_s * 1e6}
+    line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+            "warmup": max(args.warmup, 3), "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": "f16", "data": "synthetic", "config": workload_config(),
+            "clocks": clocks, "e2e": e2e, "gpu_launches": gpu_launches, "roofline": roofline,
+            "pct_of_fp16_dense_peak": 100.0 * value / world / NOMINAL_FP16_TFLOPS}
+    if world == 1:
+        line["extra"] = extras(att, bd, device, stream, peaks)
+        host_inputs = [(c, tuple(t.cpu().numpy() for t in (tq, tk, tv))) for c, tq, tk, tv, _ in sets[0]]
+        line["cpu_baseline"] = cpu_baseline(host_inputs)
+    print(json.dumps(line))
+    return 0
+
+
+def time_calls(att, bd, tensors, stream, iters, graph=False):
+    """Mean microseconds for one pass over `tensors` (a list of calls), rotating nothing: small extras."""
+    import torch
+
+    def once():
+        for c, tq, tk, tv, to in tensors:
+            rc = bd.sd_attn_forward(att.handle, tq.data_ptr(), tk.data_ptr(), tv.data_ptr(), to.data_ptr(),
+                                    c.B, c.H, c.Nq, c.Nk, c.d, float(c.scale()), bd.F16, stream)
+            if rc != bd.OK:
+                raise bd.SdAttnError(rc, "sd_attn_forward")
+    start, end = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    for _ in range(3):
+        once()
+    torch.cuda.synchronize()
+    if graph:
+        s = torch.cuda.Stream()
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.stream(s):
+            with torch.cuda.graph(g, stream=s):
+                for c, tq, tk, tv, to in tensors:
+                    bd.sd_attn_forward(att.handle, tq.data_ptr(), tk.data_ptr(), tv.data_ptr(), to.data_ptr(),
+                                       c.B, c.H, c.Nq, c.Nk, c.d, float(c.scale()), bd.F16, s.cuda_stream)
+        g.replay()
+        torch.cuda.synchronize()
+        start.record()
+        for _ in range(iters):
+            g.replay()
+        end.record()
+    else:
+        start.record()
+        for _ in range(iters):
+            once()
+        end.record()
+    torch.cuda.synchronize()
+    return 1e3 * start.elapsed_time(end) / iters
+
+
+def extras(att, bd, device, stream, peaks):
+    """Secondary numbers: the UNet-step attention set (32 calls) and the memory-bound cross-attention."""
+    import torch
+    out = {}
+    calls = workloads.config4()
+    tensors = []
+    for c in calls:
+        q, k, v = workloads.make_inputs(c)
+        tq, tk, tv = (torch.from_numpy(x).to(device) for x in (q, k, v))
+        tensors.append((c, tq, tk, tv, torch.empty_like(tq)))
+    flops = sum(c.flops for c in calls)
+    us = time_calls(att, bd, tensors, stream, 20)
+    us_graph = time_calls(att, bd, tensors, stream, 20, graph=True)
+    out["unet_step_attention_set"] = {"calls": len(calls), "us_plain_launches": us, "us_cuda_graph": us_graph,
+                                      "tflops_cuda_graph": flops / (us_graph * 1e-6) / 1e12,
+                                      "note": "512x512, B=2, H=8: 16 self + 16 cross calls (L2-warm: 285 MB of tensors)"}
+    # cross-attention at the large-latent size, rotating sets so that Q/O stream from HBM
+    c = workloads.config5()[2]
+    n_sets = 8     # 8 x 47.6 MB
+    csets = []
+    for r in range(n_sets):
+        q, k, v = workloads.make_inputs(workloads.Call(c.name, c.B, c.H, c.Nq, c.Nk, c.d, c.config_index,
+                                                       call_index=c.call_index + 10 * r, padded_text=True))
+        tq, tk, tv = (torch.from_numpy(x).to(device) for x in (q, k, v))
+        csets.append((c, tq, tk, tv, torch.empty_like(tq)))
+    us_cross = time_calls(att, bd, csets, stream, 10) / n_sets
+    gbs = c.io_bytes() / (us_cross * 1e-6) / 1e9
+    out["cross_attention_9216x77_d40"] = {"us_per_call": us_cross, "achieved_gbs": gbs, "bound": "hbm",
+                                          "peak_gbs": peaks["hbm_gbs"], "frac": gbs / peaks["hbm_gbs"],
+                                          "frac_of_nominal_8000": gbs / 8000.0,
+                                          "algorithmic_bytes": c.io_bytes(), "peak_source": peaks["source"]}
+    att.check(stream)
+    return out
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=200)
+    ap.add_argument("--warmup", type=int, default=10)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    args = ap.parse_args()
+    if args.impl == "reference":
+        return run_reference(args)
+    return run_ours(args)
+
+
+if __name__ == "__main__":
+    sys.exit(main())

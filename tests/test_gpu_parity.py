@@ -1,0 +1,394 @@
+"""GPU parity: every kernel family, through the C ABI, against the fp64 CPU oracle on the same
+seeded bytes.
+
+Tolerances (written here, as the workload statement gives them):
+  fp16 in / fp32 accumulate / fp16 out :  max |err| <= 2e-3 * max|V|
+  fp32 path                            :  max |err| <= 1e-5 * max|V|  and  ||err||2 / ||ref||2 <= 1e-5
+On top of the stated fp16 bound, a relative L2 error <= 2e-3 is self-imposed: the stated bound is
+loose for near-uniform attention (outputs of size 0.03 against max|V| of 5).
+"""
+import ctypes
+import hashlib
+
+import numpy as np
+import pytest
+
+import oracle
+from paper_2304_11267_b200 import workloads
+
+torch = pytest.importorskip("torch")
+pytestmark = pytest.mark.gpu
+
+F16_ABS = 2e-3
+F16_REL_L2 = 2e-3
+F32_TOL = 1e-5
+
+
+@pytest.fixture(scope="module")
+def bd():
+    from paper_2304_11267_b200 import binding
+    from paper_2304_11267_b200 import build
+    build.build()
+    binding.load()
+    return binding
+
+
+@pytest.fixture()
+def att(bd):
+    a = bd.Attention()
+    yield a
+    a.check()
+    a.close()
+
+
+def gpu(x):
+    return torch.from_numpy(x).cuda()
+
+
+def rand_qkv(seed, B, H, Nq, Nk, d, dtype=np.float16, qmult=1.0):
+    g = np.random.default_rng(seed)
+    q = (g.standard_normal((B, H, Nq, d), dtype=np.float32) * qmult).astype(dtype)
+    k = g.standard_normal((B, H, Nk, d), dtype=np.float32).astype(dtype)
+    v = g.standard_normal((B, H, Nk, d), dtype=np.float32).astype(dtype)
+    return q, k, v
+
+
+def check(got, ref, v, dtype=np.float16, what=""):
+    got = got.astype(np.float64)
+    assert np.all(np.isfinite(got)), "%s: non-finite output" % what
+    vmax = float(np.abs(v.astype(np.float64)).max())
+    err = float(np.abs(got - ref).max())
+    rel = float(np.linalg.norm(got - ref) / max(np.linalg.norm(ref), 1e-300))
+    if dtype == np.float16:
+        assert err <= F16_ABS * vmax, "%s: max abs err %.3e > %.3e" % (what, err, F16_ABS * vmax)
+        assert rel <= F16_REL_L2, "%s: rel L2 err %.3e" % (what, rel)
+    else:
+        assert err <= F32_TOL * vmax, "%s: max abs err %.3e > %.3e" % (what, err, F32_TOL * vmax)
+        assert rel <= F32_TOL, "%s: rel L2 err %.3e" % (what, rel)
+    return err, rel
+
+
+def run(att, bd, mode, q, k, v, scale):
+    att.set_mode(mode)
+    out = att.forward(gpu(q), gpu(k), gpu(v), scale=float(scale))
+    att.check()
+    return out.cpu().numpy()
+
+
+def sample_rows(call, n, seed=5):
+    """All rows of the first and last 128-row tile of the first (b,h) plus n random rows."""
+    total = call.B * call.H * call.Nq
+    g = np.random.default_rng(seed)
+    rows = set(g.choice(total, size=min(n, total), replace=False).tolist())
+    rows.update(range(0, min(128, call.Nq)))
+    rows.update(range(total - min(128, call.Nq), total))
+    return np.array(sorted(rows), dtype=np.int64)
+
+
+# ------------------------------------------------------------------ the named workloads
+
+def test_config1_every_mode_full_tensor(att, bd):
+    call = workloads.config1()[0]
+    q, k, v = workloads.make_inputs(call)
+    ref, L, S = oracle.forward(q, k, v, call.scale())
+    outs = {}
+    for mode in (bd.MODE_AUTO, bd.MODE_FUSED, bd.MODE_TWOPASS, bd.MODE_SIMT):
+        outs[mode] = run(att, bd, mode, q, k, v, call.scale())
+        check(outs[mode], ref, v, what="c1 mode %s" % bd.MODE_NAMES[mode])
+    assert att.last_mode == bd.MODE_SIMT
+    # variant agreement: the exact reformulations of Sec. 3.2 agree with one another
+    vmax = np.abs(v.astype(np.float64)).max()
+    for a in outs.values():
+        for b in outs.values():
+            assert np.abs(a.astype(np.float64) - b.astype(np.float64)).max() <= 2 * F16_ABS * vmax
+
+
+@pytest.mark.parametrize("idx", [0, 1], ids=["plain", "peaked"])
+def test_config2_full_size_sampled_rows(att, bd, idx):
+    call = workloads.config2()[idx]
+    q, k, v = workloads.make_inputs(call)
+    rows = sample_rows(call, 1024)
+    ref, _, _ = oracle.forward(q, k, v, call.scale(), rows=rows)
+    out = run(att, bd, bd.MODE_AUTO, q, k, v, call.scale())
+    assert att.last_mode == bd.MODE_FUSED
+    check(out.reshape(-1, call.d)[rows], ref, v, what=call.name)
+    assert np.all(np.isfinite(out.astype(np.float64)))
+    # a property that holds at any size: outputs stay inside the per-(b,h) hull of V
+    vmin = v.astype(np.float64).min(axis=2, keepdims=True) - 4e-3
+    vmax = v.astype(np.float64).max(axis=2, keepdims=True) + 4e-3
+    assert np.all(out >= vmin) and np.all(out <= vmax)
+
+
+@pytest.mark.parametrize("idx", range(4))
+def test_config3_cross_attention_full_tensor(att, bd, idx):
+    call = workloads.config3()[idx]
+    q, k, v = workloads.make_inputs(call)
+    ref, _, _ = oracle.forward(q, k, v, call.scale())
+    out = run(att, bd, bd.MODE_AUTO, q, k, v, call.scale())
+    assert att.last_mode == bd.MODE_CROSS
+    check(out, ref, v, what=call.name)
+    for mode in (bd.MODE_FUSED, bd.MODE_TWOPASS):
+        check(run(att, bd, mode, q, k, v, call.scale()), ref, v, what=call.name + bd.MODE_NAMES[mode])
+
+
+def test_config4_unet_step_all_32_calls(att, bd):
+    att.set_mode(bd.MODE_AUTO)
+    modes = []
+    for call in workloads.config4():
+        q, k, v = workloads.make_inputs(call)
+        rows = sample_rows(call, 256)
+        ref, _, _ = oracle.forward(q, k, v, call.scale(), rows=rows)
+        out = att.forward(gpu(q), gpu(k), gpu(v), scale=float(call.scale())).cpu().numpy()
+        check(out.reshape(-1, call.d)[rows], ref, v, what=call.name)
+        modes.append(att.last_mode)
+    # 15 self-attention calls take the fused kernel; the 64-token one and all cross calls fit one key tile
+    assert modes.count(bd.MODE_FUSED) == 15 and modes.count(bd.MODE_CROSS) == 17
+
+
+@pytest.mark.parametrize("idx", [0, 1, 2], ids=["self_plain", "self_peaked", "cross"])
+def test_config5_large_latent_sampled_rows(att, bd, idx):
+    call = workloads.config5()[idx]
+    q, k, v = workloads.make_inputs(call)
+    rows = sample_rows(call, 384)
+    ref, L, S = oracle.forward(q, k, v, call.scale(), rows=rows)
+    out = run(att, bd, bd.MODE_AUTO, q, k, v, call.scale())
+    check(out.reshape(-1, call.d)[rows], ref, v, what=call.name)
+    if idx == 1:
+        # the comparator that materialises the 9216 x 9216 score matrices (10.9 GB of scratch)
+        tp = run(att, bd, bd.MODE_TWOPASS, q, k, v, call.scale())
+        check(tp.reshape(-1, call.d)[rows], ref, v, what=call.name + " twopass")
+        n = call.B * call.H * call.Nq
+        ws = att._workspace
+        off = (n * call.Nk * 4 + 255) // 256 * 256
+        LS = ws[off:off + n * 8].view(torch.float32).cpu().numpy().reshape(n, 2)[rows]
+        np.testing.assert_allclose(LS[:, 0], L, rtol=0, atol=2e-5 * max(1.0, np.abs(L).max()))
+        np.testing.assert_allclose(LS[:, 1], S, rtol=2e-5)
+        att._workspace = None
+        bd.sd_attn_set_workspace(att.handle, 0, 0)
+
+
+# ------------------------------------------------------------------ awkward shapes
+
+EDGE_N = [1, 2, 15, 16, 17, 63, 64, 65, 77, 127, 128, 129, 255, 257]
+
+
+def edge_shapes(d):
+    g = np.random.default_rng(d)
+    pairs = [(n, n) for n in EDGE_N]
+    pairs += [(int(a), int(b)) for a, b in zip(g.choice(EDGE_N, 12), g.choice(EDGE_N, 12))]
+    pairs += [(300, 77), (130, 513), (1, 1000), (640, 384)]
+    return pairs
+
+
+@pytest.mark.parametrize("d", [40, 80, 160])
+@pytest.mark.parametrize("mode_name", ["auto", "fused", "twopass", "simt", "cross"])
+def test_edge_shapes(att, bd, mode_name, d):
+    mode = {v: k for k, v in bd.MODE_NAMES.items()}[mode_name]
+    att.set_mode(mode)
+    for i, (Nq, Nk) in enumerate(edge_shapes(d)):
+        if mode == bd.MODE_CROSS and Nk > bd.CROSS_MAX_NK:
+            continue
+        B, H = [(1, 1), (1, 3), (2, 8)][i % 3]
+        q, k, v = rand_qkv(1000 * d + i, B, H, Nq, Nk, d, qmult=[1.0, 4.0][i % 2])
+        scale = np.float32(1 / np.sqrt(d))
+        ref, _, _ = oracle.forward(q, k, v, scale)
+        out = att.forward(gpu(q), gpu(k), gpu(v), scale=float(scale)).cpu().numpy()
+        check(out, ref, v, what="%s d=%d Nq=%d Nk=%d BH=%d" % (mode_name, d, Nq, Nk, B * H))
+    att.check()
+
+
+@pytest.mark.parametrize("d", [8, 24, 48, 64, 96, 104, 128, 136])
+def test_other_head_dims(att, bd, d):
+    for mode in (bd.MODE_FUSED, bd.MODE_CROSS, bd.MODE_TWOPASS):
+        Nk = 100 if mode == bd.MODE_CROSS else 300
+        q, k, v = rand_qkv(d, 1, 2, 200, Nk, d, qmult=3.0)
+        ref, _, _ = oracle.forward(q, k, v, 0.2)
+        check(run(att, bd, mode, q, k, v, 0.2), ref, v, what="d=%d mode %s" % (d, bd.MODE_NAMES[mode]))
+
+
+# ------------------------------------------------------------------ fp32 path
+
+@pytest.mark.parametrize("shape", [(1, 8, 1024, 1024, 40), (2, 2, 300, 77, 80), (1, 2, 257, 513, 160),
+                                   (1, 1, 33, 65, 24), (1, 3, 64, 64, 7)])
+@pytest.mark.parametrize("qmult", [1.0, 4.0])
+def test_fp32_path(att, bd, shape, qmult):
+    B, H, Nq, Nk, d = shape
+    q, k, v = rand_qkv(7 + Nq, B, H, Nq, Nk, d, np.float32, qmult)
+    scale = np.float32(1 / np.sqrt(d))
+    ref, _, _ = oracle.forward(q, k, v, scale)
+    out = run(att, bd, bd.MODE_AUTO, q, k, v, scale)
+    assert att.last_mode == bd.MODE_SIMT
+    check(out, ref, v, np.float32, what="fp32 %s" % (shape,))
+
+
+# ------------------------------------------------------------------ degenerate and special cases
+
+@pytest.mark.parametrize("mode_name", ["fused", "cross", "twopass", "simt"])
+def test_special_cases(att, bd, mode_name):
+    mode = {v: k for k, v in bd.MODE_NAMES.items()}[mode_name]
+    # one key: out = V[0] exactly
+    q, k, v = rand_qkv(1, 1, 2, 70, 1, 40)
+    out = run(att, bd, mode, q, k, v, 0.3)
+    assert np.array_equal(out, np.broadcast_to(v, out.shape))
+    # zero scale: uniform weights -> column mean of V; negative scale = negated queries
+    q, k, v = rand_qkv(2, 1, 2, 130, 77, 80, qmult=3.0)
+    ref0, _, _ = oracle.forward(q, k, v, 0.0)
+    check(run(att, bd, mode, q, k, v, 0.0), ref0, v, what="zero scale")
+    refn, _, _ = oracle.forward(q, k, v, -0.2)
+    check(run(att, bd, mode, q, k, v, -0.2), refn, v, what="negative scale")
+    # identical keys -> mean of V; a dominant logit -> that V row
+    k2 = np.broadcast_to(k[:, :, :1], k.shape).copy()
+    refm, _, _ = oracle.forward(q, k2, v, 0.11)
+    check(run(att, bd, mode, q, k2, v, 0.11), refm, v, what="identical keys")
+    q3 = np.zeros_like(q)
+    q3[..., 0] = 8.0
+    k3 = np.zeros_like(k)
+    k3[:, :, 33, 0] = 8.0
+    out3 = run(att, bd, mode, q3, k3, v, 1.0)
+    assert np.array_equal(out3, np.broadcast_to(v[:, :, 33:34], out3.shape))
+
+
+def test_padding_rows_with_distinct_values_only_see_their_mean(att, bd):
+    call = workloads.config3()[0]
+    q, k, v = workloads.make_inputs(call)
+    v2 = v.copy()
+    v2[:, :, 57:] = np.random.default_rng(3).standard_normal(v2[:, :, 57:].shape).astype(np.float16)
+    v3 = v2.copy()
+    v3[:, :, 57:] = v2[:, :, 57:][:, :, ::-1]
+    ref, _, _ = oracle.forward(q, k, v2, call.scale())
+    a = run(att, bd, bd.MODE_CROSS, q, k, v2, call.scale())
+    b = run(att, bd, bd.MODE_CROSS, q, k, v3, call.scale())
+    check(a, ref, v2, what="distinct padding values")
+    check(b, ref, v2, what="reversed padding values")
+
+
+# ------------------------------------------------------------------ memory safety, determinism, errors
+
+@pytest.mark.parametrize("mode_name,shape", [("fused", (1, 3, 300, 333, 40)), ("cross", (2, 2, 130, 77, 80)),
+                                             ("twopass", (1, 2, 257, 200, 160)), ("simt", (1, 2, 100, 90, 40)),
+                                             ("fused", (1, 1, 64, 200, 160))])
+def test_guard_bands_inputs_untouched_and_bitwise_repeatable(att, bd, mode_name, shape):
+    mode = {v: k for k, v in bd.MODE_NAMES.items()}[mode_name]
+    B, H, Nq, Nk, d = shape
+    q, k, v = rand_qkv(11, B, H, Nq, Nk, d, qmult=4.0)
+    att.set_mode(mode)
+    n = B * H * Nq * d
+    guard = 4096
+    big = torch.full((n + 2 * guard,), float("nan"), dtype=torch.float16, device="cuda")
+    out = big[guard:guard + n].view(B, H, Nq, d)
+    tq, tk, tv = gpu(q), gpu(k), gpu(v)
+    digest = [hashlib.sha256(t.cpu().numpy().tobytes()).hexdigest() for t in (tq, tk, tv)]
+    att.forward(tq, tk, tv, scale=0.17, out=out)
+    att.check()
+    first = out.cpu().numpy().copy()
+    assert torch.isnan(big[:guard]).all() and torch.isnan(big[guard + n:]).all(), "wrote outside out"
+    assert np.all(np.isfinite(first.astype(np.float64)))
+    assert digest == [hashlib.sha256(t.cpu().numpy().tobytes()).hexdigest() for t in (tq, tk, tv)]
+    ref, _, _ = oracle.forward(q, k, v, 0.17)
+    check(first, ref, v, what="guarded " + mode_name)
+    out.fill_(float("nan"))
+    att.forward(tq, tk, tv, scale=0.17, out=out)
+    att.check()
+    assert np.array_equal(out.cpu().numpy(), first), "two runs differ bitwise"
+
+
+def test_error_codes_enqueue_nothing(att, bd):
+    h = att.handle
+    q, k, v = (gpu(x) for x in rand_qkv(1, 1, 1, 128, 200, 40))
+    out = torch.full_like(q, 7.0)
+    args = (q.data_ptr(), k.data_ptr(), v.data_ptr(), out.data_ptr())
+    before = att.launch_count
+    f = bd.sd_attn_forward
+    assert f(h, *args, 0, 1, 128, 200, 40, 0.1, bd.F16) == bd.ERR_INVALID_VALUE
+    assert f(h, *args, 1, 1, 128, 0, 40, 0.1, bd.F16) == bd.ERR_INVALID_VALUE
+    assert f(h, *args, 1, 1, -1, 200, 40, 0.1, bd.F16) == bd.ERR_INVALID_VALUE
+    assert f(h, *args, 1, 1, 128, 200, 40, float("nan"), bd.F16) == bd.ERR_INVALID_VALUE
+    assert f(h, *args, 1, 1, 128, 200, 40, float("inf"), bd.F16) == bd.ERR_INVALID_VALUE
+    assert f(h, 0, *args[1:], 1, 1, 128, 200, 40, 0.1, bd.F16) == bd.ERR_INVALID_VALUE
+    assert f(h, *args, 1, 1, 128, 200, 40, 0.1, 5) == bd.ERR_UNSUPPORTED
+    assert f(h, *args, 1, 1, 128, 200, 168, 0.1, bd.F16) == bd.ERR_UNSUPPORTED
+    assert f(h, args[0] + 2, *args[1:], 1, 1, 128, 200, 40, 0.1, bd.F16) == bd.ERR_ALIGNMENT
+    assert f(h, *args, 1, 1, 0, 200, 40, 0.1, bd.F16) == bd.OK                    # Nq == 0: no-op
+    assert bd.sd_attn_set_mode(h, 9) == bd.ERR_INVALID_VALUE
+    att.set_mode(bd.MODE_CROSS)
+    assert f(h, *args, 1, 1, 128, 200, 40, 0.1, bd.F16) == bd.ERR_UNSUPPORTED     # Nk above one tile
+    att.set_mode(bd.MODE_FUSED)
+    assert f(h, *args, 1, 1, 128, 200, 20, 0.1, bd.F16) == bd.ERR_UNSUPPORTED     # d % 8 != 0
+    assert f(h, *args, 1, 1, 128, 200, 40, 0.1, bd.F32) == bd.ERR_UNSUPPORTED     # no TF32 path
+    att.set_mode(bd.MODE_TWOPASS)
+    assert f(h, *args, 1, 1, 128, 200, 40, 0.1, bd.F16) == bd.ERR_WORKSPACE
+    assert bd.sd_attn_set_workspace(h, q.data_ptr() + 16, 64) == bd.ERR_ALIGNMENT
+    assert bd.sd_attn_set_workspace(h, 0, 64) == bd.ERR_INVALID_VALUE
+    torch.cuda.synchronize()
+    assert att.launch_count == before
+    assert torch.all(out == 7.0)
+    assert att.last_mode != bd.MODE_TWOPASS
+
+
+def test_auto_falls_back_to_cuda_cores_for_odd_head_dims(att, bd):
+    q, k, v = rand_qkv(4, 1, 2, 150, 150, 36)
+    ref, _, _ = oracle.forward(q, k, v, 0.2)
+    out = run(att, bd, bd.MODE_AUTO, q, k, v, 0.2)
+    assert att.last_mode == bd.MODE_SIMT
+    check(out, ref, v, what="d=36")
+
+
+def test_forward_host_with_pinned_buffers(att, bd):
+    call = workloads.config3()[1]
+    q, k, v = workloads.make_inputs(call)
+    ref, _, _ = oracle.forward(q, k, v, call.scale())
+    hq, hk, hv = (torch.from_numpy(x).pin_memory() for x in (q, k, v))
+    hout = torch.empty_like(hq).pin_memory()
+    need = bd.sd_attn_host_staging_bytes(call.B, call.H, call.Nq, call.Nk, call.d, bd.F16)
+    staging = torch.empty(need, dtype=torch.uint8, device="cuda")
+    stream = torch.cuda.current_stream().cuda_stream
+    args = (call.B, call.H, call.Nq, call.Nk, call.d, float(call.scale()), bd.F16, stream)
+    assert bd.sd_attn_forward_host(att.handle, hq.data_ptr(), hk.data_ptr(), hv.data_ptr(), hout.data_ptr(),
+                                   staging.data_ptr(), need - 1, *args) == bd.ERR_WORKSPACE
+    assert bd.sd_attn_forward_host(att.handle, hq.data_ptr(), hk.data_ptr(), hv.data_ptr(), hout.data_ptr(),
+                                   staging.data_ptr(), need, *args) == bd.OK
+    att.check(stream)
+    check(hout.numpy(), ref, v, what="forward_host")
+
+
+def test_forward_is_capturable_in_a_cuda_graph(att, bd):
+    calls = workloads.config4()[18:22]      # two self (256 tokens) and two cross calls
+    tensors = []
+    for c in calls:
+        q, k, v = workloads.make_inputs(c)
+        tensors.append((c, q, k, v, gpu(q), gpu(k), gpu(v), torch.zeros(q.shape, dtype=torch.float16, device="cuda")))
+    att.set_mode(bd.MODE_AUTO)
+    s = torch.cuda.Stream()
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.stream(s):
+        for c, q, k, v, tq, tk, tv, to in tensors:           # warm-up outside capture
+            att.forward(tq, tk, tv, scale=float(c.scale()), out=to, stream=s.cuda_stream)
+        s.synchronize()
+        with torch.cuda.graph(graph, stream=s):
+            for c, q, k, v, tq, tk, tv, to in tensors:
+                att.forward(tq, tk, tv, scale=float(c.scale()), out=to, stream=s.cuda_stream)
+    for t in tensors:
+        t[7].zero_()
+    graph.replay()
+    torch.cuda.synchronize()
+    att.check()
+    for c, q, k, v, tq, tk, tv, to in tensors:
+        ref, _, _ = oracle.forward(q, k, v, c.scale())
+        check(to.cpu().numpy(), ref, v, what="graph " + c.name)
+
+
+def test_twopass_score_matrix_and_row_statistics(att, bd):
+    q, k, v = rand_qkv(9, 2, 2, 300, 333, 80, qmult=4.0)
+    scale = np.float32(1 / np.sqrt(80))
+    ref, L, S = oracle.forward(q, k, v, scale)
+    run(att, bd, bd.MODE_TWOPASS, q, k, v, scale)
+    a_ptr, s_ptr = bd.sd_attn_twopass_buffers(att.handle)
+    ws = att._workspace
+    assert a_ptr == ws.data_ptr()
+    n = 2 * 2 * 300
+    A = ws[:n * 333 * 4].view(torch.float32).cpu().numpy().reshape(2, 2, 300, 333)
+    LS = ws[s_ptr - a_ptr:s_ptr - a_ptr + n * 8].view(torch.float32).cpu().numpy().reshape(2, 2, 300, 2)
+    a_ref = float(scale) * np.einsum("bhic,bhjc->bhij", q.astype(np.float64), k.astype(np.float64))
+    np.testing.assert_allclose(A, a_ref, rtol=0, atol=1e-5 * np.abs(a_ref).max())
+    np.testing.assert_allclose(LS[..., 0], L, rtol=0, atol=1e-5 * np.abs(L).max())   # L: exact to fp32 rounding
+    np.testing.assert_allclose(LS[..., 1], S, rtol=1e-5)                              # S of Eq. 4
