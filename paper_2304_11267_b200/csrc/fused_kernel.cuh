@@ -6,16 +6,20 @@
 // because its accumulators live in registers on mobile GPUs; here they live in the 512-column
 // tensor memory, so every head dim up to 160 takes the same path.
 //
-// One CTA owns TWO tiles of 128 query rows and ping-pongs between them so that the tensor pipe
-// works on one tile while the other is in its softmax:
-//   warps 0-3  softmax of tile 0 (thread = query row = TMEM lane)      warp 8  TMA producer
-//   warps 4-7  softmax of tile 1                                        warp 9  MMA issuer, TMEM owner
+// One CTA owns TWO tiles of 128 query rows, each with its own softmax warpgroup and its own MMA
+// issuer, so that the tensor pipe works for one tile while the other is in its softmax:
+//   warps 0-3  softmax of tile 0 (thread = query row = TMEM lane)      warp 8       TMA producer
+//   warps 4-7  softmax of tile 1                                        warps 9, 10  MMA issuers
 // Per key tile j and query tile t:
 //   S_t = Q_t K_j^T          tcgen05.mma, both operands from swizzled shared memory
-//   softmax warps            row max; O_t is rescaled only when the running max grew by more than
-//                            2^8 (so p <= 256 fits fp16); p = exp2(s*c - m*c); P_t as packed fp16 over
-//                            the columns of S_t
+//   softmax warps            read the row of S_t into registers (S_t is then free for tile j+1); row max;
+//                            O_t is rescaled only when the running max grew by more than 2^8 (so
+//                            p <= 256 fits fp16); p = exp2(s*c - m*c), a fixed share of them evaluated on
+//                            the FMA pipe; P_t written back to tensor memory as packed fp16
 //   O_t += P_t V_j           tcgen05.mma, P from tensor memory, V as an N-major shared-memory operand
+// When 3*BN + 2*dpad <= 512 tensor-memory columns (d <= 64) P_t has columns of its own, and the
+// next S_t is issued as soon as the row of S_t sits in registers; otherwise P_t reuses the columns
+// of S_t and the next S_t follows the P V product.
 // All waits are bounded; an expired wait raises a block-wide abort flag and the kernel returns.
 #pragma once
 #include <cuda.h>
@@ -25,10 +29,19 @@
 
 namespace sd_attn {
 
-constexpr int FUSED_THREADS = 320;
+constexpr int FUSED_THREADS = 352;
 constexpr int FUSED_MAX_STAGES = 4;
+constexpr int FUSED_MAX_KSTEPS = 10;   // MMA steps of the Q K^T contraction at the largest head dim (160)
 constexpr int FUSED_SMEM_BUDGET = 220 * 1024;
 constexpr float FUSED_RESCALE_LOG2 = 8.0f;  // rescale O only when the max grew by more than 2^8
+#ifndef SD_ATTN_POLY_PER8
+#define SD_ATTN_POLY_PER8 0
+#endif
+#ifndef SD_ATTN_TAKE_TURNS
+#define SD_ATTN_TAKE_TURNS 0
+#endif
+constexpr bool FUSED_TAKE_TURNS = SD_ATTN_TAKE_TURNS != 0;
+constexpr int FUSED_POLY_PER8 = SD_ATTN_POLY_PER8;  // of every 8 exponentials, this many use the FMA pipe
 
 struct FusedArgs {
     __half* out;  // [BH][Nq][d]
@@ -39,9 +52,24 @@ struct FusedArgs {
     float scale_log2e;
     int negate;
     int* status;
+#ifdef SD_ATTN_TRACE
+    long long* trace;   // timeline probe of block (0,0): [role][tile j < 40][8 slots] clock64 stamps
+#endif
 };
 
+#ifdef SD_ATTN_TRACE
+#define FUSED_TRACE(role, j, slot)                                                              \
+    do {                                                                                        \
+        if (args.trace && blockIdx.x == 0 && blockIdx.y == 0 && (j) < 40)                       \
+            args.trace[((role) * 40 + (j)) * 8 + (slot)] = clock64();                           \
+    } while (0)
+#else
+#define FUSED_TRACE(role, j, slot) do { } while (0)
+#endif
+
 __host__ inline int fused_block_n(int d) { return ((d + 15) / 16 * 16) <= 128 ? 128 : 64; }
+// P gets tensor-memory columns of its own when S_0 S_1 | P_0 P_1 | O_0 O_1 fit the 512 columns.
+__host__ inline bool fused_split_p(int d) { return 3 * fused_block_n(d) + 2 * ((d + 15) / 16 * 16) <= 512; }
 
 __host__ inline void fused_fill_args(FusedArgs* a, __half* out, int Nq, int Nk, int d, float scale_log2e, bool negate,
                                      int* status) {
@@ -67,17 +95,21 @@ __host__ inline size_t fused_smem_bytes(const FusedArgs& a) {
 __host__ inline size_t fused_smem_bytes_max() { return FUSED_SMEM_BUDGET + 1024; }
 
 enum {
-    SITE_F_Q = 10, SITE_F_K = 11, SITE_F_V = 12, SITE_F_EMPTY = 13, SITE_F_S = 14, SITE_F_P = 15, SITE_F_O = 16
+    SITE_F_Q = 10, SITE_F_KV = 11, SITE_F_EMPTY = 13, SITE_F_S = 14, SITE_F_P = 15, SITE_F_O = 16,
+    SITE_F_SFREE = 17, SITE_F_PFREE = 18, SITE_F_TURN = 19
 };
 
-template <int BN>
+template <int BN, bool SPLIT_P>
 __global__ void __launch_bounds__(FUSED_THREADS, 1)
 fused_attention_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__ CUtensorMap tmap_k,
                        const __grid_constant__ CUtensorMap tmap_v, const FusedArgs args) {
     extern __shared__ uint8_t fused_smem_raw[];
-    __shared__ __align__(8) uint64_t bar_q_full[2], bar_s_full[2], bar_p_full[2], bar_o_full[2];
-    __shared__ __align__(8) uint64_t bar_k_full[FUSED_MAX_STAGES], bar_v_full[FUSED_MAX_STAGES],
-        bar_kv_empty[FUSED_MAX_STAGES];
+    // per query tile: Q landed | S ready (MMA) | S consumed (softmax) | P ready (softmax) | P V done (MMA)
+    __shared__ __align__(8) uint64_t bar_q_full[2], bar_s_full[2], bar_s_free[2], bar_p_full[2], bar_pv_done[2];
+    // the two softmax warpgroups take turns on the special-function unit: bar_turn[t] lets tile t run its
+    // exponentials; while one group is there the other loads S, takes its row maximum and waits
+    __shared__ __align__(8) uint64_t bar_turn[2];
+    __shared__ __align__(8) uint64_t bar_kv_full[FUSED_MAX_STAGES], bar_kv_empty[FUSED_MAX_STAGES];
     __shared__ uint32_t tmem_base_slot;
     __shared__ int abort_flag;
 
@@ -100,13 +132,14 @@ fused_attention_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_
         for (int t = 0; t < 2; ++t) {
             mbar_init(smem_u32(&bar_q_full[t]), 1);
             mbar_init(smem_u32(&bar_s_full[t]), 1);
-            mbar_init(smem_u32(&bar_p_full[t]), TILE_M);
-            mbar_init(smem_u32(&bar_o_full[t]), 1);
+            mbar_init(smem_u32(&bar_s_free[t]), 4);    // one arrival per softmax warp
+            mbar_init(smem_u32(&bar_p_full[t]), 4);
+            mbar_init(smem_u32(&bar_pv_done[t]), 1);
+            mbar_init(smem_u32(&bar_turn[t]), 4);
         }
         for (int s = 0; s < FUSED_MAX_STAGES; ++s) {
-            mbar_init(smem_u32(&bar_k_full[s]), 1);
-            mbar_init(smem_u32(&bar_v_full[s]), 1);
-            mbar_init(smem_u32(&bar_kv_empty[s]), 1);
+            mbar_init(smem_u32(&bar_kv_full[s]), 1);
+            mbar_init(smem_u32(&bar_kv_empty[s]), n_qtiles);   // one commit per issuer
         }
         mbar_init_fence();
     }
@@ -118,12 +151,14 @@ fused_attention_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_
     __syncthreads();
     tc_fence_after_sync();
     const uint32_t tmem_base = tmem_base_slot;
-    // columns: S_0 | S_1 | O_0 | O_1 ; P_t reuses the first BN/2 columns of S_t
-    const uint32_t tmem_o0 = tmem_base + 2 * BN;
+    // columns: S_0 | S_1 | (P_0 | P_1 when split) | O_0 | O_1 ; otherwise P_t reuses the first BN/2 columns of S_t
+    const uint32_t tmem_p0 = SPLIT_P ? tmem_base + 2 * BN : tmem_base;
+    const uint32_t tmem_p_stride = SPLIT_P ? BN / 2 : BN;
+    const uint32_t tmem_o0 = tmem_base + (SPLIT_P ? 3 * BN : 2 * BN);
 
     if (warp == 8) {
         // ------------------------------------------------------------ TMA producer
-        if (lane == 0) {
+        if (elect_one()) {
             tma_prefetch_desc(&tmap_q);
             tma_prefetch_desc(&tmap_k);
             tma_prefetch_desc(&tmap_v);
@@ -140,67 +175,83 @@ fused_attention_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_
                     !mbar_wait(smem_u32(&bar_kv_empty[s]), ((j / stages) - 1) & 1, abort_p, args.status, SITE_F_EMPTY, j))
                     break;
                 const uint32_t k_dst = kv_smem + s * 2 * kv_tile_bytes, v_dst = k_dst + kv_tile_bytes;
-                const uint32_t bk = smem_u32(&bar_k_full[s]), bv = smem_u32(&bar_v_full[s]);
-                mbar_arrive_expect_tx(bk, kv_tile_bytes);
+                const uint32_t bar = smem_u32(&bar_kv_full[s]);
+                mbar_arrive_expect_tx(bar, 2 * kv_tile_bytes);
                 for (int ch = 0; ch < nch; ++ch)
-                    tma_load_3d(k_dst + ch * BN * CHUNK_ROW_BYTES, &tmap_k, bk, ch * CHUNK_COLS, j * BN, bh);
-                mbar_arrive_expect_tx(bv, kv_tile_bytes);
+                    tma_load_3d(k_dst + ch * BN * CHUNK_ROW_BYTES, &tmap_k, bar, ch * CHUNK_COLS, j * BN, bh);
                 for (int ch = 0; ch < nch; ++ch)
-                    tma_load_3d(v_dst + ch * BN * CHUNK_ROW_BYTES, &tmap_v, bv, ch * CHUNK_COLS, j * BN, bh);
+                    tma_load_3d(v_dst + ch * BN * CHUNK_ROW_BYTES, &tmap_v, bar, ch * CHUNK_COLS, j * BN, bh);
             }
         }
-    } else if (warp == 9) {
-        // ------------------------------------------------------------ MMA issuer
-        if (lane == 0) {
+    } else if (warp >= 9) {
+        // ------------------------------------------------------------ MMA issuer of query tile t
+        const int t = warp - 9;
+        if (t < n_qtiles && elect_one()) {
             const uint32_t idesc_s = idesc_f16(TILE_M, BN, false, false, args.negate != 0);
             const uint32_t idesc_o = idesc_f16(TILE_M, dpad, false, true, false);
             const int ksteps_s = (args.d + 15) / 16;
-            auto issue_s = [&](int t, int s) {   // S_t = Q_t K_s^T
-                const uint32_t qa = q_smem + t * q_tile_bytes, kb = kv_smem + s * 2 * kv_tile_bytes;
-                for (int kk = 0; kk < ksteps_s; ++kk) {
-                    const int ch = kk >> 2, within = (kk & 3) * 32;
-                    mma_f16_ss(tmem_base + t * BN,
-                               smem_desc_sw128(qa + ch * TILE_M * CHUNK_ROW_BYTES + within, 16, 1024),
-                               smem_desc_sw128(kb + ch * BN * CHUNK_ROW_BYTES + within, 16, 1024), idesc_s, kk > 0);
-                }
-                tc_commit(smem_u32(&bar_s_full[t]));
+            // descriptors differ only in their low word (the start address >> 4): precompute the offsets
+            const uint64_t q_desc = smem_desc_sw128(q_smem + t * q_tile_bytes, 16, 1024);
+            const uint64_t k_desc = smem_desc_sw128(kv_smem, 16, 1024);
+            const uint64_t v_desc = smem_desc_sw128(kv_smem + kv_tile_bytes, BN * CHUNK_ROW_BYTES, 1024);
+            uint32_t q_off[FUSED_MAX_KSTEPS], k_off[FUSED_MAX_KSTEPS];
+#pragma unroll
+            for (int kk = 0; kk < FUSED_MAX_KSTEPS; ++kk) {
+                q_off[kk] = ((kk >> 2) * TILE_M * CHUNK_ROW_BYTES + (kk & 3) * 32) >> 4;
+                k_off[kk] = ((kk >> 2) * BN * CHUNK_ROW_BYTES + (kk & 3) * 32) >> 4;
+            }
+            const uint32_t stage_off = (2 * kv_tile_bytes) >> 4;
+            const uint32_t tmem_s = tmem_base + t * BN;
+            const uint32_t tmem_p = tmem_p0 + t * tmem_p_stride;
+            const uint32_t tmem_o = tmem_o0 + t * dpad;
+            const uint32_t b_sfull = smem_u32(&bar_s_full[t]), b_sfree = smem_u32(&bar_s_free[t]);
+            const uint32_t b_pfull = smem_u32(&bar_p_full[t]), b_pvdone = smem_u32(&bar_pv_done[t]);
+
+            auto issue_s = [&](int s) {   // S_t = Q_t K_s^T
+                const uint64_t kd = k_desc + (uint64_t)(s * stage_off);
+#pragma unroll
+                for (int kk = 0; kk < FUSED_MAX_KSTEPS; ++kk)
+                    if (kk < ksteps_s) mma_f16_ss(tmem_s, q_desc + q_off[kk], kd + k_off[kk], idesc_s, kk > 0);
+                tc_commit(b_sfull);
             };
-            auto issue_o = [&](int t, int s, bool accumulate) {   // O_t (+)= P_t V_s
-                const uint32_t vb = kv_smem + s * 2 * kv_tile_bytes + kv_tile_bytes;
+            auto issue_o = [&](int s, bool accumulate) {   // O_t (+)= P_t V_s
+                const uint64_t vd = v_desc + (uint64_t)(s * stage_off);
 #pragma unroll
                 for (int kk = 0; kk < BN / 16; ++kk)
-                    mma_f16_ts(tmem_o0 + t * dpad, tmem_base + t * BN + kk * 8,
-                               smem_desc_sw128(vb + kk * 16 * CHUNK_ROW_BYTES, BN * CHUNK_ROW_BYTES, 1024), idesc_o,
+                    mma_f16_ts(tmem_o, tmem_p + kk * 8, vd + (uint64_t)(kk * ((16 * CHUNK_ROW_BYTES) >> 4)), idesc_o,
                                accumulate || kk > 0);
             };
-            bool ok = true;
-            for (int t = 0; t < n_qtiles && ok; ++t)
-                ok = mbar_wait(smem_u32(&bar_q_full[t]), 0, abort_p, args.status, SITE_F_Q, t);
-            if (ok) ok = mbar_wait(smem_u32(&bar_k_full[0]), 0, abort_p, args.status, SITE_F_K, 0);
+
+            bool ok = mbar_wait(smem_u32(&bar_q_full[t]), 0, abort_p, args.status, SITE_F_Q, t) &&
+                      mbar_wait(smem_u32(&bar_kv_full[0]), 0, abort_p, args.status, SITE_F_KV, 0);
             if (ok) {
                 tc_fence_after_sync();
-                for (int t = 0; t < n_qtiles; ++t) issue_s(t, 0);
+                issue_s(0);
             }
             for (int j = 0; j < n_kv && ok; ++j) {
                 const int s = j % stages;
-                ok = mbar_wait(smem_u32(&bar_v_full[s]), (j / stages) & 1, abort_p, args.status, SITE_F_V, j);
-                for (int t = 0; t < n_qtiles && ok; ++t) {
-                    ok = mbar_wait(smem_u32(&bar_p_full[t]), j & 1, abort_p, args.status, SITE_F_P, j);
+                const int s1 = (j + 1) % stages;
+                FUSED_TRACE(2 + t, j, 0);
+                if (j + 1 < n_kv)   // the next K/V tile landed long ago: take this wait off the critical path
+                    ok = mbar_wait(smem_u32(&bar_kv_full[s1]), ((j + 1) / stages) & 1, abort_p, args.status, SITE_F_KV, j + 1);
+                if (SPLIT_P && ok && j + 1 < n_kv) {
+                    // S_t is free once its row sits in the softmax registers: start tile j+1 right away
+                    ok = mbar_wait(b_sfree, j & 1, abort_p, args.status, SITE_F_SFREE, j);
                     if (!ok) break;
                     tc_fence_after_sync();
-                    issue_o(t, s, j > 0);
-                    if (t == n_qtiles - 1) tc_commit(smem_u32(&bar_kv_empty[s]));  // K_j and V_j fully consumed
-                    if (j + 1 < n_kv) {
-                        const int s1 = (j + 1) % stages;
-                        ok = mbar_wait(smem_u32(&bar_k_full[s1]), ((j + 1) / stages) & 1, abort_p, args.status,
-                                       SITE_F_K, j + 1);
-                        if (!ok) break;
-                        tc_fence_after_sync();
-                        issue_s(t, s1);
-                    } else {
-                        tc_commit(smem_u32(&bar_o_full[t]));
-                    }
+                    FUSED_TRACE(2 + t, j, 1);
+                    issue_s(s1);
+                    FUSED_TRACE(2 + t, j, 2);
                 }
+                if (ok) ok = mbar_wait(b_pfull, j & 1, abort_p, args.status, SITE_F_P, j);
+                if (!ok) break;
+                tc_fence_after_sync();
+                FUSED_TRACE(2 + t, j, 3);
+                issue_o(s, j > 0);
+                tc_commit(b_pvdone);                          // O_t holds tiles 0..j; P_t may be rewritten
+                tc_commit(smem_u32(&bar_kv_empty[s]));        // this issuer is done with K_j and V_j
+                if (!SPLIT_P && j + 1 < n_kv) issue_s(s1);    // P_t shares columns with S_t: S follows P V
+                FUSED_TRACE(2 + t, j, 4);
             }
         }
     } else {
@@ -210,35 +261,54 @@ fused_attention_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_
             const int r = tid & (TILE_M - 1);    // row inside the tile = TMEM lane
             const uint32_t lane_off = (uint32_t)((warp & 3) * 32) << 16;
             const uint32_t tmem_s = tmem_base + t * BN + lane_off;
+            const uint32_t tmem_p = tmem_p0 + t * tmem_p_stride + lane_off;
             const uint32_t tmem_o = tmem_o0 + t * dpad + lane_off;
+            const uint32_t b_sfull = smem_u32(&bar_s_full[t]), b_sfree = smem_u32(&bar_s_free[t]);
+            const uint32_t b_pfull = smem_u32(&bar_p_full[t]), b_pvdone = smem_u32(&bar_pv_done[t]);
+            const bool tracer = (warp & 3) == 0 && lane == 0;
             const float c2 = args.scale_log2e;
+            const bool take_turns = FUSED_TAKE_TURNS && n_qtiles == 2;
+            const uint32_t b_my_turn = smem_u32(&bar_turn[t]), b_other_turn = smem_u32(&bar_turn[t ^ 1]);
+            if (take_turns && t == 1 && lane == 0) mbar_arrive(b_other_turn);   // tile 0 goes first
             float m_run = -INFINITY;  // running max, in raw score units
             float l_run = 0.f;        // running sum of p (relative to m_run)
             bool ok = true;
             for (int j = 0; j < n_kv; ++j) {
-                ok = mbar_wait(smem_u32(&bar_s_full[t]), j & 1, abort_p, args.status, SITE_F_S, j);
+                if (tracer) FUSED_TRACE(t, j, 0);
+                ok = mbar_wait(b_sfull, j & 1, abort_p, args.status, SITE_F_S, j);
                 ok = __all_sync(0xffffffffu, ok);
                 if (!ok) break;
                 tc_fence_after_sync();
+                if (tracer) FUSED_TRACE(t, j, 1);
                 const int valid = args.Nk - j * BN;   // columns >= valid are zero-filled keys
-                float row_max = -INFINITY;
+                // the whole row of S_t into registers with one wait, then hand S_t back
+                uint32_t s[BN];
 #pragma unroll
-                for (int g = 0; g < BN / 16; ++g) {
-                    uint32_t x[16];
-                    tmem_ld16(tmem_s + g * 16, x);
-                    tmem_wait_ld();
-                    if (valid >= BN) {
+                for (int g = 0; g < BN / 32; ++g) tmem_ld32(tmem_s + g * 32, &s[g * 32]);
+                tmem_wait_ld();
+                tc_fence_before_sync();
+                if (lane == 0) mbar_arrive(b_sfree);
+                if (tracer) FUSED_TRACE(t, j, 2);
+                if (valid < BN) {
 #pragma unroll
-                        for (int c = 0; c < 16; ++c) row_max = fmaxf(row_max, __uint_as_float(x[c]));
-                    } else {
-#pragma unroll
-                        for (int c = 0; c < 16; ++c)
-                            if (g * 16 + c < valid) row_max = fmaxf(row_max, __uint_as_float(x[c]));
-                    }
+                    for (int c = 0; c < BN; ++c)
+                        if (c >= valid) s[c] = 0xff800000u;   // -inf: no part in the maximum
                 }
+                float mx[8];
+#pragma unroll
+                for (int c = 0; c < 8; ++c) mx[c] = __uint_as_float(s[c]);
+#pragma unroll
+                for (int c = 8; c < BN; ++c) mx[c & 7] = fmaxf(mx[c & 7], __uint_as_float(s[c]));
+                const float row_max = fmaxf(fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3])),
+                                            fmaxf(fmaxf(mx[4], mx[5]), fmaxf(mx[6], mx[7])));
                 if (j == 0) {
                     m_run = row_max;
                 } else {
+                    // P_t and O_t belong to the tensor pipe until the P V product of tile j-1 has completed
+                    ok = mbar_wait(b_pvdone, (j - 1) & 1, abort_p, args.status, SITE_F_PFREE, j);
+                    ok = __all_sync(0xffffffffu, ok);
+                    if (!ok) break;
+                    tc_fence_after_sync();
                     const bool grow = (row_max - m_run) * c2 > FUSED_RESCALE_LOG2;
                     if (__any_sync(0xffffffffu, grow)) {
                         const float alpha = grow ? ex2_approx((m_run - row_max) * c2) : 1.f;
@@ -255,30 +325,41 @@ fused_attention_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_
                     }
                 }
                 const float neg_mc = -m_run * c2;
-#pragma unroll
-                for (int g = 0; g < BN / 16; ++g) {
-                    uint32_t x[16], packed[8];
-                    tmem_ld16(tmem_s + g * 16, x);
-                    tmem_wait_ld();
-                    float p[16];
-#pragma unroll
-                    for (int c = 0; c < 16; ++c) p[c] = ex2_approx(fmaf(__uint_as_float(x[c]), c2, neg_mc));
-                    if (valid < BN) {
-#pragma unroll
-                        for (int c = 0; c < 16; ++c)
-                            if (g * 16 + c >= valid) p[c] = 0.f;
-                    }
-#pragma unroll
-                    for (int c = 0; c < 16; ++c) l_run += p[c];
-#pragma unroll
-                    for (int c = 0; c < 8; ++c) packed[c] = pack_half2(p[2 * c], p[2 * c + 1]);
-                    tmem_st8(tmem_s + g * 8, packed);
+                if (take_turns) {
+                    ok = mbar_wait(b_my_turn, j & 1, abort_p, args.status, SITE_F_TURN, j);
+                    ok = __all_sync(0xffffffffu, ok);
+                    if (!ok) break;
                 }
+                if (tracer) FUSED_TRACE(t, j, 3);
+                float sum[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+                for (int g = 0; g < BN / 32; ++g) {
+                    uint32_t packed[16];
+#pragma unroll
+                    for (int c = 0; c < 32; c += 2) {
+                        const float x0 = fmaf(__uint_as_float(s[g * 32 + c]), c2, neg_mc);
+                        const float x1 = fmaf(__uint_as_float(s[g * 32 + c + 1]), c2, neg_mc);
+                        // a fixed share of the exponentials runs on the FMA pipe instead of the SFU
+                        float p0 = ((c & 7) < FUSED_POLY_PER8) ? ex2_poly(x0) : ex2_approx(x0);
+                        float p1 = (((c + 1) & 7) < FUSED_POLY_PER8) ? ex2_poly(x1) : ex2_approx(x1);
+                        if (valid < BN) {   // zero-filled key rows carry no weight (also when scale == 0)
+                            if (g * 32 + c >= valid) p0 = 0.f;
+                            if (g * 32 + c + 1 >= valid) p1 = 0.f;
+                        }
+                        sum[(c >> 1) & 3] += p0 + p1;
+                        packed[c >> 1] = pack_half2(p0, p1);
+                    }
+                    tmem_st16(tmem_p + g * 16, packed);
+                }
+                l_run += (sum[0] + sum[1]) + (sum[2] + sum[3]);
+                if (take_turns && lane == 0) mbar_arrive(b_other_turn);
+                if (tracer) FUSED_TRACE(t, j, 4);
                 tmem_wait_st();
                 tc_fence_before_sync();
-                mbar_arrive(smem_u32(&bar_p_full[t]));
+                if (lane == 0) mbar_arrive(b_pfull);
+                if (tracer) FUSED_TRACE(t, j, 5);
             }
-            if (ok) ok = mbar_wait(smem_u32(&bar_o_full[t]), 0, abort_p, args.status, SITE_F_O, t);
+            if (ok) ok = mbar_wait(b_pvdone, (n_kv - 1) & 1, abort_p, args.status, SITE_F_O, t);
             ok = __all_sync(0xffffffffu, ok);
             if (ok) {
                 tc_fence_after_sync();
@@ -312,10 +393,7 @@ fused_attention_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_
     __syncthreads();
     if (warp == 8 && lane == 0 && abort_flag) {
         // gave up somewhere: give copies still in flight a bounded chance to land
-        for (int s = 0; s < stages; ++s) {
-            mbar_drain(smem_u32(&bar_k_full[s]), 0);
-            mbar_drain(smem_u32(&bar_v_full[s]), 0);
-        }
+        for (int s = 0; s < stages; ++s) mbar_drain(smem_u32(&bar_kv_full[s]), 0);
     }
     __syncthreads();
     if (warp == 9) {

@@ -14,6 +14,7 @@
 #include "../../include/sd_attn_debug.h"
 #include "cross_kernel.cuh"
 #include "fused_kernel.cuh"
+#include "fused4_kernel.cuh"
 #include "simt_kernel.cuh"
 #include "twopass_kernel.cuh"
 
@@ -37,6 +38,7 @@ struct sd_attn_handle {
     encode_tiled_fn encode_tiled;
     cudaError_t last_cuda_error;
     int sm_count;
+    int prefer_two_tile;      // SD_ATTN_FUSED_TWO_TILE=1: use the two-tile fused kernel for every head dim
 };
 
 static const float LOG2E = 1.4426950408889634f;
@@ -93,11 +95,15 @@ extern "C" int sd_attn_create(sd_attn_handle** out) {
         return cuda_fail(nullptr, e != cudaSuccess ? e : cudaErrorUnknown);
     }
     h->encode_tiled = (encode_tiled_fn)fn;
+    const char* two = getenv("SD_ATTN_FUSED_TWO_TILE");
+    h->prefer_two_tile = (two && two[0] == '1') ? 1 : 0;
 
     // dynamic shared memory ceilings of every kernel, once
     e = raise_smem_limit(cross_attention_kernel, cross_smem_bytes(3, 128));
-    if (e == cudaSuccess) e = raise_smem_limit(fused_attention_kernel<128>, fused_smem_bytes_max());
-    if (e == cudaSuccess) e = raise_smem_limit(fused_attention_kernel<64>, fused_smem_bytes_max());
+    if (e == cudaSuccess) e = raise_smem_limit(fused_attention_kernel<128, true>, fused_smem_bytes_max());
+    if (e == cudaSuccess) e = raise_smem_limit(fused_attention_kernel<128, false>, fused_smem_bytes_max());
+    if (e == cudaSuccess) e = raise_smem_limit(fused_attention_kernel<64, true>, fused_smem_bytes_max());
+    if (e == cudaSuccess) e = raise_smem_limit(fused4_attention_kernel, fused4_smem_bytes());
     if (e == cudaSuccess) e = raise_smem_limit(twopass_scores_kernel, twopass_scores_smem_bytes(3));
     if (e == cudaSuccess) e = raise_smem_limit(twopass_pv_kernel, twopass_pv_smem_bytes(3));
     if (e == cudaSuccess) e = raise_smem_limit(simt_attention_kernel<float, 5>, simt_smem_bytes(160));
@@ -255,20 +261,51 @@ static int launch_cross(sd_attn_handle* h, const Problem& p) {
     return SD_ATTN_OK;
 }
 
+// d <= 64: four query tiles per CTA over key tiles of 64 (the softmax, not the tensor pipe, is the bound)
+static int launch_fused4(sd_attn_handle* h, const Problem& p) {
+    Fused4Args a;
+    a.out = (__half*)p.out;
+    a.Nq = p.Nq; a.Nk = p.Nk; a.d = p.d;
+    a.dpad = (p.d + 15) / 16 * 16;
+    a.scale_log2e = fabsf(p.scale) * LOG2E;
+    a.negate = p.scale < 0.f;
+    a.status = h->dev_status;
+#ifdef SD_ATTN_TRACE
+    a.trace = (long long*)h->dump_scores;
+#endif
+    CUtensorMap tq, tk, tv;
+    int rc = make_tmap(h, &tq, p.q, p.BH, p.Nq, p.d, TILE_M);
+    if (rc == SD_ATTN_OK) rc = make_tmap(h, &tk, p.k, p.BH, p.Nk, p.d, F4_BN);
+    if (rc == SD_ATTN_OK) rc = make_tmap(h, &tv, p.v, p.BH, p.Nk, p.d, F4_BN);
+    if (rc != SD_ATTN_OK) return rc;
+    dim3 grid((p.Nq + F4_TILES * TILE_M - 1) / (F4_TILES * TILE_M), p.BH), block(F4_THREADS);
+    fused4_attention_kernel<<<grid, block, fused4_smem_bytes(), p.stream>>>(tq, tk, tv, a);
+    cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess) return cuda_fail(h, e);
+    h->launches += 1;
+    return SD_ATTN_OK;
+}
+
 static int launch_fused(sd_attn_handle* h, const Problem& p) {
+    if (p.d <= F4_MAX_D && !h->prefer_two_tile) return launch_fused4(h, p);
     FusedArgs a;
     const int bn = fused_block_n(p.d);
     fused_fill_args(&a, (__half*)p.out, p.Nq, p.Nk, p.d, fabsf(p.scale) * LOG2E, p.scale < 0.f, h->dev_status);
+#ifdef SD_ATTN_TRACE
+    a.trace = (long long*)h->dump_scores;   // trace builds reuse the debug pointer as the probe buffer
+#endif
     CUtensorMap tq, tk, tv;
     int rc = make_tmap(h, &tq, p.q, p.BH, p.Nq, p.d, TILE_M);
     if (rc == SD_ATTN_OK) rc = make_tmap(h, &tk, p.k, p.BH, p.Nk, p.d, bn);
     if (rc == SD_ATTN_OK) rc = make_tmap(h, &tv, p.v, p.BH, p.Nk, p.d, bn);
     if (rc != SD_ATTN_OK) return rc;
     dim3 grid((p.Nq + 2 * TILE_M - 1) / (2 * TILE_M), p.BH), block(FUSED_THREADS);
-    if (bn == 128)
-        fused_attention_kernel<128><<<grid, block, fused_smem_bytes(a), p.stream>>>(tq, tk, tv, a);
+    if (bn == 128 && fused_split_p(p.d))
+        fused_attention_kernel<128, true><<<grid, block, fused_smem_bytes(a), p.stream>>>(tq, tk, tv, a);
+    else if (bn == 128)
+        fused_attention_kernel<128, false><<<grid, block, fused_smem_bytes(a), p.stream>>>(tq, tk, tv, a);
     else
-        fused_attention_kernel<64><<<grid, block, fused_smem_bytes(a), p.stream>>>(tq, tk, tv, a);
+        fused_attention_kernel<64, true><<<grid, block, fused_smem_bytes(a), p.stream>>>(tq, tk, tv, a);
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) return cuda_fail(h, e);
     h->launches += 1;
