@@ -2,23 +2,25 @@
 //
 // At d = 40 a score element costs only 160 tensor-core FLOPs but one exponential, and the special
 // function unit retires 16 exponentials per clock per SM: the softmax, not the tensor pipe, bounds the
-// kernel.  Two softmax warps per scheduler keep that unit about 95% busy only while both are inside
-// their exponential loop; loads from tensor memory, barrier waits and the tensor-core round trip leave
-// it idle.  This kernel therefore runs FOUR query tiles of 128 rows per CTA -- four softmax warpgroups,
-// four warps per scheduler -- over key tiles of 64, so that some group is always in its exponentials:
-//   warps 0-15   softmax of tiles 0..3 (thread = query row = TMEM lane), 112 registers each
+// kernel.  Two softmax warps per scheduler keep that unit busy only while both are inside their
+// exponential sweep; loads from tensor memory, barrier waits and the tensor-core round trip leave it
+// idle.  This kernel therefore runs FOUR query tiles of 128 rows per CTA -- four softmax warpgroups,
+// four warps per scheduler -- over key tiles of 64:
+//   warps 0-15   softmax of tiles 0..3 (thread = query row = TMEM lane), 104 registers each
 //   warp 16      TMA producer          warps 17-20  MMA issuers, one per tile (32 registers each;
 //                warps 21-23 only fill the second control warpgroup so that setmaxnreg applies)
-// Tensor memory (512 columns): per tile S_t (64 columns, fp32) and O_t (dpad <= 64 columns); the packed
-// fp16 weights P_t overwrite the first 32 columns of S_t, so the next S_t is issued after the P V
-// product of the current key tile (in issue order on the same thread).
-// The running-max rescale of O_t is lazy (only when the max grew by more than 2^8) and safe without
-// an extra barrier: S_t(j) being ready implies that the P V product of tile j-1 has completed.
+// Tensor memory (512 columns): per tile S_t (64 fp32 columns) and O_t (dpad <= 64 columns); the packed
+// fp16 weights P_t overwrite the first 32 columns of S_t, so the next S_t follows the P V product of the
+// current key tile in issue order on the same thread.  (A 48-wide key tile with P_t in columns of its
+// own, which takes the tensor-core round trip off the softmax's path, measured slower: the fixed cost
+// per key tile outweighs it.)
+// The running-max rescale of O_t is lazy (only when the max grew by more than 2^8).
 #pragma once
 #include <cuda.h>
 
 #include "cross_kernel.cuh"  // TILE_M, CHUNK_COLS, CHUNK_ROW_BYTES
-#include "fused_kernel.cuh"  // FUSED_RESCALE_LOG2, FUSED_TRACE
+#include "fused_kernel.cuh"  // FUSED_RESCALE_LOG2, FUSED_TRACE, FUSED_POLY_PER8
+#include "softmax_math.cuh"
 #include "tc_common.cuh"
 
 namespace sd_attn {
@@ -47,14 +49,16 @@ __host__ inline size_t fused4_smem_bytes() {
     return (size_t)F4_TILES * TILE_M * CHUNK_ROW_BYTES + (size_t)F4_STAGES * 2 * F4_BN * CHUNK_ROW_BYTES + 1024;
 }
 
-enum { SITE_G_Q = 30, SITE_G_KV = 31, SITE_G_EMPTY = 32, SITE_G_S = 33, SITE_G_P = 34, SITE_G_O = 35 };
+enum { SITE_G_Q = 30, SITE_G_KV = 31, SITE_G_EMPTY = 32, SITE_G_S = 33, SITE_G_P = 34, SITE_G_O = 35, SITE_G_PV = 37 };
 
 __global__ void __launch_bounds__(F4_THREADS, 1)
 fused4_attention_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__ CUtensorMap tmap_k,
                         const __grid_constant__ CUtensorMap tmap_v, const Fused4Args args) {
+    constexpr int BN = F4_BN;
     extern __shared__ uint8_t f4_smem_raw[];
+    // per query tile: Q landed | S ready (MMA) | P ready (softmax) | P V done (MMA)
     __shared__ __align__(8) uint64_t bar_q_full[F4_TILES], bar_s_full[F4_TILES], bar_p_full[F4_TILES],
-        bar_o_done[F4_TILES];
+        bar_pv_done[F4_TILES];
     __shared__ __align__(8) uint64_t bar_kv_full[F4_STAGES], bar_kv_empty[F4_STAGES];
     __shared__ uint32_t tmem_base_slot;
     __shared__ int abort_flag;
@@ -64,12 +68,12 @@ fused4_attention_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid
     const int row_base = blockIdx.x * F4_TILES * TILE_M;
     int n_qtiles = (args.Nq - row_base + TILE_M - 1) / TILE_M;
     if (n_qtiles > F4_TILES) n_qtiles = F4_TILES;
-    const int n_kv = (args.Nk + F4_BN - 1) / F4_BN;
+    const int n_kv = (args.Nk + BN - 1) / BN;
     const int dpad = args.dpad;
 
     const uint32_t smem_base = (smem_u32(f4_smem_raw) + 1023u) & ~1023u;
     constexpr uint32_t q_tile_bytes = TILE_M * CHUNK_ROW_BYTES;     // one 64-column chunk (d <= 64)
-    constexpr uint32_t kv_tile_bytes = F4_BN * CHUNK_ROW_BYTES;
+    constexpr uint32_t kv_tile_bytes = BN * CHUNK_ROW_BYTES;
     const uint32_t q_smem = smem_base;                              // [4][128 rows][128 B]
     const uint32_t kv_smem = q_smem + F4_TILES * q_tile_bytes;      // [stages][K | V][64 rows][128 B]
     volatile int* abort_p = &abort_flag;
@@ -80,7 +84,7 @@ fused4_attention_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid
             mbar_init(smem_u32(&bar_q_full[t]), 1);
             mbar_init(smem_u32(&bar_s_full[t]), 1);
             mbar_init(smem_u32(&bar_p_full[t]), 4);    // one arrival per softmax warp
-            mbar_init(smem_u32(&bar_o_done[t]), 1);
+            mbar_init(smem_u32(&bar_pv_done[t]), 1);
         }
         for (int s = 0; s < F4_STAGES; ++s) {
             mbar_init(smem_u32(&bar_kv_full[s]), 1);
@@ -96,8 +100,7 @@ fused4_attention_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid
     __syncthreads();
     tc_fence_after_sync();
     const uint32_t tmem_base = tmem_base_slot;
-    // columns: S_0 S_1 S_2 S_3 (64 each) | O_0 O_1 O_2 O_3 (dpad each)
-    const uint32_t tmem_o0 = tmem_base + F4_TILES * F4_BN;
+    const uint32_t tmem_o0 = tmem_base + F4_TILES * BN;   // columns: S_0..S_3 | O_0..O_3
 
     // All four warps of a warpgroup must execute the SAME setmaxnreg instruction: one site per kind.
     if (warp >= 16) setmaxnreg_dec<F4_CONTROL_REGS>();
@@ -120,24 +123,25 @@ fused4_attention_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid
                 const uint32_t k_dst = kv_smem + s * 2 * kv_tile_bytes, v_dst = k_dst + kv_tile_bytes;
                 const uint32_t bar = smem_u32(&bar_kv_full[s]);
                 mbar_arrive_expect_tx(bar, 2 * kv_tile_bytes);
-                tma_load_3d(k_dst, &tmap_k, bar, 0, j * F4_BN, bh);
-                tma_load_3d(v_dst, &tmap_v, bar, 0, j * F4_BN, bh);
+                tma_load_3d(k_dst, &tmap_k, bar, 0, j * BN, bh);
+                tma_load_3d(v_dst, &tmap_v, bar, 0, j * BN, bh);
             }
         }
     } else if (warp > 16) {
         // ------------------------------------------------------------ MMA issuer of query tile t
         const int t = warp - 17;
         if (t < F4_TILES && t < n_qtiles && elect_one()) {
-            const uint32_t idesc_s = idesc_f16(TILE_M, F4_BN, false, false, args.negate != 0);
+            const uint32_t idesc_s = idesc_f16(TILE_M, BN, false, false, args.negate != 0);
             const uint32_t idesc_o = idesc_f16(TILE_M, dpad, false, true, false);
             const int ksteps_s = (args.d + 15) / 16;   // <= 4: all inside one swizzled 64-column chunk
             const uint64_t q_desc = smem_desc_sw128(q_smem + t * q_tile_bytes, 16, 1024);
             const uint64_t k_desc = smem_desc_sw128(kv_smem, 16, 1024);
-            const uint64_t v_desc = smem_desc_sw128(kv_smem + kv_tile_bytes, F4_BN * CHUNK_ROW_BYTES, 1024);
+            const uint64_t v_desc = smem_desc_sw128(kv_smem + kv_tile_bytes, BN * CHUNK_ROW_BYTES, 1024);
             constexpr uint32_t stage_off = (2 * kv_tile_bytes) >> 4;
-            const uint32_t tmem_s = tmem_base + t * F4_BN;
+            const uint32_t tmem_s = tmem_base + t * BN;
             const uint32_t tmem_o = tmem_o0 + t * dpad;
             const uint32_t b_sfull = smem_u32(&bar_s_full[t]), b_pfull = smem_u32(&bar_p_full[t]);
+            const uint32_t b_pvdone = smem_u32(&bar_pv_done[t]);
 
             auto issue_s = [&](int s) {   // S_t = Q_t K_s^T
                 const uint64_t kd = k_desc + (uint64_t)(s * stage_off);
@@ -146,10 +150,10 @@ fused4_attention_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid
                     if (kk < ksteps_s) mma_f16_ss(tmem_s, q_desc + (uint64_t)(kk * 2), kd + (uint64_t)(kk * 2), idesc_s, kk > 0);
                 tc_commit(b_sfull);
             };
-            auto issue_o = [&](int s, bool accumulate) {   // O_t (+)= P_t V_s
+            auto issue_o = [&](int s, bool accumulate) {   // O_t (+)= P_t V_s, P_t in the first columns of S_t
                 const uint64_t vd = v_desc + (uint64_t)(s * stage_off);
 #pragma unroll
-                for (int kk = 0; kk < F4_BN / 16; ++kk)
+                for (int kk = 0; kk < BN / 16; ++kk)
                     mma_f16_ts(tmem_o, tmem_s + kk * 8, vd + (uint64_t)(kk * ((16 * CHUNK_ROW_BYTES) >> 4)), idesc_o,
                                accumulate || kk > 0);
             };
@@ -171,9 +175,9 @@ fused4_attention_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid
                 tc_fence_after_sync();
                 if (t == 0) FUSED_TRACE(4, j, 1);
                 issue_o(s, j > 0);
-                tc_commit(smem_u32(&bar_kv_empty[s]));   // this issuer is done with K_j and V_j
-                if (j + 1 < n_kv) issue_s(s1);           // also tells the softmax that O_t holds tiles 0..j
-                else tc_commit(smem_u32(&bar_o_done[t]));
+                if (j + 1 < n_kv) issue_s(s1);                // the softmax waits for this one: commit it first
+                tc_commit(b_pvdone);                          // O_t holds tiles 0..j
+                tc_commit(smem_u32(&bar_kv_empty[s]));        // this issuer is done with K_j and V_j
                 if (t == 0) FUSED_TRACE(4, j, 2);
             }
         }
@@ -184,9 +188,10 @@ fused4_attention_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid
         if (t < n_qtiles) {
             const int r = tid & (TILE_M - 1);    // row inside the tile = TMEM lane
             const uint32_t lane_off = (uint32_t)((warp & 3) * 32) << 16;
-            const uint32_t tmem_s = tmem_base + t * F4_BN + lane_off;
+            const uint32_t tmem_s = tmem_base + t * BN + lane_off;
             const uint32_t tmem_o = tmem_o0 + t * dpad + lane_off;
             const uint32_t b_sfull = smem_u32(&bar_s_full[t]), b_pfull = smem_u32(&bar_p_full[t]);
+            const uint32_t b_pvdone = smem_u32(&bar_pv_done[t]);
             const float c2 = args.scale_log2e;
             float m_run = -INFINITY;  // running max, in raw score units
             float l_run = 0.f;        // running sum of p (relative to m_run)
@@ -199,32 +204,22 @@ fused4_attention_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid
                 if (!ok) break;
                 tc_fence_after_sync();
                 if (tracer) FUSED_TRACE(t, j, 1);
-                const int valid = args.Nk - j * F4_BN;   // columns >= valid are zero-filled keys
-                uint32_t s[F4_BN];
+                const int valid = args.Nk - j * BN;   // columns >= valid are zero-filled keys
+                uint32_t s[BN];
                 tmem_ld32(tmem_s, &s[0]);
                 tmem_ld32(tmem_s + 32, &s[32]);
                 tmem_wait_ld();
                 if (tracer) FUSED_TRACE(t, j, 2);
-                float mx[8];
-#pragma unroll
-                for (int c = 0; c < 8; ++c) mx[c] = -INFINITY;
-                if (valid >= F4_BN) {
-#pragma unroll
-                    for (int c = 0; c < F4_BN; ++c) mx[c & 7] = fmaxf(mx[c & 7], __uint_as_float(s[c]));
-                } else {   // zero-filled key rows take no part in the maximum
-#pragma unroll
-                    for (int c = 0; c < F4_BN; ++c)
-                        if (c < valid) mx[c & 7] = fmaxf(mx[c & 7], __uint_as_float(s[c]));
-                }
-                const float row_max = fmaxf(fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3])),
-                                            fmaxf(fmaxf(mx[4], mx[5]), fmaxf(mx[6], mx[7])));
+                const bool ragged = valid < BN;   // only the last key tile can be
+                const float row_max = ragged ? row_max_masked<BN>(s, valid) : row_max_bf16<BN>(s);
                 if (j == 0) {
                     m_run = row_max;
                 } else {
                     const bool grow = (row_max - m_run) * c2 > FUSED_RESCALE_LOG2;
                     if (__any_sync(0xffffffffu, grow)) {
-                        // rare: rescale O_t in 8-column pieces, then fetch the row of S_t again (its
-                        // registers are reused here to keep the common path within the register budget)
+                        // rare.  S_t(j) being ready means the P V product of tile j-1 was issued before it and has
+                        // completed, so O_t may be touched.  The first registers of the score row are borrowed
+                        // (register budget) and the row, still intact in tensor memory, is fetched again.
                         const float alpha = grow ? ex2_approx((m_run - row_max) * c2) : 1.f;
                         if (grow) m_run = row_max;
                         l_run *= alpha;
@@ -243,31 +238,31 @@ fused4_attention_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid
                 }
                 const float neg_mc = -m_run * c2;
                 if (tracer) FUSED_TRACE(t, j, 3);
-                float sum[4] = {0.f, 0.f, 0.f, 0.f};
-#pragma unroll
-                for (int g = 0; g < F4_BN / 32; ++g) {
-                    uint32_t packed[16];
-#pragma unroll
-                    for (int c = 0; c < 32; c += 2) {
-                        float p0 = ex2_approx(fmaf(__uint_as_float(s[g * 32 + c]), c2, neg_mc));
-                        float p1 = ex2_approx(fmaf(__uint_as_float(s[g * 32 + c + 1]), c2, neg_mc));
-                        if (valid < F4_BN) {   // zero-filled key rows carry no weight (also when scale == 0)
-                            if (g * 32 + c >= valid) p0 = 0.f;
-                            if (g * 32 + c + 1 >= valid) p1 = 0.f;
-                        }
-                        sum[(c >> 1) & 3] += p0 + p1;
-                        packed[c >> 1] = pack_half2(p0, p1);
-                    }
-                    tmem_st16(tmem_s + g * 16, packed);   // P_t over columns of S_t that already sit in registers
+                uint32_t packed[16];
+                if (!ragged) {
+                    const uint64_t c2c2 = pack_b64(__float_as_uint(c2), __float_as_uint(c2));
+                    const uint64_t nmnm = pack_b64(__float_as_uint(neg_mc), __float_as_uint(neg_mc));
+                    uint64_t acc[2] = {0ull, 0ull};
+                    exp2_pack_32<FUSED_POLY_PER8>(&s[0], c2c2, nmnm, packed, acc);
+                    tmem_st16(tmem_s, packed);        // P_t over columns of S_t that already sit in registers
+                    exp2_pack_32<FUSED_POLY_PER8>(&s[32], c2c2, nmnm, packed, acc);
+                    tmem_st16(tmem_s + 16, packed);
+                    l_run += sum_f32x2(acc[0], acc[1]);
+                } else {
+                    float sum = 0.f;
+                    exp2_pack_32_masked(&s[0], c2, neg_mc, 0, valid, packed, sum);
+                    tmem_st16(tmem_s, packed);
+                    exp2_pack_32_masked(&s[32], c2, neg_mc, 32, valid, packed, sum);
+                    tmem_st16(tmem_s + 16, packed);
+                    l_run += sum;
                 }
-                l_run += (sum[0] + sum[1]) + (sum[2] + sum[3]);
                 if (tracer) FUSED_TRACE(t, j, 4);
                 tmem_wait_st();
                 tc_fence_before_sync();
                 if (lane == 0) mbar_arrive(b_pfull);
                 if (tracer) FUSED_TRACE(t, j, 5);
             }
-            if (ok) ok = mbar_wait(smem_u32(&bar_o_done[t]), 0, abort_p, args.status, SITE_G_O, t);
+            if (ok) ok = mbar_wait(b_pvdone, (n_kv - 1) & 1, abort_p, args.status, SITE_G_O, t);
             ok = __all_sync(0xffffffffu, ok);
             if (ok) {
                 tc_fence_after_sync();

@@ -17,14 +17,16 @@
 //                            p <= 256 fits fp16); p = exp2(s*c - m*c), a fixed share of them evaluated on
 //                            the FMA pipe; P_t written back to tensor memory as packed fp16
 //   O_t += P_t V_j           tcgen05.mma, P from tensor memory, V as an N-major shared-memory operand
-// When 3*BN + 2*dpad <= 512 tensor-memory columns (d <= 64) P_t has columns of its own, and the
-// next S_t is issued as soon as the row of S_t sits in registers; otherwise P_t reuses the columns
-// of S_t and the next S_t follows the P V product.
+// Tensor memory (512 columns) holds S_0 S_1 | P_0 P_1 | O_0 O_1, i.e. 3*BN + 2*dpad columns: key
+// tiles are 128 wide for d <= 64 and 64 wide above.  P_t has columns of its own, so the next S_t is
+// issued as soon as the row of S_t sits in the softmax registers and the tensor-core round trip stays
+// off the softmax's path.
 // All waits are bounded; an expired wait raises a block-wide abort flag and the kernel returns.
 #pragma once
 #include <cuda.h>
 
 #include "cross_kernel.cuh"  // TILE_M, CHUNK_COLS, CHUNK_ROW_BYTES
+#include "softmax_math.cuh"
 #include "tc_common.cuh"
 
 namespace sd_attn {
@@ -37,10 +39,6 @@ constexpr float FUSED_RESCALE_LOG2 = 8.0f;  // rescale O only when the max grew 
 #ifndef SD_ATTN_POLY_PER8
 #define SD_ATTN_POLY_PER8 0
 #endif
-#ifndef SD_ATTN_TAKE_TURNS
-#define SD_ATTN_TAKE_TURNS 0
-#endif
-constexpr bool FUSED_TAKE_TURNS = SD_ATTN_TAKE_TURNS != 0;
 constexpr int FUSED_POLY_PER8 = SD_ATTN_POLY_PER8;  // of every 8 exponentials, this many use the FMA pipe
 
 struct FusedArgs {
@@ -67,9 +65,8 @@ struct FusedArgs {
 #define FUSED_TRACE(role, j, slot) do { } while (0)
 #endif
 
-__host__ inline int fused_block_n(int d) { return ((d + 15) / 16 * 16) <= 128 ? 128 : 64; }
-// P gets tensor-memory columns of its own when S_0 S_1 | P_0 P_1 | O_0 O_1 fit the 512 columns.
-__host__ inline bool fused_split_p(int d) { return 3 * fused_block_n(d) + 2 * ((d + 15) / 16 * 16) <= 512; }
+// key tiles of 128 while S_0 S_1 | P_0 P_1 | O_0 O_1 fit the 512 tensor-memory columns, else of 64
+__host__ inline int fused_block_n(int d) { return ((d + 15) / 16 * 16) <= 64 ? 128 : 64; }
 
 __host__ inline void fused_fill_args(FusedArgs* a, __half* out, int Nq, int Nk, int d, float scale_log2e, bool negate,
                                      int* status) {
@@ -96,19 +93,16 @@ __host__ inline size_t fused_smem_bytes_max() { return FUSED_SMEM_BUDGET + 1024;
 
 enum {
     SITE_F_Q = 10, SITE_F_KV = 11, SITE_F_EMPTY = 13, SITE_F_S = 14, SITE_F_P = 15, SITE_F_O = 16,
-    SITE_F_SFREE = 17, SITE_F_PFREE = 18, SITE_F_TURN = 19
+    SITE_F_SFREE = 17, SITE_F_PFREE = 18
 };
 
-template <int BN, bool SPLIT_P>
+template <int BN>
 __global__ void __launch_bounds__(FUSED_THREADS, 1)
 fused_attention_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__ CUtensorMap tmap_k,
                        const __grid_constant__ CUtensorMap tmap_v, const FusedArgs args) {
     extern __shared__ uint8_t fused_smem_raw[];
     // per query tile: Q landed | S ready (MMA) | S consumed (softmax) | P ready (softmax) | P V done (MMA)
     __shared__ __align__(8) uint64_t bar_q_full[2], bar_s_full[2], bar_s_free[2], bar_p_full[2], bar_pv_done[2];
-    // the two softmax warpgroups take turns on the special-function unit: bar_turn[t] lets tile t run its
-    // exponentials; while one group is there the other loads S, takes its row maximum and waits
-    __shared__ __align__(8) uint64_t bar_turn[2];
     __shared__ __align__(8) uint64_t bar_kv_full[FUSED_MAX_STAGES], bar_kv_empty[FUSED_MAX_STAGES];
     __shared__ uint32_t tmem_base_slot;
     __shared__ int abort_flag;
@@ -135,7 +129,6 @@ fused_attention_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_
             mbar_init(smem_u32(&bar_s_free[t]), 4);    // one arrival per softmax warp
             mbar_init(smem_u32(&bar_p_full[t]), 4);
             mbar_init(smem_u32(&bar_pv_done[t]), 1);
-            mbar_init(smem_u32(&bar_turn[t]), 4);
         }
         for (int s = 0; s < FUSED_MAX_STAGES; ++s) {
             mbar_init(smem_u32(&bar_kv_full[s]), 1);
@@ -151,10 +144,10 @@ fused_attention_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_
     __syncthreads();
     tc_fence_after_sync();
     const uint32_t tmem_base = tmem_base_slot;
-    // columns: S_0 | S_1 | (P_0 | P_1 when split) | O_0 | O_1 ; otherwise P_t reuses the first BN/2 columns of S_t
-    const uint32_t tmem_p0 = SPLIT_P ? tmem_base + 2 * BN : tmem_base;
-    const uint32_t tmem_p_stride = SPLIT_P ? BN / 2 : BN;
-    const uint32_t tmem_o0 = tmem_base + (SPLIT_P ? 3 * BN : 2 * BN);
+    // columns: S_0 | S_1 | P_0 | P_1 | O_0 | O_1
+    const uint32_t tmem_p0 = tmem_base + 2 * BN;
+    constexpr uint32_t tmem_p_stride = BN / 2;
+    const uint32_t tmem_o0 = tmem_base + 3 * BN;
 
     if (warp == 8) {
         // ------------------------------------------------------------ TMA producer
@@ -234,7 +227,7 @@ fused_attention_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_
                 FUSED_TRACE(2 + t, j, 0);
                 if (j + 1 < n_kv)   // the next K/V tile landed long ago: take this wait off the critical path
                     ok = mbar_wait(smem_u32(&bar_kv_full[s1]), ((j + 1) / stages) & 1, abort_p, args.status, SITE_F_KV, j + 1);
-                if (SPLIT_P && ok && j + 1 < n_kv) {
+                if (ok && j + 1 < n_kv) {
                     // S_t is free once its row sits in the softmax registers: start tile j+1 right away
                     ok = mbar_wait(b_sfree, j & 1, abort_p, args.status, SITE_F_SFREE, j);
                     if (!ok) break;
@@ -250,7 +243,6 @@ fused_attention_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_
                 issue_o(s, j > 0);
                 tc_commit(b_pvdone);                          // O_t holds tiles 0..j; P_t may be rewritten
                 tc_commit(smem_u32(&bar_kv_empty[s]));        // this issuer is done with K_j and V_j
-                if (!SPLIT_P && j + 1 < n_kv) issue_s(s1);    // P_t shares columns with S_t: S follows P V
                 FUSED_TRACE(2 + t, j, 4);
             }
         }
@@ -267,9 +259,6 @@ fused_attention_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_
             const uint32_t b_pfull = smem_u32(&bar_p_full[t]), b_pvdone = smem_u32(&bar_pv_done[t]);
             const bool tracer = (warp & 3) == 0 && lane == 0;
             const float c2 = args.scale_log2e;
-            const bool take_turns = FUSED_TAKE_TURNS && n_qtiles == 2;
-            const uint32_t b_my_turn = smem_u32(&bar_turn[t]), b_other_turn = smem_u32(&bar_turn[t ^ 1]);
-            if (take_turns && t == 1 && lane == 0) mbar_arrive(b_other_turn);   // tile 0 goes first
             float m_run = -INFINITY;  // running max, in raw score units
             float l_run = 0.f;        // running sum of p (relative to m_run)
             bool ok = true;
@@ -289,18 +278,8 @@ fused_attention_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_
                 tc_fence_before_sync();
                 if (lane == 0) mbar_arrive(b_sfree);
                 if (tracer) FUSED_TRACE(t, j, 2);
-                if (valid < BN) {
-#pragma unroll
-                    for (int c = 0; c < BN; ++c)
-                        if (c >= valid) s[c] = 0xff800000u;   // -inf: no part in the maximum
-                }
-                float mx[8];
-#pragma unroll
-                for (int c = 0; c < 8; ++c) mx[c] = __uint_as_float(s[c]);
-#pragma unroll
-                for (int c = 8; c < BN; ++c) mx[c & 7] = fmaxf(mx[c & 7], __uint_as_float(s[c]));
-                const float row_max = fmaxf(fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3])),
-                                            fmaxf(fmaxf(mx[4], mx[5]), fmaxf(mx[6], mx[7])));
+                const bool ragged = valid < BN;   // only the last key tile can be
+                const float row_max = ragged ? row_max_masked<BN>(s, valid) : row_max_bf16<BN>(s);
                 if (j == 0) {
                     m_run = row_max;
                 } else {
@@ -325,34 +304,28 @@ fused_attention_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_
                     }
                 }
                 const float neg_mc = -m_run * c2;
-                if (take_turns) {
-                    ok = mbar_wait(b_my_turn, j & 1, abort_p, args.status, SITE_F_TURN, j);
-                    ok = __all_sync(0xffffffffu, ok);
-                    if (!ok) break;
-                }
                 if (tracer) FUSED_TRACE(t, j, 3);
-                float sum[4] = {0.f, 0.f, 0.f, 0.f};
+                if (!ragged) {
+                    const uint64_t c2c2 = pack_b64(__float_as_uint(c2), __float_as_uint(c2));
+                    const uint64_t nmnm = pack_b64(__float_as_uint(neg_mc), __float_as_uint(neg_mc));
+                    uint64_t acc[2] = {0ull, 0ull};
 #pragma unroll
-                for (int g = 0; g < BN / 32; ++g) {
-                    uint32_t packed[16];
-#pragma unroll
-                    for (int c = 0; c < 32; c += 2) {
-                        const float x0 = fmaf(__uint_as_float(s[g * 32 + c]), c2, neg_mc);
-                        const float x1 = fmaf(__uint_as_float(s[g * 32 + c + 1]), c2, neg_mc);
-                        // a fixed share of the exponentials runs on the FMA pipe instead of the SFU
-                        float p0 = ((c & 7) < FUSED_POLY_PER8) ? ex2_poly(x0) : ex2_approx(x0);
-                        float p1 = (((c + 1) & 7) < FUSED_POLY_PER8) ? ex2_poly(x1) : ex2_approx(x1);
-                        if (valid < BN) {   // zero-filled key rows carry no weight (also when scale == 0)
-                            if (g * 32 + c >= valid) p0 = 0.f;
-                            if (g * 32 + c + 1 >= valid) p1 = 0.f;
-                        }
-                        sum[(c >> 1) & 3] += p0 + p1;
-                        packed[c >> 1] = pack_half2(p0, p1);
+                    for (int g = 0; g < BN / 32; ++g) {
+                        uint32_t packed[16];
+                        exp2_pack_32<FUSED_POLY_PER8>(&s[g * 32], c2c2, nmnm, packed, acc);
+                        tmem_st16(tmem_p + g * 16, packed);
                     }
-                    tmem_st16(tmem_p + g * 16, packed);
+                    l_run += sum_f32x2(acc[0], acc[1]);
+                } else {
+                    float sum = 0.f;
+#pragma unroll
+                    for (int g = 0; g < BN / 32; ++g) {
+                        uint32_t packed[16];
+                        exp2_pack_32_masked(&s[g * 32], c2, neg_mc, g * 32, valid, packed, sum);
+                        tmem_st16(tmem_p + g * 16, packed);
+                    }
+                    l_run += sum;
                 }
-                l_run += (sum[0] + sum[1]) + (sum[2] + sum[3]);
-                if (take_turns && lane == 0) mbar_arrive(b_other_turn);
                 if (tracer) FUSED_TRACE(t, j, 4);
                 tmem_wait_st();
                 tc_fence_before_sync();

@@ -24,7 +24,19 @@ typedef CUresult (*encode_tiled_fn)(CUtensorMap*, CUtensorMapDataType, cuuint32_
                                     const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
                                     CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
 
+// A tensor map depends only on (base address, shape, tile rows): encoding costs a few microseconds on
+// the host, so the handle remembers the most recent ones.  Entries own nothing and are never dereferenced
+// on the host; a stale entry is harmless because the key includes everything the encoding reads.
+struct TmapCacheEntry {
+    const void* base;
+    int BH, N, d, box_rows;
+    CUtensorMap map;
+};
+constexpr int TMAP_CACHE_ENTRIES = 128;
+
 struct sd_attn_handle {
+    TmapCacheEntry tmap_cache[TMAP_CACHE_ENTRIES];
+    int tmap_cache_next;
     int device;
     int mode;
     int last_mode;
@@ -100,9 +112,8 @@ extern "C" int sd_attn_create(sd_attn_handle** out) {
 
     // dynamic shared memory ceilings of every kernel, once
     e = raise_smem_limit(cross_attention_kernel, cross_smem_bytes(3, 128));
-    if (e == cudaSuccess) e = raise_smem_limit(fused_attention_kernel<128, true>, fused_smem_bytes_max());
-    if (e == cudaSuccess) e = raise_smem_limit(fused_attention_kernel<128, false>, fused_smem_bytes_max());
-    if (e == cudaSuccess) e = raise_smem_limit(fused_attention_kernel<64, true>, fused_smem_bytes_max());
+    if (e == cudaSuccess) e = raise_smem_limit(fused_attention_kernel<128>, fused_smem_bytes_max());
+    if (e == cudaSuccess) e = raise_smem_limit(fused_attention_kernel<64>, fused_smem_bytes_max());
     if (e == cudaSuccess) e = raise_smem_limit(fused4_attention_kernel, fused4_smem_bytes());
     if (e == cudaSuccess) e = raise_smem_limit(twopass_scores_kernel, twopass_scores_smem_bytes(3));
     if (e == cudaSuccess) e = raise_smem_limit(twopass_pv_kernel, twopass_pv_smem_bytes(3));
@@ -188,6 +199,13 @@ extern "C" int sd_attn_query_status(sd_attn_handle* h, void* stream, int* detail
 // A [BH][N][d] fp16 tensor seen by the TMA as (x = d, y = N, z = BH); tiles are 64 columns wide
 // (one 128-byte swizzled row) by `box_rows` rows.  Columns >= d and rows >= N read as zero.
 static int make_tmap(sd_attn_handle* h, CUtensorMap* map, const void* base, int BH, int N, int d, int box_rows) {
+    for (int i = 0; i < TMAP_CACHE_ENTRIES; ++i) {
+        const TmapCacheEntry& e = h->tmap_cache[i];
+        if (e.base == base && e.BH == BH && e.N == N && e.d == d && e.box_rows == box_rows) {
+            *map = e.map;
+            return SD_ATTN_OK;
+        }
+    }
     cuuint64_t dims[3] = {(cuuint64_t)d, (cuuint64_t)N, (cuuint64_t)BH};
     cuuint64_t strides[2] = {(cuuint64_t)d * 2, (cuuint64_t)N * d * 2};
     cuuint32_t box[3] = {(cuuint32_t)CHUNK_COLS, (cuuint32_t)box_rows, 1};
@@ -200,6 +218,10 @@ static int make_tmap(sd_attn_handle* h, CUtensorMap* map, const void* base, int 
         h->last_cuda_error = cudaErrorInvalidValue;
         return SD_ATTN_ERR_CUDA;
     }
+    TmapCacheEntry& slot = h->tmap_cache[h->tmap_cache_next];
+    h->tmap_cache_next = (h->tmap_cache_next + 1) % TMAP_CACHE_ENTRIES;
+    slot.base = base; slot.BH = BH; slot.N = N; slot.d = d; slot.box_rows = box_rows;
+    slot.map = *map;
     return SD_ATTN_OK;
 }
 
@@ -300,12 +322,10 @@ static int launch_fused(sd_attn_handle* h, const Problem& p) {
     if (rc == SD_ATTN_OK) rc = make_tmap(h, &tv, p.v, p.BH, p.Nk, p.d, bn);
     if (rc != SD_ATTN_OK) return rc;
     dim3 grid((p.Nq + 2 * TILE_M - 1) / (2 * TILE_M), p.BH), block(FUSED_THREADS);
-    if (bn == 128 && fused_split_p(p.d))
-        fused_attention_kernel<128, true><<<grid, block, fused_smem_bytes(a), p.stream>>>(tq, tk, tv, a);
-    else if (bn == 128)
-        fused_attention_kernel<128, false><<<grid, block, fused_smem_bytes(a), p.stream>>>(tq, tk, tv, a);
+    if (bn == 128)
+        fused_attention_kernel<128><<<grid, block, fused_smem_bytes(a), p.stream>>>(tq, tk, tv, a);
     else
-        fused_attention_kernel<64, true><<<grid, block, fused_smem_bytes(a), p.stream>>>(tq, tk, tv, a);
+        fused_attention_kernel<64><<<grid, block, fused_smem_bytes(a), p.stream>>>(tq, tk, tv, a);
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) return cuda_fail(h, e);
     h->launches += 1;

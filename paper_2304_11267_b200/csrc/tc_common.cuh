@@ -85,11 +85,14 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
 // waiter polls it so that one expired wait releases the whole block.  Returns false on abort.
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag,
                                           int* status, int site, int tile) {
+    // try_wait itself suspends the thread for a hardware-chosen slice, so the first polls add no
+    // sleep: a sleeping poller would see a completed phase up to a sleep period late, and that
+    // delay sits on the MMA-issue round trip of the fused kernels.
     for (uint32_t i = 0; i < WAIT_POLL_LIMIT; ++i) {
         if (mbar_try_wait(bar, parity)) return true;
-        if (i > 16) {
+        if ((i & 63) == 63) {
             if (*abort_flag) return false;
-            __nanosleep(i > 1024 ? 128 : 32);
+            if (i > (1u << 14)) __nanosleep(256);
         }
     }
     *abort_flag = 1;
