@@ -1,0 +1,354 @@
+// Persistent cross-attention kernel for the text-conditioning shape of the UNet: 65..80 keys (the 77
+// text tokens), any head dim up to 160.  Memory-bound: per tile of 128 query rows it reads Q and writes O
+// once; K and V (12-50 KB per head) stay in L2.
+//
+// cross_kernel.cuh runs one tile per CTA, start to finish, and leans on CTA-level overlap; its launch,
+// tensor-memory allocation, descriptor fetch and drain are paid per tile and HBM sits idle meanwhile.
+// Here ONE CTA per SM walks a contiguous range of (head, tile) items with every stage overlapped:
+//   warps 0 .. 4*NWG-1   NWG softmax groups; group w owns items w, w+NWG, ... (thread = query row):
+//                        row max, exp2, row sum, weights back to tensor memory, later O / sum -> global
+//   next warp            TMA producer: the Q tile of item i into ring stage i % NS (several in flight); K and V
+//                        of a head once per head, double-buffered.  (The copy engine spends about 7 clocks per
+//                        80-byte row of a d = 40 tensor, measured, so fetching K and V per item -- 160 more rows --
+//                        would make it the bound.  A single warp of 128-bit cp.async copies for Q measured slower.)
+//   two more warps       MMA issuers: one thread issues S_w = Q K^T as soon as a stage lands, another O_w = P_w V
+//                        when the weights are ready
+// Tensor memory: per group S_w (80 columns; the packed fp16 weights overwrite the first 40) and O_w
+// (dpad columns), so NWG = 512 / (80 + dpad) capped at 4: four groups at d = 40, three at 80, two at 160.
+// No running rescale is needed: all keys of a row are in the tile, so L and S of Eq. 4 are exact.
+#pragma once
+#include <cuda.h>
+
+#include "cross_kernel.cuh"  // TILE_M, CHUNK_COLS, CHUNK_ROW_BYTES
+#include "softmax_math.cuh"
+#include "tc_common.cuh"
+
+namespace sd_attn {
+
+constexpr int X2_KN = 80;            // keys rounded up to the MMA N granule; the kernel serves 65..80 keys
+constexpr int X2_MAX_STAGES = 8;
+constexpr int X2_MAX_KSTEPS = 10;
+constexpr int X2_SMEM_BUDGET = 216 * 1024;
+constexpr int X2_SOFTMAX_REGS = 112;  // four-group variant, after setmaxnreg: 512 * 112 + 128 * 32 = 61440 = 640 * 96
+constexpr int X2_CONTROL_REGS = 32;
+
+struct Cross2Args {
+    __half* out;        // [BH][Nq][d]
+    int Nq, Nk, d;
+    int dpad, nch;
+    int stages;         // depth of the Q ring
+    int tiles_per_bh;   // ceil(Nq / 128)
+    int n_items;        // BH * tiles_per_bh
+    float scale_log2e;
+    int negate;
+    int* status;
+#ifdef SD_ATTN_TRACE
+    long long* trace;   // timeline probe of block 0: [role][item < 40][8 slots] clock64 stamps
+#endif
+};
+
+#ifdef SD_ATTN_TRACE
+#define X2_TRACE(role, i, slot)                                                      \
+    do {                                                                             \
+        if (args.trace && blockIdx.x == 0 && (i) < 40)                               \
+            args.trace[((role) * 40 + (i)) * 8 + (slot)] = clock64();                \
+    } while (0)
+#else
+#define X2_TRACE(role, i, slot) do { } while (0)
+#endif
+
+__host__ inline int cross2_groups(int d) {
+    const int g = 512 / (X2_KN + (d + 15) / 16 * 16);
+    return g > 4 ? 4 : g;
+}
+__host__ inline int cross2_threads(int groups) { return groups * 128 + 128; }   // + one control warpgroup
+__host__ inline int cross2_q_bytes(int nch) { return nch * TILE_M * CHUNK_ROW_BYTES; }
+__host__ inline int cross2_kv_bytes(int nch) { return nch * X2_KN * CHUNK_ROW_BYTES; }
+// shared memory: [2 head buffers][K | V] then the Q ring
+__host__ inline int cross2_stages(int nch) {
+    int s = (X2_SMEM_BUDGET - 4 * cross2_kv_bytes(nch)) / cross2_q_bytes(nch);
+    return s > X2_MAX_STAGES ? X2_MAX_STAGES : s;
+}
+__host__ inline size_t cross2_smem_bytes(int nch) {
+    return (size_t)4 * cross2_kv_bytes(nch) + (size_t)cross2_stages(nch) * cross2_q_bytes(nch) + 1024;
+}
+__host__ inline bool cross2_supports(int Nk, int d) { return Nk > 64 && Nk <= X2_KN && d % 8 == 0 && d <= 160; }
+
+enum {
+    SITE_Y_STAGE = 40, SITE_Y_EMPTY = 41, SITE_Y_S = 42, SITE_Y_P = 43, SITE_Y_O = 44, SITE_Y_OFREE = 45,
+    SITE_Y_KV = 46, SITE_Y_KVEMPTY = 47, SITE_Y_PV = 48
+};
+
+// S = Q K^T over KS contraction steps of 16 columns, offsets folded at compile time.
+template <int KS>
+__device__ __forceinline__ void issue_qk(uint32_t tmem_s, uint64_t q_desc, uint64_t k_desc, uint32_t idesc) {
+#pragma unroll
+    for (int kk = 0; kk < KS; ++kk)
+        mma_f16_ss(tmem_s, q_desc + (uint64_t)(((kk >> 2) * TILE_M * CHUNK_ROW_BYTES + (kk & 3) * 32) >> 4),
+                   k_desc + (uint64_t)(((kk >> 2) * X2_KN * CHUNK_ROW_BYTES + (kk & 3) * 32) >> 4), idesc, kk > 0);
+}
+
+template <int NWG>
+__global__ void __launch_bounds__(NWG * 128 + 128, 1)
+cross2_attention_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__ CUtensorMap tmap_k,
+                        const __grid_constant__ CUtensorMap tmap_v, const Cross2Args args) {
+    extern __shared__ uint8_t x2_smem_raw[];
+    __shared__ __align__(8) uint64_t bar_full[X2_MAX_STAGES], bar_empty[X2_MAX_STAGES];
+    __shared__ __align__(8) uint64_t bar_kv_full[2], bar_kv_empty[2];
+    __shared__ __align__(8) uint64_t bar_s_full[NWG], bar_p_full[NWG], bar_o_full[NWG], bar_o_free[NWG], bar_pv_done[NWG];
+    __shared__ uint32_t tmem_base_slot;
+    __shared__ int abort_flag;
+
+    constexpr int LOADER_WARP = NWG * 4, S_ISSUER_WARP = NWG * 4 + 1, O_ISSUER_WARP = NWG * 4 + 2;
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int nch = args.nch, dpad = args.dpad, stages = args.stages;
+    // contiguous range of items for this CTA: consecutive items share a head, so K and V are fetched rarely
+    const int per = args.n_items / gridDim.x, extra = args.n_items % gridDim.x;
+    const int item0 = blockIdx.x * per + min((int)blockIdx.x, extra);
+    const int n_local = per + ((int)blockIdx.x < extra ? 1 : 0);
+    const int bh0 = item0 / args.tiles_per_bh;   // head of the first item; head "group" g = bh - bh0
+
+    const uint32_t smem_base = (smem_u32(x2_smem_raw) + 1023u) & ~1023u;
+    const uint32_t q_bytes = nch * TILE_M * CHUNK_ROW_BYTES, kv_bytes = nch * X2_KN * CHUNK_ROW_BYTES;
+    const uint32_t kv_smem = smem_base;                    // [2][K | V]
+    const uint32_t q_smem = smem_base + 4 * kv_bytes;      // [stages][nch][128 rows][128 B]
+    volatile int* abort_p = &abort_flag;
+
+    if (tid == 0) {
+        abort_flag = 0;
+        for (int s = 0; s < X2_MAX_STAGES; ++s) {
+            mbar_init(smem_u32(&bar_full[s]), 1);
+            mbar_init(smem_u32(&bar_empty[s]), 1);
+        }
+        for (int b = 0; b < 2; ++b) {
+            mbar_init(smem_u32(&bar_kv_full[b]), 1);
+            mbar_init(smem_u32(&bar_kv_empty[b]), 1);
+        }
+        for (int w = 0; w < NWG; ++w) {
+            mbar_init(smem_u32(&bar_s_full[w]), 1);
+            mbar_init(smem_u32(&bar_p_full[w]), 4);   // one arrival per softmax warp
+            mbar_init(smem_u32(&bar_o_full[w]), 1);
+            mbar_init(smem_u32(&bar_o_free[w]), 4);
+            mbar_init(smem_u32(&bar_pv_done[w]), 1);
+        }
+        mbar_init_fence();
+    }
+    if (warp == S_ISSUER_WARP) {
+        tmem_alloc(smem_u32(&tmem_base_slot), 512);
+        tmem_relinquish();
+    }
+    tc_fence_before_sync();
+    __syncthreads();
+    tc_fence_after_sync();
+    const uint32_t tmem_base = tmem_base_slot;
+    const uint32_t tmem_o0 = tmem_base + NWG * X2_KN;   // columns: S_0 .. S_{NWG-1} | O_0 .. O_{NWG-1}
+
+    // With four softmax groups the register file is the limit (a row of 80 scores per thread): the control
+    // warpgroup (producer, two issuers, one idle warp) hands registers over.  All four warps of a warpgroup
+    // must execute the SAME setmaxnreg instruction, hence one site per kind.
+    // setmaxnreg only moves registers INSIDE the CTA's launch allocation (threads x registers per thread as
+    // compiled): an increase that the decreases do not cover blocks for ever.  The host checks, from the
+    // compiled register count, that 512 * X2_SOFTMAX_REGS + 128 * X2_CONTROL_REGS fits before using this variant.
+    constexpr bool REBALANCE = NWG == 4;
+    if (REBALANCE && warp >= NWG * 4) setmaxnreg_dec<X2_CONTROL_REGS>();
+    if (warp == LOADER_WARP) {
+        // ------------------------------------------------------------ TMA producer
+        if (elect_one()) {
+            tma_prefetch_desc(&tmap_q);
+            tma_prefetch_desc(&tmap_k);
+            tma_prefetch_desc(&tmap_v);
+            int g_prev = -1;
+            for (int i = 0; i < n_local; ++i) {
+                const int item = item0 + i, bh = item / args.tiles_per_bh, tile = item - bh * args.tiles_per_bh;
+                const int s = i % stages, g = bh - bh0;
+                if (g != g_prev) {
+                    // a new head: its K and V go into buffer g & 1 once the head two back has been consumed
+                    if (g >= 2 && !mbar_wait(smem_u32(&bar_kv_empty[g & 1]), ((g >> 1) - 1) & 1, abort_p, args.status,
+                                             SITE_Y_KVEMPTY, i))
+                        break;
+                    const uint32_t bar = smem_u32(&bar_kv_full[g & 1]), dst = kv_smem + (g & 1) * 2 * kv_bytes;
+                    mbar_arrive_expect_tx(bar, 2 * kv_bytes);
+                    for (int ch = 0; ch < nch; ++ch)
+                        tma_load_3d(dst + ch * X2_KN * CHUNK_ROW_BYTES, &tmap_k, bar, ch * CHUNK_COLS, 0, bh);
+                    for (int ch = 0; ch < nch; ++ch)
+                        tma_load_3d(dst + kv_bytes + ch * X2_KN * CHUNK_ROW_BYTES, &tmap_v, bar, ch * CHUNK_COLS, 0, bh);
+                    g_prev = g;
+                }
+                if (i >= stages &&
+                    !mbar_wait(smem_u32(&bar_empty[s]), ((i / stages) - 1) & 1, abort_p, args.status, SITE_Y_EMPTY, i))
+                    break;
+                X2_TRACE(NWG + 1, i, 0);
+                const uint32_t bar = smem_u32(&bar_full[s]), dst = q_smem + s * q_bytes;
+                mbar_arrive_expect_tx(bar, q_bytes);
+                for (int ch = 0; ch < nch; ++ch)
+                    tma_load_3d(dst + ch * TILE_M * CHUNK_ROW_BYTES, &tmap_q, bar, ch * CHUNK_COLS, tile * TILE_M, bh);
+            }
+        }
+    } else if (warp == S_ISSUER_WARP || warp == O_ISSUER_WARP) {
+        // ------------------------------------------------------------ MMA issuers
+        // An issuer is one thread sharing a scheduler with busy softmax warps: each barrier test and each
+        // tcgen05.mma costs it tens to hundreds of clocks, and a single thread doing both products of every
+        // item became the bound of the kernel.  So two threads split the work: one issues S = Q K^T (and
+        // frees Q stages), the other O = P V (and frees K/V buffers).  S of item i+NWG reuses the columns
+        // of S/P of item i, so the S issuer waits for that item's P V product to COMPLETE (bar_pv_done).
+        if (elect_one()) {
+            struct Cursor { int i, s, sph, w, n, g, t; };
+            const int t_first = item0 - bh0 * args.tiles_per_bh;
+            auto advance = [&](Cursor& c) {   // item bookkeeping without divisions
+                ++c.i;
+                if (++c.s == stages) { c.s = 0; c.sph ^= 1; }
+                if (++c.w == NWG) { c.w = 0; ++c.n; }
+                if (++c.t == args.tiles_per_bh) { c.t = 0; ++c.g; }
+            };
+            Cursor c = {0, 0, 0, 0, 0, 0, t_first};
+            bool ok = true;
+            if (warp == S_ISSUER_WARP) {
+                const uint32_t idesc_s = idesc_f16(TILE_M, X2_KN, false, false, args.negate != 0);
+                const int ksteps_s = (args.d + 15) / 16;
+                const uint64_t q_desc0 = smem_desc_sw128(q_smem, 16, 1024);
+                const uint64_t k_desc0 = smem_desc_sw128(kv_smem, 16, 1024);
+                const uint32_t q_stage_off = q_bytes >> 4, kv_buf_off = (2 * kv_bytes) >> 4;
+                for (; c.i < n_local && ok; advance(c)) {
+                    ok = mbar_wait(smem_u32(&bar_full[c.s]), c.sph, abort_p, args.status, SITE_Y_STAGE, c.i) &&
+                         mbar_wait(smem_u32(&bar_kv_full[c.g & 1]), (c.g >> 1) & 1, abort_p, args.status, SITE_Y_KV, c.i);
+                    if (ok && c.n >= 1)   // the group's previous item no longer needs these columns
+                        ok = mbar_wait(smem_u32(&bar_pv_done[c.w]), (c.n - 1) & 1, abort_p, args.status, SITE_Y_PV, c.i);
+                    if (!ok) break;
+                    tc_fence_after_sync();
+                    X2_TRACE(NWG, c.i, 3);
+                    const uint64_t qd = q_desc0 + (uint64_t)(c.s * q_stage_off);
+                    const uint64_t kd = k_desc0 + (uint64_t)((c.g & 1) * kv_buf_off);
+                    const uint32_t ts = tmem_base + c.w * X2_KN;
+                    if (ksteps_s == 3) issue_qk<3>(ts, qd, kd, idesc_s);
+                    else if (ksteps_s == 5) issue_qk<5>(ts, qd, kd, idesc_s);
+                    else if (ksteps_s == 10) issue_qk<10>(ts, qd, kd, idesc_s);
+                    else
+                        for (int kk = 0; kk < ksteps_s; ++kk)
+                            mma_f16_ss(ts, qd + (uint64_t)(((kk >> 2) * TILE_M * CHUNK_ROW_BYTES + (kk & 3) * 32) >> 4),
+                                       kd + (uint64_t)(((kk >> 2) * X2_KN * CHUNK_ROW_BYTES + (kk & 3) * 32) >> 4), idesc_s,
+                                       kk > 0);
+                    tc_commit(smem_u32(&bar_s_full[c.w]));
+                    tc_commit(smem_u32(&bar_empty[c.s]));   // the Q stage is free once this product has read it
+                    X2_TRACE(NWG, c.i, 4);
+                }
+            } else {
+                const uint32_t idesc_o = idesc_f16(TILE_M, dpad, false, true, false);
+                const uint64_t v_desc0 = smem_desc_sw128(kv_smem + kv_bytes, X2_KN * CHUNK_ROW_BYTES, 1024);
+                const uint32_t kv_buf_off = (2 * kv_bytes) >> 4;
+                for (; c.i < n_local && ok; advance(c)) {
+                    if (c.n >= 1)   // O_w of the group's previous item must have been read out
+                        ok = mbar_wait(smem_u32(&bar_o_free[c.w]), (c.n - 1) & 1, abort_p, args.status, SITE_Y_OFREE, c.i);
+                    X2_TRACE(NWG, c.i, 0);
+                    if (ok) ok = mbar_wait(smem_u32(&bar_p_full[c.w]), c.n & 1, abort_p, args.status, SITE_Y_P, c.i);
+                    if (!ok) break;
+                    tc_fence_after_sync();
+                    X2_TRACE(NWG, c.i, 1);
+                    const uint64_t vd = v_desc0 + (uint64_t)((c.g & 1) * kv_buf_off);
+#pragma unroll
+                    for (int kk = 0; kk < X2_KN / 16; ++kk)   // O_w = P_w V, P_w in the first columns of S_w
+                        mma_f16_ts(tmem_o0 + c.w * dpad, tmem_base + c.w * X2_KN + kk * 8,
+                                   vd + (uint64_t)(kk * ((16 * CHUNK_ROW_BYTES) >> 4)), idesc_o, kk > 0);
+                    tc_commit(smem_u32(&bar_o_full[c.w]));
+                    tc_commit(smem_u32(&bar_pv_done[c.w]));
+                    // last item of its head: every S product of this head completed before its softmax ran
+                    if (c.i + 1 == n_local || c.t + 1 == args.tiles_per_bh) tc_commit(smem_u32(&bar_kv_empty[c.g & 1]));
+                    X2_TRACE(NWG, c.i, 2);
+                }
+            }
+        }
+    } else if (warp < NWG * 4) {
+        // ------------------------------------------------------------ softmax + epilogue warps
+        if (REBALANCE) setmaxnreg_inc<X2_SOFTMAX_REGS>();
+        const int w = warp >> 2;
+        const int r = tid & (TILE_M - 1);
+        const uint32_t lane_off = (uint32_t)((warp & 3) * 32) << 16;
+        const uint32_t tmem_s = tmem_base + w * X2_KN + lane_off;
+        const uint32_t tmem_o = tmem_o0 + w * dpad + lane_off;
+        const float c2 = args.scale_log2e;
+        const int valid = args.Nk;
+        bool ok = true;
+        const bool tracer = (warp & 3) == 0 && lane == 0;
+        for (int i = w; i < n_local; i += NWG) {
+            const int n = i / NWG;
+            if (tracer) X2_TRACE(w, i, 0);
+            ok = mbar_wait(smem_u32(&bar_s_full[w]), n & 1, abort_p, args.status, SITE_Y_S, i);
+            ok = __all_sync(0xffffffffu, ok);
+            if (!ok) break;
+            tc_fence_after_sync();
+            if (tracer) X2_TRACE(w, i, 1);
+            float row_sum;
+            {
+                uint32_t s[X2_KN];
+                tmem_ld32(tmem_s, &s[0]);
+                tmem_ld32(tmem_s + 32, &s[32]);
+                tmem_ld16(tmem_s + 64, *reinterpret_cast<uint32_t(*)[16]>(&s[64]));
+                tmem_wait_ld();
+                // L_i of Eq. 4 (to bf16 precision: it only anchors the exponent) over the valid keys
+                const float row_max = fmaxf(row_max_bf16<64>(s), row_max_masked<16>(&s[64], valid - 64));
+                const float neg_mc = -row_max * c2;
+                const uint64_t c2c2 = pack_b64(__float_as_uint(c2), __float_as_uint(c2));
+                const uint64_t nmnm = pack_b64(__float_as_uint(neg_mc), __float_as_uint(neg_mc));
+                uint64_t acc[2] = {0ull, 0ull};
+                uint32_t packed[16];
+                exp2_pack_32<0>(&s[0], c2c2, nmnm, packed, acc);
+                tmem_st16(tmem_s, packed);
+                exp2_pack_32<0>(&s[32], c2c2, nmnm, packed, acc);
+                tmem_st16(tmem_s + 16, packed);
+                float tail = 0.f;
+                exp2_pack_32_masked<8>(&s[64], c2, neg_mc, 64, valid, packed, tail);
+                tmem_st8(tmem_s + 32, *reinterpret_cast<uint32_t(*)[8]>(&packed[0]));
+                row_sum = sum_f32x2(acc[0], acc[1]) + tail;   // S_i of Eq. 4
+            }
+            tmem_wait_st();
+            tc_fence_before_sync();
+            if (lane == 0) mbar_arrive(smem_u32(&bar_p_full[w]));
+            if (tracer) X2_TRACE(w, i, 2);
+
+            ok = mbar_wait(smem_u32(&bar_o_full[w]), n & 1, abort_p, args.status, SITE_Y_O, i);
+            ok = __all_sync(0xffffffffu, ok);
+            if (!ok) break;
+            tc_fence_after_sync();
+            if (tracer) X2_TRACE(w, i, 3);
+            const int item = item0 + i, bh = item / args.tiles_per_bh, tile = item - bh * args.tiles_per_bh;
+            const int row = tile * TILE_M + r;
+            const float inv = 1.f / row_sum;
+            __half* orow = args.out + ((size_t)bh * args.Nq + row) * args.d;
+            // O / S_i -> fp16 -> global, 32 columns per tensor-memory round trip (dpad is a multiple of 16)
+            for (int c0 = 0; c0 < dpad; c0 += 32) {
+                uint32_t x[32];
+                tmem_ld16(tmem_o + c0, *reinterpret_cast<uint32_t(*)[16]>(&x[0]));
+                if (c0 + 16 < dpad) tmem_ld16(tmem_o + c0 + 16, *reinterpret_cast<uint32_t(*)[16]>(&x[16]));
+                tmem_wait_ld();
+                if (row < args.Nq) {
+#pragma unroll
+                    for (int g = 0; g < 4; ++g) {
+                        uint4 v8;
+                        v8.x = pack_half2(__uint_as_float(x[g * 8 + 0]) * inv, __uint_as_float(x[g * 8 + 1]) * inv);
+                        v8.y = pack_half2(__uint_as_float(x[g * 8 + 2]) * inv, __uint_as_float(x[g * 8 + 3]) * inv);
+                        v8.z = pack_half2(__uint_as_float(x[g * 8 + 4]) * inv, __uint_as_float(x[g * 8 + 5]) * inv);
+                        v8.w = pack_half2(__uint_as_float(x[g * 8 + 6]) * inv, __uint_as_float(x[g * 8 + 7]) * inv);
+                        if (c0 + g * 8 + 8 <= args.d) *reinterpret_cast<uint4*>(orow + c0 + g * 8) = v8;
+                    }
+                }
+            }
+            tc_fence_before_sync();
+            if (lane == 0) mbar_arrive(smem_u32(&bar_o_free[w]));
+            if (tracer) X2_TRACE(w, i, 4);
+        }
+    }
+
+    // ------------------------------------------------------------ teardown (every thread arrives)
+    tc_fence_before_sync();
+    __syncthreads();
+    if (warp == LOADER_WARP && lane == 0 && abort_flag) {
+        mbar_drain(smem_u32(&bar_kv_full[0]), 0);   // gave up: let a K/V fetch still in flight land
+        mbar_drain(smem_u32(&bar_kv_full[1]), 0);
+    }
+    __syncthreads();
+    if (warp == S_ISSUER_WARP) {
+        __syncwarp();
+        tmem_dealloc(tmem_base, 512);
+    }
+}
+
+}  // namespace sd_attn

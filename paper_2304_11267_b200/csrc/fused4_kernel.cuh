@@ -103,6 +103,8 @@ fused4_attention_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid
     const uint32_t tmem_o0 = tmem_base + F4_TILES * BN;   // columns: S_0..S_3 | O_0..O_3
 
     // All four warps of a warpgroup must execute the SAME setmaxnreg instruction: one site per kind.
+    // setmaxnreg only moves registers INSIDE the CTA's launch allocation (768 threads x registers per thread as
+    // compiled): an increase the decreases do not cover blocks for ever, so the host checks the compiled count.
     if (warp >= 16) setmaxnreg_dec<F4_CONTROL_REGS>();
     if (warp == 16) {
         // ------------------------------------------------------------ TMA producer

@@ -13,6 +13,7 @@
 #include "../../include/sd_attn.h"
 #include "../../include/sd_attn_debug.h"
 #include "cross_kernel.cuh"
+#include "cross2_kernel.cuh"
 #include "fused_kernel.cuh"
 #include "fused4_kernel.cuh"
 #include "simt_kernel.cuh"
@@ -47,9 +48,13 @@ struct sd_attn_handle {
     const float* tp_scores;   // where the last TWOPASS call put A and [L,S]
     const float* tp_stats;
     float* dump_scores;       // bring-up hook of the cross kernel (see sd_attn_debug.h)
+    void* trace;              // SD_ATTN_TRACE builds only: clock-stamp buffer (the address comes from SD_ATTN_TRACE_PTR)
     encode_tiled_fn encode_tiled;
     cudaError_t last_cuda_error;
     int sm_count;
+    int fused4_ok;            // the register hand-over inside these kernels fits their launch allocation
+    int cross2_four_ok;
+    int cross_one_tile_only;  // SD_ATTN_CROSS_ONE_TILE=1: never use the persistent cross-attention kernel
     int prefer_two_tile;      // SD_ATTN_FUSED_TWO_TILE=1: use the two-tile fused kernel for every head dim
 };
 
@@ -107,11 +112,20 @@ extern "C" int sd_attn_create(sd_attn_handle** out) {
         return cuda_fail(nullptr, e != cudaSuccess ? e : cudaErrorUnknown);
     }
     h->encode_tiled = (encode_tiled_fn)fn;
+#ifdef SD_ATTN_TRACE
+    const char* tr = getenv("SD_ATTN_TRACE_PTR");
+    h->trace = tr ? (void*)strtoull(tr, nullptr, 0) : nullptr;
+#endif
+    const char* one = getenv("SD_ATTN_CROSS_ONE_TILE");
+    h->cross_one_tile_only = (one && one[0] == '1') ? 1 : 0;
     const char* two = getenv("SD_ATTN_FUSED_TWO_TILE");
     h->prefer_two_tile = (two && two[0] == '1') ? 1 : 0;
 
     // dynamic shared memory ceilings of every kernel, once
     e = raise_smem_limit(cross_attention_kernel, cross_smem_bytes(3, 128));
+    if (e == cudaSuccess) e = raise_smem_limit(cross2_attention_kernel<2>, X2_SMEM_BUDGET + 1024);
+    if (e == cudaSuccess) e = raise_smem_limit(cross2_attention_kernel<3>, X2_SMEM_BUDGET + 1024);
+    if (e == cudaSuccess) e = raise_smem_limit(cross2_attention_kernel<4>, X2_SMEM_BUDGET + 1024);
     if (e == cudaSuccess) e = raise_smem_limit(fused_attention_kernel<128>, fused_smem_bytes_max());
     if (e == cudaSuccess) e = raise_smem_limit(fused_attention_kernel<64>, fused_smem_bytes_max());
     if (e == cudaSuccess) e = raise_smem_limit(fused4_attention_kernel, fused4_smem_bytes());
@@ -121,6 +135,16 @@ extern "C" int sd_attn_create(sd_attn_handle** out) {
     if (e == cudaSuccess) e = raise_smem_limit(simt_attention_kernel<__half, 5>, simt_smem_bytes(160));
     if (e == cudaSuccess) e = raise_smem_limit(simt_attention_kernel<float, 4>, simt_smem_bytes(128));
     if (e == cudaSuccess) e = raise_smem_limit(simt_attention_kernel<__half, 4>, simt_smem_bytes(128));
+    // setmaxnreg budgets (see the kernels): only use a variant whose increases are covered by its decreases
+    if (e == cudaSuccess) {
+        cudaFuncAttributes fa;
+        e = cudaFuncGetAttributes(&fa, fused4_attention_kernel);
+        if (e == cudaSuccess)
+            h->fused4_ok = F4_THREADS * fa.numRegs >= 512 * F4_SOFTMAX_REGS + 256 * F4_CONTROL_REGS;
+        if (e == cudaSuccess) e = cudaFuncGetAttributes(&fa, cross2_attention_kernel<4>);
+        if (e == cudaSuccess)
+            h->cross2_four_ok = cross2_threads(4) * fa.numRegs >= 512 * X2_SOFTMAX_REGS + 128 * X2_CONTROL_REGS;
+    }
     if (e == cudaSuccess) e = cudaMalloc((void**)&h->dev_status, sizeof(int) * DEV_STATUS_INTS);
     if (e == cudaSuccess) e = cudaMemset(h->dev_status, 0, sizeof(int) * DEV_STATUS_INTS);
     if (e != cudaSuccess) {
@@ -258,7 +282,45 @@ static int launch_simt(sd_attn_handle* h, const Problem& p) {
     return SD_ATTN_OK;
 }
 
+// 65..80 keys (the 77 text tokens): one persistent CTA per SM walks a range of (head, tile) items
+static int launch_cross2(sd_attn_handle* h, const Problem& p) {
+    Cross2Args a;
+    a.out = (__half*)p.out;
+    a.Nq = p.Nq; a.Nk = p.Nk; a.d = p.d;
+    a.dpad = (p.d + 15) / 16 * 16;
+    a.nch = (p.d + CHUNK_COLS - 1) / CHUNK_COLS;
+    a.stages = cross2_stages(a.nch);
+    a.tiles_per_bh = (p.Nq + TILE_M - 1) / TILE_M;
+    a.n_items = p.BH * a.tiles_per_bh;
+    a.scale_log2e = fabsf(p.scale) * LOG2E;
+    a.negate = p.scale < 0.f;
+    a.status = h->dev_status;
+#ifdef SD_ATTN_TRACE
+    a.trace = (long long*)h->trace;
+#endif
+    CUtensorMap tq, tk, tv;
+    int rc = make_tmap(h, &tq, p.q, p.BH, p.Nq, p.d, TILE_M);
+    if (rc == SD_ATTN_OK) rc = make_tmap(h, &tk, p.k, p.BH, p.Nk, p.d, X2_KN);
+    if (rc == SD_ATTN_OK) rc = make_tmap(h, &tv, p.v, p.BH, p.Nk, p.d, X2_KN);
+    if (rc != SD_ATTN_OK) return rc;
+    const int grid = a.n_items < h->sm_count ? a.n_items : h->sm_count;
+    int groups = cross2_groups(p.d);
+    if (groups >= 4 && !h->cross2_four_ok) groups = 3;
+    const size_t smem = cross2_smem_bytes(a.nch);
+    if (groups >= 4)
+        cross2_attention_kernel<4><<<grid, cross2_threads(4), smem, p.stream>>>(tq, tk, tv, a);
+    else if (groups == 3)
+        cross2_attention_kernel<3><<<grid, cross2_threads(3), smem, p.stream>>>(tq, tk, tv, a);
+    else
+        cross2_attention_kernel<2><<<grid, cross2_threads(2), smem, p.stream>>>(tq, tk, tv, a);
+    cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess) return cuda_fail(h, e);
+    h->launches += 1;
+    return SD_ATTN_OK;
+}
+
 static int launch_cross(sd_attn_handle* h, const Problem& p) {
+    if (cross2_supports(p.Nk, p.d) && !h->cross_one_tile_only && !h->dump_scores) return launch_cross2(h, p);
     CrossArgs a;
     a.out = (__half*)p.out;
     a.Nq = p.Nq; a.Nk = p.Nk; a.d = p.d;
@@ -293,7 +355,7 @@ static int launch_fused4(sd_attn_handle* h, const Problem& p) {
     a.negate = p.scale < 0.f;
     a.status = h->dev_status;
 #ifdef SD_ATTN_TRACE
-    a.trace = (long long*)h->dump_scores;
+    a.trace = (long long*)h->trace;
 #endif
     CUtensorMap tq, tk, tv;
     int rc = make_tmap(h, &tq, p.q, p.BH, p.Nq, p.d, TILE_M);
@@ -309,12 +371,12 @@ static int launch_fused4(sd_attn_handle* h, const Problem& p) {
 }
 
 static int launch_fused(sd_attn_handle* h, const Problem& p) {
-    if (p.d <= F4_MAX_D && !h->prefer_two_tile) return launch_fused4(h, p);
+    if (p.d <= F4_MAX_D && !h->prefer_two_tile && h->fused4_ok) return launch_fused4(h, p);
     FusedArgs a;
     const int bn = fused_block_n(p.d);
     fused_fill_args(&a, (__half*)p.out, p.Nq, p.Nk, p.d, fabsf(p.scale) * LOG2E, p.scale < 0.f, h->dev_status);
 #ifdef SD_ATTN_TRACE
-    a.trace = (long long*)h->dump_scores;   // trace builds reuse the debug pointer as the probe buffer
+    a.trace = (long long*)h->trace;
 #endif
     CUtensorMap tq, tk, tv;
     int rc = make_tmap(h, &tq, p.q, p.BH, p.Nq, p.d, TILE_M);
