@@ -135,6 +135,38 @@ int sd_attn_last_mode(const sd_attn_handle *h);
 /* How many kernels of this library the handle has launched since it was created. */
 long long sd_attn_launch_count(const sd_attn_handle *h);
 
+/*
+ * The two-pass evaluation for callers that cannot allocate device memory.  (The paper has no
+ * counterpart: this entry point exists for deployment, not for the method.)
+ *
+ * Who needs it: code that runs where cudaMalloc is unavailable or forbidden -- inside a host framework
+ * that owns the whole device heap, in a process whose device memory was carved up at start-up, or on a
+ * path where an allocation's implicit device-wide synchronisation is unacceptable.  Such callers can
+ * neither create a handle (sd_attn_create allocates) nor lend a workspace.  Here the scratch of the
+ * two-pass path (the binary32 score matrix and the [L, S] row statistics of Eq. 4) is a fixed array of
+ * SD_ATTN_STATIC_MAX_SCRATCH bytes built into the library image; every GPU that loads the library holds
+ * that array until the process exits, used or not.
+ *
+ * Arguments, layout and result are those of sd_attn_forward in TWOPASS mode with dtype SD_ATTN_F16 (q, k,
+ * v, out are caller-owned DEVICE pointers; no handle).  The call allocates nothing: no cudaMalloc, no
+ * cudaFree, no allocating library routine.
+ *   - A call whose scratch need, sd_attn_workspace_bytes(SD_ATTN_MODE_TWOPASS, ...), exceeds
+ *     SD_ATTN_STATIC_MAX_SCRATCH returns SD_ATTN_ERR_WORKSPACE and enqueues nothing (with SD_ATTN_LOG set
+ *     the two sizes are printed).  F32 data or d % 8 != 0 is SD_ATTN_ERR_UNSUPPORTED.
+ *   - The FIRST call on each device looks up the device address of the built-in array (with that device
+ *     current) and raises the kernels' shared-memory limits; make that first call outside any stream
+ *     capture.  Later calls only enqueue work on `stream`.
+ *   - All calls on a device share the one array, which keeps whatever the previous call left in it; every
+ *     call overwrites what it reads and clears its device status word first, so calls that follow one
+ *     another on a stream are independent.  Calls that OVERLAP on the GPU (different streams, or different
+ *     host threads without ordering) race on the array and produce garbage: serialise them.
+ *   - A bounded wait that expires inside a kernel cannot be reported by this entry point (there is no
+ *     handle to query); use the handle-based API where that matters.
+ */
+#define SD_ATTN_STATIC_MAX_SCRATCH ((size_t)34 * 1024 * 1024)
+int sd_attn_forward_twopass_static(const void *q, const void *k, const void *v, void *out, int B, int H,
+                                   int Nq, int Nk, int d, float scale, int dtype, void *stream);
+
 /* Static, NUL-terminated description of a status code. */
 const char *sd_attn_status_string(int status);
 

@@ -21,11 +21,13 @@ MODE_NAMES = {MODE_AUTO: "auto", MODE_FUSED: "fused", MODE_CROSS: "cross", MODE_
               MODE_SIMT: "simt"}
 CROSS_MAX_NK = 128
 MAX_D = 160
+STATIC_MAX_SCRATCH = 34 * 1024 * 1024   # SD_ATTN_STATIC_MAX_SCRATCH: built-in scratch of the no-allocation entry point
 
 EXPORTS = ["sd_attn_create", "sd_attn_forward", "sd_attn_destroy", "sd_attn_set_mode",
            "sd_attn_workspace_bytes", "sd_attn_set_workspace", "sd_attn_twopass_buffers",
            "sd_attn_query_status", "sd_attn_last_mode", "sd_attn_launch_count", "sd_attn_status_string",
-           "sd_attn_forward_host", "sd_attn_host_staging_bytes", "sd_attn_debug_dump_cross_scores"]
+           "sd_attn_forward_host", "sd_attn_host_staging_bytes", "sd_attn_debug_dump_cross_scores",
+           "sd_attn_forward_twopass_static"]
 
 _lib = None
 
@@ -73,6 +75,8 @@ def load() -> ctypes.CDLL:
     lib.sd_attn_launch_count.argtypes = [vp]
     lib.sd_attn_status_string.restype = ctypes.c_char_p
     lib.sd_attn_status_string.argtypes = [ci]
+    lib.sd_attn_forward_twopass_static.restype = ci
+    lib.sd_attn_forward_twopass_static.argtypes = [vp, vp, vp, vp, ci, ci, ci, ci, ci, cf, ci, vp]
     lib.sd_attn_debug_dump_cross_scores.restype = ci
     lib.sd_attn_debug_dump_cross_scores.argtypes = [vp, vp]
     _lib = lib
@@ -112,6 +116,17 @@ def sd_attn_forward_host(handle, q, k, v, out, staging, staging_bytes, B, H, Nq,
 
 def sd_attn_host_staging_bytes(B, H, Nq, Nk, d, dtype) -> int:
     return int(load().sd_attn_host_staging_bytes(B, H, Nq, Nk, d, dtype))
+
+
+def sd_attn_forward_twopass_static(q, k, v, out, B, H, Nq, Nk, d, scale, dtype, stream=0) -> int:
+    """Two-pass attention on the library's built-in scratch array: no handle, no allocation anywhere.
+
+    For callers that cannot call cudaMalloc (the device heap belongs to someone else).  q, k, v, out are
+    device addresses.  Returns the status code; ERR_WORKSPACE when the call needs more scratch than
+    ``STATIC_MAX_SCRATCH`` bytes.  Calls that overlap on the GPU race on the shared array.
+    """
+    return load().sd_attn_forward_twopass_static(q, k, v, out, B, H, Nq, Nk, d, ctypes.c_float(scale), dtype,
+                                                 stream or None)
 
 
 def sd_attn_set_mode(handle, mode: int) -> int:

@@ -9,6 +9,7 @@
 #include <stdio.h>
 #include <stdlib.h>
 #include <string.h>
+#include <mutex>
 
 #include "../../include/sd_attn.h"
 #include "../../include/sd_attn_debug.h"
@@ -494,4 +495,121 @@ extern "C" int sd_attn_forward_host(sd_attn_handle* h, const void* q, const void
     if (rc != SD_ATTN_OK) return rc;
     e = cudaMemcpyAsync(out, dout, q_bytes, cudaMemcpyDeviceToHost, s);
     return e == cudaSuccess ? SD_ATTN_OK : cuda_fail(h, e);
+}
+
+// ------------------------------------------------------------------------------------------------
+// Two-pass attention for callers that cannot allocate device memory.
+//
+// Some hosts of this library run where cudaMalloc is off limits: inside a framework that owns the whole
+// device heap and forbids side allocations, in a process whose memory was carved up front, or on a
+// latency path where an allocation (an implicit device synchronisation) is not acceptable.  Such a
+// caller cannot create a handle either (sd_attn_create allocates the status block), nor lend a
+// workspace it does not have.  For them the scratch of the two-pass path -- the score matrix A and
+// the [L, S] row statistics -- lives in a fixed array inside the library image.
+//
+// The array is part of every GPU's copy of the module from the moment the library is loaded until the
+// process exits, whether or not this entry point is ever called; hence the modest size.
+constexpr size_t SD_ATTN_STATIC_SCRATCH_BYTES = SD_ATTN_STATIC_MAX_SCRATCH;
+static __device__ __align__(256) unsigned char g_static_scratch[SD_ATTN_STATIC_SCRATCH_BYTES];
+static __device__ __align__(256) int g_static_status[DEV_STATUS_INTS];
+
+// In host code the names above are only host-side handles of the device symbols, not device addresses:
+// the real addresses are looked up once per device (with that device current) and kept here.
+constexpr int STATIC_MAX_DEVICES = 64;
+struct StaticDeviceState {
+    int ready;
+    unsigned char* scratch;
+    int* status;
+    encode_tiled_fn encode_tiled;
+};
+static StaticDeviceState g_static_state[STATIC_MAX_DEVICES];
+static std::mutex g_static_mutex;   // two host threads may make their first call on a device together
+
+static int static_setup(int dev, StaticDeviceState** out) {
+    if (dev < 0 || dev >= STATIC_MAX_DEVICES) return SD_ATTN_ERR_UNSUPPORTED;
+    StaticDeviceState* st = &g_static_state[dev];
+    std::lock_guard<std::mutex> lock(g_static_mutex);
+    if (!st->ready) {
+        int major = 0;
+        cudaError_t e = cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev);
+        if (e != cudaSuccess) return cuda_fail(nullptr, e);
+        if (major != 10) return SD_ATTN_ERR_ARCH;
+        void* scratch = nullptr;
+        void* status = nullptr;
+        e = cudaGetSymbolAddress(&scratch, g_static_scratch);
+        if (e == cudaSuccess) e = cudaGetSymbolAddress(&status, g_static_status);
+        if (e != cudaSuccess || !scratch || !status) return cuda_fail(nullptr, e != cudaSuccess ? e : cudaErrorUnknown);
+        void* fn = nullptr;
+        cudaDriverEntryPointQueryResult qres;
+        e = cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres);
+        if (e != cudaSuccess || qres != cudaDriverEntryPointSuccess || !fn)
+            return cuda_fail(nullptr, e != cudaSuccess ? e : cudaErrorUnknown);
+        e = raise_smem_limit(twopass_scores_kernel, twopass_scores_smem_bytes(3));
+        if (e == cudaSuccess) e = raise_smem_limit(twopass_pv_kernel, twopass_pv_smem_bytes(3));
+        if (e != cudaSuccess) return cuda_fail(nullptr, e);
+        st->scratch = (unsigned char*)scratch;
+        st->status = (int*)status;
+        st->encode_tiled = (encode_tiled_fn)fn;
+        st->ready = 1;
+    }
+    *out = st;
+    return SD_ATTN_OK;
+}
+
+static int static_tmap(encode_tiled_fn enc, CUtensorMap* map, const void* base, int BH, int N, int d, int box_rows) {
+    cuuint64_t dims[3] = {(cuuint64_t)d, (cuuint64_t)N, (cuuint64_t)BH};
+    cuuint64_t strides[2] = {(cuuint64_t)d * 2, (cuuint64_t)N * d * 2};
+    cuuint32_t box[3] = {(cuuint32_t)CHUNK_COLS, (cuuint32_t)box_rows, 1};
+    cuuint32_t estr[3] = {1, 1, 1};
+    CUresult r = enc(map, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 3, const_cast<void*>(base), dims, strides, box, estr,
+                     CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                     CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    return r == CUDA_SUCCESS ? SD_ATTN_OK : SD_ATTN_ERR_CUDA;
+}
+
+extern "C" int sd_attn_forward_twopass_static(const void* q, const void* k, const void* v, void* out, int B, int H,
+                                              int Nq, int Nk, int d, float scale, int dtype, void* stream) {
+    if (B <= 0 || H <= 0 || Nq < 0 || Nk <= 0 || d <= 0) return SD_ATTN_ERR_INVALID_VALUE;
+    if (!isfinite(scale)) return SD_ATTN_ERR_INVALID_VALUE;
+    if (dtype != SD_ATTN_F16 || d > SD_ATTN_MAX_D || d % 8 != 0) return SD_ATTN_ERR_UNSUPPORTED;
+    if ((long long)B * H > 65535) return SD_ATTN_ERR_UNSUPPORTED;
+    if (Nq == 0) return SD_ATTN_OK;
+    if (!q || !k || !v || !out) return SD_ATTN_ERR_INVALID_VALUE;
+    if ((((uintptr_t)q | (uintptr_t)k | (uintptr_t)v | (uintptr_t)out) & 15u) != 0) return SD_ATTN_ERR_ALIGNMENT;
+    const size_t need = sd_attn_workspace_bytes(SD_ATTN_MODE_TWOPASS, B, H, Nq, Nk, d, dtype);
+    if (need > SD_ATTN_STATIC_SCRATCH_BYTES) {
+        if (getenv("SD_ATTN_LOG"))
+            fprintf(stderr, "[sd_attn] static two-pass scratch: call needs %zu bytes, the built-in array holds %zu\n", need,
+                    (size_t)SD_ATTN_STATIC_SCRATCH_BYTES);
+        return SD_ATTN_ERR_WORKSPACE;
+    }
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return cuda_fail(nullptr, e);
+    StaticDeviceState* st = nullptr;
+    int rc = static_setup(dev, &st);
+    if (rc != SD_ATTN_OK) return rc;
+
+    const int BH = B * H;
+    const size_t rows = (size_t)BH * Nq;
+    float* scores = (float*)st->scratch;
+    float* stats = (float*)(st->scratch + ((rows * (size_t)Nk * sizeof(float) + 255) & ~(size_t)255));
+    cudaStream_t s = (cudaStream_t)stream;
+    // the status block is shared by every call and keeps the last call's contents: start from zero
+    e = cudaMemsetAsync(st->status, 0, sizeof(int) * DEV_STATUS_INTS, s);
+    if (e != cudaSuccess) return cuda_fail(nullptr, e);
+    TwoPassArgs a;
+    twopass_fill_args(&a, scores, stats, (__half*)out, Nq, Nk, d, scale, st->status);
+    CUtensorMap tq, tk, tv;
+    rc = static_tmap(st->encode_tiled, &tq, q, BH, Nq, d, TILE_M);
+    if (rc == SD_ATTN_OK) rc = static_tmap(st->encode_tiled, &tk, k, BH, Nk, d, TWOPASS_BN);
+    if (rc == SD_ATTN_OK) rc = static_tmap(st->encode_tiled, &tv, v, BH, Nk, d, TWOPASS_BN);
+    if (rc != SD_ATTN_OK) return rc;
+    dim3 grid((Nq + TILE_M - 1) / TILE_M, BH);
+    twopass_scores_kernel<<<grid, TWOPASS_THREADS, twopass_scores_smem_bytes(a.nch), s>>>(tq, tk, a);
+    e = cudaGetLastError();
+    if (e != cudaSuccess) return cuda_fail(nullptr, e);
+    twopass_pv_kernel<<<grid, TWOPASS_THREADS, twopass_pv_smem_bytes(a.nch), s>>>(tv, a);
+    e = cudaGetLastError();
+    return e == cudaSuccess ? SD_ATTN_OK : cuda_fail(nullptr, e);
 }
