@@ -14,12 +14,16 @@
 // current key tile in issue order on the same thread.  (A 48-wide key tile with P_t in columns of its
 // own, which takes the tensor-core round trip off the softmax's path, measured slower: the fixed cost
 // per key tile outweighs it.)
-// The running-max rescale of O_t is lazy (only when the max grew by more than 2^8).
+// No per-tile maximum is taken.  The exponent is anchored FUSED_HEADROOM_LOG2 above the maximum of the row's
+// first key tile; a later tile is evaluated against that anchor as it stands, and only when its weights sum to
+// more than FUSED_TILE_SUM_LIMIT (a score far above the anchor: rare) is the tile's maximum taken, O_t and the
+// row sum rescaled and the tile redone.  Any anchor gives the same result in exact arithmetic; this one keeps
+// every weight inside binary16's normal range where it matters.
 #pragma once
 #include <cuda.h>
 
 #include "cross_kernel.cuh"  // TILE_M, CHUNK_COLS, CHUNK_ROW_BYTES
-#include "fused_kernel.cuh"  // FUSED_RESCALE_LOG2, FUSED_TRACE, FUSED_POLY_PER8
+#include "fused_kernel.cuh"  // FUSED_HEADROOM_LOG2, FUSED_TILE_SUM_LIMIT, FUSED_TRACE, FUSED_POLY_PER8
 #include "softmax_math.cuh"
 #include "tc_common.cuh"
 
@@ -28,7 +32,7 @@ namespace sd_attn {
 constexpr int F4_TILES = 4;
 constexpr int F4_BN = 64;
 constexpr int F4_THREADS = 24 * 32;   // 16 softmax warps + 8 control warps (producer, 4 issuers, 3 idle)
-constexpr int F4_SOFTMAX_REGS = 104;  // after setmaxnreg: 512 * 104 + 256 * 32 = 61440 of the 65536 registers
+constexpr int F4_SOFTMAX_REGS = 104;  // after setmaxnreg: 512 * 104 + 256 * 32 = 768 * 80, the launch allocation
 constexpr int F4_CONTROL_REGS = 32;
 constexpr int F4_STAGES = 8;
 constexpr int F4_MAX_D = 64;
@@ -195,7 +199,7 @@ fused4_attention_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid
             const uint32_t b_sfull = smem_u32(&bar_s_full[t]), b_pfull = smem_u32(&bar_p_full[t]);
             const uint32_t b_pvdone = smem_u32(&bar_pv_done[t]);
             const float c2 = args.scale_log2e;
-            float m_run = -INFINITY;  // running max, in raw score units
+            float m_run = 0.f;        // anchor of the exponent: a bound on the running max, times scale*log2(e)
             float l_run = 0.f;        // running sum of p (relative to m_run)
             bool ok = true;
             const bool tracer = (warp & 3) == 0 && lane == 0;
@@ -213,18 +217,45 @@ fused4_attention_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid
                 tmem_wait_ld();
                 if (tracer) FUSED_TRACE(t, j, 2);
                 const bool ragged = valid < BN;   // only the last key tile can be
-                const float row_max = ragged ? row_max_masked<BN>(s, valid) : row_max_bf16<BN>(s);
                 if (j == 0) {
-                    m_run = row_max;
-                } else {
-                    const bool grow = (row_max - m_run) * c2 > FUSED_RESCALE_LOG2;
-                    if (__any_sync(0xffffffffu, grow)) {
-                        // rare.  S_t(j) being ready means the P V product of tile j-1 was issued before it and has
-                        // completed, so O_t may be touched.  The first registers of the score row are borrowed
-                        // (register budget) and the row, still intact in tensor memory, is fetched again.
-                        const float alpha = grow ? ex2_approx((m_run - row_max) * c2) : 1.f;
-                        if (grow) m_run = row_max;
-                        l_run *= alpha;
+                    const float row_max = ragged ? row_max_masked<BN>(s, valid) : row_max_bf16<BN>(s);
+                    m_run = row_max * c2 + FUSED_HEADROOM_LOG2;
+                }
+                if (tracer) FUSED_TRACE(t, j, 3);
+                // The weights of this tile are taken against the anchor as it stands; the tile's own maximum is
+                // NOT computed.  A row whose weights sum to more than FUSED_TILE_SUM_LIMIT has met a score far above
+                // its anchor: only then (rare) is the maximum taken, O_t and the row sum rescaled and the tile redone.
+                uint32_t packed[BN / 2];
+                float tile_sum;
+#pragma unroll 1
+                for (int attempt = 0; attempt < 2; ++attempt) {
+                    const float neg_mc = -m_run;
+                    if (!ragged) {
+                        const uint64_t c2c2 = pack_b64(__float_as_uint(c2), __float_as_uint(c2));
+                        const uint64_t nmnm = pack_b64(__float_as_uint(neg_mc), __float_as_uint(neg_mc));
+                        uint64_t acc[2] = {0ull, 0ull};
+                        exp2_pack_32<FUSED_POLY_PER8>(&s[0], c2c2, nmnm, &packed[0], acc);
+                        exp2_pack_32<FUSED_POLY_PER8>(&s[32], c2c2, nmnm, &packed[16], acc);
+                        tile_sum = sum_f32x2(acc[0], acc[1]);
+                    } else {
+                        tile_sum = 0.f;
+                        exp2_pack_32_masked(&s[0], c2, neg_mc, 0, valid, &packed[0], tile_sum);
+                        exp2_pack_32_masked(&s[32], c2, neg_mc, 32, valid, &packed[16], tile_sum);
+                    }
+                    const bool over = !(tile_sum <= FUSED_TILE_SUM_LIMIT);
+                    if (attempt == 1 || !__any_sync(0xffffffffu, over)) break;
+                    // S_t(j) being ready means the P V product of tile j-1 was issued before it and has completed,
+                    // so O_t may be touched; nothing of P_t(j) has been stored yet, so the scores are still in
+                    // tensor memory.  The first registers of the score row are borrowed for O_t (register budget).
+                    tmem_ld32(tmem_s, &s[0]);
+                    tmem_ld32(tmem_s + 32, &s[32]);
+                    tmem_wait_ld();
+                    const float row_max = ragged ? row_max_masked<BN>(s, valid) : row_max_bf16<BN>(s);
+                    const float m_new = row_max * c2 + FUSED_HEADROOM_LOG2;
+                    const float alpha = over ? ex2_approx(m_run - m_new) : 1.f;
+                    if (over) m_run = m_new;
+                    l_run *= alpha;
+                    if (j > 0) {
                         for (int g = 0; g < (dpad >> 4); ++g) {
                             tmem_ld16(tmem_o + g * 16, *reinterpret_cast<uint32_t(*)[16]>(&s[0]));
                             tmem_wait_ld();
@@ -233,31 +264,13 @@ fused4_attention_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid
                             tmem_st16(tmem_o + g * 16, *reinterpret_cast<uint32_t(*)[16]>(&s[0]));
                         }
                         tmem_wait_st();
-                        tmem_ld32(tmem_s, &s[0]);
-                        tmem_ld32(tmem_s + 32, &s[32]);
-                        tmem_wait_ld();
                     }
+                    tmem_ld32(tmem_s, &s[0]);
+                    tmem_ld32(tmem_s + 32, &s[32]);
+                    tmem_wait_ld();
                 }
-                const float neg_mc = -m_run * c2;
-                if (tracer) FUSED_TRACE(t, j, 3);
-                uint32_t packed[16];
-                if (!ragged) {
-                    const uint64_t c2c2 = pack_b64(__float_as_uint(c2), __float_as_uint(c2));
-                    const uint64_t nmnm = pack_b64(__float_as_uint(neg_mc), __float_as_uint(neg_mc));
-                    uint64_t acc[2] = {0ull, 0ull};
-                    exp2_pack_32<FUSED_POLY_PER8>(&s[0], c2c2, nmnm, packed, acc);
-                    tmem_st16(tmem_s, packed);        // P_t over columns of S_t that already sit in registers
-                    exp2_pack_32<FUSED_POLY_PER8>(&s[32], c2c2, nmnm, packed, acc);
-                    tmem_st16(tmem_s + 16, packed);
-                    l_run += sum_f32x2(acc[0], acc[1]);
-                } else {
-                    float sum = 0.f;
-                    exp2_pack_32_masked(&s[0], c2, neg_mc, 0, valid, packed, sum);
-                    tmem_st16(tmem_s, packed);
-                    exp2_pack_32_masked(&s[32], c2, neg_mc, 32, valid, packed, sum);
-                    tmem_st16(tmem_s + 16, packed);
-                    l_run += sum;
-                }
+                l_run += tile_sum;
+                tmem_st32(tmem_s, packed);   // P_t over the first columns of S_t, whose scores sit in registers
                 if (tracer) FUSED_TRACE(t, j, 4);
                 tmem_wait_st();
                 tc_fence_before_sync();

@@ -35,7 +35,20 @@ constexpr int FUSED_THREADS = 352;
 constexpr int FUSED_MAX_STAGES = 4;
 constexpr int FUSED_MAX_KSTEPS = 10;   // MMA steps of the Q K^T contraction at the largest head dim (160)
 constexpr int FUSED_SMEM_BUDGET = 220 * 1024;
-constexpr float FUSED_RESCALE_LOG2 = 8.0f;  // rescale O only when the max grew by more than 2^8
+// The anchor of the exponent starts FUSED_HEADROOM_LOG2 above the first tile's row max (weights <= 2^-3,
+// still 11 bits below which binary16 stays normal) and O is rescaled only when a later row max exceeds
+// the anchor by more than FUSED_RESCALE_LOG2 (weights <= 2^12, far inside binary16's range).
+#ifndef SD_ATTN_RESCALE_LOG2
+#define SD_ATTN_RESCALE_LOG2 12.0f
+#endif
+#ifndef SD_ATTN_HEADROOM_LOG2
+#define SD_ATTN_HEADROOM_LOG2 3.0f
+#endif
+constexpr float FUSED_RESCALE_LOG2 = SD_ATTN_RESCALE_LOG2;
+constexpr float FUSED_HEADROOM_LOG2 = SD_ATTN_HEADROOM_LOG2;
+// The four-tile kernel does not take a key tile's maximum at all: it re-anchors a row only when the weights of
+// one tile sum to more than this (so no weight exceeds it: 2^12 is far inside binary16's range).
+constexpr float FUSED_TILE_SUM_LIMIT = 4096.0f;
 #ifndef SD_ATTN_POLY_PER8
 #define SD_ATTN_POLY_PER8 0
 #endif
@@ -259,7 +272,7 @@ fused_attention_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_
             const uint32_t b_pfull = smem_u32(&bar_p_full[t]), b_pvdone = smem_u32(&bar_pv_done[t]);
             const bool tracer = (warp & 3) == 0 && lane == 0;
             const float c2 = args.scale_log2e;
-            float m_run = -INFINITY;  // running max, in raw score units
+            float m_run = -INFINITY;  // anchor of the exponent: a bound on the running max, times scale*log2(e)
             float l_run = 0.f;        // running sum of p (relative to m_run)
             bool ok = true;
             for (int j = 0; j < n_kv; ++j) {
@@ -280,18 +293,20 @@ fused_attention_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_
                 if (tracer) FUSED_TRACE(t, j, 2);
                 const bool ragged = valid < BN;   // only the last key tile can be
                 const float row_max = ragged ? row_max_masked<BN>(s, valid) : row_max_bf16<BN>(s);
+                const float row_max2 = row_max * c2;   // in log2 units, as the exponent sees it
                 if (j == 0) {
-                    m_run = row_max;
+                    m_run = row_max2 + FUSED_HEADROOM_LOG2;
                 } else {
                     // P_t and O_t belong to the tensor pipe until the P V product of tile j-1 has completed
                     ok = mbar_wait(b_pvdone, (j - 1) & 1, abort_p, args.status, SITE_F_PFREE, j);
                     ok = __all_sync(0xffffffffu, ok);
                     if (!ok) break;
                     tc_fence_after_sync();
-                    const bool grow = (row_max - m_run) * c2 > FUSED_RESCALE_LOG2;
+                    const bool grow = row_max2 - m_run > FUSED_RESCALE_LOG2;
                     if (__any_sync(0xffffffffu, grow)) {
-                        const float alpha = grow ? ex2_approx((m_run - row_max) * c2) : 1.f;
-                        if (grow) m_run = row_max;
+                        const float m_new = row_max2 + FUSED_HEADROOM_LOG2;
+                        const float alpha = grow ? ex2_approx(m_run - m_new) : 1.f;
+                        if (grow) m_run = m_new;
                         l_run *= alpha;
                         for (int g = 0; g < (dpad >> 4); ++g) {
                             uint32_t x[16];
@@ -303,7 +318,7 @@ fused_attention_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_
                         }
                     }
                 }
-                const float neg_mc = -m_run * c2;
+                const float neg_mc = -m_run;
                 if (tracer) FUSED_TRACE(t, j, 3);
                 if (!ragged) {
                     const uint64_t c2c2 = pack_b64(__float_as_uint(c2), __float_as_uint(c2));

@@ -248,6 +248,34 @@ def test_special_cases(att, bd, mode_name):
     assert np.array_equal(out3, np.broadcast_to(v[:, :, 33:34], out3.shape))
 
 
+@pytest.mark.parametrize("d", [40, 80, 160])
+@pytest.mark.parametrize("order", ["rising", "falling", "steps"])
+def test_running_anchor_follows_scores_that_grow_along_the_keys(att, bd, d, order):
+    """The online form (Sec. 3.2.2) must re-anchor its exponent when later key tiles hold far larger scores.
+
+    rising: the key norm grows 30-fold along the sequence, so the row maximum keeps moving (many re-anchorings,
+    different rows of a warp at different tiles); falling: the largest scores come first and the rest underflow
+    against them; steps: three isolated keys, each dominating everything before it by e^20 or more.
+    """
+    B, H, Nq, Nk = 1, 2, 520, 1000
+    q, k, v = rand_qkv(900 + d, B, H, Nq, Nk, d, qmult=2.0)
+    k32 = k.astype(np.float32)
+    if order == "steps":
+        for pos, gain in ((130, 3.0), (515, 6.0), (940, 9.0)):
+            k32[:, :, pos] = gain * np.sign(q.astype(np.float32).mean(axis=2, keepdims=False))[:, :, :] + k32[:, :, pos]
+    else:
+        ramp = np.geomspace(0.2, 6.0, Nk, dtype=np.float32)
+        if order == "falling":
+            ramp = ramp[::-1]
+        k32 = k32 * ramp[None, None, :, None]
+    k = k32.astype(np.float16)
+    scale = float(np.float32(1.0 / np.sqrt(d)))
+    ref, L, _ = oracle.forward(q, k, v, scale)
+    assert (L.max() - L.min()) * 1.4427 > 12.0          # the logits span far more than one fixed anchor covers
+    for mode in (bd.MODE_FUSED, bd.MODE_TWOPASS):
+        check(run(att, bd, mode, q, k, v, scale), ref, v, what="%s d=%d mode %s" % (order, d, bd.MODE_NAMES[mode]))
+
+
 def test_padding_rows_with_distinct_values_only_see_their_mean(att, bd):
     call = workloads.config3()[0]
     q, k, v = workloads.make_inputs(call)
