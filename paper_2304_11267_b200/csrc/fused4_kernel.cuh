@@ -67,7 +67,10 @@ fused4_attention_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid
     __shared__ uint32_t tmem_base_slot;
     __shared__ int abort_flag;
 
-    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int tid = threadIdx.x, lane = tid & 31;
+    // through a shuffle so that the compiler knows the warp index is warp-uniform (descriptor arithmetic of the
+    // issuer then lives in uniform registers)
+    const int warp = __shfl_sync(0xffffffffu, tid >> 5, 0);
     const int bh = blockIdx.y;
     const int row_base = blockIdx.x * F4_TILES * TILE_M;
     int n_qtiles = (args.Nq - row_base + TILE_M - 1) / TILE_M;

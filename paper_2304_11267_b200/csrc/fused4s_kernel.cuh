@@ -1,0 +1,340 @@
+// Fused single-pass attention for head dims up to 48 (the d = 40 layers of the UNet): the four-tile kernel
+// of fused4_kernel.cuh with one SPARE score buffer that takes the tensor-core round trip off the softmax's path.
+//
+// In the four-tile kernel the weights P_t(j) overwrite the scores S_t(j), so S_t(j+1) can only follow the
+// product P_t(j) V(j): after every key tile a softmax warpgroup idles for the round trip softmax -> MMA issue ->
+// tensor pipe -> softmax (450-550 clocks of 2500), and four warps per scheduler do not hide it.  With d <= 48 the
+// four output accumulators need 192 of the 512 tensor-memory columns, which leaves room for FIVE 64-column score
+// buffers for the four tiles.  The (tile, key tile) steps are put in one global order k = T*j + t (T tiles);
+// step k uses buffer k mod (T+1); S(k + T + 1) is issued right behind P(k) V(k) -- into the buffer that product
+// frees -- and belongs to the tile that comes NEXT in the rotation, not to the tile that just finished.  So when a
+// tile finishes key tile j its scores for j+1 were requested a quarter of a period earlier, by its neighbour's
+// hand-off, and are normally there.
+//
+//   warps 0-15   softmax of tiles 0..3 (thread = query row = TMEM lane)
+//   warp 16      TMA producer          warps 17-20  MMA issuers: issuer t multiplies P_t V and then requests the
+//                scores of tile t+1 (32 registers each; warps 21-23 only fill the control warpgroup)
+//
+// The anchor scheme of the exponent (no per-tile maximum) is that of fused4_kernel.cuh.
+#pragma once
+#include <cuda.h>
+
+#include "fused4_kernel.cuh"  // Fused4Args, F4_* constants, SITE_G_*
+
+namespace sd_attn {
+
+constexpr int F4S_MAX_DPAD = 48;
+constexpr int F4S_BUFFERS = F4_TILES + 1;
+constexpr int F4S_SOFTMAX_REGS = 104;   // 512 * 104 + 256 * 32 = 768 * 80, the launch allocation
+constexpr int F4S_CONTROL_REGS = 32;
+
+__global__ void __launch_bounds__(F4_THREADS, 1)
+fused4s_attention_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__ CUtensorMap tmap_k,
+                         const __grid_constant__ CUtensorMap tmap_v, const Fused4Args args) {
+    constexpr int BN = F4_BN;
+    extern __shared__ uint8_t f4s_smem_raw[];
+    // per (tile, buffer): S ready (MMA) | P ready (softmax).  per tile: Q landed | P V of key tile j done | all of
+    // O_t done.  The score barriers are per tile AND buffer so that every barrier has ONE consumer that takes its
+    // phases in order (a parity wait is only sound for a waiter exactly one phase behind): tile t meets buffer b
+    // every NB key tiles, and the buffer cannot come back to it before its previous contents were consumed.
+    __shared__ __align__(8) uint64_t bar_s_full[F4_TILES][F4S_BUFFERS], bar_p_full[F4_TILES][F4S_BUFFERS];
+    __shared__ __align__(8) uint64_t bar_q_full[F4_TILES], bar_pv_done[F4_TILES], bar_o_final[F4_TILES];
+    __shared__ __align__(8) uint64_t bar_kv_full[F4_STAGES], bar_kv_empty[F4_STAGES];
+    __shared__ uint32_t tmem_base_slot;
+    __shared__ int abort_flag;
+
+    const int tid = threadIdx.x, lane = tid & 31;
+    const int warp = __shfl_sync(0xffffffffu, tid >> 5, 0);   // warp-uniform for the compiler
+    const int bh = blockIdx.y;
+    const int row_base = blockIdx.x * F4_TILES * TILE_M;
+    int T = (args.Nq - row_base + TILE_M - 1) / TILE_M;   // query tiles of this CTA
+    if (T > F4_TILES) T = F4_TILES;
+    const int NB = T + 1;                                 // score buffers in the rotation
+    const int n_kv = (args.Nk + BN - 1) / BN;
+    const int dpad = args.dpad;
+
+    const uint32_t smem_base = (smem_u32(f4s_smem_raw) + 1023u) & ~1023u;
+    constexpr uint32_t q_tile_bytes = TILE_M * CHUNK_ROW_BYTES;     // one 64-column chunk (d <= 48)
+    constexpr uint32_t kv_tile_bytes = BN * CHUNK_ROW_BYTES;
+    const uint32_t q_smem = smem_base;                              // [4][128 rows][128 B]
+    const uint32_t kv_smem = q_smem + F4_TILES * q_tile_bytes;      // [stages][K | V][64 rows][128 B]
+    volatile int* abort_p = &abort_flag;
+
+    if (tid == 0) {
+        abort_flag = 0;
+        for (int t = 0; t < F4_TILES; ++t) {
+            for (int b = 0; b < F4S_BUFFERS; ++b) {
+                mbar_init(smem_u32(&bar_s_full[t][b]), 1);
+                mbar_init(smem_u32(&bar_p_full[t][b]), 4);    // one arrival per softmax warp of the tile
+            }
+            mbar_init(smem_u32(&bar_q_full[t]), 1);
+            mbar_init(smem_u32(&bar_pv_done[t]), 1);
+            mbar_init(smem_u32(&bar_o_final[t]), 1);
+        }
+        for (int s = 0; s < F4_STAGES; ++s) {
+            mbar_init(smem_u32(&bar_kv_full[s]), 1);
+            mbar_init(smem_u32(&bar_kv_empty[s]), T);   // one commit per issuer
+        }
+        mbar_init_fence();
+    }
+    if (warp == 16) {
+        tmem_alloc(smem_u32(&tmem_base_slot), 512);
+        tmem_relinquish();
+    }
+    tc_fence_before_sync();
+    __syncthreads();
+    tc_fence_after_sync();
+    const uint32_t tmem_base = tmem_base_slot;
+    const uint32_t tmem_o0 = tmem_base + F4S_BUFFERS * BN;   // columns: five score buffers | O_0..O_3
+
+    // One setmaxnreg site per kind, executed by whole warpgroups; the budget is the CTA's launch allocation.
+    if (warp >= 16) setmaxnreg_dec<F4S_CONTROL_REGS>();
+    if (warp == 16) {
+        // ------------------------------------------------------------ TMA producer
+        if (elect_one()) {
+            tma_prefetch_desc(&tmap_q);
+            tma_prefetch_desc(&tmap_k);
+            tma_prefetch_desc(&tmap_v);
+            for (int t = 0; t < T; ++t) {
+                const uint32_t bar = smem_u32(&bar_q_full[t]);
+                mbar_arrive_expect_tx(bar, q_tile_bytes);
+                tma_load_3d(q_smem + t * q_tile_bytes, &tmap_q, bar, 0, row_base + t * TILE_M, bh);
+            }
+            for (int j = 0; j < n_kv; ++j) {
+                const int s = j % F4_STAGES;
+                if (j >= F4_STAGES && !mbar_wait(smem_u32(&bar_kv_empty[s]), ((j / F4_STAGES) - 1) & 1, abort_p,
+                                                 args.status, SITE_G_EMPTY, j))
+                    break;
+                const uint32_t k_dst = kv_smem + s * 2 * kv_tile_bytes, v_dst = k_dst + kv_tile_bytes;
+                const uint32_t bar = smem_u32(&bar_kv_full[s]);
+                mbar_arrive_expect_tx(bar, 2 * kv_tile_bytes);
+                tma_load_3d(k_dst, &tmap_k, bar, 0, j * BN, bh);
+                tma_load_3d(v_dst, &tmap_v, bar, 0, j * BN, bh);
+            }
+        }
+    } else if (warp > 16 && warp <= 16 + F4_TILES) {
+        // ------------------------------------------------------------ MMA issuer of the steps of query tile t
+        // Issuer t waits for P of its own tile's step k = T*j + t, issues O_t += P V(j), and then -- behind that
+        // product, on the same thread, into the buffer it frees -- the scores of step k + NB, which belong to the
+        // NEXT tile of the rotation.
+        const int t = warp - 17;
+        if (t < T && elect_one()) {
+            const uint32_t idesc_s = idesc_f16(TILE_M, BN, false, false, args.negate != 0);
+            const uint32_t idesc_o = idesc_f16(TILE_M, dpad, false, true, false);
+            const int ksteps_s = (args.d + 15) / 16;   // <= 3: inside one swizzled 64-column chunk
+            const int tn = (t + 1 == T) ? 0 : t + 1;   // the tile whose scores this thread requests
+            const uint64_t q_desc = smem_desc_sw128(q_smem + tn * q_tile_bytes, 16, 1024);
+            const uint64_t q_desc_own = smem_desc_sw128(q_smem + t * q_tile_bytes, 16, 1024);
+            const uint64_t k_desc0 = smem_desc_sw128(kv_smem, 16, 1024);
+            const uint64_t v_desc0 = smem_desc_sw128(kv_smem + kv_tile_bytes, BN * CHUNK_ROW_BYTES, 1024);
+            constexpr uint32_t stage_off = (2 * kv_tile_bytes) >> 4;
+            const uint32_t tmem_o = tmem_o0 + t * dpad;
+            const uint32_t b_pvdone = smem_u32(&bar_pv_done[t]);
+
+            auto issue_s = [&](uint64_t qd, int tile, int j, int b) {   // scores of (tile, key tile j) into buffer b
+                const uint64_t kd = k_desc0 + (uint64_t)((j % F4_STAGES) * stage_off);
+                const uint32_t ts = tmem_base + b * BN;
+#pragma unroll
+                for (int kk = 0; kk < 3; ++kk)
+                    if (kk < ksteps_s) mma_f16_ss(ts, qd + (uint64_t)(kk * 2), kd + (uint64_t)(kk * 2), idesc_s, kk > 0);
+                tc_commit(smem_u32(&bar_s_full[tile][b]));
+            };
+            auto issue_o = [&](int j, int b) {   // O_t (+)= P V(j), P in the first 32 columns of score buffer b
+                const uint64_t vd = v_desc0 + (uint64_t)((j % F4_STAGES) * stage_off);
+                const uint32_t tp = tmem_base + b * BN;
+#pragma unroll
+                for (int kk = 0; kk < BN / 16; ++kk)
+                    mma_f16_ts(tmem_o, tp + kk * 8, vd + (uint64_t)(kk * ((16 * CHUNK_ROW_BYTES) >> 4)), idesc_o, j > 0 || kk > 0);
+            };
+
+            bool ok = mbar_wait(smem_u32(&bar_kv_full[0]), 0, abort_p, args.status, SITE_G_KV, 0) &&
+                      mbar_wait(smem_u32(&bar_q_full[t]), 0, abort_p, args.status, SITE_G_Q, t) &&
+                      mbar_wait(smem_u32(&bar_q_full[tn]), 0, abort_p, args.status, SITE_G_Q, tn);
+            if (ok) {
+                // the first T+1 steps fill the buffers: step t (own tile, key tile 0) into buffer t; the last issuer
+                // also requests step T (tile 0, key tile 1) into the spare buffer T
+                tc_fence_after_sync();
+                issue_s(q_desc_own, t, 0, t);
+                if (t == T - 1 && n_kv > 1) {
+                    ok = mbar_wait(smem_u32(&bar_kv_full[1]), 0, abort_p, args.status, SITE_G_KV, 1);
+                    if (ok) {
+                        tc_fence_after_sync();
+                        issue_s(q_desc, tn, 1, T);
+                    }
+                }
+            }
+            // own step k = T*j + t: buffer b = k % NB, which tile t meets for the (j / NB)-th time (as in the softmax
+            // warps); it requests step k + NB = (tn, jn) into the same buffer
+            int b = t, ph = 0, jm = 0;
+            const int jn_off = (t + 1 == T) ? 2 : 1;
+            for (int j = 0; j < n_kv && ok; ++j) {
+                const int jn = j + jn_off;
+                const bool more = jn < n_kv;
+                if (more)   // landed long ago: keep this wait off the critical path
+                    ok = mbar_wait(smem_u32(&bar_kv_full[jn % F4_STAGES]), (jn / F4_STAGES) & 1, abort_p, args.status,
+                                   SITE_G_KV, jn);
+                if (t == 0) FUSED_TRACE(4, j, 0);
+                if (ok) ok = mbar_wait(smem_u32(&bar_p_full[t][b]), ph, abort_p, args.status, SITE_G_P, j);
+                if (!ok) break;
+                tc_fence_after_sync();
+                if (t == 0) FUSED_TRACE(4, j, 1);
+                issue_o(j, b);
+                if (more) issue_s(q_desc, tn, jn, b);               // into the buffer P is read from: behind it, in order
+                tc_commit(b_pvdone);                                // O_t holds key tiles 0..j
+                tc_commit(smem_u32(&bar_kv_empty[j % F4_STAGES]));  // this issuer is done with K(j), V(j)
+                if (j == n_kv - 1) tc_commit(smem_u32(&bar_o_final[t]));
+                if (t == 0) FUSED_TRACE(4, j, 2);
+                b = (b == 0) ? NB - 1 : b - 1;              // k += NB - 1
+                if (++jm == NB) { jm = 0; ph ^= 1; }
+            }
+        }
+    } else if (warp < 16) {
+        // ------------------------------------------------------------ softmax warps
+        setmaxnreg_inc<F4S_SOFTMAX_REGS>();
+        const int t = warp >> 2;                 // query tile of this warpgroup
+        if (t < T) {
+            const int r = tid & (TILE_M - 1);    // row inside the tile = TMEM lane
+            const uint32_t lane_off = (uint32_t)((warp & 3) * 32) << 16;
+            const uint32_t tmem_o = tmem_o0 + t * dpad + lane_off;
+            const uint32_t b_pvdone = smem_u32(&bar_pv_done[t]);
+            const float c2 = args.scale_log2e;
+            float m_run = 0.f;   // anchor of the exponent: a bound on the running max, times scale*log2(e)
+            float l_run = 0.f;   // running sum of p (relative to m_run)
+            bool ok = true;
+            const bool tracer = (warp & 3) == 0 && lane == 0;
+            // step k = T*j + t uses buffer k % NB; k grows by T = NB - 1 per key tile, so the buffer index walks down and
+            // tile t meets each buffer every NB key tiles: phase (j / NB) & 1 of that (tile, buffer) barrier pair
+            int b = t % NB, ph = 0, jm = 0;
+            for (int j = 0; j < n_kv; ++j) {
+                const uint32_t tmem_s = tmem_base + b * BN + lane_off;
+                if (tracer) FUSED_TRACE(t, j, 0);
+                ok = mbar_wait(smem_u32(&bar_s_full[t][b]), ph, abort_p, args.status, SITE_G_S, j);
+                ok = __all_sync(0xffffffffu, ok);
+                if (!ok) break;
+                tc_fence_after_sync();
+                if (tracer) FUSED_TRACE(t, j, 1);
+                const int valid = args.Nk - j * BN;   // columns >= valid are zero-filled keys
+                uint32_t s[BN];
+                tmem_ld32(tmem_s, &s[0]);
+                tmem_ld32(tmem_s + 32, &s[32]);
+                tmem_wait_ld();
+                if (tracer) FUSED_TRACE(t, j, 2);
+                const bool ragged = valid < BN;   // only the last key tile can be
+                if (j == 0) {
+                    const float row_max = ragged ? row_max_masked<BN>(s, valid) : row_max_bf16<BN>(s);
+                    m_run = row_max * c2 + FUSED_HEADROOM_LOG2;
+                }
+                uint32_t packed[BN / 2];
+                float tile_sum;
+#pragma unroll 1
+                for (int attempt = 0; attempt < 2; ++attempt) {
+                    const float neg_mc = -m_run;
+                    if (!ragged) {
+                        const uint64_t c2c2 = pack_b64(__float_as_uint(c2), __float_as_uint(c2));
+                        const uint64_t nmnm = pack_b64(__float_as_uint(neg_mc), __float_as_uint(neg_mc));
+                        uint64_t acc[2] = {0ull, 0ull};
+                        exp2_pack_32<FUSED_POLY_PER8>(&s[0], c2c2, nmnm, &packed[0], acc);
+                        exp2_pack_32<FUSED_POLY_PER8>(&s[32], c2c2, nmnm, &packed[16], acc);
+                        tile_sum = sum_f32x2(acc[0], acc[1]);
+                    } else {
+                        tile_sum = 0.f;
+                        exp2_pack_32_masked(&s[0], c2, neg_mc, 0, valid, &packed[0], tile_sum);
+                        exp2_pack_32_masked(&s[32], c2, neg_mc, 32, valid, &packed[16], tile_sum);
+                    }
+                    const bool over = !(tile_sum <= FUSED_TILE_SUM_LIMIT);
+                    if (attempt == 1 || !__any_sync(0xffffffffu, over)) break;
+                    // Rare: a row of this warp met a score far above its anchor.  O_t may be touched once the P V
+                    // product of key tile j-1 has completed (that of j-2 has: see the wait before the hand-off below);
+                    // nothing of P_t(j) has been stored yet, so the scores are still in tensor memory.  The first
+                    // registers of the row are borrowed for O_t.
+                    if (j > 0) {
+                        ok = mbar_wait(b_pvdone, (j - 1) & 1, abort_p, args.status, SITE_G_PV, j);
+                        ok = __all_sync(0xffffffffu, ok);
+                        if (!ok) break;
+                        tc_fence_after_sync();
+                    }
+                    tmem_ld32(tmem_s, &s[0]);
+                    tmem_ld32(tmem_s + 32, &s[32]);
+                    tmem_wait_ld();
+                    const float row_max = ragged ? row_max_masked<BN>(s, valid) : row_max_bf16<BN>(s);
+                    const float m_new = row_max * c2 + FUSED_HEADROOM_LOG2;
+                    const float alpha = over ? ex2_approx(m_run - m_new) : 1.f;
+                    if (over) m_run = m_new;
+                    l_run *= alpha;
+                    if (j > 0) {
+                        for (int g = 0; g < (dpad >> 4); ++g) {
+                            tmem_ld16(tmem_o + g * 16, *reinterpret_cast<uint32_t(*)[16]>(&s[0]));
+                            tmem_wait_ld();
+#pragma unroll
+                            for (int c = 0; c < 16; ++c) s[c] = __float_as_uint(__uint_as_float(s[c]) * alpha);
+                            tmem_st16(tmem_o + g * 16, *reinterpret_cast<uint32_t(*)[16]>(&s[0]));
+                        }
+                        tmem_wait_st();
+                    }
+                    tmem_ld32(tmem_s, &s[0]);
+                    tmem_ld32(tmem_s + 32, &s[32]);
+                    tmem_wait_ld();
+                }
+                if (!ok) break;
+                l_run += tile_sum;
+                tmem_st32(tmem_s, packed);   // P_t(j) over the first columns of the buffer, whose scores sit in registers
+                if (tracer) FUSED_TRACE(t, j, 4);
+                tmem_wait_st();
+                // A parity wait is only sound while the waiter is at most one phase behind.  The scores of this tile
+                // are requested by ANOTHER issuer than the one that multiplies P_t V, so nothing else orders this
+                // warp against its own tile's products: it consumes every phase of pv_done here, before it hands
+                // P_t(j) over (P V(j) cannot complete earlier), when P V(j-1) has had a whole step to finish.
+                if (j > 0) {
+                    ok = mbar_wait(b_pvdone, (j - 1) & 1, abort_p, args.status, SITE_G_PV, j);
+                    ok = __all_sync(0xffffffffu, ok);
+                    if (!ok) break;
+                }
+                tc_fence_before_sync();
+                if (lane == 0) mbar_arrive(smem_u32(&bar_p_full[t][b]));
+                if (tracer) FUSED_TRACE(t, j, 5);
+                b = (b == 0) ? NB - 1 : b - 1;              // k += NB - 1
+                if (++jm == NB) { jm = 0; ph ^= 1; }
+            }
+            if (ok) ok = mbar_wait(smem_u32(&bar_o_final[t]), 0, abort_p, args.status, SITE_G_O, t);
+            ok = __all_sync(0xffffffffu, ok);
+            if (ok) {
+                tc_fence_after_sync();
+                const float inv = 1.f / l_run;
+                const int row = row_base + t * TILE_M + r;
+                __half* orow = args.out + ((size_t)bh * args.Nq + row) * args.d;
+                for (int g = 0; g < (dpad >> 4); ++g) {
+                    uint32_t x[16];
+                    tmem_ld16(tmem_o + g * 16, x);
+                    tmem_wait_ld();
+                    uint4 lo, hi;
+                    lo.x = pack_half2(__uint_as_float(x[0]) * inv, __uint_as_float(x[1]) * inv);
+                    lo.y = pack_half2(__uint_as_float(x[2]) * inv, __uint_as_float(x[3]) * inv);
+                    lo.z = pack_half2(__uint_as_float(x[4]) * inv, __uint_as_float(x[5]) * inv);
+                    lo.w = pack_half2(__uint_as_float(x[6]) * inv, __uint_as_float(x[7]) * inv);
+                    hi.x = pack_half2(__uint_as_float(x[8]) * inv, __uint_as_float(x[9]) * inv);
+                    hi.y = pack_half2(__uint_as_float(x[10]) * inv, __uint_as_float(x[11]) * inv);
+                    hi.z = pack_half2(__uint_as_float(x[12]) * inv, __uint_as_float(x[13]) * inv);
+                    hi.w = pack_half2(__uint_as_float(x[14]) * inv, __uint_as_float(x[15]) * inv);
+                    if (row < args.Nq) {
+                        if (g * 16 + 8 <= args.d) *reinterpret_cast<uint4*>(orow + g * 16) = lo;
+                        if (g * 16 + 16 <= args.d) *reinterpret_cast<uint4*>(orow + g * 16 + 8) = hi;
+                    }
+                }
+            }
+        }
+    }
+
+    // ------------------------------------------------------------ teardown (every thread arrives)
+    tc_fence_before_sync();
+    __syncthreads();
+    if (warp == 16 && lane == 0 && abort_flag) {
+        for (int s = 0; s < F4_STAGES; ++s) mbar_drain(smem_u32(&bar_kv_full[s]), 0);
+    }
+    __syncthreads();
+    if (warp == 16) {
+        __syncwarp();
+        tmem_dealloc(tmem_base, 512);
+    }
+}
+
+}  // namespace sd_attn

@@ -17,6 +17,7 @@
 #include "cross2_kernel.cuh"
 #include "fused_kernel.cuh"
 #include "fused4_kernel.cuh"
+#include "fused4s_kernel.cuh"
 #include "simt_kernel.cuh"
 #include "twopass_kernel.cuh"
 
@@ -54,6 +55,8 @@ struct sd_attn_handle {
     cudaError_t last_cuda_error;
     int sm_count;
     int fused4_ok;            // the register hand-over inside these kernels fits their launch allocation
+    int fused4s_ok;
+    int no_spare;             // SD_ATTN_FUSED_NO_SPARE=1: the four-tile kernel without the spare score buffer
     int cross2_four_ok;
     int cross_one_tile_only;  // SD_ATTN_CROSS_ONE_TILE=1: never use the persistent cross-attention kernel
     int prefer_two_tile;      // SD_ATTN_FUSED_TWO_TILE=1: use the two-tile fused kernel for every head dim
@@ -119,6 +122,8 @@ extern "C" int sd_attn_create(sd_attn_handle** out) {
 #endif
     const char* one = getenv("SD_ATTN_CROSS_ONE_TILE");
     h->cross_one_tile_only = (one && one[0] == '1') ? 1 : 0;
+    const char* nsp = getenv("SD_ATTN_FUSED_NO_SPARE");
+    h->no_spare = (nsp && nsp[0] == '1') ? 1 : 0;
     const char* two = getenv("SD_ATTN_FUSED_TWO_TILE");
     h->prefer_two_tile = (two && two[0] == '1') ? 1 : 0;
 
@@ -130,6 +135,7 @@ extern "C" int sd_attn_create(sd_attn_handle** out) {
     if (e == cudaSuccess) e = raise_smem_limit(fused_attention_kernel<128>, fused_smem_bytes_max());
     if (e == cudaSuccess) e = raise_smem_limit(fused_attention_kernel<64>, fused_smem_bytes_max());
     if (e == cudaSuccess) e = raise_smem_limit(fused4_attention_kernel, fused4_smem_bytes());
+    if (e == cudaSuccess) e = raise_smem_limit(fused4s_attention_kernel, fused4_smem_bytes());
     if (e == cudaSuccess) e = raise_smem_limit(twopass_scores_kernel, twopass_scores_smem_bytes(3));
     if (e == cudaSuccess) e = raise_smem_limit(twopass_pv_kernel, twopass_pv_smem_bytes(3));
     if (e == cudaSuccess) e = raise_smem_limit(simt_attention_kernel<float, 5>, simt_smem_bytes(160));
@@ -142,6 +148,9 @@ extern "C" int sd_attn_create(sd_attn_handle** out) {
         e = cudaFuncGetAttributes(&fa, fused4_attention_kernel);
         if (e == cudaSuccess)
             h->fused4_ok = F4_THREADS * fa.numRegs >= 512 * F4_SOFTMAX_REGS + 256 * F4_CONTROL_REGS;
+        if (e == cudaSuccess) e = cudaFuncGetAttributes(&fa, fused4s_attention_kernel);
+        if (e == cudaSuccess)
+            h->fused4s_ok = F4_THREADS * fa.numRegs >= 512 * F4S_SOFTMAX_REGS + 256 * F4S_CONTROL_REGS;
         if (e == cudaSuccess) e = cudaFuncGetAttributes(&fa, cross2_attention_kernel<4>);
         if (e == cudaSuccess)
             h->cross2_four_ok = cross2_threads(4) * fa.numRegs >= 512 * X2_SOFTMAX_REGS + 128 * X2_CONTROL_REGS;
@@ -364,7 +373,10 @@ static int launch_fused4(sd_attn_handle* h, const Problem& p) {
     if (rc == SD_ATTN_OK) rc = make_tmap(h, &tv, p.v, p.BH, p.Nk, p.d, F4_BN);
     if (rc != SD_ATTN_OK) return rc;
     dim3 grid((p.Nq + F4_TILES * TILE_M - 1) / (F4_TILES * TILE_M), p.BH), block(F4_THREADS);
-    fused4_attention_kernel<<<grid, block, fused4_smem_bytes(), p.stream>>>(tq, tk, tv, a);
+    if (a.dpad <= F4S_MAX_DPAD && h->fused4s_ok && !h->no_spare)
+        fused4s_attention_kernel<<<grid, block, fused4_smem_bytes(), p.stream>>>(tq, tk, tv, a);
+    else
+        fused4_attention_kernel<<<grid, block, fused4_smem_bytes(), p.stream>>>(tq, tk, tv, a);
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) return cuda_fail(h, e);
     h->launches += 1;
