@@ -41,6 +41,7 @@ struct Fused4Args {
     __half* out;  // [BH][Nq][d]
     int Nq, Nk, d;
     int dpad;     // d rounded up to 16 (<= 64)
+    int tiles_per_cta;   // spare-buffer kernel only: 1..4 query tiles per CTA (small problems spread over more SMs)
     float scale_log2e;
     int negate;
     int* status;

@@ -15,6 +15,8 @@
 //   warp 16      TMA producer          warps 17-20  MMA issuers: issuer t multiplies P_t V and then requests the
 //                scores of tile t+1 (32 registers each; warps 21-23 only fill the control warpgroup)
 //
+// A CTA takes 1 to 4 query tiles (Fused4Args::tiles_per_cta): the host gives a small problem fewer tiles per CTA so
+// that it spreads over more SMs; with one tile the rotation degenerates to two alternating score buffers.
 // The anchor scheme of the exponent (no per-tile maximum) is that of fused4_kernel.cuh.
 #pragma once
 #include <cuda.h>
@@ -23,7 +25,28 @@
 
 namespace sd_attn {
 
+#ifdef SD_ATTN_TRACE
+#define F4S_MARK(i)                                                                                   \
+    do {                                                                                              \
+        if (args.trace && blockIdx.x == 0 && blockIdx.y == 0) {                                       \
+            unsigned long long gt_;                                                                   \
+            asm volatile("mov.u64 %0, %globaltimer;" : "=l"(gt_));                                    \
+            args.trace[5 * 40 * 8 + 1024 + (i)] = (long long)gt_;                                     \
+            args.trace[5 * 40 * 8 + 1024 + 16 + (i)] = clock64();                                     \
+        }                                                                                             \
+    } while (0)
+#else
+#define F4S_MARK(i) do { } while (0)
+#endif
+
 constexpr int F4S_MAX_DPAD = 48;
+// Of every 8 exponentials this many are evaluated by the degree-3 polynomial on the FMA pipe instead of the
+// special function unit, which is the busiest unit of this kernel (measured: 0 -> 100 us, 2 -> 95 us, 3 -> 96 us on
+// the 4096-token d = 40 call).
+#ifndef SD_ATTN_F4S_POLY_PER8
+#define SD_ATTN_F4S_POLY_PER8 2
+#endif
+constexpr int F4S_POLY_PER8 = SD_ATTN_F4S_POLY_PER8;
 constexpr int F4S_BUFFERS = F4_TILES + 1;
 constexpr int F4S_SOFTMAX_REGS = 104;   // 512 * 104 + 256 * 32 = 768 * 80, the launch allocation
 constexpr int F4S_CONTROL_REGS = 32;
@@ -46,9 +69,18 @@ fused4s_attention_kernel(const __grid_constant__ CUtensorMap tmap_q, const __gri
     const int tid = threadIdx.x, lane = tid & 31;
     const int warp = __shfl_sync(0xffffffffu, tid >> 5, 0);   // warp-uniform for the compiler
     const int bh = blockIdx.y;
-    const int row_base = blockIdx.x * F4_TILES * TILE_M;
+    const int row_base = blockIdx.x * args.tiles_per_cta * TILE_M;
+#ifdef SD_ATTN_TRACE
+    if (args.trace && tid == 0) {   // per-CTA start stamp and SM id
+        unsigned long long gt; unsigned smid;
+        asm volatile("mov.u64 %0, %globaltimer;" : "=l"(gt));
+        asm volatile("mov.u32 %0, %smid;" : "=r"(smid));
+        const int cta = blockIdx.y * gridDim.x + blockIdx.x;
+        if (cta < 256) { args.trace[5 * 40 * 8 + cta * 4] = (long long)gt; args.trace[5 * 40 * 8 + cta * 4 + 2] = smid; }
+    }
+#endif
     int T = (args.Nq - row_base + TILE_M - 1) / TILE_M;   // query tiles of this CTA
-    if (T > F4_TILES) T = F4_TILES;
+    if (T > args.tiles_per_cta) T = args.tiles_per_cta;
     const int NB = T + 1;                                 // score buffers in the rotation
     const int n_kv = (args.Nk + BN - 1) / BN;
     const int dpad = args.dpad;
@@ -84,6 +116,7 @@ fused4s_attention_kernel(const __grid_constant__ CUtensorMap tmap_q, const __gri
     tc_fence_before_sync();
     __syncthreads();
     tc_fence_after_sync();
+    if (tid == 0) F4S_MARK(0);
     const uint32_t tmem_base = tmem_base_slot;
     const uint32_t tmem_o0 = tmem_base + F4S_BUFFERS * BN;   // columns: five score buffers | O_0..O_3
 
@@ -95,11 +128,14 @@ fused4s_attention_kernel(const __grid_constant__ CUtensorMap tmap_q, const __gri
             tma_prefetch_desc(&tmap_q);
             tma_prefetch_desc(&tmap_k);
             tma_prefetch_desc(&tmap_v);
-            for (int t = 0; t < T; ++t) {
+            // In the order the issuers need them: Q_0 and the first key tile first (a tile of 80-byte rows costs the
+            // TMA unit about 7 clocks per row, so the order decides when the first scores can start).
+            auto load_q = [&](int t) {
                 const uint32_t bar = smem_u32(&bar_q_full[t]);
                 mbar_arrive_expect_tx(bar, q_tile_bytes);
                 tma_load_3d(q_smem + t * q_tile_bytes, &tmap_q, bar, 0, row_base + t * TILE_M, bh);
-            }
+            };
+            load_q(0);
             for (int j = 0; j < n_kv; ++j) {
                 const int s = j % F4_STAGES;
                 if (j >= F4_STAGES && !mbar_wait(smem_u32(&bar_kv_empty[s]), ((j / F4_STAGES) - 1) & 1, abort_p,
@@ -110,7 +146,11 @@ fused4s_attention_kernel(const __grid_constant__ CUtensorMap tmap_q, const __gri
                 mbar_arrive_expect_tx(bar, 2 * kv_tile_bytes);
                 tma_load_3d(k_dst, &tmap_k, bar, 0, j * BN, bh);
                 tma_load_3d(v_dst, &tmap_v, bar, 0, j * BN, bh);
+                if (j == 0)
+                    for (int t = 1; t < T; ++t) load_q(t);
             }
+            if (n_kv == 0)
+                for (int t = 1; t < T; ++t) load_q(t);
         }
     } else if (warp > 16 && warp <= 16 + F4_TILES) {
         // ------------------------------------------------------------ MMA issuer of the steps of query tile t
@@ -148,14 +188,14 @@ fused4s_attention_kernel(const __grid_constant__ CUtensorMap tmap_q, const __gri
             };
 
             bool ok = mbar_wait(smem_u32(&bar_kv_full[0]), 0, abort_p, args.status, SITE_G_KV, 0) &&
-                      mbar_wait(smem_u32(&bar_q_full[t]), 0, abort_p, args.status, SITE_G_Q, t) &&
-                      mbar_wait(smem_u32(&bar_q_full[tn]), 0, abort_p, args.status, SITE_G_Q, tn);
+                      mbar_wait(smem_u32(&bar_q_full[t]), 0, abort_p, args.status, SITE_G_Q, t);
             if (ok) {
                 // the first T+1 steps fill the buffers: step t (own tile, key tile 0) into buffer t; the last issuer
                 // also requests step T (tile 0, key tile 1) into the spare buffer T
                 tc_fence_after_sync();
                 issue_s(q_desc_own, t, 0, t);
-                if (t == T - 1 && n_kv > 1) {
+                ok = mbar_wait(smem_u32(&bar_q_full[tn]), 0, abort_p, args.status, SITE_G_Q, tn);
+                if (ok && t == T - 1 && n_kv > 1) {
                     ok = mbar_wait(smem_u32(&bar_kv_full[1]), 0, abort_p, args.status, SITE_G_KV, 1);
                     if (ok) {
                         tc_fence_after_sync();
@@ -201,7 +241,7 @@ fused4s_attention_kernel(const __grid_constant__ CUtensorMap tmap_q, const __gri
             float m_run = 0.f;   // anchor of the exponent: a bound on the running max, times scale*log2(e)
             float l_run = 0.f;   // running sum of p (relative to m_run)
             bool ok = true;
-            const bool tracer = (warp & 3) == 0 && lane == 0;
+            const bool tracer = false;
             // step k = T*j + t uses buffer k % NB; k grows by T = NB - 1 per key tile, so the buffer index walks down and
             // tile t meets each buffer every NB key tiles: phase (j / NB) & 1 of that (tile, buffer) barrier pair
             int b = t % NB, ph = 0, jm = 0;
@@ -213,6 +253,7 @@ fused4s_attention_kernel(const __grid_constant__ CUtensorMap tmap_q, const __gri
                 if (!ok) break;
                 tc_fence_after_sync();
                 if (tracer) FUSED_TRACE(t, j, 1);
+                if (tid == 0 && (j == 0 || j == 1 || j == 32 || j == n_kv - 1)) F4S_MARK(j == 0 ? 1 : j == 1 ? 2 : j == 32 ? 3 : 4);
                 const int valid = args.Nk - j * BN;   // columns >= valid are zero-filled keys
                 uint32_t s[BN];
                 tmem_ld32(tmem_s, &s[0]);
@@ -233,8 +274,8 @@ fused4s_attention_kernel(const __grid_constant__ CUtensorMap tmap_q, const __gri
                         const uint64_t c2c2 = pack_b64(__float_as_uint(c2), __float_as_uint(c2));
                         const uint64_t nmnm = pack_b64(__float_as_uint(neg_mc), __float_as_uint(neg_mc));
                         uint64_t acc[2] = {0ull, 0ull};
-                        exp2_pack_32<FUSED_POLY_PER8>(&s[0], c2c2, nmnm, &packed[0], acc);
-                        exp2_pack_32<FUSED_POLY_PER8>(&s[32], c2c2, nmnm, &packed[16], acc);
+                        exp2_pack_32<F4S_POLY_PER8>(&s[0], c2c2, nmnm, &packed[0], acc);
+                        exp2_pack_32<F4S_POLY_PER8>(&s[32], c2c2, nmnm, &packed[16], acc);
                         tile_sum = sum_f32x2(acc[0], acc[1]);
                     } else {
                         tile_sum = 0.f;
@@ -295,8 +336,10 @@ fused4s_attention_kernel(const __grid_constant__ CUtensorMap tmap_q, const __gri
                 b = (b == 0) ? NB - 1 : b - 1;              // k += NB - 1
                 if (++jm == NB) { jm = 0; ph ^= 1; }
             }
+            if (tid == 0) F4S_MARK(5);
             if (ok) ok = mbar_wait(smem_u32(&bar_o_final[t]), 0, abort_p, args.status, SITE_G_O, t);
             ok = __all_sync(0xffffffffu, ok);
+            if (tid == 0) F4S_MARK(6);
             if (ok) {
                 tc_fence_after_sync();
                 const float inv = 1.f / l_run;
@@ -325,8 +368,10 @@ fused4s_attention_kernel(const __grid_constant__ CUtensorMap tmap_q, const __gri
     }
 
     // ------------------------------------------------------------ teardown (every thread arrives)
+    if (tid == 0) F4S_MARK(7);
     tc_fence_before_sync();
     __syncthreads();
+    if (tid == 0) F4S_MARK(8);
     if (warp == 16 && lane == 0 && abort_flag) {
         for (int s = 0; s < F4_STAGES; ++s) mbar_drain(smem_u32(&bar_kv_full[s]), 0);
     }
@@ -335,6 +380,14 @@ fused4s_attention_kernel(const __grid_constant__ CUtensorMap tmap_q, const __gri
         __syncwarp();
         tmem_dealloc(tmem_base, 512);
     }
+#ifdef SD_ATTN_TRACE
+    if (args.trace && tid == 0) {
+        unsigned long long gt;
+        asm volatile("mov.u64 %0, %globaltimer;" : "=l"(gt));
+        const int cta = blockIdx.y * gridDim.x + blockIdx.x;
+        if (cta < 256) args.trace[5 * 40 * 8 + cta * 4 + 1] = (long long)gt;
+    }
+#endif
 }
 
 }  // namespace sd_attn

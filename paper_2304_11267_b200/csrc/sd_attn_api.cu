@@ -57,6 +57,7 @@ struct sd_attn_handle {
     int fused4_ok;            // the register hand-over inside these kernels fits their launch allocation
     int fused4s_ok;
     int no_spare;             // SD_ATTN_FUSED_NO_SPARE=1: the four-tile kernel without the spare score buffer
+    int fused4_tiles_override;   // SD_ATTN_FUSED_TILES=1..4: fixed query tiles per CTA of the spare-buffer kernel (tests)
     int cross2_four_ok;
     int cross_one_tile_only;  // SD_ATTN_CROSS_ONE_TILE=1: never use the persistent cross-attention kernel
     int prefer_two_tile;      // SD_ATTN_FUSED_TWO_TILE=1: use the two-tile fused kernel for every head dim
@@ -124,6 +125,8 @@ extern "C" int sd_attn_create(sd_attn_handle** out) {
     h->cross_one_tile_only = (one && one[0] == '1') ? 1 : 0;
     const char* nsp = getenv("SD_ATTN_FUSED_NO_SPARE");
     h->no_spare = (nsp && nsp[0] == '1') ? 1 : 0;
+    const char* ftl = getenv("SD_ATTN_FUSED_TILES");
+    h->fused4_tiles_override = (ftl && ftl[0] >= '1' && ftl[0] <= '4' && !ftl[1]) ? ftl[0] - '0' : 0;
     const char* two = getenv("SD_ATTN_FUSED_TWO_TILE");
     h->prefer_two_tile = (two && two[0] == '1') ? 1 : 0;
 
@@ -373,10 +376,27 @@ static int launch_fused4(sd_attn_handle* h, const Problem& p) {
     if (rc == SD_ATTN_OK) rc = make_tmap(h, &tv, p.v, p.BH, p.Nk, p.d, F4_BN);
     if (rc != SD_ATTN_OK) return rc;
     dim3 grid((p.Nq + F4_TILES * TILE_M - 1) / (F4_TILES * TILE_M), p.BH), block(F4_THREADS);
-    if (a.dpad <= F4S_MAX_DPAD && h->fused4s_ok && !h->no_spare)
+    a.tiles_per_cta = F4_TILES;
+    if (a.dpad <= F4S_MAX_DPAD && h->fused4s_ok && !h->no_spare) {
+        // Tiles per CTA: the fewest waves of CTAs times the cost of one key-tile step of a CTA with that many tiles
+        // (clocks, measured: four tiles share the exponential unit, one tile alone is bound by its hand-off chain).
+        static const int step_cost[F4_TILES + 1] = {0, 1000, 1400, 1900, 2400};
+        const int tiles_per_head = (p.Nq + TILE_M - 1) / TILE_M;
+        long best = -1;
+        for (int tpc = 1; tpc <= F4_TILES; ++tpc) {
+            const long ctas = (long)((tiles_per_head + tpc - 1) / tpc) * p.BH;
+            const long cost = ((ctas + h->sm_count - 1) / h->sm_count) * step_cost[tpc];
+            if (best < 0 || cost < best) {
+                best = cost;
+                a.tiles_per_cta = tpc;
+            }
+        }
+        if (h->fused4_tiles_override > 0) a.tiles_per_cta = h->fused4_tiles_override;
+        grid.x = (tiles_per_head + a.tiles_per_cta - 1) / a.tiles_per_cta;
         fused4s_attention_kernel<<<grid, block, fused4_smem_bytes(), p.stream>>>(tq, tk, tv, a);
-    else
+    } else {
         fused4_attention_kernel<<<grid, block, fused4_smem_bytes(), p.stream>>>(tq, tk, tv, a);
+    }
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) return cuda_fail(h, e);
     h->launches += 1;

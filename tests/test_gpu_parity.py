@@ -276,6 +276,33 @@ def test_running_anchor_follows_scores_that_grow_along_the_keys(att, bd, d, orde
         check(run(att, bd, mode, q, k, v, scale), ref, v, what="%s d=%d mode %s" % (order, d, bd.MODE_NAMES[mode]))
 
 
+@pytest.mark.parametrize("env", [{"SD_ATTN_FUSED_TILES": "1"}, {"SD_ATTN_FUSED_TILES": "2"}, {"SD_ATTN_FUSED_TILES": "3"},
+                                 {"SD_ATTN_FUSED_TILES": "4"}, {"SD_ATTN_FUSED_NO_SPARE": "1"},
+                                 {"SD_ATTN_FUSED_TWO_TILE": "1"}],
+                         ids=lambda e: "-".join("%s=%s" % kv for kv in e.items()))
+def test_every_variant_of_the_small_head_dim_kernel(bd, env, monkeypatch):
+    """The d <= 48 path picks 1 to 4 query tiles per CTA by problem size and has two fallbacks; force each of them.
+
+    Shapes: ragged in rows and keys, more key tiles than the K/V ring has stages (so stages are reused), and both
+    fewer and more query tiles per head than a CTA takes.
+    """
+    for k, v in env.items():
+        monkeypatch.setenv(k, v)
+    a = bd.Attention()        # the variant switches are read when the handle is created
+    try:
+        for n, (B, H, Nq, Nk, d, qmult) in enumerate([(1, 2, 600, 1100, 40, 1.0), (2, 1, 129, 700, 40, 4.0),
+                                                       (1, 1, 1300, 130, 24, 1.0)]):
+            q, k, v = rand_qkv(4100 + n, B, H, Nq, Nk, d, qmult=qmult)
+            scale = float(np.float32(1.0 / np.sqrt(d)))
+            ref, _, _ = oracle.forward(q, k, v, scale)
+            a.set_mode(bd.MODE_FUSED)
+            out = a.forward(gpu(q), gpu(k), gpu(v), scale=scale)
+            a.check()
+            check(out.cpu().numpy(), ref, v, what="%s shape %d" % (env, n))
+    finally:
+        a.close()
+
+
 def test_padding_rows_with_distinct_values_only_see_their_mean(att, bd):
     call = workloads.config3()[0]
     q, k, v = workloads.make_inputs(call)
