@@ -42,6 +42,8 @@ struct Fused4Args {
     int Nq, Nk, d;
     int dpad;     // d rounded up to 16 (<= 64)
     int tiles_per_cta;   // spare-buffer kernel only: 1..4 query tiles per CTA (small problems spread over more SMs)
+    int nch;             // spare-buffer kernel only: 64-column chunks per row (1..3)
+    int stages;          // spare-buffer kernel only: K/V ring depth (2..8)
     float scale_log2e;
     int negate;
     int* status;

@@ -1,5 +1,7 @@
-// Fused single-pass attention for head dims up to 48 (the d = 40 layers of the UNet): the four-tile kernel
-// of fused4_kernel.cuh with one SPARE score buffer that takes the tensor-core round trip off the softmax's path.
+// Fused single-pass attention with one SPARE score buffer that takes the tensor-core round trip off the
+// softmax's path: T query tiles per CTA share T + 1 score buffers.  T is at most 4 at d <= 48 (the d = 40 layers of
+// the UNet), 3 at d <= 80, 2 at d <= 160: (T + 1) * 64 score columns and T * dpad output columns fill the 512
+// columns of tensor memory.
 //
 // In the four-tile kernel the weights P_t(j) overwrite the scores S_t(j), so S_t(j+1) can only follow the
 // product P_t(j) V(j): after every key tile a softmax warpgroup idles for the round trip softmax -> MMA issue ->
@@ -39,7 +41,13 @@ namespace sd_attn {
 #define F4S_MARK(i) do { } while (0)
 #endif
 
-constexpr int F4S_MAX_DPAD = 48;
+constexpr int F4S_MAX_DPAD = 160;
+constexpr int F4S_MAX_KSTEPS = 10;          // MMA steps of Q K^T at the largest head dim
+constexpr int F4S_SMEM_BUDGET = 220 * 1024;
+__host__ inline int f4s_max_tiles(int dpad) {   // (T + 1) * 64 + T * dpad <= 512
+    const int t = (512 - F4_BN) / (F4_BN + dpad);
+    return t > F4_TILES ? F4_TILES : t;
+}
 // Of every 8 exponentials this many are evaluated by the degree-3 polynomial on the FMA pipe instead of the
 // special function unit, which is the busiest unit of this kernel (measured: 0 -> 100 us, 2 -> 95 us, 3 -> 96 us on
 // the 4096-token d = 40 call).
@@ -51,6 +59,7 @@ constexpr int F4S_BUFFERS = F4_TILES + 1;
 constexpr int F4S_SOFTMAX_REGS = 104;   // 512 * 104 + 256 * 32 = 768 * 80, the launch allocation
 constexpr int F4S_CONTROL_REGS = 32;
 
+template <int POLY, int NCH>   // NCH: 64-column chunks per row (head dim <= 64 * NCH)
 __global__ void __launch_bounds__(F4_THREADS, 1)
 fused4s_attention_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__ CUtensorMap tmap_k,
                          const __grid_constant__ CUtensorMap tmap_v, const Fused4Args args) {
@@ -84,12 +93,14 @@ fused4s_attention_kernel(const __grid_constant__ CUtensorMap tmap_q, const __gri
     const int NB = T + 1;                                 // score buffers in the rotation
     const int n_kv = (args.Nk + BN - 1) / BN;
     const int dpad = args.dpad;
+    constexpr int nch = NCH;
+    const int stages = args.stages;   // K/V ring depth
 
     const uint32_t smem_base = (smem_u32(f4s_smem_raw) + 1023u) & ~1023u;
-    constexpr uint32_t q_tile_bytes = TILE_M * CHUNK_ROW_BYTES;     // one 64-column chunk (d <= 48)
-    constexpr uint32_t kv_tile_bytes = BN * CHUNK_ROW_BYTES;
-    const uint32_t q_smem = smem_base;                              // [4][128 rows][128 B]
-    const uint32_t kv_smem = q_smem + F4_TILES * q_tile_bytes;      // [stages][K | V][64 rows][128 B]
+    constexpr uint32_t q_tile_bytes = nch * TILE_M * CHUNK_ROW_BYTES;   // [chunk][128 rows][128 B]
+    constexpr uint32_t kv_tile_bytes = nch * BN * CHUNK_ROW_BYTES;      // [chunk][64 rows][128 B]
+    const uint32_t q_smem = smem_base;                              // [tiles per CTA] query tiles
+    const uint32_t kv_smem = q_smem + args.tiles_per_cta * q_tile_bytes;   // [stages][K | V]
     volatile int* abort_p = &abort_flag;
 
     if (tid == 0) {
@@ -118,7 +129,7 @@ fused4s_attention_kernel(const __grid_constant__ CUtensorMap tmap_q, const __gri
     tc_fence_after_sync();
     if (tid == 0) F4S_MARK(0);
     const uint32_t tmem_base = tmem_base_slot;
-    const uint32_t tmem_o0 = tmem_base + F4S_BUFFERS * BN;   // columns: five score buffers | O_0..O_3
+    const uint32_t tmem_o0 = tmem_base + (args.tiles_per_cta + 1) * BN;   // columns: the score buffers | O_0 .. O_{T-1}
 
     // One setmaxnreg site per kind, executed by whole warpgroups; the budget is the CTA's launch allocation.
     if (warp >= 16) setmaxnreg_dec<F4S_CONTROL_REGS>();
@@ -133,19 +144,23 @@ fused4s_attention_kernel(const __grid_constant__ CUtensorMap tmap_q, const __gri
             auto load_q = [&](int t) {
                 const uint32_t bar = smem_u32(&bar_q_full[t]);
                 mbar_arrive_expect_tx(bar, q_tile_bytes);
-                tma_load_3d(q_smem + t * q_tile_bytes, &tmap_q, bar, 0, row_base + t * TILE_M, bh);
+                for (int ch = 0; ch < nch; ++ch)
+                    tma_load_3d(q_smem + t * q_tile_bytes + ch * TILE_M * CHUNK_ROW_BYTES, &tmap_q, bar, ch * CHUNK_COLS,
+                                row_base + t * TILE_M, bh);
             };
             load_q(0);
-            for (int j = 0; j < n_kv; ++j) {
-                const int s = j % F4_STAGES;
-                if (j >= F4_STAGES && !mbar_wait(smem_u32(&bar_kv_empty[s]), ((j / F4_STAGES) - 1) & 1, abort_p,
-                                                 args.status, SITE_G_EMPTY, j))
+            int s = 0, pe = 1;   // stage of key tile j; parity of the kv_empty phase that frees it (from j = stages on)
+            for (int j = 0; j < n_kv; ++j, ++s) {
+                if (s == stages) { s = 0; pe ^= 1; }
+                if (j >= stages && !mbar_wait(smem_u32(&bar_kv_empty[s]), pe, abort_p, args.status, SITE_G_EMPTY, j))
                     break;
                 const uint32_t k_dst = kv_smem + s * 2 * kv_tile_bytes, v_dst = k_dst + kv_tile_bytes;
                 const uint32_t bar = smem_u32(&bar_kv_full[s]);
                 mbar_arrive_expect_tx(bar, 2 * kv_tile_bytes);
-                tma_load_3d(k_dst, &tmap_k, bar, 0, j * BN, bh);
-                tma_load_3d(v_dst, &tmap_v, bar, 0, j * BN, bh);
+                for (int ch = 0; ch < nch; ++ch)
+                    tma_load_3d(k_dst + ch * BN * CHUNK_ROW_BYTES, &tmap_k, bar, ch * CHUNK_COLS, j * BN, bh);
+                for (int ch = 0; ch < nch; ++ch)
+                    tma_load_3d(v_dst + ch * BN * CHUNK_ROW_BYTES, &tmap_v, bar, ch * CHUNK_COLS, j * BN, bh);
                 if (j == 0)
                     for (int t = 1; t < T; ++t) load_q(t);
             }
@@ -161,7 +176,7 @@ fused4s_attention_kernel(const __grid_constant__ CUtensorMap tmap_q, const __gri
         if (t < T && elect_one()) {
             const uint32_t idesc_s = idesc_f16(TILE_M, BN, false, false, args.negate != 0);
             const uint32_t idesc_o = idesc_f16(TILE_M, dpad, false, true, false);
-            const int ksteps_s = (args.d + 15) / 16;   // <= 3: inside one swizzled 64-column chunk
+            const int ksteps_s = (args.d + 15) / 16;   // 16 columns each; four to a swizzled 64-column chunk
             const int tn = (t + 1 == T) ? 0 : t + 1;   // the tile whose scores this thread requests
             const uint64_t q_desc = smem_desc_sw128(q_smem + tn * q_tile_bytes, 16, 1024);
             const uint64_t q_desc_own = smem_desc_sw128(q_smem + t * q_tile_bytes, 16, 1024);
@@ -171,16 +186,18 @@ fused4s_attention_kernel(const __grid_constant__ CUtensorMap tmap_q, const __gri
             const uint32_t tmem_o = tmem_o0 + t * dpad;
             const uint32_t b_pvdone = smem_u32(&bar_pv_done[t]);
 
-            auto issue_s = [&](uint64_t qd, int tile, int j, int b) {   // scores of (tile, key tile j) into buffer b
-                const uint64_t kd = k_desc0 + (uint64_t)((j % F4_STAGES) * stage_off);
+            auto issue_s = [&](uint64_t qd, int tile, int st, int b) {   // scores of (tile, K in stage st) into buffer b
+                const uint64_t kd = k_desc0 + (uint64_t)(st * stage_off);
                 const uint32_t ts = tmem_base + b * BN;
 #pragma unroll
-                for (int kk = 0; kk < 3; ++kk)
-                    if (kk < ksteps_s) mma_f16_ss(ts, qd + (uint64_t)(kk * 2), kd + (uint64_t)(kk * 2), idesc_s, kk > 0);
+                for (int kk = 0; kk < 4 * NCH; ++kk)
+                    if (kk < ksteps_s)
+                        mma_f16_ss(ts, qd + (uint64_t)(((kk >> 2) * TILE_M * CHUNK_ROW_BYTES + (kk & 3) * 32) >> 4),
+                                   kd + (uint64_t)(((kk >> 2) * BN * CHUNK_ROW_BYTES + (kk & 3) * 32) >> 4), idesc_s, kk > 0);
                 tc_commit(smem_u32(&bar_s_full[tile][b]));
             };
-            auto issue_o = [&](int j, int b) {   // O_t (+)= P V(j), P in the first 32 columns of score buffer b
-                const uint64_t vd = v_desc0 + (uint64_t)((j % F4_STAGES) * stage_off);
+            auto issue_o = [&](int j, int st, int b) {   // O_t (+)= P V(j), V in stage st, P in the first 32 columns of buffer b
+                const uint64_t vd = v_desc0 + (uint64_t)(st * stage_off);
                 const uint32_t tp = tmem_base + b * BN;
 #pragma unroll
                 for (int kk = 0; kk < BN / 16; ++kk)
@@ -193,13 +210,13 @@ fused4s_attention_kernel(const __grid_constant__ CUtensorMap tmap_q, const __gri
                 // the first T+1 steps fill the buffers: step t (own tile, key tile 0) into buffer t; the last issuer
                 // also requests step T (tile 0, key tile 1) into the spare buffer T
                 tc_fence_after_sync();
-                issue_s(q_desc_own, t, 0, t);
+                issue_s(q_desc_own, t, 0, t);   // stage 0
                 ok = mbar_wait(smem_u32(&bar_q_full[tn]), 0, abort_p, args.status, SITE_G_Q, tn);
                 if (ok && t == T - 1 && n_kv > 1) {
-                    ok = mbar_wait(smem_u32(&bar_kv_full[1]), 0, abort_p, args.status, SITE_G_KV, 1);
+                    ok = mbar_wait(smem_u32(&bar_kv_full[1]), 0, abort_p, args.status, SITE_G_KV, 1);   // stages >= 2
                     if (ok) {
                         tc_fence_after_sync();
-                        issue_s(q_desc, tn, 1, T);
+                        issue_s(q_desc, tn, 1, T);   // stage 1
                     }
                 }
             }
@@ -207,25 +224,28 @@ fused4s_attention_kernel(const __grid_constant__ CUtensorMap tmap_q, const __gri
             // warps); it requests step k + NB = (tn, jn) into the same buffer
             int b = t, ph = 0, jm = 0;
             const int jn_off = (t + 1 == T) ? 2 : 1;
+            int sj = 0;                                 // stage of key tile j
+            int sn = jn_off % stages, pn = (jn_off / stages) & 1;   // stage and phase of key tile jn = j + jn_off
             for (int j = 0; j < n_kv && ok; ++j) {
                 const int jn = j + jn_off;
                 const bool more = jn < n_kv;
                 if (more)   // landed long ago: keep this wait off the critical path
-                    ok = mbar_wait(smem_u32(&bar_kv_full[jn % F4_STAGES]), (jn / F4_STAGES) & 1, abort_p, args.status,
-                                   SITE_G_KV, jn);
+                    ok = mbar_wait(smem_u32(&bar_kv_full[sn]), pn, abort_p, args.status, SITE_G_KV, jn);
                 if (t == 0) FUSED_TRACE(4, j, 0);
                 if (ok) ok = mbar_wait(smem_u32(&bar_p_full[t][b]), ph, abort_p, args.status, SITE_G_P, j);
                 if (!ok) break;
                 tc_fence_after_sync();
                 if (t == 0) FUSED_TRACE(4, j, 1);
-                issue_o(j, b);
-                if (more) issue_s(q_desc, tn, jn, b);               // into the buffer P is read from: behind it, in order
+                issue_o(j, sj, b);
+                if (more) issue_s(q_desc, tn, sn, b);               // into the buffer P is read from: behind it, in order
                 tc_commit(b_pvdone);                                // O_t holds key tiles 0..j
-                tc_commit(smem_u32(&bar_kv_empty[j % F4_STAGES]));  // this issuer is done with K(j), V(j)
+                tc_commit(smem_u32(&bar_kv_empty[sj]));             // this issuer is done with K(j), V(j)
                 if (j == n_kv - 1) tc_commit(smem_u32(&bar_o_final[t]));
                 if (t == 0) FUSED_TRACE(4, j, 2);
                 b = (b == 0) ? NB - 1 : b - 1;              // k += NB - 1
                 if (++jm == NB) { jm = 0; ph ^= 1; }
+                if (++sj == stages) sj = 0;
+                if (++sn == stages) { sn = 0; pn ^= 1; }
             }
         }
     } else if (warp < 16) {
@@ -274,8 +294,8 @@ fused4s_attention_kernel(const __grid_constant__ CUtensorMap tmap_q, const __gri
                         const uint64_t c2c2 = pack_b64(__float_as_uint(c2), __float_as_uint(c2));
                         const uint64_t nmnm = pack_b64(__float_as_uint(neg_mc), __float_as_uint(neg_mc));
                         uint64_t acc[2] = {0ull, 0ull};
-                        exp2_pack_32<F4S_POLY_PER8>(&s[0], c2c2, nmnm, &packed[0], acc);
-                        exp2_pack_32<F4S_POLY_PER8>(&s[32], c2c2, nmnm, &packed[16], acc);
+                        exp2_pack_32<POLY>(&s[0], c2c2, nmnm, &packed[0], acc);
+                        exp2_pack_32<POLY>(&s[32], c2c2, nmnm, &packed[16], acc);
                         tile_sum = sum_f32x2(acc[0], acc[1]);
                     } else {
                         tile_sum = 0.f;

@@ -60,6 +60,7 @@ struct FusedArgs {
     int dpad;     // d rounded up to 16
     int nch;      // 64-column chunks per row
     int stages;   // K/V ring depth
+    int tiles_per_cta;   // 1 or 2 query tiles per CTA (one when the problem has too few tiles to fill the SMs)
     float scale_log2e;
     int negate;
     int* status;
@@ -96,6 +97,7 @@ __host__ inline void fused_fill_args(FusedArgs* a, __half* out, int Nq, int Nk, 
     a->scale_log2e = scale_log2e;
     a->negate = negate ? 1 : 0;
     a->status = status;
+    a->tiles_per_cta = 2;
 }
 
 __host__ inline size_t fused_smem_bytes(const FusedArgs& a) {
@@ -122,8 +124,8 @@ fused_attention_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int bh = blockIdx.y;
-    const int row_base = blockIdx.x * 2 * TILE_M;
-    const int n_qtiles = (row_base + TILE_M < args.Nq) ? 2 : 1;
+    const int row_base = blockIdx.x * args.tiles_per_cta * TILE_M;
+    const int n_qtiles = (args.tiles_per_cta == 2 && row_base + TILE_M < args.Nq) ? 2 : 1;
     const int n_kv = (args.Nk + BN - 1) / BN;
     const int nch = args.nch, dpad = args.dpad, stages = args.stages;
 

@@ -138,7 +138,10 @@ extern "C" int sd_attn_create(sd_attn_handle** out) {
     if (e == cudaSuccess) e = raise_smem_limit(fused_attention_kernel<128>, fused_smem_bytes_max());
     if (e == cudaSuccess) e = raise_smem_limit(fused_attention_kernel<64>, fused_smem_bytes_max());
     if (e == cudaSuccess) e = raise_smem_limit(fused4_attention_kernel, fused4_smem_bytes());
-    if (e == cudaSuccess) e = raise_smem_limit(fused4s_attention_kernel, fused4_smem_bytes());
+    if (e == cudaSuccess) e = raise_smem_limit(fused4s_attention_kernel<F4S_POLY_PER8, 1>, F4S_SMEM_BUDGET + 1024);
+    if (e == cudaSuccess) e = raise_smem_limit(fused4s_attention_kernel<0, 1>, F4S_SMEM_BUDGET + 1024);
+    if (e == cudaSuccess) e = raise_smem_limit(fused4s_attention_kernel<0, 2>, F4S_SMEM_BUDGET + 1024);
+    if (e == cudaSuccess) e = raise_smem_limit(fused4s_attention_kernel<0, 3>, F4S_SMEM_BUDGET + 1024);
     if (e == cudaSuccess) e = raise_smem_limit(twopass_scores_kernel, twopass_scores_smem_bytes(3));
     if (e == cudaSuccess) e = raise_smem_limit(twopass_pv_kernel, twopass_pv_smem_bytes(3));
     if (e == cudaSuccess) e = raise_smem_limit(simt_attention_kernel<float, 5>, simt_smem_bytes(160));
@@ -151,9 +154,13 @@ extern "C" int sd_attn_create(sd_attn_handle** out) {
         e = cudaFuncGetAttributes(&fa, fused4_attention_kernel);
         if (e == cudaSuccess)
             h->fused4_ok = F4_THREADS * fa.numRegs >= 512 * F4_SOFTMAX_REGS + 256 * F4_CONTROL_REGS;
-        if (e == cudaSuccess) e = cudaFuncGetAttributes(&fa, fused4s_attention_kernel);
-        if (e == cudaSuccess)
-            h->fused4s_ok = F4_THREADS * fa.numRegs >= 512 * F4S_SOFTMAX_REGS + 256 * F4S_CONTROL_REGS;
+        h->fused4s_ok = 1;
+        const void* f4s[4] = {(const void*)fused4s_attention_kernel<F4S_POLY_PER8, 1>, (const void*)fused4s_attention_kernel<0, 1>,
+                              (const void*)fused4s_attention_kernel<0, 2>, (const void*)fused4s_attention_kernel<0, 3>};
+        for (int i = 0; i < 4 && e == cudaSuccess; ++i) {
+            e = cudaFuncGetAttributes(&fa, f4s[i]);
+            if (e == cudaSuccess && F4_THREADS * fa.numRegs < 512 * F4S_SOFTMAX_REGS + 256 * F4S_CONTROL_REGS) h->fused4s_ok = 0;
+        }
         if (e == cudaSuccess) e = cudaFuncGetAttributes(&fa, cross2_attention_kernel<4>);
         if (e == cudaSuccess)
             h->cross2_four_ok = cross2_threads(4) * fa.numRegs >= 512 * X2_SOFTMAX_REGS + 128 * X2_CONTROL_REGS;
@@ -377,26 +384,65 @@ static int launch_fused4(sd_attn_handle* h, const Problem& p) {
     if (rc != SD_ATTN_OK) return rc;
     dim3 grid((p.Nq + F4_TILES * TILE_M - 1) / (F4_TILES * TILE_M), p.BH), block(F4_THREADS);
     a.tiles_per_cta = F4_TILES;
-    if (a.dpad <= F4S_MAX_DPAD && h->fused4s_ok && !h->no_spare) {
-        // Tiles per CTA: the fewest waves of CTAs times the cost of one key-tile step of a CTA with that many tiles
-        // (clocks, measured: four tiles share the exponential unit, one tile alone is bound by its hand-off chain).
-        static const int step_cost[F4_TILES + 1] = {0, 1000, 1400, 1900, 2400};
-        const int tiles_per_head = (p.Nq + TILE_M - 1) / TILE_M;
-        long best = -1;
-        for (int tpc = 1; tpc <= F4_TILES; ++tpc) {
-            const long ctas = (long)((tiles_per_head + tpc - 1) / tpc) * p.BH;
-            const long cost = ((ctas + h->sm_count - 1) / h->sm_count) * step_cost[tpc];
-            if (best < 0 || cost < best) {
-                best = cost;
-                a.tiles_per_cta = tpc;
-            }
+    a.nch = 1;
+    a.stages = F4_STAGES;
+    fused4_attention_kernel<<<grid, block, fused4_smem_bytes(), p.stream>>>(tq, tk, tv, a);
+    cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess) return cuda_fail(h, e);
+    h->launches += 1;
+    return SD_ATTN_OK;
+}
+
+// The spare-buffer kernel: any head dim up to 160, 1..4 query tiles per CTA.
+static int launch_fused4s(sd_attn_handle* h, const Problem& p) {
+    Fused4Args a;
+    a.out = (__half*)p.out;
+    a.Nq = p.Nq; a.Nk = p.Nk; a.d = p.d;
+    a.dpad = (p.d + 15) / 16 * 16;
+    a.nch = (p.d + CHUNK_COLS - 1) / CHUNK_COLS;
+    a.scale_log2e = fabsf(p.scale) * LOG2E;
+    a.negate = p.scale < 0.f;
+    a.status = h->dev_status;
+#ifdef SD_ATTN_TRACE
+    a.trace = (long long*)h->trace;
+#endif
+    const int q_tile_bytes = a.nch * TILE_M * CHUNK_ROW_BYTES, stage_bytes = 2 * a.nch * F4_BN * CHUNK_ROW_BYTES;
+    // Tiles per CTA: the fewest waves of CTAs times the cost of one key-tile step of a CTA with that many tiles
+    // (clocks, measured at d = 40: four tiles share the exponential unit, one tile alone is bound by its hand-off
+    // chain), among the counts tensor memory and shared memory (at least two K/V stages) have room for.
+    static const int step_cost[F4_TILES + 1] = {0, 1000, 1400, 1900, 2400};
+    const int tiles_per_head = (p.Nq + TILE_M - 1) / TILE_M;
+    int max_tiles = f4s_max_tiles(a.dpad);
+    while (max_tiles > 1 && F4S_SMEM_BUDGET - max_tiles * q_tile_bytes < 2 * stage_bytes) --max_tiles;
+    long best = -1;
+    a.tiles_per_cta = 1;
+    for (int tpc = 1; tpc <= max_tiles; ++tpc) {
+        const long ctas = (long)((tiles_per_head + tpc - 1) / tpc) * p.BH;
+        const long cost = ((ctas + h->sm_count - 1) / h->sm_count) * step_cost[tpc];
+        if (best < 0 || cost < best) {
+            best = cost;
+            a.tiles_per_cta = tpc;
         }
-        if (h->fused4_tiles_override > 0) a.tiles_per_cta = h->fused4_tiles_override;
-        grid.x = (tiles_per_head + a.tiles_per_cta - 1) / a.tiles_per_cta;
-        fused4s_attention_kernel<<<grid, block, fused4_smem_bytes(), p.stream>>>(tq, tk, tv, a);
-    } else {
-        fused4_attention_kernel<<<grid, block, fused4_smem_bytes(), p.stream>>>(tq, tk, tv, a);
     }
+    if (h->fused4_tiles_override > 0 && h->fused4_tiles_override <= max_tiles) a.tiles_per_cta = h->fused4_tiles_override;
+    a.stages = (F4S_SMEM_BUDGET - a.tiles_per_cta * q_tile_bytes) / stage_bytes;
+    if (a.stages > F4_STAGES) a.stages = F4_STAGES;
+    const size_t smem = (size_t)a.tiles_per_cta * q_tile_bytes + (size_t)a.stages * stage_bytes + 1024;
+    CUtensorMap tq, tk, tv;
+    int rc = make_tmap(h, &tq, p.q, p.BH, p.Nq, p.d, TILE_M);
+    if (rc == SD_ATTN_OK) rc = make_tmap(h, &tk, p.k, p.BH, p.Nk, p.d, F4_BN);
+    if (rc == SD_ATTN_OK) rc = make_tmap(h, &tv, p.v, p.BH, p.Nk, p.d, F4_BN);
+    if (rc != SD_ATTN_OK) return rc;
+    dim3 grid((tiles_per_head + a.tiles_per_cta - 1) / a.tiles_per_cta, p.BH), block(F4_THREADS);
+    // the polynomial share of the exponentials only pays where four tiles saturate the special function unit
+    if (a.dpad <= 48)
+        fused4s_attention_kernel<F4S_POLY_PER8, 1><<<grid, block, smem, p.stream>>>(tq, tk, tv, a);
+    else if (a.nch == 1)
+        fused4s_attention_kernel<0, 1><<<grid, block, smem, p.stream>>>(tq, tk, tv, a);
+    else if (a.nch == 2)
+        fused4s_attention_kernel<0, 2><<<grid, block, smem, p.stream>>>(tq, tk, tv, a);
+    else
+        fused4s_attention_kernel<0, 3><<<grid, block, smem, p.stream>>>(tq, tk, tv, a);
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) return cuda_fail(h, e);
     h->launches += 1;
@@ -404,6 +450,7 @@ static int launch_fused4(sd_attn_handle* h, const Problem& p) {
 }
 
 static int launch_fused(sd_attn_handle* h, const Problem& p) {
+    if (h->fused4s_ok && !h->no_spare && !h->prefer_two_tile) return launch_fused4s(h, p);
     if (p.d <= F4_MAX_D && !h->prefer_two_tile && h->fused4_ok) return launch_fused4(h, p);
     FusedArgs a;
     const int bn = fused_block_n(p.d);
@@ -416,7 +463,11 @@ static int launch_fused(sd_attn_handle* h, const Problem& p) {
     if (rc == SD_ATTN_OK) rc = make_tmap(h, &tk, p.k, p.BH, p.Nk, p.d, bn);
     if (rc == SD_ATTN_OK) rc = make_tmap(h, &tv, p.v, p.BH, p.Nk, p.d, bn);
     if (rc != SD_ATTN_OK) return rc;
-    dim3 grid((p.Nq + 2 * TILE_M - 1) / (2 * TILE_M), p.BH), block(FUSED_THREADS);
+    // two query tiles per CTA share the K/V loads; a problem that would leave SMs idle that way takes one per CTA
+    // (measured: 24 -> 22.8 us at 1024 tokens d = 80; at d = 160, 256 tokens, one per CTA is slower, 13.5 -> 15.4 us)
+    const int tiles_per_head = (p.Nq + TILE_M - 1) / TILE_M;
+    a.tiles_per_cta = ((long)((tiles_per_head + 1) / 2) * p.BH >= h->sm_count || a.dpad > 96) ? 2 : 1;
+    dim3 grid((tiles_per_head + a.tiles_per_cta - 1) / a.tiles_per_cta, p.BH), block(FUSED_THREADS);
     if (bn == 128)
         fused_attention_kernel<128><<<grid, block, fused_smem_bytes(a), p.stream>>>(tq, tk, tv, a);
     else
