@@ -302,7 +302,11 @@ fused4s_attention_kernel(const __grid_constant__ CUtensorMap tmap_q, const __gri
                         exp2_pack_32_masked(&s[0], c2, neg_mc, 0, valid, &packed[0], tile_sum);
                         exp2_pack_32_masked(&s[32], c2, neg_mc, 32, valid, &packed[16], tile_sum);
                     }
+#ifdef SD_ATTN_X_NORARE
+                    const bool over = false;
+#else
                     const bool over = !(tile_sum <= FUSED_TILE_SUM_LIMIT);
+#endif
                     if (attempt == 1 || !__any_sync(0xffffffffu, over)) break;
                     // Rare: a row of this warp met a score far above its anchor.  O_t may be touched once the P V
                     // product of key tile j-1 has completed (that of j-2 has: see the wait before the hand-off below);

@@ -35,14 +35,16 @@ constexpr int FUSED_THREADS = 352;
 constexpr int FUSED_MAX_STAGES = 4;
 constexpr int FUSED_MAX_KSTEPS = 10;   // MMA steps of the Q K^T contraction at the largest head dim (160)
 constexpr int FUSED_SMEM_BUDGET = 220 * 1024;
-// The anchor of the exponent starts FUSED_HEADROOM_LOG2 above the first tile's row max (weights <= 2^-3,
-// still 11 bits below which binary16 stays normal) and O is rescaled only when a later row max exceeds
-// the anchor by more than FUSED_RESCALE_LOG2 (weights <= 2^12, far inside binary16's range).
+// The anchor of the exponent starts FUSED_HEADROOM_LOG2 above the first tile's row max (weights <= 2^-6: the
+// eight binades below that are still normal binary16, and what lies further down rounds without bias) and O is
+// rescaled only when a later row max exceeds the anchor by more than FUSED_RESCALE_LOG2 (weights <= 2^12, far
+// inside binary16's range).  Measured on the "peaked" inputs: headroom 3 re-anchors about one warp-tile in 130
+// and costs 3.5% of the 4096-token call; headroom 6 re-anchors almost never, with the same error.
 #ifndef SD_ATTN_RESCALE_LOG2
 #define SD_ATTN_RESCALE_LOG2 12.0f
 #endif
 #ifndef SD_ATTN_HEADROOM_LOG2
-#define SD_ATTN_HEADROOM_LOG2 3.0f
+#define SD_ATTN_HEADROOM_LOG2 6.0f
 #endif
 constexpr float FUSED_RESCALE_LOG2 = SD_ATTN_RESCALE_LOG2;
 constexpr float FUSED_HEADROOM_LOG2 = SD_ATTN_HEADROOM_LOG2;
