@@ -33,9 +33,9 @@ UNIT = "TFLOP/s"
 NOMINAL_FP16_TFLOPS = 2250.0
 ROTATING_SETS = 8   # 8 x 42 MB of q/k/v/out for the two variants = 336 MB, above the 126 MB L2
 # DRAM bytes per launch of the fused kernel on this workload: dram__bytes_read.sum + dram__bytes_write.sum of one
-# ncu capture (profiles/fused4_c2_self_4096_d40.md): 15.78 MB read (q, k, v once: 15.73 MB algorithmic) and
+# ncu capture (profiles/fused4s_c2_self_4096_d40.md): 15.79 MB read (q, k, v once: 15.73 MB algorithmic) and
 # nothing written during the launch -- the 5.2 MB of output are still in the 126 MB L2 when the kernel ends.
-FUSED_TRAFFIC_BYTES_PER_LAUNCH = 15776512
+FUSED_TRAFFIC_BYTES_PER_LAUNCH = 15790592
 
 
 def measured_peaks():
@@ -316,17 +316,18 @@ def run_ours(args):
     # the step's only kernel is the fused one, so its mean launch duration is the timed region / launches
     exps_per_launch = calls[0].B * calls[0].H * calls[0].Nq * calls[0].Nk
     sfu_peak = 16.0 * 148 * (clocks.get("sm_max_mhz") or 1965) * 1e6 / 1e12     # ex2: 16 per clock per SM
-    roofline = {"bound": "tensor", "kernel": "fused4_attention_kernel", "achieved": achieved,
+    roofline = {"bound": "tensor", "kernel": "fused4s_attention_kernel", "achieved": achieved,
                 "peak": peaks["tflops"], "unit": "TFLOP/s", "frac": achieved / peaks["tflops"],
                 "peak_source": "%s cuBLAS bf16 burst (fp16 peak = bf16 peak, nominal ratio 1.0)" % peaks["source"],
                 "frac_of_nominal_2250": achieved / NOMINAL_FP16_TFLOPS,
                 "traffic": FUSED_TRAFFIC_BYTES_PER_LAUNCH, "algorithmic_bytes": calls[0].io_bytes(),
                 "us_per_launch": per_launch_s * 1e6,
-                "note": "one exponential per score on the special-function unit (16/clk/SM, measured) caps this "
-                        "d=40 shape near 0.33 of the nominal tensor peak; see roofline_alu",
+                "note": "one exponential per score: the special-function unit alone (16/clk/SM, measured) would cap this "
+                        "d=40 shape at 0.33 of the nominal tensor peak; the kernel sends a quarter of them to the FMA pipe; "
+                        "see roofline_alu",
                 "roofline_alu": {"bound": "alu", "unit": "Texp/s", "achieved": exps_per_launch / per_launch_s / 1e12,
                                  "peak": sfu_peak, "frac": exps_per_launch / per_launch_s / 1e12 / sfu_peak,
-                                 "peak_source": "16 ex2/clk/SM x 148 SMs x max SM clock"}}
+                                 "peak_source": "16 ex2/clk/SM x 148 SMs x max SM clock (special-function unit only)"}}
     line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
             "warmup": max(args.warmup, 3), "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
             "vs_baseline": None, "dtype": "f16", "data": "synthetic", "config": workload_config(),
