@@ -100,7 +100,16 @@ cross2_attention_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid
     __shared__ int abort_flag;
 
     constexpr int LOADER_WARP = NWG * 4, S_ISSUER_WARP = NWG * 4 + 1, O_ISSUER_WARP = NWG * 4 + 2;
+#ifdef SD_ATTN_TRACE
+    if (args.trace && blockIdx.x == 0 && threadIdx.x == 0) {
+        unsigned long long gt;
+        asm volatile("mov.u64 %0, %globaltimer;" : "=l"(gt));
+        args.trace[((NWG + 1) * 40 + 39) * 8 + 1] = clock64();
+        args.trace[((NWG + 1) * 40 + 39) * 8 + 4] = (long long)gt;
+    }
+#endif
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    if (threadIdx.x == 0) pdl_launch_dependents();   // the next kernel of the stream may start its set-up
     const int nch = args.nch, dpad = args.dpad, stages = args.stages;
     // contiguous range of items for this CTA: consecutive items share a head, so K and V are fetched rarely
     const int per = args.n_items / gridDim.x, extra = args.n_items % gridDim.x;
@@ -139,6 +148,12 @@ cross2_attention_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid
     }
     tc_fence_before_sync();
     __syncthreads();
+    // Set-up (barriers, tensor memory) overlapped the tail of the previous kernel of the stream; global memory and
+    // every bounded wait come after it has completed.
+    pdl_wait();
+#ifdef SD_ATTN_TRACE
+    if (args.trace && blockIdx.x == 0 && threadIdx.x == 0) args.trace[((NWG + 1) * 40 + 39) * 8 + 2] = clock64();
+#endif
     tc_fence_after_sync();
     const uint32_t tmem_base = tmem_base_slot;
     const uint32_t tmem_o0 = tmem_base + NWG * X2_KN;   // columns: S_0 .. S_{NWG-1} | O_0 .. O_{NWG-1}
@@ -179,6 +194,9 @@ cross2_attention_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid
                     break;
                 X2_TRACE(NWG + 1, i, 0);
                 const uint32_t bar = smem_u32(&bar_full[s]), dst = q_smem + s * q_bytes;
+#ifdef SD_ATTN_X_NOQ
+                if (i >= stages) { mbar_arrive(bar); continue; }
+#endif
                 mbar_arrive_expect_tx(bar, q_bytes);
                 for (int ch = 0; ch < nch; ++ch)
                     tma_load_3d(dst + ch * TILE_M * CHUNK_ROW_BYTES, &tmap_q, bar, ch * CHUNK_COLS, tile * TILE_M, bh);
@@ -349,6 +367,14 @@ cross2_attention_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid
         __syncwarp();
         tmem_dealloc(tmem_base, 512);
     }
+#ifdef SD_ATTN_TRACE
+    if (args.trace && blockIdx.x == 0 && threadIdx.x == 0) {
+        unsigned long long gt;
+        asm volatile("mov.u64 %0, %globaltimer;" : "=l"(gt));
+        args.trace[((NWG + 1) * 40 + 39) * 8 + 3] = clock64();
+        args.trace[((NWG + 1) * 40 + 39) * 8 + 5] = (long long)gt;
+    }
+#endif
 }
 
 }  // namespace sd_attn

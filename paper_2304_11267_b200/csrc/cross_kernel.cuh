@@ -51,6 +51,7 @@ cross_attention_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_
     __shared__ int abort_flag;
 
     const int tid = threadIdx.x, warp = tid >> 5;
+    if (threadIdx.x == 0) pdl_launch_dependents();   // the next kernel of the stream may start its set-up
     const int tile = blockIdx.x, bh = blockIdx.y;
     const int row0 = tile * TILE_M;
     const int kn = args.kn, nch = args.nch, dpad = args.dpad;
@@ -80,6 +81,9 @@ cross_attention_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_
     tc_fence_before_sync();
     __syncthreads();
     tc_fence_after_sync();
+    // Set-up (barriers, tensor memory) overlapped the tail of the previous kernel of the stream; global memory and
+    // every bounded wait come after it has completed.
+    pdl_wait();
     const uint32_t tmem_base = tmem_base_slot;
     const uint32_t tmem_s = tmem_base;          // S: kn fp32 columns; P (packed fp16) reuses them
     const uint32_t tmem_o = tmem_base + kn;     // O: dpad fp32 columns

@@ -77,6 +77,7 @@ fused4s_attention_kernel(const __grid_constant__ CUtensorMap tmap_q, const __gri
 
     const int tid = threadIdx.x, lane = tid & 31;
     const int warp = __shfl_sync(0xffffffffu, tid >> 5, 0);   // warp-uniform for the compiler
+    if (threadIdx.x == 0) pdl_launch_dependents();   // the next kernel of the stream may start its set-up
     const int bh = blockIdx.y;
     const int row_base = blockIdx.x * args.tiles_per_cta * TILE_M;
 #ifdef SD_ATTN_TRACE
@@ -127,6 +128,9 @@ fused4s_attention_kernel(const __grid_constant__ CUtensorMap tmap_q, const __gri
     tc_fence_before_sync();
     __syncthreads();
     tc_fence_after_sync();
+    // Set-up (barriers, tensor memory) overlapped the tail of the previous kernel of the stream; global memory and
+    // every bounded wait come after it has completed.
+    pdl_wait();
     if (tid == 0) F4S_MARK(0);
     const uint32_t tmem_base = tmem_base_slot;
     const uint32_t tmem_o0 = tmem_base + (args.tiles_per_cta + 1) * BN;   // columns: the score buffers | O_0 .. O_{T-1}

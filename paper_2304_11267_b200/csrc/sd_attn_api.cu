@@ -56,6 +56,7 @@ struct sd_attn_handle {
     int sm_count;
     int fused4_ok;            // the register hand-over inside these kernels fits their launch allocation
     int fused4s_ok;
+    int no_pdl;               // SD_ATTN_NO_PDL=1: ordinary launches (no overlap of a kernel's set-up with its predecessor)
     int no_spare;             // SD_ATTN_FUSED_NO_SPARE=1: the four-tile kernel without the spare score buffer
     int fused4_tiles_override;   // SD_ATTN_FUSED_TILES=1..4: fixed query tiles per CTA of the spare-buffer kernel (tests)
     int cross2_four_ok;
@@ -83,6 +84,25 @@ static int cuda_fail(sd_attn_handle* h, cudaError_t e) {
     if (h) h->last_cuda_error = e;
     if (getenv("SD_ATTN_LOG")) fprintf(stderr, "[sd_attn] CUDA error: %s\n", cudaGetErrorString(e));
     return SD_ATTN_ERR_CUDA;
+}
+
+// Launch with the programmatic-stream-serialization attribute: the kernel may begin its set-up while the previous
+// kernel of the stream is still running and waits for it (griddepcontrol.wait) before it touches global memory.
+// Only the kernels that contain that wait are launched this way.
+template <typename... KArgs, typename... Args>
+static cudaError_t launch_overlapped(const sd_attn_handle* h, void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem,
+                                     cudaStream_t stream, Args&&... args) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid;
+    cfg.blockDim = block;
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = h->no_pdl ? 0 : 1;
+    return cudaLaunchKernelEx(&cfg, kernel, KArgs(args)...);
 }
 
 template <typename K>
@@ -123,6 +143,8 @@ extern "C" int sd_attn_create(sd_attn_handle** out) {
 #endif
     const char* one = getenv("SD_ATTN_CROSS_ONE_TILE");
     h->cross_one_tile_only = (one && one[0] == '1') ? 1 : 0;
+    const char* npd = getenv("SD_ATTN_NO_PDL");
+    h->no_pdl = (npd && npd[0] == '1') ? 1 : 0;
     const char* nsp = getenv("SD_ATTN_FUSED_NO_SPARE");
     h->no_spare = (nsp && nsp[0] == '1') ? 1 : 0;
     const char* ftl = getenv("SD_ATTN_FUSED_TILES");
@@ -328,11 +350,11 @@ static int launch_cross2(sd_attn_handle* h, const Problem& p) {
     if (groups >= 4 && !h->cross2_four_ok) groups = 3;
     const size_t smem = cross2_smem_bytes(a.nch);
     if (groups >= 4)
-        cross2_attention_kernel<4><<<grid, cross2_threads(4), smem, p.stream>>>(tq, tk, tv, a);
+        launch_overlapped(h, cross2_attention_kernel<4>, dim3(grid), dim3(cross2_threads(4)), smem, p.stream, tq, tk, tv, a);
     else if (groups == 3)
-        cross2_attention_kernel<3><<<grid, cross2_threads(3), smem, p.stream>>>(tq, tk, tv, a);
+        launch_overlapped(h, cross2_attention_kernel<3>, dim3(grid), dim3(cross2_threads(3)), smem, p.stream, tq, tk, tv, a);
     else
-        cross2_attention_kernel<2><<<grid, cross2_threads(2), smem, p.stream>>>(tq, tk, tv, a);
+        launch_overlapped(h, cross2_attention_kernel<2>, dim3(grid), dim3(cross2_threads(2)), smem, p.stream, tq, tk, tv, a);
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) return cuda_fail(h, e);
     h->launches += 1;
@@ -358,7 +380,7 @@ static int launch_cross(sd_attn_handle* h, const Problem& p) {
     if (rc == SD_ATTN_OK) rc = make_tmap(h, &tv, p.v, p.BH, p.Nk, p.d, a.kn);
     if (rc != SD_ATTN_OK) return rc;
     dim3 grid((p.Nq + TILE_M - 1) / TILE_M, p.BH), block(CROSS_THREADS);
-    cross_attention_kernel<<<grid, block, cross_smem_bytes(a.nch, a.kn), p.stream>>>(tq, tk, tv, a);
+    launch_overlapped(h, cross_attention_kernel, grid, block, cross_smem_bytes(a.nch, a.kn), p.stream, tq, tk, tv, a);
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) return cuda_fail(h, e);
     h->launches += 1;
@@ -436,13 +458,13 @@ static int launch_fused4s(sd_attn_handle* h, const Problem& p) {
     dim3 grid((tiles_per_head + a.tiles_per_cta - 1) / a.tiles_per_cta, p.BH), block(F4_THREADS);
     // the polynomial share of the exponentials only pays where four tiles saturate the special function unit
     if (a.dpad <= 48)
-        fused4s_attention_kernel<F4S_POLY_PER8, 1><<<grid, block, smem, p.stream>>>(tq, tk, tv, a);
+        launch_overlapped(h, fused4s_attention_kernel<F4S_POLY_PER8, 1>, grid, block, smem, p.stream, tq, tk, tv, a);
     else if (a.nch == 1)
-        fused4s_attention_kernel<0, 1><<<grid, block, smem, p.stream>>>(tq, tk, tv, a);
+        launch_overlapped(h, fused4s_attention_kernel<0, 1>, grid, block, smem, p.stream, tq, tk, tv, a);
     else if (a.nch == 2)
-        fused4s_attention_kernel<0, 2><<<grid, block, smem, p.stream>>>(tq, tk, tv, a);
+        launch_overlapped(h, fused4s_attention_kernel<0, 2>, grid, block, smem, p.stream, tq, tk, tv, a);
     else
-        fused4s_attention_kernel<0, 3><<<grid, block, smem, p.stream>>>(tq, tk, tv, a);
+        launch_overlapped(h, fused4s_attention_kernel<0, 3>, grid, block, smem, p.stream, tq, tk, tv, a);
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) return cuda_fail(h, e);
     h->launches += 1;
