@@ -66,6 +66,17 @@ typedef enum {
  * compute capability 10.x), resolves the driver's tensor-map encoder, raises the kernels'
  * dynamic shared-memory limits and allocates one 64-byte device status block.  No stream
  * work.  *out receives the handle (NULL on failure).
+ *
+ * Switches read from the environment at this call (all default off; they select slower variants that exist
+ * for comparison and testing, results are the same within the tolerance):
+ *   SD_ATTN_NO_PDL=1            launch every kernel the ordinary way.  By default the tensor-core kernels are
+ *                               launched with programmatic stream serialization: a kernel may run its set-up
+ *                               while the previous kernel of the stream finishes, and waits for that kernel to
+ *                               complete before it reads or writes global memory, so stream order is kept.
+ *   SD_ATTN_FUSED_TILES=1..4    fixed number of query tiles per CTA of the FUSED kernel (default: by problem size)
+ *   SD_ATTN_FUSED_NO_SPARE=1    FUSED: the four-tile kernel without the spare score buffer (d <= 64)
+ *   SD_ATTN_FUSED_TWO_TILE=1    FUSED: the two-tile kernel
+ *   SD_ATTN_CROSS_ONE_TILE=1    CROSS: one tile per CTA also for 65..80 keys
  */
 int sd_attn_create(sd_attn_handle **out);
 

@@ -303,6 +303,34 @@ def test_every_variant_of_the_small_head_dim_kernel(bd, env, monkeypatch):
         a.close()
 
 
+@pytest.mark.parametrize("shape", [(1, 4, 512, 512, 40), (2, 2, 256, 77, 80), (1, 2, 130, 300, 160)])
+def test_back_to_back_calls_that_depend_on_one_another(att, bd, shape):
+    """Calls queued on one stream without synchronisation, each reading what the previous one wrote and writing
+    over what the previous one read: a kernel may start its set-up while its predecessor still runs, but must not
+    touch global memory before the predecessor has finished."""
+    B, H, Nq, Nk, d = shape
+    q, k, v = rand_qkv(5200 + d, B, H, Nq, Nk, d)
+    scale = float(np.float32(1.0 / np.sqrt(d)))
+    att.set_mode(bd.MODE_AUTO)
+    ta, tk, tv = gpu(q), gpu(k), gpu(v)
+    tb = torch.empty_like(ta)
+    stream = torch.cuda.current_stream().cuda_stream
+    chain = 6
+    for n in range(chain):        # a -> b -> a -> b ...: queries of call n are the output of call n-1
+        src, dst = (ta, tb) if n % 2 == 0 else (tb, ta)
+        rc = bd.sd_attn_forward(att.handle, src.data_ptr(), tk.data_ptr(), tv.data_ptr(), dst.data_ptr(),
+                                B, H, Nq, Nk, d, scale, bd.F16, stream)
+        assert rc == bd.OK
+    att.check()
+    got = (ta if chain % 2 == 0 else tb).cpu().numpy()
+    cur = q
+    for n in range(chain):        # the same chain on the CPU, rounding to fp16 between the links as the GPU does
+        ref, _, _ = oracle.forward(cur, k, v, scale)
+        cur = ref.astype(np.float16)
+    vmax = float(np.abs(v.astype(np.float64)).max())
+    assert np.abs(got.astype(np.float64) - ref).max() <= chain * F16_ABS * vmax
+
+
 def test_padding_rows_with_distinct_values_only_see_their_mean(att, bd):
     call = workloads.config3()[0]
     q, k, v = workloads.make_inputs(call)
