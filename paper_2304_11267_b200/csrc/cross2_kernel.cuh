@@ -5,8 +5,11 @@
 // cross_kernel.cuh runs one tile per CTA, start to finish, and leans on CTA-level overlap; its launch,
 // tensor-memory allocation, descriptor fetch and drain are paid per tile and HBM sits idle meanwhile.
 // Here ONE CTA per SM walks a contiguous range of (head, tile) items with every stage overlapped:
-//   warps 0 .. 4*NWG-1   NWG softmax groups; group w owns items w, w+NWG, ... (thread = query row):
-//                        row max, exp2, row sum, weights back to tensor memory, later O / sum -> global
+//   warps 0 .. 4*NWG-1   NWG softmax groups; group w owns items w, w+NWG, ... (thread = query row): exp2, row sum,
+//                        weights back to tensor memory, 1 / row sum to shared memory -- and on to its next item
+//   next 4 warps         the epilogue warpgroup: for every item in turn, O_w / row sum -> fp16 -> global.  (With the
+//                        softmax warps doing their own epilogue a group spent a third of an item waiting for the
+//                        P V product and writing out, and four groups did not hide it.)
 //   next warp            TMA producer: the Q tile of item i into ring stage i % NS (several in flight); K and V
 //                        of a head once per head, double-buffered.  (The copy engine spends about 7 clocks per
 //                        80-byte row of a d = 40 tensor, measured, so fetching K and V per item -- 160 more rows --
@@ -15,7 +18,11 @@
 //                        when the weights are ready
 // Tensor memory: per group S_w (80 columns; the packed fp16 weights overwrite the first 40) and O_w
 // (dpad columns), so NWG = 512 / (80 + dpad) capped at 4: four groups at d = 40, three at 80, two at 160.
-// No running rescale is needed: all keys of a row are in the tile, so L and S of Eq. 4 are exact.
+// No running rescale is needed: all keys of a row are in the tile.  The exponent is anchored X2_HEADROOM_LOG2 above
+// the score of the row's FIRST key instead of the row maximum (any anchor gives the same weights in exact
+// arithmetic); only if the weights of a row then sum to more than X2_SUM_LIMIT -- its maximum lies far above its
+// first score: rare -- does the warp take the true maximum and redo the row.  That keeps the maximum off the path
+// and lets a row be processed in two pieces (48 + 32 columns) with half the registers.
 #pragma once
 #include <cuda.h>
 
@@ -29,8 +36,12 @@ constexpr int X2_KN = 80;            // keys rounded up to the MMA N granule; th
 constexpr int X2_MAX_STAGES = 8;
 constexpr int X2_MAX_KSTEPS = 10;
 constexpr int X2_SMEM_BUDGET = 216 * 1024;
-constexpr int X2_SOFTMAX_REGS = 112;  // four-group variant, after setmaxnreg: 512 * 112 + 128 * 32 = 61440 = 640 * 96
+// four-group variant, after setmaxnreg: 512 * 96 + 128 * 64 + 128 * 32 = 61440 = 768 * 80, the launch allocation
+constexpr int X2_SOFTMAX_REGS = 96;
+constexpr int X2_EPILOGUE_REGS = 64;
 constexpr int X2_CONTROL_REGS = 32;
+constexpr float X2_HEADROOM_LOG2 = 8.0f;   // weights of the first key: 2^-8
+constexpr float X2_SUM_LIMIT = 4096.0f;    // no weight above 2^12 reaches the binary16 pack
 
 struct Cross2Args {
     __half* out;        // [BH][Nq][d]
@@ -61,7 +72,7 @@ __host__ inline int cross2_groups(int d) {
     const int g = 512 / (X2_KN + (d + 15) / 16 * 16);
     return g > 4 ? 4 : g;
 }
-__host__ inline int cross2_threads(int groups) { return groups * 128 + 128; }   // + one control warpgroup
+__host__ inline int cross2_threads(int groups) { return groups * 128 + 256; }   // + epilogue and control warpgroups
 __host__ inline int cross2_q_bytes(int nch) { return nch * TILE_M * CHUNK_ROW_BYTES; }
 __host__ inline int cross2_kv_bytes(int nch) { return nch * X2_KN * CHUNK_ROW_BYTES; }
 // shared memory: [2 head buffers][K | V] then the Q ring
@@ -89,17 +100,19 @@ __device__ __forceinline__ void issue_qk(uint32_t tmem_s, uint64_t q_desc, uint6
 }
 
 template <int NWG>
-__global__ void __launch_bounds__(NWG * 128 + 128, 1)
+__global__ void __launch_bounds__(NWG * 128 + 256, 1)
 cross2_attention_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__ CUtensorMap tmap_k,
                         const __grid_constant__ CUtensorMap tmap_v, const Cross2Args args) {
     extern __shared__ uint8_t x2_smem_raw[];
     __shared__ __align__(8) uint64_t bar_full[X2_MAX_STAGES], bar_empty[X2_MAX_STAGES];
     __shared__ __align__(8) uint64_t bar_kv_full[2], bar_kv_empty[2];
     __shared__ __align__(8) uint64_t bar_s_full[NWG], bar_p_full[NWG], bar_o_full[NWG], bar_o_free[NWG], bar_pv_done[NWG];
+    __shared__ float inv_sum[NWG][2][TILE_M];   // 1 / row sum of the group's current and previous item
     __shared__ uint32_t tmem_base_slot;
     __shared__ int abort_flag;
 
-    constexpr int LOADER_WARP = NWG * 4, S_ISSUER_WARP = NWG * 4 + 1, O_ISSUER_WARP = NWG * 4 + 2;
+    constexpr int EPILOGUE_WARP0 = NWG * 4;
+    constexpr int LOADER_WARP = NWG * 4 + 4, S_ISSUER_WARP = NWG * 4 + 5, O_ISSUER_WARP = NWG * 4 + 6;
 #ifdef SD_ATTN_TRACE
     if (args.trace && blockIdx.x == 0 && threadIdx.x == 0) {
         unsigned long long gt;
@@ -165,7 +178,7 @@ cross2_attention_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid
     // compiled): an increase that the decreases do not cover blocks for ever.  The host checks, from the
     // compiled register count, that 512 * X2_SOFTMAX_REGS + 128 * X2_CONTROL_REGS fits before using this variant.
     constexpr bool REBALANCE = NWG == 4;
-    if (REBALANCE && warp >= NWG * 4) setmaxnreg_dec<X2_CONTROL_REGS>();
+    if (REBALANCE && warp >= LOADER_WARP) setmaxnreg_dec<X2_CONTROL_REGS>();
     if (warp == LOADER_WARP) {
         // ------------------------------------------------------------ TMA producer
         if (elect_one()) {
@@ -275,13 +288,12 @@ cross2_attention_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid
             }
         }
     } else if (warp < NWG * 4) {
-        // ------------------------------------------------------------ softmax + epilogue warps
+        // ------------------------------------------------------------ softmax warps
         if (REBALANCE) setmaxnreg_inc<X2_SOFTMAX_REGS>();
         const int w = warp >> 2;
         const int r = tid & (TILE_M - 1);
         const uint32_t lane_off = (uint32_t)((warp & 3) * 32) << 16;
         const uint32_t tmem_s = tmem_base + w * X2_KN + lane_off;
-        const uint32_t tmem_o = tmem_o0 + w * dpad + lane_off;
         const float c2 = args.scale_log2e;
         const int valid = args.Nk;
         bool ok = true;
@@ -294,42 +306,84 @@ cross2_attention_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid
             if (!ok) break;
             tc_fence_after_sync();
             if (tracer) X2_TRACE(w, i, 1);
-            float row_sum;
-            {
-                uint32_t s[X2_KN];
-                tmem_ld32(tmem_s, &s[0]);
-                tmem_ld32(tmem_s + 32, &s[32]);
-                tmem_ld16(tmem_s + 64, *reinterpret_cast<uint32_t(*)[16]>(&s[64]));
-                tmem_wait_ld();
-                // L_i of Eq. 4 (to bf16 precision: it only anchors the exponent) over the valid keys
-                const float row_max = fmaxf(row_max_bf16<64>(s), row_max_masked<16>(&s[64], valid - 64));
-                const float neg_mc = -row_max * c2;
-                const uint64_t c2c2 = pack_b64(__float_as_uint(c2), __float_as_uint(c2));
-                const uint64_t nmnm = pack_b64(__float_as_uint(neg_mc), __float_as_uint(neg_mc));
+            uint32_t packed[X2_KN / 2];
+            float row_sum, anchor = 0.f;
+#pragma unroll 1
+            for (int attempt = 0; attempt < 2; ++attempt) {
                 uint64_t acc[2] = {0ull, 0ull};
-                uint32_t packed[16];
-                exp2_pack_32<0>(&s[0], c2c2, nmnm, packed, acc);
-                tmem_st16(tmem_s, packed);
-                exp2_pack_32<0>(&s[32], c2c2, nmnm, packed, acc);
-                tmem_st16(tmem_s + 16, packed);
                 float tail = 0.f;
-                exp2_pack_32_masked<8>(&s[64], c2, neg_mc, 64, valid, packed, tail);
-                tmem_st8(tmem_s + 32, *reinterpret_cast<uint32_t(*)[8]>(&packed[0]));
-                row_sum = sum_f32x2(acc[0], acc[1]) + tail;   // S_i of Eq. 4
+                {   // columns 0..47
+                    uint32_t s[48];
+                    tmem_ld32(tmem_s, &s[0]);
+                    tmem_ld16(tmem_s + 32, *reinterpret_cast<uint32_t(*)[16]>(&s[32]));
+                    tmem_wait_ld();
+                    if (attempt == 0) anchor = __uint_as_float(s[0]) * c2 + X2_HEADROOM_LOG2;
+                    const float neg_mc = -anchor;
+                    const uint64_t c2c2 = pack_b64(__float_as_uint(c2), __float_as_uint(c2));
+                    const uint64_t nmnm = pack_b64(__float_as_uint(neg_mc), __float_as_uint(neg_mc));
+                    exp2_pack_32<0>(&s[0], c2c2, nmnm, &packed[0], acc);
+                    exp2_pack_16<0>(&s[32], c2c2, nmnm, &packed[16], acc);
+                }
+                {   // columns 48..79: the last 16 hold the keys past Nk (zero-filled) and are masked
+                    uint32_t s[32];
+                    tmem_ld32(tmem_s + 48, &s[0]);
+                    tmem_wait_ld();
+                    const float neg_mc = -anchor;
+                    const uint64_t c2c2 = pack_b64(__float_as_uint(c2), __float_as_uint(c2));
+                    const uint64_t nmnm = pack_b64(__float_as_uint(neg_mc), __float_as_uint(neg_mc));
+                    exp2_pack_16<0>(&s[0], c2c2, nmnm, &packed[24], acc);
+                    exp2_pack_32_masked<8>(&s[16], c2, neg_mc, 64, valid, &packed[32], tail);
+                }
+                row_sum = sum_f32x2(acc[0], acc[1]) + tail;   // S_i of Eq. 4, relative to the anchor
+                const bool over = !(row_sum <= X2_SUM_LIMIT);
+                if (attempt == 1 || !__any_sync(0xffffffffu, over)) break;
+                // rare: the row maximum lies far above the first score.  Nothing has been stored yet: take L_i of
+                // Eq. 4 (to bf16 precision: it only anchors the exponent) from the scores and redo the row.
+                float row_max;
+                {
+                    uint32_t s[32];
+                    tmem_ld32(tmem_s, &s[0]);
+                    tmem_wait_ld();
+                    row_max = row_max_bf16<32>(s);
+                    tmem_ld32(tmem_s + 32, &s[0]);
+                    tmem_wait_ld();
+                    row_max = fmaxf(row_max, row_max_bf16<32>(s));
+                    tmem_ld16(tmem_s + 64, *reinterpret_cast<uint32_t(*)[16]>(&s[0]));
+                    tmem_wait_ld();
+                    row_max = fmaxf(row_max, row_max_masked<16>(s, valid - 64));
+                }
+                anchor = row_max * c2;
             }
+            tmem_st32(tmem_s, &packed[0]);    // P_w over the first 40 columns of S_w
+            tmem_st8(tmem_s + 32, *reinterpret_cast<uint32_t(*)[8]>(&packed[32]));
+            inv_sum[w][n & 1][r] = 1.f / row_sum;   // for the epilogue warpgroup
             tmem_wait_st();
             tc_fence_before_sync();
+            __syncwarp();                           // every lane's store before lane 0's arrival
             if (lane == 0) mbar_arrive(smem_u32(&bar_p_full[w]));
             if (tracer) X2_TRACE(w, i, 2);
-
+        }
+    } else if (warp < LOADER_WARP) {
+        // ------------------------------------------------------------ epilogue warpgroup: every item in turn
+        if (REBALANCE) setmaxnreg_dec<X2_EPILOGUE_REGS>();
+        const int r = tid & (TILE_M - 1);
+        const uint32_t lane_off = (uint32_t)((warp & 3) * 32) << 16;
+        bool ok = true;
+        int w = 0, n = 0;
+        int bh = bh0, tile = item0 - bh0 * args.tiles_per_bh;
+        const bool tracer = warp == EPILOGUE_WARP0 && lane == 0;
+        for (int i = 0; i < n_local; ++i) {
+            const uint32_t tmem_o = tmem_o0 + w * dpad + lane_off;
+            // bar_o_full[w] completes after the O issuer saw bar_p_full[w], which the softmax warps arrived on after
+            // writing inv_sum: the values are in shared memory by then.  (bar_p_full itself must not be waited on
+            // here: a second consumer may fall two phases behind, and a parity wait cannot tell.)
             ok = mbar_wait(smem_u32(&bar_o_full[w]), n & 1, abort_p, args.status, SITE_Y_O, i);
             ok = __all_sync(0xffffffffu, ok);
             if (!ok) break;
             tc_fence_after_sync();
             if (tracer) X2_TRACE(w, i, 3);
-            const int item = item0 + i, bh = item / args.tiles_per_bh, tile = item - bh * args.tiles_per_bh;
+            const float inv = inv_sum[w][n & 1][r];
             const int row = tile * TILE_M + r;
-            const float inv = 1.f / row_sum;
             __half* orow = args.out + ((size_t)bh * args.Nq + row) * args.d;
             // O / S_i -> fp16 -> global, 32 columns per tensor-memory round trip (dpad is a multiple of 16)
             for (int c0 = 0; c0 < dpad; c0 += 32) {
@@ -337,6 +391,10 @@ cross2_attention_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid
                 tmem_ld16(tmem_o + c0, *reinterpret_cast<uint32_t(*)[16]>(&x[0]));
                 if (c0 + 16 < dpad) tmem_ld16(tmem_o + c0 + 16, *reinterpret_cast<uint32_t(*)[16]>(&x[16]));
                 tmem_wait_ld();
+                if (c0 + 32 >= dpad) {   // all of O_w is in registers: the next product of this group may overwrite it
+                    tc_fence_before_sync();
+                    if (lane == 0) mbar_arrive(smem_u32(&bar_o_free[w]));
+                }
                 if (row < args.Nq) {
 #pragma unroll
                     for (int g = 0; g < 4; ++g) {
@@ -349,9 +407,9 @@ cross2_attention_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid
                     }
                 }
             }
-            tc_fence_before_sync();
-            if (lane == 0) mbar_arrive(smem_u32(&bar_o_free[w]));
             if (tracer) X2_TRACE(w, i, 4);
+            if (++w == NWG) { w = 0; ++n; }
+            if (++tile == args.tiles_per_bh) { tile = 0; ++bh; }
         }
     }
 

@@ -185,7 +185,7 @@ extern "C" int sd_attn_create(sd_attn_handle** out) {
         }
         if (e == cudaSuccess) e = cudaFuncGetAttributes(&fa, cross2_attention_kernel<4>);
         if (e == cudaSuccess)
-            h->cross2_four_ok = cross2_threads(4) * fa.numRegs >= 512 * X2_SOFTMAX_REGS + 128 * X2_CONTROL_REGS;
+            h->cross2_four_ok = cross2_threads(4) * fa.numRegs >= 512 * X2_SOFTMAX_REGS + 128 * X2_EPILOGUE_REGS + 128 * X2_CONTROL_REGS;
     }
     if (e == cudaSuccess) e = cudaMalloc((void**)&h->dev_status, sizeof(int) * DEV_STATUS_INTS);
     if (e == cudaSuccess) e = cudaMemset(h->dev_status, 0, sizeof(int) * DEV_STATUS_INTS);
