@@ -10,12 +10,17 @@
 //   next 4 warps         the epilogue warpgroup: for every item in turn, O_w / row sum -> fp16 -> global.  (With the
 //                        softmax warps doing their own epilogue a group spent a third of an item waiting for the
 //                        P V product and writing out, and four groups did not hide it.)
-//   next warp            TMA producer: the Q tile of item i into ring stage i % NS (several in flight); K and V
+//   next warp            producer: the Q tile of item i into ring stage i % NS (several in flight); K and V
 //                        of a head once per head, double-buffered.  (The copy engine spends about 7 clocks per
 //                        80-byte row of a d = 40 tensor, measured, so fetching K and V per item -- 160 more rows --
 //                        would make it the bound.  A single warp of 128-bit cp.async copies for Q measured slower.)
 //   two more warps       MMA issuers: one thread issues S_w = Q K^T as soon as a stage lands, another O_w = P_w V
 //                        when the weights are ready
+// Q at head dims up to 48 (four groups): a tiled TMA load of 128 rows of 80 bytes keeps the copy engine busy for
+// 900-1300 clocks, which became the bound of the kernel once the softmax no longer was.  The tile is 10 KB of
+// CONTIGUOUS global memory, so it is fetched with one untiled bulk copy into a raw ring stage instead, and the softmax
+// group that will use it rewrites it (thread = row: five 16-byte loads, six swizzled 16-byte stores, columns 40..47
+// zeroed) into its own MMA-layout buffer while it waits for tensor-core work anyway.
 // Tensor memory: per group S_w (80 columns; the packed fp16 weights overwrite the first 40) and O_w
 // (dpad columns), so NWG = 512 / (80 + dpad) capped at 4: four groups at d = 40, three at 80, two at 160.
 // No running rescale is needed: all keys of a row are in the tile.  The exponent is anchored X2_HEADROOM_LOG2 above
@@ -44,6 +49,7 @@ constexpr float X2_HEADROOM_LOG2 = 8.0f;   // weights of the first key: 2^-8
 constexpr float X2_SUM_LIMIT = 4096.0f;    // no weight above 2^12 reaches the binary16 pack
 
 struct Cross2Args {
+    const __half* q;    // [BH][Nq][d]: the four-group variant fetches Q tiles with untiled bulk copies
     __half* out;        // [BH][Nq][d]
     int Nq, Nk, d;
     int dpad, nch;
@@ -83,6 +89,16 @@ __host__ inline int cross2_stages(int nch) {
 __host__ inline size_t cross2_smem_bytes(int nch) {
     return (size_t)4 * cross2_kv_bytes(nch) + (size_t)cross2_stages(nch) * cross2_q_bytes(nch) + 1024;
 }
+// four-group variant (d <= 48): [2 head buffers][K | V], four MMA-layout Q buffers, then the ring of raw Q tiles
+__host__ inline int cross2_raw_bytes(int d) { return (TILE_M * d * 2 + 127) & ~127; }
+__host__ inline int cross2_dense_stages(int d) {   // a multiple of 4: a stage then always serves the same group
+    int s = (X2_SMEM_BUDGET - 4 * cross2_kv_bytes(1) - 4 * cross2_q_bytes(1)) / cross2_raw_bytes(d);
+    s = s > X2_MAX_STAGES ? X2_MAX_STAGES : s;
+    return s / 4 * 4;
+}
+__host__ inline size_t cross2_dense_smem_bytes(int d) {
+    return (size_t)4 * cross2_kv_bytes(1) + (size_t)4 * cross2_q_bytes(1) + (size_t)cross2_dense_stages(d) * cross2_raw_bytes(d) + 1024;
+}
 __host__ inline bool cross2_supports(int Nk, int d) { return Nk > 64 && Nk <= X2_KN && d % 8 == 0 && d <= 160; }
 
 enum {
@@ -107,6 +123,7 @@ cross2_attention_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid
     __shared__ __align__(8) uint64_t bar_full[X2_MAX_STAGES], bar_empty[X2_MAX_STAGES];
     __shared__ __align__(8) uint64_t bar_kv_full[2], bar_kv_empty[2];
     __shared__ __align__(8) uint64_t bar_s_full[NWG], bar_p_full[NWG], bar_o_full[NWG], bar_o_free[NWG], bar_pv_done[NWG];
+    __shared__ __align__(8) uint64_t bar_q_ready[NWG];   // four-group variant: the group's MMA-layout Q buffer is written
     __shared__ float inv_sum[NWG][2][TILE_M];   // 1 / row sum of the group's current and previous item
     __shared__ uint32_t tmem_base_slot;
     __shared__ int abort_flag;
@@ -132,15 +149,18 @@ cross2_attention_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid
 
     const uint32_t smem_base = (smem_u32(x2_smem_raw) + 1023u) & ~1023u;
     const uint32_t q_bytes = nch * TILE_M * CHUNK_ROW_BYTES, kv_bytes = nch * X2_KN * CHUNK_ROW_BYTES;
+    constexpr bool DENSE_Q = NWG == 4;                     // d <= 48: one chunk, Q by untiled bulk copy + rewrite
     const uint32_t kv_smem = smem_base;                    // [2][K | V]
-    const uint32_t q_smem = smem_base + 4 * kv_bytes;      // [stages][nch][128 rows][128 B]
+    const uint32_t q_smem = smem_base + 4 * kv_bytes;      // [stages][nch][128 rows][128 B]; DENSE_Q: [NWG] of them
+    const uint32_t raw_bytes = (TILE_M * args.d * 2 + 127) & ~127;
+    const uint32_t raw_smem = q_smem + NWG * q_bytes;      // DENSE_Q: [stages] raw tiles of 128 rows x 2d bytes
     volatile int* abort_p = &abort_flag;
 
     if (tid == 0) {
         abort_flag = 0;
         for (int s = 0; s < X2_MAX_STAGES; ++s) {
             mbar_init(smem_u32(&bar_full[s]), 1);
-            mbar_init(smem_u32(&bar_empty[s]), 1);
+            mbar_init(smem_u32(&bar_empty[s]), DENSE_Q ? 4 : 1);   // DENSE_Q: the four warps that read the raw tile
         }
         for (int b = 0; b < 2; ++b) {
             mbar_init(smem_u32(&bar_kv_full[b]), 1);
@@ -152,6 +172,7 @@ cross2_attention_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid
             mbar_init(smem_u32(&bar_o_full[w]), 1);
             mbar_init(smem_u32(&bar_o_free[w]), 4);
             mbar_init(smem_u32(&bar_pv_done[w]), 1);
+            mbar_init(smem_u32(&bar_q_ready[w]), 4);
         }
         mbar_init_fence();
     }
@@ -210,6 +231,14 @@ cross2_attention_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid
 #ifdef SD_ATTN_X_NOQ
                 if (i >= stages) { mbar_arrive(bar); continue; }
 #endif
+                if (DENSE_Q) {
+                    int rows = args.Nq - tile * TILE_M;
+                    if (rows > TILE_M) rows = TILE_M;
+                    const uint32_t bytes = (uint32_t)rows * args.d * 2;   // d % 8 == 0: a multiple of 16
+                    mbar_arrive_expect_tx(bar, bytes);
+                    bulk_load(raw_smem + s * raw_bytes, args.q + ((size_t)bh * args.Nq + (size_t)tile * TILE_M) * args.d, bytes, bar);
+                    continue;
+                }
                 mbar_arrive_expect_tx(bar, q_bytes);
                 for (int ch = 0; ch < nch; ++ch)
                     tma_load_3d(dst + ch * TILE_M * CHUNK_ROW_BYTES, &tmap_q, bar, ch * CHUNK_COLS, tile * TILE_M, bh);
@@ -240,14 +269,15 @@ cross2_attention_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid
                 const uint64_t k_desc0 = smem_desc_sw128(kv_smem, 16, 1024);
                 const uint32_t q_stage_off = q_bytes >> 4, kv_buf_off = (2 * kv_bytes) >> 4;
                 for (; c.i < n_local && ok; advance(c)) {
-                    ok = mbar_wait(smem_u32(&bar_full[c.s]), c.sph, abort_p, args.status, SITE_Y_STAGE, c.i) &&
+                    ok = (DENSE_Q ? mbar_wait(smem_u32(&bar_q_ready[c.w]), c.n & 1, abort_p, args.status, SITE_Y_STAGE, c.i)
+                                  : mbar_wait(smem_u32(&bar_full[c.s]), c.sph, abort_p, args.status, SITE_Y_STAGE, c.i)) &&
                          mbar_wait(smem_u32(&bar_kv_full[c.g & 1]), (c.g >> 1) & 1, abort_p, args.status, SITE_Y_KV, c.i);
                     if (ok && c.n >= 1)   // the group's previous item no longer needs these columns
                         ok = mbar_wait(smem_u32(&bar_pv_done[c.w]), (c.n - 1) & 1, abort_p, args.status, SITE_Y_PV, c.i);
                     if (!ok) break;
                     tc_fence_after_sync();
                     X2_TRACE(NWG, c.i, 3);
-                    const uint64_t qd = q_desc0 + (uint64_t)(c.s * q_stage_off);
+                    const uint64_t qd = q_desc0 + (uint64_t)((DENSE_Q ? c.w : c.s) * q_stage_off);
                     const uint64_t kd = k_desc0 + (uint64_t)((c.g & 1) * kv_buf_off);
                     const uint32_t ts = tmem_base + c.w * X2_KN;
                     if (ksteps_s == 3) issue_qk<3>(ts, qd, kd, idesc_s);
@@ -259,7 +289,7 @@ cross2_attention_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid
                                        kd + (uint64_t)(((kk >> 2) * X2_KN * CHUNK_ROW_BYTES + (kk & 3) * 32) >> 4), idesc_s,
                                        kk > 0);
                     tc_commit(smem_u32(&bar_s_full[c.w]));
-                    tc_commit(smem_u32(&bar_empty[c.s]));   // the Q stage is free once this product has read it
+                    if (!DENSE_Q) tc_commit(smem_u32(&bar_empty[c.s]));   // the Q stage is free once this product has read it
                     X2_TRACE(NWG, c.i, 4);
                 }
             } else {
@@ -298,7 +328,31 @@ cross2_attention_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid
         const int valid = args.Nk;
         bool ok = true;
         const bool tracer = (warp & 3) == 0 && lane == 0;
-        for (int i = w; i < n_local; i += NWG) {
+        // DENSE_Q: rewrite the raw Q tile of item j (ring stage j % stages; j = w mod NWG and stages is a multiple of
+        // NWG, so this group is the only consumer of that stage's barrier) into the group's MMA-layout buffer: row r
+        // is 128 bytes at r * 128, its 16-byte chunk c at position c ^ (r & 7) (the 128-byte swizzle).
+        auto rewrite_q = [&](int j) -> bool {
+            const int s = j % stages;
+            bool good = mbar_wait(smem_u32(&bar_full[s]), (j / stages) & 1, abort_p, args.status, SITE_Y_STAGE, j);
+            good = __all_sync(0xffffffffu, good);
+            if (!good) return false;
+            const uint32_t src = raw_smem + s * raw_bytes + r * (args.d * 2);
+            const uint32_t dst = q_smem + w * q_bytes + r * CHUNK_ROW_BYTES;
+            const int chunks = args.d >> 3;   // 16-byte chunks of real data per row (<= 6)
+            uint4 v[6];
+#pragma unroll
+            for (int c = 0; c < 6; ++c) v[c] = c < chunks ? ld_shared_v4(src + c * 16) : make_uint4(0u, 0u, 0u, 0u);
+            __syncwarp();
+            if (lane == 0) mbar_arrive(smem_u32(&bar_empty[s]));   // the raw stage may be refilled
+#pragma unroll
+            for (int c = 0; c < 6; ++c) st_shared_v4(dst + ((c ^ (r & 7)) << 4), v[c]);
+            fence_proxy_async_smem();   // generic-proxy stores before the tensor core reads them
+            __syncwarp();
+            if (lane == 0) mbar_arrive(smem_u32(&bar_q_ready[w]));
+            return true;
+        };
+        if (DENSE_Q && w < n_local) ok = rewrite_q(w);
+        for (int i = w; i < n_local && ok; i += NWG) {
             const int n = i / NWG;
             if (tracer) X2_TRACE(w, i, 0);
             ok = mbar_wait(smem_u32(&bar_s_full[w]), n & 1, abort_p, args.status, SITE_Y_S, i);
@@ -306,6 +360,10 @@ cross2_attention_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid
             if (!ok) break;
             tc_fence_after_sync();
             if (tracer) X2_TRACE(w, i, 1);
+            if (DENSE_Q && i + NWG < n_local) {   // S of this item is done: the Q buffer may take the next one
+                ok = rewrite_q(i + NWG);
+                if (!ok) break;
+            }
             uint32_t packed[X2_KN / 2];
             float row_sum, anchor = 0.f;
 #pragma unroll 1

@@ -327,6 +327,7 @@ static int launch_simt(sd_attn_handle* h, const Problem& p) {
 // 65..80 keys (the 77 text tokens): one persistent CTA per SM walks a range of (head, tile) items
 static int launch_cross2(sd_attn_handle* h, const Problem& p) {
     Cross2Args a;
+    a.q = (const __half*)p.q;
     a.out = (__half*)p.out;
     a.Nq = p.Nq; a.Nk = p.Nk; a.d = p.d;
     a.dpad = (p.d + 15) / 16 * 16;
@@ -348,7 +349,11 @@ static int launch_cross2(sd_attn_handle* h, const Problem& p) {
     const int grid = a.n_items < h->sm_count ? a.n_items : h->sm_count;
     int groups = cross2_groups(p.d);
     if (groups >= 4 && !h->cross2_four_ok) groups = 3;
-    const size_t smem = cross2_smem_bytes(a.nch);
+    size_t smem = cross2_smem_bytes(a.nch);
+    if (groups >= 4) {   // d <= 48: Q tiles arrive as raw bulk copies and are rewritten in shared memory
+        a.stages = cross2_dense_stages(p.d);
+        smem = cross2_dense_smem_bytes(p.d);
+    }
     if (groups >= 4)
         launch_overlapped(h, cross2_attention_kernel<4>, dim3(grid), dim3(cross2_threads(4)), smem, p.stream, tq, tk, tv, a);
     else if (groups == 3)
