@@ -92,12 +92,13 @@ __host__ inline size_t cross2_smem_bytes(int nch) {
 // four-group variant (d <= 48): [2 head buffers][K | V], four MMA-layout Q buffers, then the ring of raw Q tiles
 __host__ inline int cross2_raw_bytes(int d) { return (TILE_M * d * 2 + 127) & ~127; }
 __host__ inline int cross2_dense_stages(int d) {   // a multiple of 4: a stage then always serves the same group
-    int s = (X2_SMEM_BUDGET - 4 * cross2_kv_bytes(1) - 4 * cross2_q_bytes(1)) / cross2_raw_bytes(d);
+    int s = (X2_SMEM_BUDGET - 4 * cross2_kv_bytes(1) - 4 * cross2_q_bytes(1)) / cross2_raw_bytes(d) - 2;
     s = s > X2_MAX_STAGES ? X2_MAX_STAGES : s;
     return s / 4 * 4;
 }
-__host__ inline size_t cross2_dense_smem_bytes(int d) {
-    return (size_t)4 * cross2_kv_bytes(1) + (size_t)4 * cross2_q_bytes(1) + (size_t)cross2_dense_stages(d) * cross2_raw_bytes(d) + 1024;
+__host__ inline size_t cross2_dense_smem_bytes(int d) {   // ... and two output staging tiles of the raw size
+    return (size_t)4 * cross2_kv_bytes(1) + (size_t)4 * cross2_q_bytes(1) +
+           (size_t)(cross2_dense_stages(d) + 2) * cross2_raw_bytes(d) + 1024;
 }
 __host__ inline bool cross2_supports(int Nk, int d) { return Nk > 64 && Nk <= X2_KN && d % 8 == 0 && d <= 160; }
 
@@ -130,6 +131,7 @@ cross2_attention_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid
 
     constexpr int EPILOGUE_WARP0 = NWG * 4;
     constexpr int LOADER_WARP = NWG * 4 + 4, S_ISSUER_WARP = NWG * 4 + 5, O_ISSUER_WARP = NWG * 4 + 6;
+    constexpr int S2_ISSUER_WARP = NWG * 4 + 7;   // second S issuer: the odd items
 #ifdef SD_ATTN_TRACE
     if (args.trace && blockIdx.x == 0 && threadIdx.x == 0) {
         unsigned long long gt;
@@ -154,6 +156,7 @@ cross2_attention_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid
     const uint32_t q_smem = smem_base + 4 * kv_bytes;      // [stages][nch][128 rows][128 B]; DENSE_Q: [NWG] of them
     const uint32_t raw_bytes = (TILE_M * args.d * 2 + 127) & ~127;
     const uint32_t raw_smem = q_smem + NWG * q_bytes;      // DENSE_Q: [stages] raw tiles of 128 rows x 2d bytes
+    const uint32_t out_smem = raw_smem + stages * raw_bytes;   // DENSE_Q: [2] output tiles in the same dense layout
     volatile int* abort_p = &abort_flag;
 
     if (tid == 0) {
@@ -244,13 +247,15 @@ cross2_attention_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid
                     tma_load_3d(dst + ch * TILE_M * CHUNK_ROW_BYTES, &tmap_q, bar, ch * CHUNK_COLS, tile * TILE_M, bh);
             }
         }
-    } else if (warp == S_ISSUER_WARP || warp == O_ISSUER_WARP) {
+    } else if (warp == S_ISSUER_WARP || warp == S2_ISSUER_WARP || warp == O_ISSUER_WARP) {
         // ------------------------------------------------------------ MMA issuers
         // An issuer is one thread sharing a scheduler with busy softmax warps: each barrier test and each
         // tcgen05.mma costs it tens to hundreds of clocks, and a single thread doing both products of every
-        // item became the bound of the kernel.  So two threads split the work: one issues S = Q K^T (and
-        // frees Q stages), the other O = P V (and frees K/V buffers).  S of item i+NWG reuses the columns
-        // of S/P of item i, so the S issuer waits for that item's P V product to COMPLETE (bar_pv_done).
+        // item became the bound of the kernel.  So the work is split: two threads issue S = Q K^T (even and odd
+        // items: nothing orders the scores of different items; each satisfied wait and each MMA costs such a thread
+        // about 250 clocks, 1300 per item, which alone set the pace of the kernel with one thread) and free Q stages,
+        // a third issues O = P V (and frees K/V buffers).  S of item i+NWG reuses the columns of S/P of item i, so
+        // an S issuer waits for that item's P V product to COMPLETE (bar_pv_done).
         if (elect_one()) {
             struct Cursor { int i, s, sph, w, n, g, t; };
             const int t_first = item0 - bh0 * args.tiles_per_bh;
@@ -262,16 +267,25 @@ cross2_attention_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid
             };
             Cursor c = {0, 0, 0, 0, 0, 0, t_first};
             bool ok = true;
-            if (warp == S_ISSUER_WARP) {
+            if (warp != O_ISSUER_WARP) {
+                const int parity = warp == S_ISSUER_WARP ? 0 : 1;
                 const uint32_t idesc_s = idesc_f16(TILE_M, X2_KN, false, false, args.negate != 0);
                 const int ksteps_s = (args.d + 15) / 16;
                 const uint64_t q_desc0 = smem_desc_sw128(q_smem, 16, 1024);
                 const uint64_t k_desc0 = smem_desc_sw128(kv_smem, 16, 1024);
                 const uint32_t q_stage_off = q_bytes >> 4, kv_buf_off = (2 * kv_bytes) >> 4;
+                int g_waited = -1;   // K and V of this head have been seen to land
                 for (; c.i < n_local && ok; advance(c)) {
+                    if ((c.i & 1) != parity) continue;
+                    X2_TRACE(NWG, c.i, 5);
                     ok = (DENSE_Q ? mbar_wait(smem_u32(&bar_q_ready[c.w]), c.n & 1, abort_p, args.status, SITE_Y_STAGE, c.i)
-                                  : mbar_wait(smem_u32(&bar_full[c.s]), c.sph, abort_p, args.status, SITE_Y_STAGE, c.i)) &&
-                         mbar_wait(smem_u32(&bar_kv_full[c.g & 1]), (c.g >> 1) & 1, abort_p, args.status, SITE_Y_KV, c.i);
+                                  : mbar_wait(smem_u32(&bar_full[c.s]), c.sph, abort_p, args.status, SITE_Y_STAGE, c.i));
+                    X2_TRACE(NWG, c.i, 6);
+                    if (ok && c.g != g_waited) {
+                        ok = mbar_wait(smem_u32(&bar_kv_full[c.g & 1]), (c.g >> 1) & 1, abort_p, args.status, SITE_Y_KV, c.i);
+                        g_waited = c.g;
+                    }
+                    X2_TRACE(NWG, c.i, 7);
                     if (ok && c.n >= 1)   // the group's previous item no longer needs these columns
                         ok = mbar_wait(smem_u32(&bar_pv_done[c.w]), (c.n - 1) & 1, abort_p, args.status, SITE_Y_PV, c.i);
                     if (!ok) break;
@@ -435,14 +449,52 @@ cross2_attention_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid
             // bar_o_full[w] completes after the O issuer saw bar_p_full[w], which the softmax warps arrived on after
             // writing inv_sum: the values are in shared memory by then.  (bar_p_full itself must not be waited on
             // here: a second consumer may fall two phases behind, and a parity wait cannot tell.)
+            if (DENSE_Q && tid == EPILOGUE_WARP0 * 32) bulk_wait_read<1>();   // staging tile i & 1 has been read out
             ok = mbar_wait(smem_u32(&bar_o_full[w]), n & 1, abort_p, args.status, SITE_Y_O, i);
-            ok = __all_sync(0xffffffffu, ok);
+            // one verdict for the whole warpgroup (its warps meet at a named barrier below: none may leave alone);
+            // the barrier also publishes the bulk_wait_read above
+            ok = DENSE_Q ? named_barrier_and(1, 128, ok) : __all_sync(0xffffffffu, ok);
             if (!ok) break;
             tc_fence_after_sync();
             if (tracer) X2_TRACE(w, i, 3);
             const float inv = inv_sum[w][n & 1][r];
             const int row = tile * TILE_M + r;
             __half* orow = args.out + ((size_t)bh * args.Nq + row) * args.d;
+            if (DENSE_Q) {
+                // The tile is one contiguous piece of global memory: rows go to a dense staging tile in shared memory
+                // (thread = row) and ONE bulk copy writes it out -- full lines instead of five strided 16-byte stores
+                // per thread.  Two staging tiles: the copy of the item before last must have read its tile.
+                const uint32_t stage = out_smem + (i & 1) * raw_bytes;
+                uint32_t x[48];
+                tmem_ld32(tmem_o, &x[0]);
+                if (dpad > 32) tmem_ld16(tmem_o + 32, *reinterpret_cast<uint32_t(*)[16]>(&x[32]));
+                tmem_wait_ld();
+                tc_fence_before_sync();
+                if (lane == 0) mbar_arrive(smem_u32(&bar_o_free[w]));   // O_w is in registers
+                const uint32_t dst = stage + r * (args.d * 2);
+#pragma unroll
+                for (int g = 0; g < 6; ++g) {
+                    uint4 v8;
+                    v8.x = pack_half2(__uint_as_float(x[g * 8 + 0]) * inv, __uint_as_float(x[g * 8 + 1]) * inv);
+                    v8.y = pack_half2(__uint_as_float(x[g * 8 + 2]) * inv, __uint_as_float(x[g * 8 + 3]) * inv);
+                    v8.z = pack_half2(__uint_as_float(x[g * 8 + 4]) * inv, __uint_as_float(x[g * 8 + 5]) * inv);
+                    v8.w = pack_half2(__uint_as_float(x[g * 8 + 6]) * inv, __uint_as_float(x[g * 8 + 7]) * inv);
+                    if (g * 8 + 8 <= args.d) st_shared_v4(dst + g * 16, v8);
+                }
+                fence_proxy_async_smem();   // generic-proxy stores before the bulk copy reads them
+                named_barrier(1, 128);
+                if (tid == EPILOGUE_WARP0 * 32) {
+                    int rows = args.Nq - tile * TILE_M;
+                    if (rows > TILE_M) rows = TILE_M;
+                    bulk_store(args.out + ((size_t)bh * args.Nq + (size_t)tile * TILE_M) * args.d, stage,
+                               (uint32_t)rows * args.d * 2);
+                    bulk_commit();
+                }
+                if (tracer) X2_TRACE(w, i, 4);
+                if (++w == NWG) { w = 0; ++n; }
+                if (++tile == args.tiles_per_bh) { tile = 0; ++bh; }
+                continue;
+            }
             // O / S_i -> fp16 -> global, 32 columns per tensor-memory round trip (dpad is a multiple of 16)
             for (int c0 = 0; c0 < dpad; c0 += 32) {
                 uint32_t x[32];
@@ -469,6 +521,7 @@ cross2_attention_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid
             if (++w == NWG) { w = 0; ++n; }
             if (++tile == args.tiles_per_bh) { tile = 0; ++bh; }
         }
+        if (DENSE_Q && tid == EPILOGUE_WARP0 * 32) bulk_wait_all();   // shared memory must outlive the copies
     }
 
     // ------------------------------------------------------------ teardown (every thread arrives)
