@@ -231,9 +231,6 @@ cross2_attention_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid
                     break;
                 X2_TRACE(NWG + 1, i, 0);
                 const uint32_t bar = smem_u32(&bar_full[s]), dst = q_smem + s * q_bytes;
-#ifdef SD_ATTN_X_NOQ
-                if (i >= stages) { mbar_arrive(bar); continue; }
-#endif
                 if (DENSE_Q) {
                     int rows = args.Nq - tile * TILE_M;
                     if (rows > TILE_M) rows = TILE_M;

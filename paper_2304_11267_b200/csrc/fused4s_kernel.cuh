@@ -27,6 +27,7 @@
 
 namespace sd_attn {
 
+// Trace builds only: coarse timeline of CTA (0, 0) -- globaltimer and clock64 at mark i -- behind the per-role stamps.
 #ifdef SD_ATTN_TRACE
 #define F4S_MARK(i)                                                                                   \
     do {                                                                                              \
@@ -265,7 +266,7 @@ fused4s_attention_kernel(const __grid_constant__ CUtensorMap tmap_q, const __gri
             float m_run = 0.f;   // anchor of the exponent: a bound on the running max, times scale*log2(e)
             float l_run = 0.f;   // running sum of p (relative to m_run)
             bool ok = true;
-            const bool tracer = false;
+            const bool tracer = (warp & 3) == 0 && lane == 0;
             // step k = T*j + t uses buffer k % NB; k grows by T = NB - 1 per key tile, so the buffer index walks down and
             // tile t meets each buffer every NB key tiles: phase (j / NB) & 1 of that (tile, buffer) barrier pair
             int b = t % NB, ph = 0, jm = 0;
@@ -306,11 +307,7 @@ fused4s_attention_kernel(const __grid_constant__ CUtensorMap tmap_q, const __gri
                         exp2_pack_32_masked(&s[0], c2, neg_mc, 0, valid, &packed[0], tile_sum);
                         exp2_pack_32_masked(&s[32], c2, neg_mc, 32, valid, &packed[16], tile_sum);
                     }
-#ifdef SD_ATTN_X_NORARE
-                    const bool over = false;
-#else
                     const bool over = !(tile_sum <= FUSED_TILE_SUM_LIMIT);
-#endif
                     if (attempt == 1 || !__any_sync(0xffffffffu, over)) break;
                     // Rare: a row of this warp met a score far above its anchor.  O_t may be touched once the P V
                     // product of key tile j-1 has completed (that of j-2 has: see the wait before the hand-off below);
