@@ -452,9 +452,11 @@ static int launch_fused4s(sd_attn_handle* h, const Problem& p) {
         }
     }
     if (h->fused4_tiles_override > 0 && h->fused4_tiles_override <= max_tiles) a.tiles_per_cta = h->fused4_tiles_override;
-    a.stages = (F4S_SMEM_BUDGET - a.tiles_per_cta * q_tile_bytes) / stage_bytes;
+    // one chunk per row: the kernel lays out four tile slots and eight stages whatever tiles_per_cta is (192 KB)
+    const int tile_slots = a.nch == 1 ? F4_TILES : a.tiles_per_cta;
+    a.stages = (F4S_SMEM_BUDGET - tile_slots * q_tile_bytes) / stage_bytes;
     if (a.stages > F4_STAGES) a.stages = F4_STAGES;
-    const size_t smem = (size_t)a.tiles_per_cta * q_tile_bytes + (size_t)a.stages * stage_bytes + 1024;
+    const size_t smem = (size_t)tile_slots * q_tile_bytes + (size_t)a.stages * stage_bytes + 1024;
     CUtensorMap tq, tk, tv;
     int rc = make_tmap(h, &tq, p.q, p.BH, p.Nq, p.d, TILE_M);
     if (rc == SD_ATTN_OK) rc = make_tmap(h, &tk, p.k, p.BH, p.Nk, p.d, F4_BN);

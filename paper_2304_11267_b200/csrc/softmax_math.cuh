@@ -126,9 +126,7 @@ __device__ __forceinline__ void exp2_pack_32(const uint32_t* s, uint64_t c2c2, u
             p0 = ex2_approx(__uint_as_float(x0));
             p1 = ex2_approx(__uint_as_float(x1));
         }
-#ifndef SD_ATTN_X_NOSUM
         acc[k & 1] = add_f32x2(acc[k & 1], pack_b64(__float_as_uint(p0), __float_as_uint(p1)));
-#endif
         packed[k] = pack_half2(p0, p1);
     }
 }
