@@ -448,7 +448,7 @@ cross2_attention_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid
             // here: a second consumer may fall two phases behind, and a parity wait cannot tell.)
             if (DENSE_Q && tid == EPILOGUE_WARP0 * 32) bulk_wait_read<1>();   // staging tile i & 1 has been read out
             ok = mbar_wait(smem_u32(&bar_o_full[w]), n & 1, abort_p, args.status, SITE_Y_O, i);
-            // one verdict for the whole warpgroup (its warps meet at a named barrier below: none may leave alone);
+            // one decision for the whole warpgroup (its warps meet at a named barrier below: none may leave alone);
             // the barrier also publishes the bulk_wait_read above
             ok = DENSE_Q ? named_barrier_and(1, 128, ok) : __all_sync(0xffffffffu, ok);
             if (!ok) break;

@@ -303,6 +303,35 @@ def test_every_variant_of_the_small_head_dim_kernel(bd, env, monkeypatch):
         a.close()
 
 
+@pytest.mark.parametrize("env", [{"SD_ATTN_CROSS_ONE_TILE": "1"}, {"SD_ATTN_NO_PDL": "1"}, {}],
+                         ids=lambda e: "-".join("%s=%s" % kv for kv in e.items()) or "default")
+def test_cross_attention_variants_over_head_dims_and_ragged_rows(bd, env, monkeypatch):
+    """77 and other key counts of one tile, every head-dim class (four, three, two softmax groups), row counts that
+    leave a CTA with a partial tile, fewer items than SMs and more: the persistent kernel and its one-tile fallback."""
+    for k, v in env.items():
+        monkeypatch.setenv(k, v)
+    a = bd.Attention()
+    try:
+        for n, (B, H, Nq, Nk, d, qmult) in enumerate([(2, 8, 4096, 77, 40, 1.0), (1, 3, 1000, 77, 40, 4.0),
+                                                       (2, 2, 333, 70, 80, 1.0), (1, 2, 130, 80, 160, 4.0),
+                                                       (1, 1, 64, 66, 48, 1.0), (3, 50, 129, 77, 24, 1.0)]):
+            q, k, v = rand_qkv(6100 + n, B, H, Nq, Nk, d, qmult=qmult)
+            scale = float(np.float32(1.0 / np.sqrt(d)))
+            rows = None
+            if B * H * Nq > 40000:
+                rows = np.arange(0, B * H * Nq, 7, dtype=np.int64)
+            ref, _, _ = oracle.forward(q, k, v, scale, rows=rows)
+            out = a.forward(gpu(q), gpu(k), gpu(v), scale=scale)
+            a.check()
+            assert a.last_mode == bd.MODE_CROSS
+            got = out.cpu().numpy()
+            if rows is not None:
+                got = got.reshape(-1, d)[rows]
+            check(got, ref, v, what="%s shape %d" % (env, n))
+    finally:
+        a.close()
+
+
 @pytest.mark.parametrize("shape", [(1, 4, 512, 512, 40), (2, 2, 256, 77, 80), (1, 2, 130, 300, 160)])
 def test_back_to_back_calls_that_depend_on_one_another(att, bd, shape):
     """Calls queued on one stream without synchronisation, each reading what the previous one wrote and writing
