@@ -142,6 +142,11 @@ cross2_attention_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid
 #endif
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     if (threadIdx.x == 0) pdl_launch_dependents();   // the next kernel of the stream may start its set-up
+    if (threadIdx.x == 32) {   // the tensor maps are kernel parameters: their fetch need not wait for anything
+        tma_prefetch_desc(&tmap_q);
+        tma_prefetch_desc(&tmap_k);
+        tma_prefetch_desc(&tmap_v);
+    }
     const int nch = args.nch, dpad = args.dpad, stages = args.stages;
     // contiguous range of items for this CTA: consecutive items share a head, so K and V are fetched rarely
     const int per = args.n_items / gridDim.x, extra = args.n_items % gridDim.x;
@@ -206,9 +211,6 @@ cross2_attention_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid
     if (warp == LOADER_WARP) {
         // ------------------------------------------------------------ TMA producer
         if (elect_one()) {
-            tma_prefetch_desc(&tmap_q);
-            tma_prefetch_desc(&tmap_k);
-            tma_prefetch_desc(&tmap_v);
             int g_prev = -1;
             for (int i = 0; i < n_local; ++i) {
                 const int item = item0 + i, bh = item / args.tiles_per_bh, tile = item - bh * args.tiles_per_bh;

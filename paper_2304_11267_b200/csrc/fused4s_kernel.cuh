@@ -79,6 +79,11 @@ fused4s_attention_kernel(const __grid_constant__ CUtensorMap tmap_q, const __gri
     const int tid = threadIdx.x, lane = tid & 31;
     const int warp = __shfl_sync(0xffffffffu, tid >> 5, 0);   // warp-uniform for the compiler
     if (threadIdx.x == 0) pdl_launch_dependents();   // the next kernel of the stream may start its set-up
+    if (threadIdx.x == 32) {   // the tensor maps are kernel parameters: their fetch need not wait for anything
+        tma_prefetch_desc(&tmap_q);
+        tma_prefetch_desc(&tmap_k);
+        tma_prefetch_desc(&tmap_v);
+    }
     const int bh = blockIdx.y;
     const int row_base = blockIdx.x * args.tiles_per_cta * TILE_M;
 #ifdef SD_ATTN_TRACE
@@ -141,9 +146,6 @@ fused4s_attention_kernel(const __grid_constant__ CUtensorMap tmap_q, const __gri
     if (warp == 16) {
         // ------------------------------------------------------------ TMA producer
         if (elect_one()) {
-            tma_prefetch_desc(&tmap_q);
-            tma_prefetch_desc(&tmap_k);
-            tma_prefetch_desc(&tmap_v);
             // In the order the issuers need them: Q_0 and the first key tile first (a tile of 80-byte rows costs the
             // TMA unit about 7 clocks per row, so the order decides when the first scores can start).
             auto load_q = [&](int t) {
