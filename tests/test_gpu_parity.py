@@ -360,6 +360,36 @@ def test_back_to_back_calls_that_depend_on_one_another(att, bd, shape):
     assert np.abs(got.astype(np.float64) - ref).max() <= chain * F16_ABS * vmax
 
 
+@pytest.mark.parametrize("Nk", [129, 130, 191, 192, 193, 255, 257, 4095, 4097])
+def test_every_ragged_tail_of_the_key_tiles(att, bd, Nk):
+    """Key counts around the 64-key tile boundaries: the zero-filled keys of the last tile must get weight zero."""
+    q, k, v = rand_qkv(7000 + Nk, 1, 2, 150, Nk, 40, qmult=2.0)
+    scale = float(np.float32(1.0 / np.sqrt(40)))
+    ref, _, _ = oracle.forward(q, k, v, scale)
+    check(run(att, bd, bd.MODE_FUSED, q, k, v, scale), ref, v, what="Nk=%d" % Nk)
+
+
+def test_many_heads_and_bitwise_agreement_between_tile_counts(bd, monkeypatch):
+    """640 (batch, head) problems in one call; and the number of query tiles a CTA takes changes the schedule, not
+    the arithmetic of a row: the outputs of the variants must agree bit for bit."""
+    q, k, v = rand_qkv(7100, 16, 40, 130, 200, 40)
+    scale = float(np.float32(1.0 / np.sqrt(40)))
+    rows = np.arange(0, 16 * 40 * 130, 11, dtype=np.int64)
+    ref, _, _ = oracle.forward(q, k, v, scale, rows=rows)
+    outs = []
+    for tiles in ("1", "2", "4"):
+        monkeypatch.setenv("SD_ATTN_FUSED_TILES", tiles)
+        a = bd.Attention(bd.MODE_FUSED)
+        try:
+            out = a.forward(gpu(q), gpu(k), gpu(v), scale=scale)
+            a.check()
+            outs.append(out.cpu().numpy())
+        finally:
+            a.close()
+        check(outs[-1].reshape(-1, 40)[rows], ref, v, what="tiles per CTA %s" % tiles)
+    assert np.array_equal(outs[0], outs[1]) and np.array_equal(outs[0], outs[2])
+
+
 def test_padding_rows_with_distinct_values_only_see_their_mean(att, bd):
     call = workloads.config3()[0]
     q, k, v = workloads.make_inputs(call)
