@@ -57,8 +57,13 @@ __host__ inline int f4s_max_tiles(int dpad) {   // (T + 1) * 64 + T * dpad <= 51
 #endif
 constexpr int F4S_POLY_PER8 = SD_ATTN_F4S_POLY_PER8;
 constexpr int F4S_BUFFERS = F4_TILES + 1;
-constexpr int F4S_SOFTMAX_REGS = 104;   // 512 * 104 + 256 * 32 = 768 * 80, the launch allocation
-constexpr int F4S_CONTROL_REGS = 32;
+#ifndef SD_ATTN_F4S_SOFTMAX_REGS
+#define SD_ATTN_F4S_SOFTMAX_REGS 104   // 512 * 104 + 256 * 32 = 768 * 80, the launch allocation
+#define SD_ATTN_F4S_CONTROL_REGS 32
+#endif
+constexpr int F4S_SOFTMAX_REGS = SD_ATTN_F4S_SOFTMAX_REGS;
+constexpr int F4S_CONTROL_REGS = SD_ATTN_F4S_CONTROL_REGS;
+static_assert(512 * F4S_SOFTMAX_REGS + 256 * F4S_CONTROL_REGS == 768 * 80, "setmaxnreg budget");
 
 template <int POLY, int NCH>   // NCH: 64-column chunks per row (head dim <= 64 * NCH)
 __global__ void __launch_bounds__(F4_THREADS, 1)
