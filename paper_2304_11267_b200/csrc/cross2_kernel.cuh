@@ -211,7 +211,7 @@ cross2_attention_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid
     if (warp == LOADER_WARP) {
         // ------------------------------------------------------------ TMA producer
         if (elect_one()) {
-            int g_prev = -1;
+            int g_prev = 0;   // K and V of the first head: fetched by the first S issuer, at the same time as Q here
             for (int i = 0; i < n_local; ++i) {
                 const int item = item0 + i, bh = item / args.tiles_per_bh, tile = item - bh * args.tiles_per_bh;
                 const int s = i % stages, g = bh - bh0;
@@ -266,6 +266,16 @@ cross2_attention_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid
             };
             Cursor c = {0, 0, 0, 0, 0, 0, t_first};
             bool ok = true;
+            if (warp == S_ISSUER_WARP && n_local > 0) {
+                // K and V of the CTA's first head, while the producer thread fetches the first Q tiles: a copy
+                // instruction holds its thread for several hundred clocks, and the first scores wait for all three.
+                const uint32_t bar = smem_u32(&bar_kv_full[0]);
+                mbar_arrive_expect_tx(bar, 2 * kv_bytes);
+                for (int ch = 0; ch < nch; ++ch)
+                    tma_load_3d(kv_smem + ch * X2_KN * CHUNK_ROW_BYTES, &tmap_k, bar, ch * CHUNK_COLS, 0, bh0);
+                for (int ch = 0; ch < nch; ++ch)
+                    tma_load_3d(kv_smem + kv_bytes + ch * X2_KN * CHUNK_ROW_BYTES, &tmap_v, bar, ch * CHUNK_COLS, 0, bh0);
+            }
             if (warp != O_ISSUER_WARP) {
                 const int parity = warp == S_ISSUER_WARP ? 0 : 1;
                 const uint32_t idesc_s = idesc_f16(TILE_M, X2_KN, false, false, args.negate != 0);
