@@ -64,8 +64,9 @@ typedef enum {
 /*
  * Create a handle on the CURRENT CUDA device.  Checks the architecture (ERR_ARCH unless
  * compute capability 10.x), resolves the driver's tensor-map encoder, raises the kernels'
- * dynamic shared-memory limits and allocates one 64-byte device status block.  No stream
- * work.  *out receives the handle (NULL on failure).
+ * dynamic shared-memory limits, allocates one 64-byte device status block and creates the two
+ * copy streams and ten events sd_attn_forward_host uses.  No stream work.  *out receives the
+ * handle (NULL on failure).
  *
  * Switches read from the environment at this call (all default off; they select slower variants that exist
  * for comparison and testing, results are the same within the tolerance):
@@ -77,6 +78,7 @@ typedef enum {
  *   SD_ATTN_FUSED_NO_SPARE=1    FUSED: the four-tile kernel without the spare score buffer (d <= 64)
  *   SD_ATTN_FUSED_TWO_TILE=1    FUSED: the two-tile kernel
  *   SD_ATTN_CROSS_ONE_TILE=1    CROSS: one tile per CTA also for 65..80 keys
+ *   SD_ATTN_HOST_ONE_SLICE=1    sd_attn_forward_host: one slice, copies and kernel all on the caller's stream
  */
 int sd_attn_create(sd_attn_handle **out);
 
@@ -98,10 +100,14 @@ int sd_attn_forward(sd_attn_handle *h, const void *q, const void *k, const void 
  * The same operation (Eq. 3) for callers whose tensors live in HOST memory: q, k, v, out are HOST
  * pointers (pinned memory makes the copies asynchronous; pageable memory works but serialises).
  * `staging` is caller-owned DEVICE scratch of at least sd_attn_host_staging_bytes(...) bytes,
- * 256-byte aligned.  Enqueues on `stream`: three host-to-device copies, sd_attn_forward on the
- * staged tensors, one device-to-host copy of the result.  Does not synchronise: `out` is valid
- * once the stream has drained.  Errors as sd_attn_forward, plus WORKSPACE if `staging` is NULL,
- * misaligned or too small.
+ * 256-byte aligned.  The work is the host-to-device copies of q, k and v, sd_attn_forward on the
+ * staged tensors and the device-to-host copy of the result.  The (batch, head) range is cut into up
+ * to four slices (independent problems) whose copies run on two streams owned by the handle, so that
+ * the copies of one slice overlap the kernel of another; the slices are forked from `stream` and
+ * joined back into it by events, so for the caller the call is one piece of stream-ordered work on
+ * `stream`.  (One slice, everything on `stream`, in TWOPASS mode or when a head of q or k is not a
+ * multiple of 16 bytes.)  Does not synchronise: `out` is valid once the stream has drained.  Errors
+ * as sd_attn_forward, plus WORKSPACE if `staging` is NULL, misaligned or too small.
  */
 int sd_attn_forward_host(sd_attn_handle *h, const void *q, const void *k, const void *v, void *out,
                          void *staging, size_t staging_bytes, int B, int H, int Nq, int Nk, int d,

@@ -37,6 +37,8 @@ struct TmapCacheEntry {
 };
 constexpr int TMAP_CACHE_ENTRIES = 128;
 
+constexpr int HOST_SLICES = 4;   // sd_attn_forward_host cuts the (batch, head) range into at most this many slices
+
 struct sd_attn_handle {
     TmapCacheEntry tmap_cache[TMAP_CACHE_ENTRIES];
     int tmap_cache_next;
@@ -62,6 +64,10 @@ struct sd_attn_handle {
     int cross2_four_ok;
     int cross_one_tile_only;  // SD_ATTN_CROSS_ONE_TILE=1: never use the persistent cross-attention kernel
     int prefer_two_tile;      // SD_ATTN_FUSED_TWO_TILE=1: use the two-tile fused kernel for every head dim
+    // sd_attn_forward_host: copies of one slice of heads overlap the kernel of another (see there)
+    cudaStream_t copy_in, copy_out;
+    cudaEvent_t ev_fork, ev_join, ev_in[HOST_SLICES], ev_done[HOST_SLICES];
+    int host_overlap;         // the streams and events above exist
 };
 
 static const float LOG2E = 1.4426950408889634f;
@@ -108,6 +114,33 @@ static cudaError_t launch_overlapped(const sd_attn_handle* h, void (*kernel)(KAr
 template <typename K>
 static cudaError_t raise_smem_limit(K kernel, size_t bytes) {
     return cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bytes);
+}
+
+// Two copy streams and the events that tie them to the caller's stream in sd_attn_forward_host.
+static cudaError_t create_host_overlap(sd_attn_handle* h) {
+    cudaError_t e = cudaStreamCreateWithFlags(&h->copy_in, cudaStreamNonBlocking);
+    if (e == cudaSuccess) e = cudaStreamCreateWithFlags(&h->copy_out, cudaStreamNonBlocking);
+    if (e == cudaSuccess) e = cudaEventCreateWithFlags(&h->ev_fork, cudaEventDisableTiming);
+    if (e == cudaSuccess) e = cudaEventCreateWithFlags(&h->ev_join, cudaEventDisableTiming);
+    for (int c = 0; c < HOST_SLICES && e == cudaSuccess; ++c) {
+        e = cudaEventCreateWithFlags(&h->ev_in[c], cudaEventDisableTiming);
+        if (e == cudaSuccess) e = cudaEventCreateWithFlags(&h->ev_done[c], cudaEventDisableTiming);
+    }
+    const char* one = getenv("SD_ATTN_HOST_ONE_SLICE");
+    h->host_overlap = e == cudaSuccess && !(one && one[0] == '1');
+    return e;
+}
+
+static void destroy_host_overlap(sd_attn_handle* h) {   // the handle was calloc'ed: what was never created is null
+    for (int c = 0; c < HOST_SLICES; ++c) {
+        if (h->ev_in[c]) cudaEventDestroy(h->ev_in[c]);
+        if (h->ev_done[c]) cudaEventDestroy(h->ev_done[c]);
+    }
+    if (h->ev_fork) cudaEventDestroy(h->ev_fork);
+    if (h->ev_join) cudaEventDestroy(h->ev_join);
+    if (h->copy_in) cudaStreamDestroy(h->copy_in);
+    if (h->copy_out) cudaStreamDestroy(h->copy_out);
+    h->host_overlap = 0;
 }
 
 extern "C" int sd_attn_create(sd_attn_handle** out) {
@@ -189,7 +222,9 @@ extern "C" int sd_attn_create(sd_attn_handle** out) {
     }
     if (e == cudaSuccess) e = cudaMalloc((void**)&h->dev_status, sizeof(int) * DEV_STATUS_INTS);
     if (e == cudaSuccess) e = cudaMemset(h->dev_status, 0, sizeof(int) * DEV_STATUS_INTS);
+    if (e == cudaSuccess) e = create_host_overlap(h);
     if (e != cudaSuccess) {
+        destroy_host_overlap(h);
         if (h->dev_status) cudaFree(h->dev_status);
         free(h);
         return cuda_fail(nullptr, e);
@@ -201,6 +236,7 @@ extern "C" int sd_attn_create(sd_attn_handle** out) {
 extern "C" int sd_attn_destroy(sd_attn_handle* h) {
     if (!h) return SD_ATTN_OK;
     cudaError_t e = cudaSuccess;
+    destroy_host_overlap(h);
     if (h->dev_status) e = cudaFree(h->dev_status);
     free(h);
     return e == cudaSuccess ? SD_ATTN_OK : SD_ATTN_ERR_CUDA;
@@ -599,6 +635,46 @@ extern "C" int sd_attn_forward_host(sd_attn_handle* h, const void* q, const void
     char* dv = dk + round256(k_bytes);
     char* dout = dv + round256(k_bytes);
     cudaStream_t s = (cudaStream_t)stream;
+    // Slices of the (batch, head) range are independent problems.  With more than one, the copies run on two streams
+    // of the handle -- host to device of slice c + 1 and device to host of slice c - 1 while the kernel of slice c
+    // runs on the caller's stream -- forked from and joined back into the caller's stream by events, so that for the
+    // caller the call is still one piece of stream-ordered work.  (Not in TWOPASS mode: its workspace and the
+    // pointers sd_attn_twopass_buffers returns describe one whole call.)
+    const int BH = B * H;
+    const size_t q_head = (size_t)Nq * d * es, k_head = (size_t)Nk * d * es;
+    const bool sliceable = h->host_overlap && h->mode != SD_ATTN_MODE_TWOPASS &&
+                           q_head % 16 == 0 && k_head % 16 == 0;   // every slice starts 16-byte aligned
+    const int slices = sliceable ? (BH < HOST_SLICES ? BH : HOST_SLICES) : 1;
+    if (slices > 1) {
+        cudaError_t e = cudaEventRecord(h->ev_fork, s);
+        if (e == cudaSuccess) e = cudaStreamWaitEvent(h->copy_in, h->ev_fork, 0);
+        if (e == cudaSuccess) e = cudaStreamWaitEvent(h->copy_out, h->ev_fork, 0);
+        if (e != cudaSuccess) return cuda_fail(h, e);
+        int rc = SD_ATTN_OK;
+        for (int c = 0; c < slices && e == cudaSuccess && rc == SD_ATTN_OK; ++c) {
+            const int h0 = (int)((long long)BH * c / slices), h1 = (int)((long long)BH * (c + 1) / slices);
+            const size_t qo = q_head * h0, ko = k_head * h0, qn = q_head * (h1 - h0), kn = k_head * (h1 - h0);
+            e = cudaMemcpyAsync(dq + qo, (const char*)q + qo, qn, cudaMemcpyHostToDevice, h->copy_in);
+            if (e == cudaSuccess) e = cudaMemcpyAsync(dk + ko, (const char*)k + ko, kn, cudaMemcpyHostToDevice, h->copy_in);
+            if (e == cudaSuccess) e = cudaMemcpyAsync(dv + ko, (const char*)v + ko, kn, cudaMemcpyHostToDevice, h->copy_in);
+            if (e == cudaSuccess) e = cudaEventRecord(h->ev_in[c], h->copy_in);
+            if (e == cudaSuccess) e = cudaStreamWaitEvent(s, h->ev_in[c], 0);
+            if (e != cudaSuccess) break;
+            rc = sd_attn_forward(h, dq + qo, dk + ko, dv + ko, dout + qo, 1, h1 - h0, Nq, Nk, d, scale, dtype, stream);
+            if (rc != SD_ATTN_OK) break;
+            e = cudaEventRecord(h->ev_done[c], s);
+            if (e == cudaSuccess) e = cudaStreamWaitEvent(h->copy_out, h->ev_done[c], 0);
+            if (e == cudaSuccess) e = cudaMemcpyAsync((char*)out + qo, dout + qo, qn, cudaMemcpyDeviceToHost, h->copy_out);
+        }
+        // join in every case: the caller's stream must not run ahead of copies that were enqueued
+        cudaError_t ej = cudaEventRecord(h->ev_join, h->copy_out);
+        if (ej == cudaSuccess) ej = cudaStreamWaitEvent(s, h->ev_join, 0);
+        if (ej == cudaSuccess) ej = cudaEventRecord(h->ev_join, h->copy_in);
+        if (ej == cudaSuccess) ej = cudaStreamWaitEvent(s, h->ev_join, 0);
+        if (rc != SD_ATTN_OK) return rc;
+        if (e != cudaSuccess || ej != cudaSuccess) return cuda_fail(h, e != cudaSuccess ? e : ej);
+        return SD_ATTN_OK;
+    }
     cudaError_t e = cudaMemcpyAsync(dq, q, q_bytes, cudaMemcpyHostToDevice, s);
     if (e == cudaSuccess) e = cudaMemcpyAsync(dk, k, k_bytes, cudaMemcpyHostToDevice, s);
     if (e == cudaSuccess) e = cudaMemcpyAsync(dv, v, k_bytes, cudaMemcpyHostToDevice, s);

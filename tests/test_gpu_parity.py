@@ -493,6 +493,64 @@ def test_forward_host_with_pinned_buffers(att, bd):
     check(hout.numpy(), ref, v, what="forward_host")
 
 
+@pytest.mark.parametrize("B,H,Nq,Nk,d,dtype", [
+    (1, 1, 200, 200, 40, "f16"),     # one head: one slice, everything on the caller's stream
+    (1, 3, 300, 77, 40, "f16"),      # fewer heads than slices
+    (2, 5, 260, 260, 80, "f16"),     # ten heads in four uneven slices
+    (1, 6, 70, 90, 36, "f32"),       # fp32, heads of 16-byte multiples
+    (1, 4, 3, 5, 5, "f32"),          # heads that are not multiples of 16 bytes: not sliced
+])
+def test_forward_host_slices_on_a_side_stream(att, bd, B, H, Nq, Nk, d, dtype):
+    """The host-buffer call cuts (batch, head) into slices whose copies overlap other slices' kernels on the handle's
+    own streams; to the caller it must still behave as stream-ordered work: back-to-back calls that reuse the same
+    staging and host buffers, on a stream that is not the default one, each give their own result."""
+    np_t, code = (np.float16, bd.F16) if dtype == "f16" else (np.float32, bd.F32)
+    side = torch.cuda.Stream()
+    need = bd.sd_attn_host_staging_bytes(B, H, Nq, Nk, d, code)
+    staging = torch.empty(need, dtype=torch.uint8, device="cuda")
+    results, refs, vs = [], [], []
+    with torch.cuda.stream(side):
+        for seed in (11, 12, 13):
+            q, k, v = rand_qkv(seed, B, H, Nq, Nk, d, dtype=np_t)
+            hq, hk, hv = (torch.from_numpy(x).pin_memory() for x in (q, k, v))
+            hout = torch.zeros(q.shape, dtype=hq.dtype).pin_memory()
+            rc = bd.sd_attn_forward_host(att.handle, hq.data_ptr(), hk.data_ptr(), hv.data_ptr(), hout.data_ptr(),
+                                         staging.data_ptr(), need, B, H, Nq, Nk, d, 0.3, code, side.cuda_stream)
+            assert rc == bd.OK
+            results.append((hq, hk, hv, hout))
+            refs.append(oracle.forward(q, k, v, 0.3)[0])
+            vs.append(v)
+    att.check(side.cuda_stream)
+    for (_, _, _, hout), ref, v in zip(results, refs, vs):
+        check(hout.numpy(), ref, v, dtype=np_t, what="forward_host slices")
+
+
+def test_forward_host_in_twopass_mode_is_one_call(att, bd):
+    call = workloads.config1()[0]
+    q, k, v = workloads.make_inputs(call)
+    ref, _, _ = oracle.forward(q, k, v, call.scale())
+    hq, hk, hv = (torch.from_numpy(x).pin_memory() for x in (q, k, v))
+    hout = torch.empty_like(hq).pin_memory()
+    need = bd.sd_attn_host_staging_bytes(call.B, call.H, call.Nq, call.Nk, call.d, bd.F16)
+    staging = torch.empty(need, dtype=torch.uint8, device="cuda")
+    ws_bytes = bd.sd_attn_workspace_bytes(bd.MODE_TWOPASS, call.B, call.H, call.Nq, call.Nk, call.d, bd.F16)
+    ws = torch.empty(ws_bytes, dtype=torch.uint8, device="cuda")
+    stream = torch.cuda.current_stream().cuda_stream
+    assert bd.sd_attn_set_mode(att.handle, bd.MODE_TWOPASS) == bd.OK
+    assert bd.sd_attn_set_workspace(att.handle, ws.data_ptr(), ws_bytes) == bd.OK
+    try:
+        before = att.launch_count
+        assert bd.sd_attn_forward_host(att.handle, hq.data_ptr(), hk.data_ptr(), hv.data_ptr(), hout.data_ptr(),
+                                       staging.data_ptr(), need, call.B, call.H, call.Nq, call.Nk, call.d,
+                                       float(call.scale()), bd.F16, stream) == bd.OK
+        att.check(stream)
+        assert att.launch_count - before == 2      # one scores kernel, one P V kernel: the call was not cut up
+    finally:
+        bd.sd_attn_set_workspace(att.handle, 0, 0)
+        bd.sd_attn_set_mode(att.handle, bd.MODE_AUTO)
+    check(hout.numpy(), ref, v, what="forward_host twopass")
+
+
 def test_forward_is_capturable_in_a_cuda_graph(att, bd):
     calls = workloads.config4()[18:22]      # two self (256 tokens) and two cross calls
     tensors = []
