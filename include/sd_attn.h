@@ -75,6 +75,8 @@ typedef enum {
  *                               while the previous kernel of the stream finishes, and waits for that kernel to
  *                               complete before it reads or writes global memory, so stream order is kept.
  *   SD_ATTN_FUSED_TILES=1..4    fixed number of query tiles per CTA of the FUSED kernel (default: by problem size)
+ *   SD_ATTN_FUSED_NO_SPLIT=1    FUSED, one query tile per CTA: the tile's score columns stay with one warpgroup
+ *   SD_ATTN_FUSED_SPLIT=2|4     FUSED, one query tile per CTA: that many warpgroups share them (default: by head dim)
  *   SD_ATTN_FUSED_NO_SPARE=1    FUSED: the four-tile kernel without the spare score buffer (d <= 64)
  *   SD_ATTN_FUSED_TWO_TILE=1    FUSED: the two-tile kernel
  *   SD_ATTN_CROSS_ONE_TILE=1    CROSS: one tile per CTA also for 65..80 keys

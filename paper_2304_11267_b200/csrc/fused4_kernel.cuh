@@ -44,6 +44,7 @@ struct Fused4Args {
     int tiles_per_cta;   // spare-buffer kernel only: 1..4 query tiles per CTA (small problems spread over more SMs)
     int nch;             // spare-buffer kernel only: 64-column chunks per row (1..3)
     int stages;          // spare-buffer kernel only: K/V ring depth (2..8)
+    int split_buffers;   // spare-buffer kernel, split variant only: score buffers of the lone tile (2..5)
     float scale_log2e;
     int negate;
     int* status;

@@ -19,6 +19,8 @@
 //
 // A CTA takes 1 to 4 query tiles (Fused4Args::tiles_per_cta): the host gives a small problem fewer tiles per CTA so
 // that it spreads over more SMs; with one tile the rotation degenerates to two alternating score buffers.
+// One tile per CTA normally runs the SPLIT variant instead (template parameter, see below): the other softmax
+// warpgroups, idle otherwise, take a share of the tile's score columns each.
 // The anchor scheme of the exponent (no per-tile maximum) is that of fused4_kernel.cuh.
 #pragma once
 #include <cuda.h>
@@ -65,7 +67,13 @@ constexpr int F4S_SOFTMAX_REGS = SD_ATTN_F4S_SOFTMAX_REGS;
 constexpr int F4S_CONTROL_REGS = SD_ATTN_F4S_CONTROL_REGS;
 static_assert(512 * F4S_SOFTMAX_REGS + 256 * F4S_CONTROL_REGS == 768 * 80, "setmaxnreg budget");
 
-template <int POLY, int NCH>   // NCH: 64-column chunks per row (head dim <= 64 * NCH)
+// SPLIT > 1 (only with ONE query tile per CTA): the 64 columns of every score tile are shared out among SPLIT
+// warpgroups, each with an exponent anchor, a row sum and an accumulator O_g of its own over ITS keys (16 or 32 of
+// every 64), combined once at the end.  A lone tile is bound by the chain of latencies of one warp per scheduler
+// (tcgen05.ld -> exp2 -> tcgen05.st -> hand-over: 1400-1500 clocks per key tile, measured, against 600 per tile
+// with four tiles resident); the parts need no agreement on an anchor because their products never share an
+// accumulator.
+template <int POLY, int NCH, int SPLIT = 1>   // NCH: 64-column chunks per row (head dim <= 64 * NCH)
 __global__ void __launch_bounds__(F4_THREADS, 1)
 fused4s_attention_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__ CUtensorMap tmap_k,
                          const __grid_constant__ CUtensorMap tmap_v, const Fused4Args args) {
@@ -78,8 +86,10 @@ fused4s_attention_kernel(const __grid_constant__ CUtensorMap tmap_q, const __gri
     __shared__ __align__(8) uint64_t bar_s_full[F4_TILES][F4S_BUFFERS], bar_p_full[F4_TILES][F4S_BUFFERS];
     __shared__ __align__(8) uint64_t bar_q_full[F4_TILES], bar_pv_done[F4_TILES], bar_o_final[F4_TILES];
     __shared__ __align__(8) uint64_t bar_kv_full[F4_STAGES], bar_kv_empty[F4_STAGES];
+    __shared__ __align__(8) uint64_t bar_buf_free[F4S_BUFFERS];   // SPLIT > 1: the products reading a buffer's weights are done
     __shared__ uint32_t tmem_base_slot;
     __shared__ int abort_flag;
+    __shared__ float2 part_ml[SPLIT > 1 ? SPLIT : 1][SPLIT > 1 ? TILE_M : 1];   // SPLIT > 1: (anchor, row sum) of every part
 
     const int tid = threadIdx.x, lane = tid & 31;
     const int warp = __shfl_sync(0xffffffffu, tid >> 5, 0);   // warp-uniform for the compiler
@@ -102,7 +112,7 @@ fused4s_attention_kernel(const __grid_constant__ CUtensorMap tmap_q, const __gri
 #endif
     int T = (args.Nq - row_base + TILE_M - 1) / TILE_M;   // query tiles of this CTA
     if (T > args.tiles_per_cta) T = args.tiles_per_cta;
-    const int NB = T + 1;                                 // score buffers in the rotation
+    const int NB = SPLIT > 1 ? args.split_buffers : T + 1;   // score buffers in the rotation
     const int n_kv = (args.Nk + BN - 1) / BN;
     const int dpad = args.dpad;
     constexpr int nch = NCH;
@@ -120,12 +130,13 @@ fused4s_attention_kernel(const __grid_constant__ CUtensorMap tmap_q, const __gri
         for (int t = 0; t < F4_TILES; ++t) {
             for (int b = 0; b < F4S_BUFFERS; ++b) {
                 mbar_init(smem_u32(&bar_s_full[t][b]), 1);
-                mbar_init(smem_u32(&bar_p_full[t][b]), 4);    // one arrival per softmax warp of the tile
+                mbar_init(smem_u32(&bar_p_full[t][b]), 4 * SPLIT);    // one arrival per softmax warp of the tile
             }
             mbar_init(smem_u32(&bar_q_full[t]), 1);
             mbar_init(smem_u32(&bar_pv_done[t]), 1);
             mbar_init(smem_u32(&bar_o_final[t]), 1);
         }
+        for (int b = 0; b < F4S_BUFFERS; ++b) mbar_init(smem_u32(&bar_buf_free[b]), 1);
         for (int s = 0; s < F4_STAGES; ++s) {
             mbar_init(smem_u32(&bar_kv_full[s]), 1);
             mbar_init(smem_u32(&bar_kv_empty[s]), T);   // one commit per issuer
@@ -144,7 +155,8 @@ fused4s_attention_kernel(const __grid_constant__ CUtensorMap tmap_q, const __gri
     pdl_wait();
     if (tid == 0) F4S_MARK(0);
     const uint32_t tmem_base = tmem_base_slot;
-    const uint32_t tmem_o0 = tmem_base + (args.tiles_per_cta + 1) * BN;   // columns: the score buffers | O_0 .. O_{T-1}
+    // columns: the score buffers | O_0 .. O_{T-1} (SPLIT > 1: the parts' O_0 .. O_{SPLIT-1})
+    const uint32_t tmem_o0 = tmem_base + (SPLIT > 1 ? args.split_buffers : args.tiles_per_cta + 1) * BN;
 
     // One setmaxnreg site per kind, executed by whole warpgroups; the budget is the CTA's launch allocation.
     if (warp >= 16) setmaxnreg_dec<F4S_CONTROL_REGS>();
@@ -185,13 +197,14 @@ fused4s_attention_kernel(const __grid_constant__ CUtensorMap tmap_q, const __gri
         // product, on the same thread, into the buffer it frees -- the scores of step k + NB, which belong to the
         // NEXT tile of the rotation.
         const int t = warp - 17;
-        if (t < T && elect_one()) {
+        if ((t < T || (SPLIT > 1 && t == 1)) && elect_one()) {
             const uint32_t idesc_s = idesc_f16(TILE_M, BN, false, false, args.negate != 0);
             const uint32_t idesc_o = idesc_f16(TILE_M, dpad, false, true, false);
             const int ksteps_s = (args.d + 15) / 16;   // 16 columns each; four to a swizzled 64-column chunk
             const int tn = (t + 1 == T) ? 0 : t + 1;   // the tile whose scores this thread requests
             const uint64_t q_desc = smem_desc_sw128(q_smem + tn * q_tile_bytes, 16, 1024);
             const uint64_t q_desc_own = smem_desc_sw128(q_smem + t * q_tile_bytes, 16, 1024);
+            const uint64_t q_desc_own_split = smem_desc_sw128(q_smem, 16, 1024);   // SPLIT > 1: the one tile
             const uint64_t k_desc0 = smem_desc_sw128(kv_smem, 16, 1024);
             const uint64_t v_desc0 = smem_desc_sw128(kv_smem + kv_tile_bytes, BN * CHUNK_ROW_BYTES, 1024);
             constexpr uint32_t stage_off = (2 * kv_tile_bytes) >> 4;
@@ -221,12 +234,61 @@ fused4s_attention_kernel(const __grid_constant__ CUtensorMap tmap_q, const __gri
             auto issue_o = [&](int j, int st, int b) {   // O_t (+)= P V(j), V in stage st, P in the first 32 columns of buffer b
                 const uint64_t vd = v_desc0 + (uint64_t)(st * stage_off);
                 const uint32_t tp = tmem_base + b * BN;
+                if (SPLIT > 1) {
+                    // part g: O_g (+)= P_g V(j)[keys of g]; its weights sit at the start of its own score columns
+                    constexpr int KPP = (BN / 16) / SPLIT;   // 16-key MMA steps per part
 #pragma unroll
-                for (int kk = 0; kk < BN / 16; ++kk)
-                    mma_f16_ts(tmem_o, tp + kk * 8, vd + (uint64_t)(kk * ((16 * CHUNK_ROW_BYTES) >> 4)), idesc_o, j > 0 || kk > 0);
+                    for (int kk = 0; kk < BN / 16; ++kk)
+                        mma_f16_ts(tmem_o + (kk / KPP) * dpad, tp + (kk / KPP) * (BN / SPLIT) + (kk % KPP) * 8,
+                                   vd + (uint64_t)(kk * ((16 * CHUNK_ROW_BYTES) >> 4)), idesc_o, j > 0 || (kk % KPP) > 0);
+                } else {
+#pragma unroll
+                    for (int kk = 0; kk < BN / 16; ++kk)
+                        mma_f16_ts(tmem_o, tp + kk * 8, vd + (uint64_t)(kk * ((16 * CHUNK_ROW_BYTES) >> 4)), idesc_o, j > 0 || kk > 0);
+                }
             };
 
-            bool ok = mbar_wait(smem_u32(&bar_kv_full[0]), 0, abort_p, args.status, SITE_G_KV, 0) &&
+            if (SPLIT > 1) {
+                // One tile, NB score buffers: step j uses buffer j % NB.  A lone issuing thread needs about 1000 clocks
+                // per key tile (two waits, seven to nine MMAs, three commits) and would pace the kernel, so the work
+                // is split: thread 0 issues the products O_g (+)= P_g V(j), thread 1 the scores of key tile j + NB
+                // into the buffer those products free.  MMAs of different threads are not ordered by the tensor pipe,
+                // so thread 1 waits for the products' COMPLETION (bar_buf_free of that buffer); with NB >= 3 that
+                // round trip is off everybody's path: the parts may run NB - 1 key tiles ahead of the products.
+                bool ok = true;
+                if (t == 1) {
+                    ok = mbar_wait(smem_u32(&bar_q_full[0]), 0, abort_p, args.status, SITE_G_Q, 0);
+                    int b = 0, ph = 0;                 // buffer and its bar_buf_free phase
+                    int sn = 0, pn = 0;                // stage and phase of the key tile whose scores are requested
+                    for (int jn = 0; jn < n_kv && ok; ++jn) {
+                        ok = mbar_wait(smem_u32(&bar_kv_full[sn]), pn, abort_p, args.status, SITE_G_KV, jn);
+                        if (ok && jn >= NB) {          // the products of key tile jn - NB have read their weights
+                            ok = mbar_wait(smem_u32(&bar_buf_free[b]), ph, abort_p, args.status, SITE_G_PV, jn);
+                        }
+                        if (!ok) break;
+                        tc_fence_after_sync();
+                        issue_s(q_desc_own_split, 0, sn, b);
+                        if (++b == NB) { b = 0; if (jn >= NB) ph ^= 1; }
+                        if (++sn == stages) { sn = 0; pn ^= 1; }
+                    }
+                } else {
+                    int b = 0, ph = 0;
+                    int sj = 0;                        // stage of key tile j
+                    for (int j = 0; j < n_kv && ok; ++j) {
+                        ok = mbar_wait(smem_u32(&bar_p_full[0][b]), ph, abort_p, args.status, SITE_G_P, j);
+                        if (!ok) break;
+                        tc_fence_after_sync();
+                        issue_o(j, sj, b);
+                        tc_commit(smem_u32(&bar_pv_done[j & 1]));           // every O_g holds key tiles 0..j
+                        tc_commit(smem_u32(&bar_buf_free[b]));              // buffer b may take new scores
+                        tc_commit(smem_u32(&bar_kv_empty[sj]));             // done with K(j), V(j): S(j) completed long ago
+                        if (j == n_kv - 1) tc_commit(smem_u32(&bar_o_final[0]));
+                        if (++b == NB) { b = 0; ph ^= 1; }
+                        if (++sj == stages) sj = 0;
+                    }
+                }
+            }
+            bool ok = SPLIT == 1 && mbar_wait(smem_u32(&bar_kv_full[0]), 0, abort_p, args.status, SITE_G_KV, 0) &&
                       mbar_wait(smem_u32(&bar_q_full[t]), 0, abort_p, args.status, SITE_G_Q, t);
             if (ok) {
                 // the first T+1 steps fill the buffers: step t (own tile, key tile 0) into buffer t; the last issuer
@@ -274,7 +336,153 @@ fused4s_attention_kernel(const __grid_constant__ CUtensorMap tmap_q, const __gri
         // ------------------------------------------------------------ softmax warps
         setmaxnreg_inc<F4S_SOFTMAX_REGS>();
         const int t = warp >> 2;                 // query tile of this warpgroup
-        if (t < T) {
+        if (SPLIT > 1) {
+            // ---- one query tile, SPLIT parts: warpgroup g takes columns [g W, (g + 1) W) of every score tile
+            constexpr int W = BN / SPLIT;
+            const int g = t;
+            if (g < SPLIT) {
+                const int r = tid & (TILE_M - 1);    // row inside the tile = TMEM lane
+                const uint32_t lane_off = (uint32_t)((warp & 3) * 32) << 16;
+                const uint32_t tmem_og = tmem_o0 + g * dpad + lane_off;
+                const float c2 = args.scale_log2e;
+                float m_run = 0.f, l_run = 0.f;   // anchor and row sum of THIS part's keys
+                bool ok = true;
+                auto load_scores = [&](uint32_t taddr, uint32_t* s) {
+                    if (W == 32) tmem_ld32(taddr, s);
+                    else tmem_ld16(taddr, *reinterpret_cast<uint32_t(*)[16]>(s));
+                    tmem_wait_ld();
+                };
+                int b = 0, ph = 0;   // buffer j % NB, met for the (j / NB)-th time
+                for (int j = 0; j < n_kv; ++j) {
+                    const uint32_t tmem_s = tmem_base + b * BN + g * W + lane_off;
+                    ok = mbar_wait(smem_u32(&bar_s_full[0][b]), ph, abort_p, args.status, SITE_G_S, j);
+                    ok = __all_sync(0xffffffffu, ok);
+                    if (!ok) break;
+                    tc_fence_after_sync();
+                    if (tid == 0 && (j == 0 || j == 1 || j == 32 || j == n_kv - 1)) F4S_MARK(j == 0 ? 1 : j == 1 ? 2 : j == 32 ? 3 : 4);
+                    const int valid = args.Nk - j * BN - g * W;   // this part's columns >= valid are zero-filled keys
+                    uint32_t s[W];
+                    load_scores(tmem_s, s);
+                    const bool ragged = valid < W;   // only in the last key tile
+                    if (j == 0) {
+                        // a part without a single key (fewer keys than g W in all) keeps anchor 0 and weight 0
+                        const float row_max = valid <= 0 ? 0.f : ragged ? row_max_masked<W>(s, valid) : row_max_bf16<W>(s);
+                        m_run = row_max * c2 + FUSED_HEADROOM_LOG2;
+                    }
+                    uint32_t packed[W / 2];
+                    float tile_sum;
+#pragma unroll 1
+                    for (int attempt = 0; attempt < 2; ++attempt) {
+                        const float neg_mc = -m_run;
+                        if (!ragged) {
+                            const uint64_t c2c2 = pack_b64(__float_as_uint(c2), __float_as_uint(c2));
+                            const uint64_t nmnm = pack_b64(__float_as_uint(neg_mc), __float_as_uint(neg_mc));
+                            uint64_t acc[2] = {0ull, 0ull};
+                            exp2_pack_32<POLY, W / 2>(&s[0], c2c2, nmnm, &packed[0], acc);
+                            tile_sum = sum_f32x2(acc[0], acc[1]);
+                        } else {
+                            tile_sum = 0.f;
+                            exp2_pack_32_masked<W / 2>(&s[0], c2, neg_mc, 0, valid, &packed[0], tile_sum);
+                        }
+                        const bool over = !(tile_sum <= FUSED_TILE_SUM_LIMIT);
+                        if (attempt == 1 || !__any_sync(0xffffffffu, over)) break;
+                        // Rare: a score far above the anchor (see the unsplit path below).  O_g may be touched once
+                        // the products of key tile j-1 have completed; nothing of this tile's weights is stored yet.
+                        if (j > 0) {   // products of key tile j - 1: barrier (j - 1) & 1, its ((j - 1) / 2)-th phase
+                            ok = mbar_wait(smem_u32(&bar_pv_done[(j - 1) & 1]), ((j - 1) >> 1) & 1, abort_p, args.status, SITE_G_PV, j);
+                            ok = __all_sync(0xffffffffu, ok);
+                            if (!ok) break;
+                            tc_fence_after_sync();
+                        }
+                        load_scores(tmem_s, s);
+                        const float row_max = valid <= 0 ? 0.f : ragged ? row_max_masked<W>(s, valid) : row_max_bf16<W>(s);
+                        const float m_new = row_max * c2 + FUSED_HEADROOM_LOG2;
+                        const float alpha = over ? ex2_approx(m_run - m_new) : 1.f;
+                        if (over) m_run = m_new;
+                        l_run *= alpha;
+                        if (j > 0) {
+                            for (int cg = 0; cg < (dpad >> 4); ++cg) {
+                                uint32_t o[16];
+                                tmem_ld16(tmem_og + cg * 16, o);
+                                tmem_wait_ld();
+#pragma unroll
+                                for (int c = 0; c < 16; ++c) o[c] = __float_as_uint(__uint_as_float(o[c]) * alpha);
+                                tmem_st16(tmem_og + cg * 16, o);
+                            }
+                            tmem_wait_st();
+                        }
+                    }
+                    if (!ok) break;
+                    l_run += tile_sum;
+                    // P_g(j) over the first columns of the part's OWN score columns (the other parts may still be
+                    // reading theirs)
+                    if (W == 32) tmem_st16(tmem_s, *reinterpret_cast<const uint32_t(*)[16]>(&packed[0]));
+                    else tmem_st8(tmem_s, *reinterpret_cast<const uint32_t(*)[8]>(&packed[0]));
+                    tmem_wait_st();
+                    // The issuer signals the completion of key tile j's products on barrier j & 1.  Every warp consumes
+                    // every phase of both barriers in order (a parity wait is only sound one phase behind), two key
+                    // tiles late: before handing over P(j) it waits for tile j - 2, the phase before the one that
+                    // P(j) itself leads to -- so the wait is sound and, the tensor pipe being that far along anyway,
+                    // costs nothing.  (The rare path above waits for tile j - 1 on the other barrier, its next phase.)
+                    if (j > 1) {
+                        ok = mbar_wait(smem_u32(&bar_pv_done[j & 1]), ((j - 2) >> 1) & 1, abort_p, args.status, SITE_G_PV, j);
+                        ok = __all_sync(0xffffffffu, ok);
+                        if (!ok) break;
+                    }
+                    tc_fence_before_sync();
+                    if (lane == 0) mbar_arrive(smem_u32(&bar_p_full[0][b]));
+                    if (++b == NB) { b = 0; ph ^= 1; }
+                }
+                if (tid == 0) F4S_MARK(5);
+                // ---- combine the parts: o = sum_g 2^(m_g - m) O_g / sum_g 2^(m_g - m) l_g, m = max_g m_g
+                part_ml[g][r] = make_float2(m_run, l_run);
+                if (ok) ok = mbar_wait(smem_u32(&bar_o_final[0]), 0, abort_p, args.status, SITE_G_O, g);
+                ok = named_barrier_and(1, SPLIT * 128, ok);   // every part's (m, l) is in shared memory, every product done
+                if (tid == 0) F4S_MARK(6);
+                if (ok) {
+                    tc_fence_after_sync();
+                    float f[SPLIT];
+                    float m_all = -INFINITY, l_all = 0.f;
+#pragma unroll
+                    for (int p2 = 0; p2 < SPLIT; ++p2)
+                        if (part_ml[p2][r].y > 0.f) m_all = fmaxf(m_all, part_ml[p2][r].x);
+#pragma unroll
+                    for (int p2 = 0; p2 < SPLIT; ++p2) {
+                        const float2 ml = part_ml[p2][r];
+                        f[p2] = ml.y > 0.f ? ex2_approx(ml.x - m_all) : 0.f;   // a part without keys counts nothing
+                        l_all += f[p2] * ml.y;
+                    }
+                    const float inv = 1.f / l_all;
+#pragma unroll
+                    for (int p2 = 0; p2 < SPLIT; ++p2) f[p2] *= inv;
+                    const int row = row_base + r;
+                    __half* orow = args.out + ((size_t)bh * args.Nq + row) * args.d;
+                    // the column groups of 16 are shared out among the parts; a thread reads its row of every O_p
+                    for (int cg = g; cg < (dpad >> 4); cg += SPLIT) {
+                        float acc[16];
+#pragma unroll
+                        for (int c = 0; c < 16; ++c) acc[c] = 0.f;
+#pragma unroll
+                        for (int p2 = 0; p2 < SPLIT; ++p2) {
+                            uint32_t x[16];
+                            tmem_ld16(tmem_o0 + p2 * dpad + lane_off + cg * 16, x);
+                            tmem_wait_ld();
+#pragma unroll
+                            for (int c = 0; c < 16; ++c) acc[c] = fmaf(__uint_as_float(x[c]), f[p2], acc[c]);
+                        }
+                        uint4 lo, hi;
+                        lo.x = pack_half2(acc[0], acc[1]);   lo.y = pack_half2(acc[2], acc[3]);
+                        lo.z = pack_half2(acc[4], acc[5]);   lo.w = pack_half2(acc[6], acc[7]);
+                        hi.x = pack_half2(acc[8], acc[9]);   hi.y = pack_half2(acc[10], acc[11]);
+                        hi.z = pack_half2(acc[12], acc[13]); hi.w = pack_half2(acc[14], acc[15]);
+                        if (row < args.Nq) {
+                            if (cg * 16 + 8 <= args.d) *reinterpret_cast<uint4*>(orow + cg * 16) = lo;
+                            if (cg * 16 + 16 <= args.d) *reinterpret_cast<uint4*>(orow + cg * 16 + 8) = hi;
+                        }
+                    }
+                }
+            }
+        } else if (t < T) {
             const int r = tid & (TILE_M - 1);    // row inside the tile = TMEM lane
             const uint32_t lane_off = (uint32_t)((warp & 3) * 32) << 16;
             const uint32_t tmem_o = tmem_o0 + t * dpad + lane_off;

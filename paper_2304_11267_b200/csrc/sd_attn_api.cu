@@ -64,6 +64,8 @@ struct sd_attn_handle {
     int cross2_four_ok;
     int cross_one_tile_only;  // SD_ATTN_CROSS_ONE_TILE=1: never use the persistent cross-attention kernel
     int prefer_two_tile;      // SD_ATTN_FUSED_TWO_TILE=1: use the two-tile fused kernel for every head dim
+    int fused_no_split;       // SD_ATTN_FUSED_NO_SPLIT=1: a lone query tile keeps all 64 score columns in one warpgroup
+    int fused_split_override; // SD_ATTN_FUSED_SPLIT=2|4: that many parts wherever one tile per CTA is chosen (tests)
     // sd_attn_forward_host: copies of one slice of heads overlap the kernel of another (see there)
     cudaStream_t copy_in, copy_out;
     cudaEvent_t ev_fork, ev_join, ev_in[HOST_SLICES], ev_done[HOST_SLICES];
@@ -182,6 +184,10 @@ extern "C" int sd_attn_create(sd_attn_handle** out) {
     h->no_spare = (nsp && nsp[0] == '1') ? 1 : 0;
     const char* ftl = getenv("SD_ATTN_FUSED_TILES");
     h->fused4_tiles_override = (ftl && ftl[0] >= '1' && ftl[0] <= '4' && !ftl[1]) ? ftl[0] - '0' : 0;
+    const char* nsl = getenv("SD_ATTN_FUSED_NO_SPLIT");
+    h->fused_no_split = (nsl && nsl[0] == '1') ? 1 : 0;
+    const char* spl = getenv("SD_ATTN_FUSED_SPLIT");
+    h->fused_split_override = (spl && (spl[0] == '2' || spl[0] == '4') && !spl[1]) ? spl[0] - '0' : 0;
     const char* two = getenv("SD_ATTN_FUSED_TWO_TILE");
     h->prefer_two_tile = (two && two[0] == '1') ? 1 : 0;
 
@@ -197,6 +203,11 @@ extern "C" int sd_attn_create(sd_attn_handle** out) {
     if (e == cudaSuccess) e = raise_smem_limit(fused4s_attention_kernel<0, 1>, F4S_SMEM_BUDGET + 1024);
     if (e == cudaSuccess) e = raise_smem_limit(fused4s_attention_kernel<0, 2>, F4S_SMEM_BUDGET + 1024);
     if (e == cudaSuccess) e = raise_smem_limit(fused4s_attention_kernel<0, 3>, F4S_SMEM_BUDGET + 1024);
+    if (e == cudaSuccess) e = raise_smem_limit(fused4s_attention_kernel<0, 1, 4>, F4S_SMEM_BUDGET + 1024);
+    if (e == cudaSuccess) e = raise_smem_limit(fused4s_attention_kernel<0, 1, 2>, F4S_SMEM_BUDGET + 1024);
+    if (e == cudaSuccess) e = raise_smem_limit(fused4s_attention_kernel<0, 2, 4>, F4S_SMEM_BUDGET + 1024);
+    if (e == cudaSuccess) e = raise_smem_limit(fused4s_attention_kernel<0, 2, 2>, F4S_SMEM_BUDGET + 1024);
+    if (e == cudaSuccess) e = raise_smem_limit(fused4s_attention_kernel<0, 3, 2>, F4S_SMEM_BUDGET + 1024);
     if (e == cudaSuccess) e = raise_smem_limit(twopass_scores_kernel, twopass_scores_smem_bytes(3));
     if (e == cudaSuccess) e = raise_smem_limit(twopass_pv_kernel, twopass_pv_smem_bytes(3));
     if (e == cudaSuccess) e = raise_smem_limit(simt_attention_kernel<float, 5>, simt_smem_bytes(160));
@@ -210,9 +221,12 @@ extern "C" int sd_attn_create(sd_attn_handle** out) {
         if (e == cudaSuccess)
             h->fused4_ok = F4_THREADS * fa.numRegs >= 512 * F4_SOFTMAX_REGS + 256 * F4_CONTROL_REGS;
         h->fused4s_ok = 1;
-        const void* f4s[4] = {(const void*)fused4s_attention_kernel<F4S_POLY_PER8, 1>, (const void*)fused4s_attention_kernel<0, 1>,
-                              (const void*)fused4s_attention_kernel<0, 2>, (const void*)fused4s_attention_kernel<0, 3>};
-        for (int i = 0; i < 4 && e == cudaSuccess; ++i) {
+        const void* f4s[9] = {(const void*)fused4s_attention_kernel<F4S_POLY_PER8, 1>, (const void*)fused4s_attention_kernel<0, 1>,
+                              (const void*)fused4s_attention_kernel<0, 2>, (const void*)fused4s_attention_kernel<0, 3>,
+                              (const void*)fused4s_attention_kernel<0, 1, 4>, (const void*)fused4s_attention_kernel<0, 1, 2>,
+                              (const void*)fused4s_attention_kernel<0, 2, 4>, (const void*)fused4s_attention_kernel<0, 2, 2>,
+                              (const void*)fused4s_attention_kernel<0, 3, 2>};
+        for (int i = 0; i < 9 && e == cudaSuccess; ++i) {
             e = cudaFuncGetAttributes(&fa, f4s[i]);
             if (e == cudaSuccess && F4_THREADS * fa.numRegs < 512 * F4S_SOFTMAX_REGS + 256 * F4S_CONTROL_REGS) h->fused4s_ok = 0;
         }
@@ -499,8 +513,29 @@ static int launch_fused4s(sd_attn_handle* h, const Problem& p) {
     if (rc == SD_ATTN_OK) rc = make_tmap(h, &tv, p.v, p.BH, p.Nk, p.d, F4_BN);
     if (rc != SD_ATTN_OK) return rc;
     dim3 grid((tiles_per_head + a.tiles_per_cta - 1) / a.tiles_per_cta, p.BH), block(F4_THREADS);
+    // One tile per CTA: its score columns are shared out among as many warpgroups as tensor memory has accumulators
+    // for (two score buffers + split * dpad columns <= 512).
+    int split = 1;
+    if (a.tiles_per_cta == 1 && !h->fused_no_split) split = 2 * F4_BN + 4 * a.dpad <= 512 ? 4 : 2 * F4_BN + 2 * a.dpad <= 512 ? 2 : 1;
+    if (h->fused_split_override) split = a.tiles_per_cta == 1 && 2 * F4_BN + h->fused_split_override * a.dpad <= 512 ? h->fused_split_override : 1;
+    // ... and as many score buffers as the rest of tensor memory holds, the K/V ring permitting (a buffer ahead is a
+    // key tile ahead)
+    a.split_buffers = (512 - split * a.dpad) / F4_BN;
+    if (a.split_buffers > F4S_BUFFERS) a.split_buffers = F4S_BUFFERS;
+    if (a.split_buffers > a.stages - 1) a.split_buffers = a.stages - 1;
+    if (a.split_buffers < 2) split = 1;
+    if (split == 4 && a.nch == 1)
+        launch_overlapped(h, fused4s_attention_kernel<0, 1, 4>, grid, block, smem, p.stream, tq, tk, tv, a);
+    else if (split == 2 && a.nch == 1)
+        launch_overlapped(h, fused4s_attention_kernel<0, 1, 2>, grid, block, smem, p.stream, tq, tk, tv, a);
+    else if (split == 4 && a.nch == 2)
+        launch_overlapped(h, fused4s_attention_kernel<0, 2, 4>, grid, block, smem, p.stream, tq, tk, tv, a);
+    else if (split == 2 && a.nch == 2)
+        launch_overlapped(h, fused4s_attention_kernel<0, 2, 2>, grid, block, smem, p.stream, tq, tk, tv, a);
+    else if (split == 2 && a.nch == 3)
+        launch_overlapped(h, fused4s_attention_kernel<0, 3, 2>, grid, block, smem, p.stream, tq, tk, tv, a);
     // the polynomial share of the exponentials only pays where four tiles saturate the special function unit
-    if (a.dpad <= 48)
+    else if (a.dpad <= 48)
         launch_overlapped(h, fused4s_attention_kernel<F4S_POLY_PER8, 1>, grid, block, smem, p.stream, tq, tk, tv, a);
     else if (a.nch == 1)
         launch_overlapped(h, fused4s_attention_kernel<0, 1>, grid, block, smem, p.stream, tq, tk, tv, a);

@@ -371,11 +371,13 @@ def test_every_ragged_tail_of_the_key_tiles(att, bd, Nk):
 
 def test_many_heads_and_bitwise_agreement_between_tile_counts(bd, monkeypatch):
     """640 (batch, head) problems in one call; and the number of query tiles a CTA takes changes the schedule, not
-    the arithmetic of a row: the outputs of the variants must agree bit for bit."""
+    the arithmetic of a row: the outputs of the variants must agree bit for bit -- as long as a lone tile is not cut
+    into parts, which changes the partial sums (checked against the oracle and the others within rounding)."""
     q, k, v = rand_qkv(7100, 16, 40, 130, 200, 40)
     scale = float(np.float32(1.0 / np.sqrt(40)))
     rows = np.arange(0, 16 * 40 * 130, 11, dtype=np.int64)
     ref, _, _ = oracle.forward(q, k, v, scale, rows=rows)
+    monkeypatch.setenv("SD_ATTN_FUSED_NO_SPLIT", "1")   # a lone tile in one piece: the same arithmetic as with company
     outs = []
     for tiles in ("1", "2", "4"):
         monkeypatch.setenv("SD_ATTN_FUSED_TILES", tiles)
@@ -388,6 +390,47 @@ def test_many_heads_and_bitwise_agreement_between_tile_counts(bd, monkeypatch):
             a.close()
         check(outs[-1].reshape(-1, 40)[rows], ref, v, what="tiles per CTA %s" % tiles)
     assert np.array_equal(outs[0], outs[1]) and np.array_equal(outs[0], outs[2])
+    # one tile per CTA with its score columns shared out among 2 or 4 warpgroups: other partial sums, same result
+    monkeypatch.delenv("SD_ATTN_FUSED_NO_SPLIT")
+    monkeypatch.setenv("SD_ATTN_FUSED_TILES", "1")
+    for parts in ("2", "4"):
+        monkeypatch.setenv("SD_ATTN_FUSED_SPLIT", parts)
+        a = bd.Attention(bd.MODE_FUSED)
+        try:
+            out = a.forward(gpu(q), gpu(k), gpu(v), scale=scale).cpu().numpy()
+            a.check()
+        finally:
+            a.close()
+        check(out.reshape(-1, 40)[rows], ref, v, what="%s parts" % parts)
+        assert not np.array_equal(out, outs[0])          # it is the other kernel that ran
+        assert np.abs(out.astype(np.float64) - outs[0].astype(np.float64)).max() <= 2 * F16_ABS * np.abs(v).max()
+
+
+@pytest.mark.parametrize("parts", ["0", "2", "4"])
+@pytest.mark.parametrize("d", [40, 64, 80, 128, 160])
+def test_lone_tile_in_parts(bd, monkeypatch, parts, d):
+    """One query tile per CTA: every warpgroup of the CTA takes a share of the 64 columns of each score tile, with an
+    anchor, a row sum and an accumulator of its own (combined at the end).  Key counts around the shares' boundaries
+    (a part without a single key, a part with one), several score-buffer rounds, and rows whose large scores come
+    late (every part re-anchors on its own)."""
+    if parts != "0":
+        monkeypatch.setenv("SD_ATTN_FUSED_SPLIT", parts)
+    monkeypatch.setenv("SD_ATTN_FUSED_TILES", "1")
+    a = bd.Attention(bd.MODE_FUSED)
+    try:
+        for i, (Nq, Nk) in enumerate([(128, 129), (100, 130), (5, 145), (130, 161), (128, 177), (64, 192), (129, 449),
+                                      (257, 1000), (128, 2048)]):
+            q, k, v = rand_qkv(9000 + 13 * d + i, 1, 3, Nq, Nk, d)
+            if i % 3 == 2:   # scores rising along the keys: later tiles exceed the first tile's anchor by far
+                ramp = np.linspace(0.0, 6.0, Nk, dtype=np.float32)[None, None, :, None]
+                k = (k.astype(np.float32) + ramp * np.sign(q.astype(np.float32).mean(axis=2, keepdims=True))).astype(np.float16)
+            scale = float(np.float32(1.0 / np.sqrt(d)))
+            ref, _, _ = oracle.forward(q, k, v, scale)
+            out = a.forward(gpu(q), gpu(k), gpu(v), scale=scale).cpu().numpy()
+            a.check()
+            check(out, ref, v, what="parts=%s d=%d Nq=%d Nk=%d" % (parts, d, Nq, Nk))
+    finally:
+        a.close()
 
 
 def test_padding_rows_with_distinct_values_only_see_their_mean(att, bd):

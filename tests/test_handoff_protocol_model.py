@@ -144,3 +144,118 @@ def test_one_barrier_per_buffer_is_not_enough():
     """Different tiles consuming successive phases of ONE barrier per buffer can start waiting a phase early."""
     outcomes = {simulate(4, 17, 8, seed, per_tile_barriers=False) for seed in range(12)}
     assert outcomes != {"ok"}
+
+
+# ---------------------------------------------------------------------------------------------------------------
+# The variant for ONE query tile per CTA: the columns of every score tile are shared out among several warpgroups
+# ("parts"), NB score buffers run ahead of the products, and the MMAs come from TWO threads -- the products
+# O_g (+)= P_g V(j) from one, the scores of key tile j + NB from the other -- whose instructions the tensor pipe does
+# not order against each other.
+
+def simulate_parts(NB, n_kv, stages, seed, warps=8, pv_ring=2, wait_buf_free=True, limit=400000):
+    rnd = random.Random(seed)
+    s_full = [Bar(1) for _ in range(NB)]
+    p_full = [Bar(warps) for _ in range(NB)]
+    buf_free = [Bar(1) for _ in range(NB)]
+    pv_done = [Bar(1) for _ in range(pv_ring)]
+    o_final = Bar(1)
+    q_full = Bar(1)
+    kv_full = [Bar(1) for _ in range(stages)]
+    kv_empty = [Bar(1) for _ in range(stages)]
+    pipe_a, pipe_b = [], []                      # per issuing thread, each retired in order
+    buf = {b: {} for b in range(NB)}             # per buffer and warp: what its columns hold
+    stage, errors = {}, []
+
+    def check(cond, what):
+        if not cond:
+            errors.append(what)
+
+    def producer():
+        q_full.arrive()
+        yield
+        for j in range(n_kv):
+            s = j % stages
+            if j >= stages:
+                while not kv_empty[s].done(((j // stages) - 1) & 1):
+                    yield
+            stage[s] = j
+            kv_full[s].arrive()
+            yield
+
+    def score_thread():
+        while not q_full.done(0):
+            yield
+        for jn in range(n_kv):
+            b = jn % NB
+            while not kv_full[jn % stages].done((jn // stages) & 1):
+                yield
+            if jn >= NB and wait_buf_free:
+                while not buf_free[b].done(((jn // NB) - 1) & 1):
+                    yield
+            check(stage.get(jn % stages) == jn, ("S reads a stale stage", jn))
+            pipe_b.append(("S", jn, b, [s_full[b]]))
+            yield
+
+    def product_thread():
+        for j in range(n_kv):
+            b = j % NB
+            while not p_full[b].done((j // NB) & 1):
+                yield
+            check(stage.get(j % stages) == j, ("P V reads a stale stage", j))
+            pipe_a.append(("PV", j, b, [pv_done[j % pv_ring], buf_free[b], kv_empty[j % stages]] +
+                           ([o_final] if j == n_kv - 1 else [])))
+            yield
+
+    def part_warp(w):
+        for j in range(n_kv):
+            b = j % NB
+            while not s_full[b].done((j // NB) & 1):
+                yield
+            check(buf[b].get(w) == ("S", j), ("a part reads the wrong scores", w, j, b, buf[b].get(w)))
+            yield
+            buf[b][w] = ("P", j)
+            if j >= pv_ring:   # products of key tile j - pv_ring: the phase before the one P(j) leads to
+                jj = j - pv_ring
+                while not pv_done[jj % pv_ring].done((jj // pv_ring) & 1):
+                    yield
+            p_full[b].arrive()
+            yield
+        while not o_final.done(0):
+            yield
+
+    procs = [producer(), score_thread(), product_thread()] + [part_warp(w) for w in range(warps)]
+    steps = 0
+    while procs and not errors:
+        steps += 1
+        if steps > limit:
+            return "deadlock"
+        for pipe in (pipe_a, pipe_b):        # two in-order queues, retired independently of one another
+            if pipe and rnd.random() < 0.4:
+                kind, j, b, bars = pipe.pop(0)
+                if kind == "S":
+                    for w in range(warps):
+                        buf[b][w] = ("S", j)
+                else:
+                    check(all(buf[b].get(w) == ("P", j) for w in range(warps)), ("P V reads the wrong weights", j, b))
+                for x in bars:
+                    x.arrive()
+        i = rnd.randrange(len(procs))
+        try:
+            next(procs[i])
+        except StopIteration:
+            procs.pop(i)
+    return errors[0] if errors else "ok"
+
+
+@pytest.mark.parametrize("NB", [2, 3, 4, 5])
+@pytest.mark.parametrize("n_kv", [1, 2, 3, 5, 8, 16, 17])
+def test_lone_tile_in_parts_protocol(NB, n_kv):
+    for seed in range(4):
+        assert simulate_parts(NB, n_kv, 8, seed) == "ok"
+        assert simulate_parts(NB, n_kv, NB + 1, seed, warps=16) == "ok"
+
+
+def test_scores_must_wait_for_the_completion_of_the_products_they_overwrite():
+    """Without the per-buffer completion barrier the second thread's scores can land on weights not yet read."""
+    outcomes = {simulate_parts(3, 17, 8, seed, wait_buf_free=False) for seed in range(12)}
+    assert outcomes != {"ok"}
