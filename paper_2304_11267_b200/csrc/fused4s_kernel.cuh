@@ -67,12 +67,14 @@ constexpr int F4S_SOFTMAX_REGS = SD_ATTN_F4S_SOFTMAX_REGS;
 constexpr int F4S_CONTROL_REGS = SD_ATTN_F4S_CONTROL_REGS;
 static_assert(512 * F4S_SOFTMAX_REGS + 256 * F4S_CONTROL_REGS == 768 * 80, "setmaxnreg budget");
 
-// SPLIT > 1 (only with ONE query tile per CTA): the 64 columns of every score tile are shared out among SPLIT
-// warpgroups, each with an exponent anchor, a row sum and an accumulator O_g of its own over ITS keys (16 or 32 of
-// every 64), combined once at the end.  A lone tile is bound by the chain of latencies of one warp per scheduler
+// SPLIT > 1 (only with ONE query tile per CTA): the key tiles are dealt out among SPLIT warpgroups ("parts": part g
+// takes key tiles g, g + SPLIT, ...), each with an exponent anchor, a row sum and an accumulator O_g of its own over
+// ITS keys, combined once at the end.  A lone tile is bound by the chain of latencies of one warp per scheduler
 // (tcgen05.ld -> exp2 -> tcgen05.st -> hand-over: 1400-1500 clocks per key tile, measured, against 600 per tile
-// with four tiles resident); the parts need no agreement on an anchor because their products never share an
-// accumulator.
+// with four tiles resident); the parts work on different key tiles at the same time, so their chains overlap as
+// those of four query tiles do, and they need no agreement on an anchor because their products never share an
+// accumulator.  The score buffers run ahead of the products (NB of them, a multiple of SPLIT), and the MMAs come from
+// two threads: the products of key tile j from one, the scores of key tile j + NB from the other.
 template <int POLY, int NCH, int SPLIT = 1>   // NCH: 64-column chunks per row (head dim <= 64 * NCH)
 __global__ void __launch_bounds__(F4_THREADS, 1)
 fused4s_attention_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__ CUtensorMap tmap_k,
@@ -130,7 +132,7 @@ fused4s_attention_kernel(const __grid_constant__ CUtensorMap tmap_q, const __gri
         for (int t = 0; t < F4_TILES; ++t) {
             for (int b = 0; b < F4S_BUFFERS; ++b) {
                 mbar_init(smem_u32(&bar_s_full[t][b]), 1);
-                mbar_init(smem_u32(&bar_p_full[t][b]), 4 * SPLIT);    // one arrival per softmax warp of the tile
+                mbar_init(smem_u32(&bar_p_full[t][b]), 4);    // one arrival per softmax warp of the tile (SPLIT > 1: of the part)
             }
             mbar_init(smem_u32(&bar_q_full[t]), 1);
             mbar_init(smem_u32(&bar_pv_done[t]), 1);
@@ -217,7 +219,7 @@ fused4s_attention_kernel(const __grid_constant__ CUtensorMap tmap_q, const __gri
                 // The issuer's instruction stream is on the hand-off path (one predicated-off MMA per step cost 4% on
                 // the 9216-token call; hoisting the address arithmetic above the wait cost registers and 1%): the variant
                 // for head dims up to 48 issues at most three steps, and exactly three without predicates for d = 40.
-                constexpr int KS_MAX = (NCH == 1 && POLY != 0) ? 3 : 4 * NCH;
+                constexpr int KS_MAX = (NCH == 1 && POLY != 0 && SPLIT == 1) ? 3 : 4 * NCH;   // (POLY != 0, SPLIT == 1: the d <= 48 variant)
                 if (KS_MAX == 3 && ksteps_s == 3) {
 #pragma unroll
                     for (int kk = 0; kk < 3; ++kk)
@@ -235,12 +237,11 @@ fused4s_attention_kernel(const __grid_constant__ CUtensorMap tmap_q, const __gri
                 const uint64_t vd = v_desc0 + (uint64_t)(st * stage_off);
                 const uint32_t tp = tmem_base + b * BN;
                 if (SPLIT > 1) {
-                    // part g: O_g (+)= P_g V(j)[keys of g]; its weights sit at the start of its own score columns
-                    constexpr int KPP = (BN / 16) / SPLIT;   // 16-key MMA steps per part
+                    // key tile j belongs to part j % SPLIT: O_g (+)= P(j) V(j), the first of the part's tiles overwrites
+                    const uint32_t to = tmem_o + (j % SPLIT) * dpad;
 #pragma unroll
                     for (int kk = 0; kk < BN / 16; ++kk)
-                        mma_f16_ts(tmem_o + (kk / KPP) * dpad, tp + (kk / KPP) * (BN / SPLIT) + (kk % KPP) * 8,
-                                   vd + (uint64_t)(kk * ((16 * CHUNK_ROW_BYTES) >> 4)), idesc_o, j > 0 || (kk % KPP) > 0);
+                        mma_f16_ts(to, tp + kk * 8, vd + (uint64_t)(kk * ((16 * CHUNK_ROW_BYTES) >> 4)), idesc_o, j >= SPLIT || kk > 0);
                 } else {
 #pragma unroll
                     for (int kk = 0; kk < BN / 16; ++kk)
@@ -279,7 +280,7 @@ fused4s_attention_kernel(const __grid_constant__ CUtensorMap tmap_q, const __gri
                         if (!ok) break;
                         tc_fence_after_sync();
                         issue_o(j, sj, b);
-                        tc_commit(smem_u32(&bar_pv_done[j & 1]));           // every O_g holds key tiles 0..j
+                        tc_commit(smem_u32(&bar_pv_done[j % SPLIT]));       // the part's O_g holds its key tiles up to j
                         tc_commit(smem_u32(&bar_buf_free[b]));              // buffer b may take new scores
                         tc_commit(smem_u32(&bar_kv_empty[sj]));             // done with K(j), V(j): S(j) completed long ago
                         if (j == n_kv - 1) tc_commit(smem_u32(&bar_o_final[0]));
@@ -337,39 +338,37 @@ fused4s_attention_kernel(const __grid_constant__ CUtensorMap tmap_q, const __gri
         setmaxnreg_inc<F4S_SOFTMAX_REGS>();
         const int t = warp >> 2;                 // query tile of this warpgroup
         if (SPLIT > 1) {
-            // ---- one query tile, SPLIT parts: warpgroup g takes columns [g W, (g + 1) W) of every score tile
-            constexpr int W = BN / SPLIT;
+            // ---- one query tile, SPLIT parts: warpgroup g takes the key tiles j = g, g + SPLIT, ... whole
             const int g = t;
             if (g < SPLIT) {
                 const int r = tid & (TILE_M - 1);    // row inside the tile = TMEM lane
                 const uint32_t lane_off = (uint32_t)((warp & 3) * 32) << 16;
                 const uint32_t tmem_og = tmem_o0 + g * dpad + lane_off;
+                const uint32_t b_pvdone = smem_u32(&bar_pv_done[g]);   // products of THIS part's key tiles
                 const float c2 = args.scale_log2e;
-                float m_run = 0.f, l_run = 0.f;   // anchor and row sum of THIS part's keys
+                float m_run = 0.f, l_run = 0.f;   // anchor and row sum over this part's keys
                 bool ok = true;
-                auto load_scores = [&](uint32_t taddr, uint32_t* s) {
-                    if (W == 32) tmem_ld32(taddr, s);
-                    else tmem_ld16(taddr, *reinterpret_cast<uint32_t(*)[16]>(s));
-                    tmem_wait_ld();
-                };
-                int b = 0, ph = 0;   // buffer j % NB, met for the (j / NB)-th time
-                for (int j = 0; j < n_kv; ++j) {
-                    const uint32_t tmem_s = tmem_base + b * BN + g * W + lane_off;
+                // NB is a multiple of SPLIT, so buffer b = j % NB always meets the same part: one consumer per barrier.
+                // The part's i-th key tile uses buffer (g + SPLIT i) % NB, phase ((g + SPLIT i) / NB) & 1.
+                int b = g, ph = 0;
+                for (int j = g, i = 0; j < n_kv; j += SPLIT, ++i) {
+                    const uint32_t tmem_s = tmem_base + b * BN + lane_off;
                     ok = mbar_wait(smem_u32(&bar_s_full[0][b]), ph, abort_p, args.status, SITE_G_S, j);
                     ok = __all_sync(0xffffffffu, ok);
                     if (!ok) break;
                     tc_fence_after_sync();
-                    if (tid == 0 && (j == 0 || j == 1 || j == 32 || j == n_kv - 1)) F4S_MARK(j == 0 ? 1 : j == 1 ? 2 : j == 32 ? 3 : 4);
-                    const int valid = args.Nk - j * BN - g * W;   // this part's columns >= valid are zero-filled keys
-                    uint32_t s[W];
-                    load_scores(tmem_s, s);
-                    const bool ragged = valid < W;   // only in the last key tile
-                    if (j == 0) {
-                        // a part without a single key (fewer keys than g W in all) keeps anchor 0 and weight 0
-                        const float row_max = valid <= 0 ? 0.f : ragged ? row_max_masked<W>(s, valid) : row_max_bf16<W>(s);
+                    if (tid == 0 && (j == 0 || j == 32 || j == n_kv - 1)) F4S_MARK(j == 0 ? 1 : j == 32 ? 3 : 4);
+                    const int valid = args.Nk - j * BN;   // columns >= valid are zero-filled keys
+                    uint32_t s[BN];
+                    tmem_ld32(tmem_s, &s[0]);
+                    tmem_ld32(tmem_s + 32, &s[32]);
+                    tmem_wait_ld();
+                    const bool ragged = valid < BN;   // only the last key tile can be
+                    if (i == 0) {
+                        const float row_max = ragged ? row_max_masked<BN>(s, valid) : row_max_bf16<BN>(s);
                         m_run = row_max * c2 + FUSED_HEADROOM_LOG2;
                     }
-                    uint32_t packed[W / 2];
+                    uint32_t packed[BN / 2];
                     float tile_sum;
 #pragma unroll 1
                     for (int attempt = 0; attempt < 2; ++attempt) {
@@ -378,60 +377,59 @@ fused4s_attention_kernel(const __grid_constant__ CUtensorMap tmap_q, const __gri
                             const uint64_t c2c2 = pack_b64(__float_as_uint(c2), __float_as_uint(c2));
                             const uint64_t nmnm = pack_b64(__float_as_uint(neg_mc), __float_as_uint(neg_mc));
                             uint64_t acc[2] = {0ull, 0ull};
-                            exp2_pack_32<POLY, W / 2>(&s[0], c2c2, nmnm, &packed[0], acc);
+                            exp2_pack_32<POLY>(&s[0], c2c2, nmnm, &packed[0], acc);
+                            exp2_pack_32<POLY>(&s[32], c2c2, nmnm, &packed[16], acc);
                             tile_sum = sum_f32x2(acc[0], acc[1]);
                         } else {
                             tile_sum = 0.f;
-                            exp2_pack_32_masked<W / 2>(&s[0], c2, neg_mc, 0, valid, &packed[0], tile_sum);
+                            exp2_pack_32_masked(&s[0], c2, neg_mc, 0, valid, &packed[0], tile_sum);
+                            exp2_pack_32_masked(&s[32], c2, neg_mc, 32, valid, &packed[16], tile_sum);
                         }
                         const bool over = !(tile_sum <= FUSED_TILE_SUM_LIMIT);
                         if (attempt == 1 || !__any_sync(0xffffffffu, over)) break;
-                        // Rare: a score far above the anchor (see the unsplit path below).  O_g may be touched once
-                        // the products of key tile j-1 have completed; nothing of this tile's weights is stored yet.
-                        if (j > 0) {   // products of key tile j - 1: barrier (j - 1) & 1, its ((j - 1) / 2)-th phase
-                            ok = mbar_wait(smem_u32(&bar_pv_done[(j - 1) & 1]), ((j - 1) >> 1) & 1, abort_p, args.status, SITE_G_PV, j);
+                        // Rare: a score far above the anchor (see the unsplit path below).  O_g may be touched once the
+                        // product of this part's previous key tile has completed; nothing of this tile's weights is
+                        // stored yet.  The first registers of the row are borrowed for O_g.
+                        if (i > 0) {
+                            ok = mbar_wait(b_pvdone, (i - 1) & 1, abort_p, args.status, SITE_G_PV, j);
                             ok = __all_sync(0xffffffffu, ok);
                             if (!ok) break;
                             tc_fence_after_sync();
                         }
-                        load_scores(tmem_s, s);
-                        const float row_max = valid <= 0 ? 0.f : ragged ? row_max_masked<W>(s, valid) : row_max_bf16<W>(s);
+                        const float row_max = ragged ? row_max_masked<BN>(s, valid) : row_max_bf16<BN>(s);
                         const float m_new = row_max * c2 + FUSED_HEADROOM_LOG2;
                         const float alpha = over ? ex2_approx(m_run - m_new) : 1.f;
                         if (over) m_run = m_new;
                         l_run *= alpha;
-                        if (j > 0) {
+                        if (i > 0) {
                             for (int cg = 0; cg < (dpad >> 4); ++cg) {
-                                uint32_t o[16];
-                                tmem_ld16(tmem_og + cg * 16, o);
+                                tmem_ld16(tmem_og + cg * 16, *reinterpret_cast<uint32_t(*)[16]>(&s[0]));
                                 tmem_wait_ld();
 #pragma unroll
-                                for (int c = 0; c < 16; ++c) o[c] = __float_as_uint(__uint_as_float(o[c]) * alpha);
-                                tmem_st16(tmem_og + cg * 16, o);
+                                for (int c = 0; c < 16; ++c) s[c] = __float_as_uint(__uint_as_float(s[c]) * alpha);
+                                tmem_st16(tmem_og + cg * 16, *reinterpret_cast<uint32_t(*)[16]>(&s[0]));
                             }
                             tmem_wait_st();
                         }
+                        tmem_ld32(tmem_s, &s[0]);
+                        tmem_ld32(tmem_s + 32, &s[32]);
+                        tmem_wait_ld();
                     }
                     if (!ok) break;
                     l_run += tile_sum;
-                    // P_g(j) over the first columns of the part's OWN score columns (the other parts may still be
-                    // reading theirs)
-                    if (W == 32) tmem_st16(tmem_s, *reinterpret_cast<const uint32_t(*)[16]>(&packed[0]));
-                    else tmem_st8(tmem_s, *reinterpret_cast<const uint32_t(*)[8]>(&packed[0]));
+                    tmem_st32(tmem_s, packed);   // P(j) over the first columns of the buffer, whose scores sit in registers
                     tmem_wait_st();
-                    // The issuer signals the completion of key tile j's products on barrier j & 1.  Every warp consumes
-                    // every phase of both barriers in order (a parity wait is only sound one phase behind), two key
-                    // tiles late: before handing over P(j) it waits for tile j - 2, the phase before the one that
-                    // P(j) itself leads to -- so the wait is sound and, the tensor pipe being that far along anyway,
-                    // costs nothing.  (The rare path above waits for tile j - 1 on the other barrier, its next phase.)
-                    if (j > 1) {
-                        ok = mbar_wait(smem_u32(&bar_pv_done[j & 1]), ((j - 2) >> 1) & 1, abort_p, args.status, SITE_G_PV, j);
+                    // every phase of the part's completion barrier is consumed in order, one own key tile late: the
+                    // product of key tile j - SPLIT has had SPLIT tiles' time to finish
+                    if (i > 0) {
+                        ok = mbar_wait(b_pvdone, (i - 1) & 1, abort_p, args.status, SITE_G_PV, j);
                         ok = __all_sync(0xffffffffu, ok);
                         if (!ok) break;
                     }
                     tc_fence_before_sync();
                     if (lane == 0) mbar_arrive(smem_u32(&bar_p_full[0][b]));
-                    if (++b == NB) { b = 0; ph ^= 1; }
+                    b += SPLIT;
+                    if (b >= NB) { b -= NB; ph ^= 1; }
                 }
                 if (tid == 0) F4S_MARK(5);
                 // ---- combine the parts: o = sum_g 2^(m_g - m) O_g / sum_g 2^(m_g - m) l_g, m = max_g m_g
@@ -464,6 +462,7 @@ fused4s_attention_kernel(const __grid_constant__ CUtensorMap tmap_q, const __gri
                         for (int c = 0; c < 16; ++c) acc[c] = 0.f;
 #pragma unroll
                         for (int p2 = 0; p2 < SPLIT; ++p2) {
+                            if (p2 >= n_kv) continue;   // a part without a key tile never wrote its accumulator
                             uint32_t x[16];
                             tmem_ld16(tmem_o0 + p2 * dpad + lane_off + cg * 16, x);
                             tmem_wait_ld();

@@ -203,11 +203,10 @@ extern "C" int sd_attn_create(sd_attn_handle** out) {
     if (e == cudaSuccess) e = raise_smem_limit(fused4s_attention_kernel<0, 1>, F4S_SMEM_BUDGET + 1024);
     if (e == cudaSuccess) e = raise_smem_limit(fused4s_attention_kernel<0, 2>, F4S_SMEM_BUDGET + 1024);
     if (e == cudaSuccess) e = raise_smem_limit(fused4s_attention_kernel<0, 3>, F4S_SMEM_BUDGET + 1024);
-    if (e == cudaSuccess) e = raise_smem_limit(fused4s_attention_kernel<0, 1, 4>, F4S_SMEM_BUDGET + 1024);
-    if (e == cudaSuccess) e = raise_smem_limit(fused4s_attention_kernel<0, 1, 2>, F4S_SMEM_BUDGET + 1024);
-    if (e == cudaSuccess) e = raise_smem_limit(fused4s_attention_kernel<0, 2, 4>, F4S_SMEM_BUDGET + 1024);
-    if (e == cudaSuccess) e = raise_smem_limit(fused4s_attention_kernel<0, 2, 2>, F4S_SMEM_BUDGET + 1024);
-    if (e == cudaSuccess) e = raise_smem_limit(fused4s_attention_kernel<0, 3, 2>, F4S_SMEM_BUDGET + 1024);
+    if (e == cudaSuccess) e = raise_smem_limit(fused4s_attention_kernel<F4S_POLY_PER8, 1, 4>, F4S_SMEM_BUDGET + 1024);
+    if (e == cudaSuccess) e = raise_smem_limit(fused4s_attention_kernel<F4S_POLY_PER8, 1, 2>, F4S_SMEM_BUDGET + 1024);
+    if (e == cudaSuccess) e = raise_smem_limit(fused4s_attention_kernel<F4S_POLY_PER8, 2, 2>, F4S_SMEM_BUDGET + 1024);
+    if (e == cudaSuccess) e = raise_smem_limit(fused4s_attention_kernel<F4S_POLY_PER8, 3, 2>, F4S_SMEM_BUDGET + 1024);
     if (e == cudaSuccess) e = raise_smem_limit(twopass_scores_kernel, twopass_scores_smem_bytes(3));
     if (e == cudaSuccess) e = raise_smem_limit(twopass_pv_kernel, twopass_pv_smem_bytes(3));
     if (e == cudaSuccess) e = raise_smem_limit(simt_attention_kernel<float, 5>, simt_smem_bytes(160));
@@ -221,12 +220,12 @@ extern "C" int sd_attn_create(sd_attn_handle** out) {
         if (e == cudaSuccess)
             h->fused4_ok = F4_THREADS * fa.numRegs >= 512 * F4_SOFTMAX_REGS + 256 * F4_CONTROL_REGS;
         h->fused4s_ok = 1;
-        const void* f4s[9] = {(const void*)fused4s_attention_kernel<F4S_POLY_PER8, 1>, (const void*)fused4s_attention_kernel<0, 1>,
+        const void* f4s[8] = {(const void*)fused4s_attention_kernel<F4S_POLY_PER8, 1>, (const void*)fused4s_attention_kernel<0, 1>,
                               (const void*)fused4s_attention_kernel<0, 2>, (const void*)fused4s_attention_kernel<0, 3>,
-                              (const void*)fused4s_attention_kernel<0, 1, 4>, (const void*)fused4s_attention_kernel<0, 1, 2>,
-                              (const void*)fused4s_attention_kernel<0, 2, 4>, (const void*)fused4s_attention_kernel<0, 2, 2>,
-                              (const void*)fused4s_attention_kernel<0, 3, 2>};
-        for (int i = 0; i < 9 && e == cudaSuccess; ++i) {
+                              (const void*)fused4s_attention_kernel<F4S_POLY_PER8, 1, 4>, (const void*)fused4s_attention_kernel<F4S_POLY_PER8, 1, 2>,
+                              (const void*)fused4s_attention_kernel<F4S_POLY_PER8, 2, 2>,
+                              (const void*)fused4s_attention_kernel<F4S_POLY_PER8, 3, 2>};
+        for (int i = 0; i < 8 && e == cudaSuccess; ++i) {
             e = cudaFuncGetAttributes(&fa, f4s[i]);
             if (e == cudaSuccess && F4_THREADS * fa.numRegs < 512 * F4S_SOFTMAX_REGS + 256 * F4S_CONTROL_REGS) h->fused4s_ok = 0;
         }
@@ -513,27 +512,25 @@ static int launch_fused4s(sd_attn_handle* h, const Problem& p) {
     if (rc == SD_ATTN_OK) rc = make_tmap(h, &tv, p.v, p.BH, p.Nk, p.d, F4_BN);
     if (rc != SD_ATTN_OK) return rc;
     dim3 grid((tiles_per_head + a.tiles_per_cta - 1) / a.tiles_per_cta, p.BH), block(F4_THREADS);
-    // One tile per CTA: its score columns are shared out among as many warpgroups as tensor memory has accumulators
-    // for (two score buffers + split * dpad columns <= 512).
+    // One tile per CTA: its key tiles are dealt out among 4 or 2 warpgroups (parts), each with an accumulator of its
+    // own in tensor memory next to the score buffers, whose number is a multiple of the parts (a buffer then always
+    // meets the same part) and smaller than the K/V ring (a buffer ahead is a key tile ahead).
     int split = 1;
-    if (a.tiles_per_cta == 1 && !h->fused_no_split) split = 2 * F4_BN + 4 * a.dpad <= 512 ? 4 : 2 * F4_BN + 2 * a.dpad <= 512 ? 2 : 1;
-    if (h->fused_split_override) split = a.tiles_per_cta == 1 && 2 * F4_BN + h->fused_split_override * a.dpad <= 512 ? h->fused_split_override : 1;
-    // ... and as many score buffers as the rest of tensor memory holds, the K/V ring permitting (a buffer ahead is a
-    // key tile ahead)
-    a.split_buffers = (512 - split * a.dpad) / F4_BN;
-    if (a.split_buffers > F4S_BUFFERS) a.split_buffers = F4S_BUFFERS;
-    if (a.split_buffers > a.stages - 1) a.split_buffers = a.stages - 1;
-    if (a.split_buffers < 2) split = 1;
+    a.split_buffers = 2;
+    if (a.tiles_per_cta == 1 && !h->fused_no_split) {
+        split = 4 * F4_BN + 4 * a.dpad <= 512 ? 4 : 2;
+        if (h->fused_split_override == 2) split = 2;
+        a.split_buffers = (4 * F4_BN + split * a.dpad <= 512 && a.stages >= 5) ? 4 : 2;
+        if (a.split_buffers < split || 2 * F4_BN + 2 * a.dpad > 512) split = 1;   // (no room: d > 192)
+    }
     if (split == 4 && a.nch == 1)
-        launch_overlapped(h, fused4s_attention_kernel<0, 1, 4>, grid, block, smem, p.stream, tq, tk, tv, a);
+        launch_overlapped(h, fused4s_attention_kernel<F4S_POLY_PER8, 1, 4>, grid, block, smem, p.stream, tq, tk, tv, a);
     else if (split == 2 && a.nch == 1)
-        launch_overlapped(h, fused4s_attention_kernel<0, 1, 2>, grid, block, smem, p.stream, tq, tk, tv, a);
-    else if (split == 4 && a.nch == 2)
-        launch_overlapped(h, fused4s_attention_kernel<0, 2, 4>, grid, block, smem, p.stream, tq, tk, tv, a);
+        launch_overlapped(h, fused4s_attention_kernel<F4S_POLY_PER8, 1, 2>, grid, block, smem, p.stream, tq, tk, tv, a);
     else if (split == 2 && a.nch == 2)
-        launch_overlapped(h, fused4s_attention_kernel<0, 2, 2>, grid, block, smem, p.stream, tq, tk, tv, a);
+        launch_overlapped(h, fused4s_attention_kernel<F4S_POLY_PER8, 2, 2>, grid, block, smem, p.stream, tq, tk, tv, a);
     else if (split == 2 && a.nch == 3)
-        launch_overlapped(h, fused4s_attention_kernel<0, 3, 2>, grid, block, smem, p.stream, tq, tk, tv, a);
+        launch_overlapped(h, fused4s_attention_kernel<F4S_POLY_PER8, 3, 2>, grid, block, smem, p.stream, tq, tk, tv, a);
     // the polynomial share of the exponentials only pays where four tiles saturate the special function unit
     else if (a.dpad <= 48)
         launch_overlapped(h, fused4s_attention_kernel<F4S_POLY_PER8, 1>, grid, block, smem, p.stream, tq, tk, tv, a);

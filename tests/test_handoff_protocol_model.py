@@ -147,23 +147,23 @@ def test_one_barrier_per_buffer_is_not_enough():
 
 
 # ---------------------------------------------------------------------------------------------------------------
-# The variant for ONE query tile per CTA: the columns of every score tile are shared out among several warpgroups
-# ("parts"), NB score buffers run ahead of the products, and the MMAs come from TWO threads -- the products
-# O_g (+)= P_g V(j) from one, the scores of key tile j + NB from the other -- whose instructions the tensor pipe does
-# not order against each other.
+# The variant for ONE query tile per CTA: the key tiles are dealt out among SPLIT warpgroups ("parts": part g takes
+# key tiles g, g + SPLIT, ...), NB score buffers run ahead of the products, and the MMAs come from TWO threads -- the
+# products O_g (+)= P(j) V(j) from one, the scores of key tile j + NB from the other -- whose instructions the tensor
+# pipe does not order against each other.
 
-def simulate_parts(NB, n_kv, stages, seed, warps=8, pv_ring=2, wait_buf_free=True, limit=400000):
+def simulate_parts(SPLIT, NB, n_kv, stages, seed, warps=4, wait_buf_free=True, limit=400000):
     rnd = random.Random(seed)
     s_full = [Bar(1) for _ in range(NB)]
     p_full = [Bar(warps) for _ in range(NB)]
     buf_free = [Bar(1) for _ in range(NB)]
-    pv_done = [Bar(1) for _ in range(pv_ring)]
+    pv_done = [Bar(1) for _ in range(SPLIT)]
     o_final = Bar(1)
     q_full = Bar(1)
     kv_full = [Bar(1) for _ in range(stages)]
     kv_empty = [Bar(1) for _ in range(stages)]
     pipe_a, pipe_b = [], []                      # per issuing thread, each retired in order
-    buf = {b: {} for b in range(NB)}             # per buffer and warp: what its columns hold
+    buf = {b: {} for b in range(NB)}             # per buffer and warp: what it holds
     stage, errors = {}, []
 
     def check(cond, what):
@@ -202,28 +202,27 @@ def simulate_parts(NB, n_kv, stages, seed, warps=8, pv_ring=2, wait_buf_free=Tru
             while not p_full[b].done((j // NB) & 1):
                 yield
             check(stage.get(j % stages) == j, ("P V reads a stale stage", j))
-            pipe_a.append(("PV", j, b, [pv_done[j % pv_ring], buf_free[b], kv_empty[j % stages]] +
+            pipe_a.append(("PV", j, b, [pv_done[j % SPLIT], buf_free[b], kv_empty[j % stages]] +
                            ([o_final] if j == n_kv - 1 else [])))
             yield
 
-    def part_warp(w):
-        for j in range(n_kv):
+    def part_warp(g, w):
+        for i, j in enumerate(range(g, n_kv, SPLIT)):
             b = j % NB
             while not s_full[b].done((j // NB) & 1):
                 yield
-            check(buf[b].get(w) == ("S", j), ("a part reads the wrong scores", w, j, b, buf[b].get(w)))
+            check(buf[b].get(w) == ("S", j), ("a part reads the wrong scores", g, w, j, b, buf[b].get(w)))
             yield
             buf[b][w] = ("P", j)
-            if j >= pv_ring:   # products of key tile j - pv_ring: the phase before the one P(j) leads to
-                jj = j - pv_ring
-                while not pv_done[jj % pv_ring].done((jj // pv_ring) & 1):
+            if i > 0:          # the product of the part's previous key tile
+                while not pv_done[g].done((i - 1) & 1):
                     yield
             p_full[b].arrive()
             yield
         while not o_final.done(0):
             yield
 
-    procs = [producer(), score_thread(), product_thread()] + [part_warp(w) for w in range(warps)]
+    procs = [producer(), score_thread(), product_thread()] + [part_warp(g, w) for g in range(SPLIT) for w in range(warps)]
     steps = 0
     while procs and not errors:
         steps += 1
@@ -247,15 +246,15 @@ def simulate_parts(NB, n_kv, stages, seed, warps=8, pv_ring=2, wait_buf_free=Tru
     return errors[0] if errors else "ok"
 
 
-@pytest.mark.parametrize("NB", [2, 3, 4, 5])
-@pytest.mark.parametrize("n_kv", [1, 2, 3, 5, 8, 16, 17])
-def test_lone_tile_in_parts_protocol(NB, n_kv):
+@pytest.mark.parametrize("SPLIT,NB", [(2, 2), (2, 4), (4, 4)])
+@pytest.mark.parametrize("n_kv", [1, 2, 3, 4, 5, 8, 16, 17])
+def test_lone_tile_in_parts_protocol(SPLIT, NB, n_kv):
     for seed in range(4):
-        assert simulate_parts(NB, n_kv, 8, seed) == "ok"
-        assert simulate_parts(NB, n_kv, NB + 1, seed, warps=16) == "ok"
+        assert simulate_parts(SPLIT, NB, n_kv, 8, seed) == "ok"
+        assert simulate_parts(SPLIT, NB, n_kv, NB + 1, seed) == "ok"
 
 
 def test_scores_must_wait_for_the_completion_of_the_products_they_overwrite():
     """Without the per-buffer completion barrier the second thread's scores can land on weights not yet read."""
-    outcomes = {simulate_parts(3, 17, 8, seed, wait_buf_free=False) for seed in range(12)}
+    outcomes = {simulate_parts(2, 4, 17, 8, seed, wait_buf_free=False) for seed in range(12)}
     assert outcomes != {"ok"}
