@@ -217,7 +217,8 @@ def run_ours(args):
     att = bd.Attention(mode)
     calls = {"c2": workloads.config2, "c5-cross": lambda: [workloads.config5()[2]],
              "c3-cross": workloads.config3, "c4": workloads.config4,
-             "c1-twopass": workloads.config1}[args.workload]()
+             "c4-d80": lambda: [c for c in workloads.config4() if c.kind == "self" and c.d == 80][:1],
+             "c1": workloads.config1, "c1-twopass": workloads.config1}[args.workload]()
     sets = make_sets(calls, ROTATING_SETS, device, rank)
     if mode == bd.MODE_TWOPASS:   # the comparator borrows its scratch from the caller
         need_ws = max(bd.sd_attn_workspace_bytes(mode, c.B, c.H, c.Nq, c.Nk, c.d, bd.F16) for c in calls)
@@ -419,7 +420,7 @@ def main():
     ap.add_argument("--steps", type=int, default=200)
     ap.add_argument("--warmup", type=int, default=10)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--workload", default="c2", choices=["c2", "c5-cross", "c3-cross", "c4", "c1-twopass"],
+    ap.add_argument("--workload", default="c2", choices=["c2", "c5-cross", "c3-cross", "c4", "c4-d80", "c1", "c1-twopass"],
                     help="with --kernel-loop-only: which calls the loop runs (the bench line is always c2)")
     ap.add_argument("--kernel-loop-only", action="store_true",
                     help="run only the warm-up and the timed loop (for ncu captures)")
