@@ -24,6 +24,10 @@ _lib = None
 
 F16, F32 = 0, 1
 
+_GEGLU_SRC = os.path.join(_HERE, "sd_geglu_oracle.c")
+_GEGLU_LIB = os.path.join(_HERE, "libsd_geglu_oracle.so")
+_geglu_lib = None
+
 
 def build(force: bool = False) -> str:
     """Compile the C oracle with gcc (plain -O2, OpenMP, no fast-math, no FP contraction)."""
@@ -119,3 +123,55 @@ def forward(q: np.ndarray, k: np.ndarray, v: np.ndarray, scale, rows=None, want_
     if rc != 0:
         raise RuntimeError("sd_attn_oracle_forward failed with code %d" % rc)
     return (out, L, S, P) if want_probs else (out, L, S)
+
+
+# ---------------------------------------------------------------------------------------------------------------
+# Fused GEGLU (Sec. 3.1, Eq. 2): out = x[:, :C] * GELU(x[:, C:]).  The arithmetic lives in sd_geglu_oracle.c.
+
+def build_geglu(force: bool = False) -> str:
+    stale = (not os.path.exists(_GEGLU_LIB)) or os.path.getmtime(_GEGLU_LIB) < os.path.getmtime(_GEGLU_SRC)
+    if force or stale:
+        tmp = _GEGLU_LIB + ".tmp.%d" % os.getpid()
+        cmd = ["gcc", "-O2", "-std=c11", "-fopenmp", "-ffp-contract=off", "-fPIC", "-shared", "-o", tmp, _GEGLU_SRC, "-lm"]
+        subprocess.run(cmd, check=True, capture_output=True)
+        os.replace(tmp, _GEGLU_LIB)
+    return _GEGLU_LIB
+
+
+def _load_geglu():
+    global _geglu_lib
+    with _lock:
+        if _geglu_lib is None:
+            lib = ctypes.CDLL(build_geglu())
+            lib.sd_geglu_oracle_forward.restype = ctypes.c_int
+            lib.sd_geglu_oracle_forward.argtypes = [ctypes.c_void_p, ctypes.c_void_p, ctypes.c_int64, ctypes.c_int64,
+                                                    ctypes.c_int]
+            lib.sd_geglu_oracle_gelu.restype = ctypes.c_double
+            lib.sd_geglu_oracle_gelu.argtypes = [ctypes.c_double]
+            _geglu_lib = lib
+    return _geglu_lib
+
+
+def gelu(g: float) -> float:
+    """GELU of Eq. 2 for one double."""
+    return float(_load_geglu().sd_geglu_oracle_gelu(float(g)))
+
+
+def geglu_forward(x: np.ndarray) -> np.ndarray:
+    """x: [..., 2C] float16 or float32 -> [..., C] float64, out = x[..., :C] * GELU(x[..., C:])."""
+    if x.dtype == np.float16:
+        dtype = F16
+    elif x.dtype == np.float32:
+        dtype = F32
+    else:
+        raise TypeError("x must be float16 or float32")
+    if x.shape[-1] % 2:
+        raise ValueError("the last dimension holds both halves: it must be even")
+    x = np.ascontiguousarray(x)
+    C = x.shape[-1] // 2
+    rows = x.size // (2 * C) if C else 0
+    out = np.empty(x.shape[:-1] + (C,), dtype=np.float64)
+    rc = _load_geglu().sd_geglu_oracle_forward(x.ctypes.data, out.ctypes.data, rows, C, dtype)
+    if rc != 0:
+        raise ValueError("sd_geglu_oracle_forward rejected its arguments")
+    return out
