@@ -27,7 +27,7 @@ EXPORTS = ["sd_attn_create", "sd_attn_forward", "sd_attn_destroy", "sd_attn_set_
            "sd_attn_workspace_bytes", "sd_attn_set_workspace", "sd_attn_twopass_buffers",
            "sd_attn_query_status", "sd_attn_last_mode", "sd_attn_launch_count", "sd_attn_status_string",
            "sd_attn_forward_host", "sd_attn_host_staging_bytes", "sd_attn_debug_dump_cross_scores",
-           "sd_attn_forward_twopass_static"]
+           "sd_attn_forward_twopass_static", "sd_geglu_forward"]
 
 _lib = None
 
@@ -77,6 +77,8 @@ def load() -> ctypes.CDLL:
     lib.sd_attn_status_string.argtypes = [ci]
     lib.sd_attn_forward_twopass_static.restype = ci
     lib.sd_attn_forward_twopass_static.argtypes = [vp, vp, vp, vp, ci, ci, ci, ci, ci, cf, ci, vp]
+    lib.sd_geglu_forward.restype = ci
+    lib.sd_geglu_forward.argtypes = [vp, vp, ctypes.c_longlong, ci, ci, vp]
     lib.sd_attn_debug_dump_cross_scores.restype = ci
     lib.sd_attn_debug_dump_cross_scores.argtypes = [vp, vp]
     _lib = lib
@@ -127,6 +129,32 @@ def sd_attn_forward_twopass_static(q, k, v, out, B, H, Nq, Nk, d, scale, dtype, 
     """
     return load().sd_attn_forward_twopass_static(q, k, v, out, B, H, Nq, Nk, d, ctypes.c_float(scale), dtype,
                                                  stream or None)
+
+
+def sd_geglu_forward(x, out, rows: int, C: int, dtype: int, stream=0) -> int:
+    """Fused GEGLU (Sec. 3.1, Eq. 2): out[r][c] = x[r][c] * GELU(x[r][C + c]); x is [rows][2C], out [rows][C].
+
+    x and out are device addresses; returns the status code.  No handle: the operation has no state.
+    """
+    return load().sd_geglu_forward(x or None, out or None, rows, C, dtype, stream or None)
+
+
+def geglu(x, out=None, stream=None):
+    """Marshalling helper for torch tensors: x [..., 2C] (float16 or float32, contiguous, CUDA) -> [..., C]."""
+    import torch
+    if not x.is_cuda or not x.is_contiguous():
+        raise ValueError("x must be a contiguous CUDA tensor")
+    if x.dtype not in (torch.float16, torch.float32) or x.shape[-1] % 2:
+        raise ValueError("x must be float16 or float32 with an even last dimension")
+    C = x.shape[-1] // 2
+    if out is None:
+        out = torch.empty(x.shape[:-1] + (C,), dtype=x.dtype, device=x.device)
+    rows = x.numel() // (2 * C) if C else 0
+    s = stream if stream is not None else torch.cuda.current_stream().cuda_stream
+    rc = sd_geglu_forward(x.data_ptr(), out.data_ptr(), rows, C, F16 if x.dtype == torch.float16 else F32, s)
+    if rc != OK:
+        raise SdAttnError(rc, "sd_geglu_forward")
+    return out
 
 
 def sd_attn_set_mode(handle, mode: int) -> int:

@@ -13,8 +13,10 @@
 
 #include "../../include/sd_attn.h"
 #include "../../include/sd_attn_debug.h"
+#include "../../include/sd_geglu.h"
 #include "cross_kernel.cuh"
 #include "cross2_kernel.cuh"
+#include "geglu_kernel.cuh"
 #include "fused_kernel.cuh"
 #include "fused4_kernel.cuh"
 #include "fused4s_kernel.cuh"
@@ -830,6 +832,48 @@ extern "C" int sd_attn_forward_twopass_static(const void* q, const void* k, cons
     e = cudaGetLastError();
     if (e != cudaSuccess) return cuda_fail(nullptr, e);
     twopass_pv_kernel<<<grid, TWOPASS_THREADS, twopass_pv_smem_bytes(a.nch), s>>>(tv, a);
+    e = cudaGetLastError();
+    return e == cudaSuccess ? SD_ATTN_OK : cuda_fail(nullptr, e);
+}
+
+// ------------------------------------------------------------------------------------------------
+// Fused GEGLU (Sec. 3.1, Eq. 2): stateless, one kernel.
+extern "C" int sd_geglu_forward(const void* x, void* out, long long rows, int C, int dtype, void* stream) {
+    if (rows < 0 || C <= 0) return SD_ATTN_ERR_INVALID_VALUE;
+    if (dtype != SD_ATTN_F16 && dtype != SD_ATTN_F32) return SD_ATTN_ERR_UNSUPPORTED;
+    if (rows == 0) return SD_ATTN_OK;
+    if (!x || !out) return SD_ATTN_ERR_INVALID_VALUE;
+    if (rows > (1ll << 40) / C) return SD_ATTN_ERR_INVALID_VALUE;
+    if (((uintptr_t)x & 15u) || ((uintptr_t)out & 15u)) return SD_ATTN_ERR_ALIGNMENT;
+    int dev = 0, major = 0, sms = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e == cudaSuccess) e = cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev);
+    if (e == cudaSuccess) e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+    if (e != cudaSuccess) return cuda_fail(nullptr, e);
+    if (major != 10) return SD_ATTN_ERR_ARCH;
+    cudaStream_t s = (cudaStream_t)stream;
+    const long long elems = rows * C;
+    const int vec = dtype == SD_ATTN_F16 ? 8 : 4;
+    // a small multiple of the SM count walks the tensor with a stride; fewer blocks for a small tensor
+    auto blocks_for = [&](long long work_items) {
+        long long b = (work_items + GEGLU_THREADS - 1) / GEGLU_THREADS;
+        const long long cap = (long long)sms * 8;
+        return (unsigned)(b < cap ? b : cap);
+    };
+    if (C % vec == 0) {
+        const long long pieces = elems / vec;
+        const unsigned blocks = blocks_for((pieces + GEGLU_UNROLL - 1) / GEGLU_UNROLL);
+        if (dtype == SD_ATTN_F16)
+            geglu_vector_kernel<__half, 8><<<blocks, GEGLU_THREADS, 0, s>>>((const __half*)x, (__half*)out, pieces, C / 8);
+        else
+            geglu_vector_kernel<float, 4><<<blocks, GEGLU_THREADS, 0, s>>>((const float*)x, (float*)out, pieces, C / 4);
+    } else {
+        const unsigned blocks = blocks_for(elems);
+        if (dtype == SD_ATTN_F16)
+            geglu_scalar_kernel<__half><<<blocks, GEGLU_THREADS, 0, s>>>((const __half*)x, (__half*)out, elems, C);
+        else
+            geglu_scalar_kernel<float><<<blocks, GEGLU_THREADS, 0, s>>>((const float*)x, (float*)out, elems, C);
+    }
     e = cudaGetLastError();
     return e == cudaSuccess ? SD_ATTN_OK : cuda_fail(nullptr, e);
 }
