@@ -857,7 +857,7 @@ extern "C" int sd_geglu_forward(const void* x, void* out, long long rows, int C,
     // a small multiple of the SM count walks the tensor with a stride; fewer blocks for a small tensor
     auto blocks_for = [&](long long work_items) {
         long long b = (work_items + GEGLU_THREADS - 1) / GEGLU_THREADS;
-        const long long cap = (long long)sms * 8;
+        const long long cap = (long long)sms * GEGLU_BLOCKS_PER_SM;
         return (unsigned)(b < cap ? b : cap);
     };
     if (C % vec == 0) {
