@@ -27,6 +27,9 @@ F16, F32 = 0, 1
 _GEGLU_SRC = os.path.join(_HERE, "sd_geglu_oracle.c")
 _GEGLU_LIB = os.path.join(_HERE, "libsd_geglu_oracle.so")
 _geglu_lib = None
+_GN_SRC = os.path.join(_HERE, "sd_groupnorm_oracle.c")
+_GN_LIB = os.path.join(_HERE, "libsd_groupnorm_oracle.so")
+_gn_lib = None
 
 
 def build(force: bool = False) -> str:
@@ -175,3 +178,58 @@ def geglu_forward(x: np.ndarray) -> np.ndarray:
     if rc != 0:
         raise ValueError("sd_geglu_oracle_forward rejected its arguments")
     return out
+
+
+# ---------------------------------------------------------------------------------------------------------------
+# Fused group normalisation (Sec. 3.1, Eq. 1).  The arithmetic lives in sd_groupnorm_oracle.c.
+
+def build_groupnorm(force: bool = False) -> str:
+    stale = (not os.path.exists(_GN_LIB)) or os.path.getmtime(_GN_LIB) < os.path.getmtime(_GN_SRC)
+    if force or stale:
+        tmp = _GN_LIB + ".tmp.%d" % os.getpid()
+        cmd = ["gcc", "-O2", "-std=c11", "-fopenmp", "-ffp-contract=off", "-fPIC", "-shared", "-o", tmp, _GN_SRC, "-lm"]
+        subprocess.run(cmd, check=True, capture_output=True)
+        os.replace(tmp, _GN_LIB)
+    return _GN_LIB
+
+
+def _load_groupnorm():
+    global _gn_lib
+    with _lock:
+        if _gn_lib is None:
+            lib = ctypes.CDLL(build_groupnorm())
+            lib.sd_groupnorm_oracle_forward.restype = ctypes.c_int
+            lib.sd_groupnorm_oracle_forward.argtypes = [ctypes.c_void_p] * 6 + [ctypes.c_int64] * 4 + [ctypes.c_double,
+                                                                                                      ctypes.c_int]
+            _gn_lib = lib
+    return _gn_lib
+
+
+def groupnorm_forward(x: np.ndarray, groups: int, eps: float, gamma=None, beta=None):
+    """x: [N, C, ...] float16 or float32 (spatial dimensions flattened); returns (y, mean, rstd) in float64:
+    y like x, mean and rstd [N, groups]."""
+    if x.dtype == np.float16:
+        dtype = F16
+    elif x.dtype == np.float32:
+        dtype = F32
+    else:
+        raise TypeError("x must be float16 or float32")
+    if x.ndim < 2:
+        raise ValueError("x must be [N, C, ...]")
+    x = np.ascontiguousarray(x)
+    N, C = x.shape[0], x.shape[1]
+    HW = int(np.prod(x.shape[2:])) if x.ndim > 2 else 1
+    for name, t in (("gamma", gamma), ("beta", beta)):
+        if t is not None and (t.dtype != x.dtype or t.shape != (C,)):
+            raise ValueError("%s must be [C] in x's dtype" % name)
+    ga = np.ascontiguousarray(gamma) if gamma is not None else None
+    be = np.ascontiguousarray(beta) if beta is not None else None
+    y = np.empty(x.shape, dtype=np.float64)
+    mean = np.empty((N, groups), dtype=np.float64)
+    rstd = np.empty((N, groups), dtype=np.float64)
+    rc = _load_groupnorm().sd_groupnorm_oracle_forward(
+        x.ctypes.data, ga.ctypes.data if ga is not None else None, be.ctypes.data if be is not None else None,
+        y.ctypes.data, mean.ctypes.data, rstd.ctypes.data, N, C, HW, groups, float(eps), dtype)
+    if rc != 0:
+        raise ValueError("sd_groupnorm_oracle_forward rejected its arguments")
+    return y, mean, rstd
