@@ -27,7 +27,7 @@ EXPORTS = ["sd_attn_create", "sd_attn_forward", "sd_attn_destroy", "sd_attn_set_
            "sd_attn_workspace_bytes", "sd_attn_set_workspace", "sd_attn_twopass_buffers",
            "sd_attn_query_status", "sd_attn_last_mode", "sd_attn_launch_count", "sd_attn_status_string",
            "sd_attn_forward_host", "sd_attn_host_staging_bytes", "sd_attn_debug_dump_cross_scores",
-           "sd_attn_forward_twopass_static", "sd_geglu_forward"]
+           "sd_attn_forward_twopass_static", "sd_geglu_forward", "sd_groupnorm_forward"]
 
 _lib = None
 
@@ -79,6 +79,8 @@ def load() -> ctypes.CDLL:
     lib.sd_attn_forward_twopass_static.argtypes = [vp, vp, vp, vp, ci, ci, ci, ci, ci, cf, ci, vp]
     lib.sd_geglu_forward.restype = ci
     lib.sd_geglu_forward.argtypes = [vp, vp, ctypes.c_longlong, ci, ci, vp]
+    lib.sd_groupnorm_forward.restype = ci
+    lib.sd_groupnorm_forward.argtypes = [vp, vp, vp, vp, ci, ci, ctypes.c_longlong, ci, cf, ci, vp]
     lib.sd_attn_debug_dump_cross_scores.restype = ci
     lib.sd_attn_debug_dump_cross_scores.argtypes = [vp, vp]
     _lib = lib
@@ -154,6 +156,38 @@ def geglu(x, out=None, stream=None):
     rc = sd_geglu_forward(x.data_ptr(), out.data_ptr(), rows, C, F16 if x.dtype == torch.float16 else F32, s)
     if rc != OK:
         raise SdAttnError(rc, "sd_geglu_forward")
+    return out
+
+
+def sd_groupnorm_forward(x, gamma, beta, y, N: int, C: int, HW: int, G: int, eps: float, dtype: int, stream=0) -> int:
+    """Fused group normalisation (Sec. 3.1, Eq. 1) of x [N][C][HW] into y; gamma and beta are [C] or 0 (none).
+
+    All pointers are device addresses; returns the status code.  No handle: the operation has no state.
+    """
+    return load().sd_groupnorm_forward(x or None, gamma or None, beta or None, y or None, N, C, HW, G,
+                                       ctypes.c_float(eps), dtype, stream or None)
+
+
+def groupnorm(x, groups: int, eps: float = 1e-5, gamma=None, beta=None, out=None, stream=None):
+    """Marshalling helper for torch tensors: x [N, C, ...] (float16 or float32, contiguous, CUDA)."""
+    import torch
+    if not x.is_cuda or not x.is_contiguous() or x.dim() < 2:
+        raise ValueError("x must be a contiguous CUDA tensor [N, C, ...]")
+    if x.dtype not in (torch.float16, torch.float32):
+        raise ValueError("x must be float16 or float32")
+    N, C = x.shape[0], x.shape[1]
+    HW = x.numel() // (N * C) if N * C else 1
+    for t in (gamma, beta):
+        if t is not None and (t.dtype != x.dtype or tuple(t.shape) != (C,) or not t.is_cuda or not t.is_contiguous()):
+            raise ValueError("gamma and beta must be contiguous CUDA tensors [C] of x's dtype")
+    if out is None:
+        out = torch.empty_like(x)
+    s = stream if stream is not None else torch.cuda.current_stream().cuda_stream
+    rc = sd_groupnorm_forward(x.data_ptr(), gamma.data_ptr() if gamma is not None else 0,
+                              beta.data_ptr() if beta is not None else 0, out.data_ptr(), N, C, HW, groups, eps,
+                              F16 if x.dtype == torch.float16 else F32, s)
+    if rc != OK:
+        raise SdAttnError(rc, "sd_groupnorm_forward")
     return out
 
 

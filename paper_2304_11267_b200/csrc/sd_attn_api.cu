@@ -14,9 +14,11 @@
 #include "../../include/sd_attn.h"
 #include "../../include/sd_attn_debug.h"
 #include "../../include/sd_geglu.h"
+#include "../../include/sd_groupnorm.h"
 #include "cross_kernel.cuh"
 #include "cross2_kernel.cuh"
 #include "geglu_kernel.cuh"
+#include "groupnorm_kernel.cuh"
 #include "fused_kernel.cuh"
 #include "fused4_kernel.cuh"
 #include "fused4s_kernel.cuh"
@@ -874,6 +876,59 @@ extern "C" int sd_geglu_forward(const void* x, void* out, long long rows, int C,
         else
             geglu_scalar_kernel<float><<<blocks, GEGLU_THREADS, 0, s>>>((const float*)x, (float*)out, elems, C);
     }
+    e = cudaGetLastError();
+    return e == cudaSuccess ? SD_ATTN_OK : cuda_fail(nullptr, e);
+}
+
+// ------------------------------------------------------------------------------------------------
+// Fused group normalisation (Sec. 3.1, Eq. 1): stateless, one kernel, one thread block per (sample, group).
+static std::mutex g_gn_mutex;
+static int g_gn_limits_raised[STATIC_MAX_DEVICES];
+
+extern "C" int sd_groupnorm_forward(const void* x, const void* gamma, const void* beta, void* y, int N, int C,
+                                    long long HW, int G, float eps, int dtype, void* stream) {
+    if (N < 0 || C <= 0 || HW <= 0 || G <= 0 || C % G != 0) return SD_ATTN_ERR_INVALID_VALUE;
+    if (!(eps >= 0.f) || !isfinite(eps)) return SD_ATTN_ERR_INVALID_VALUE;
+    if (dtype != SD_ATTN_F16 && dtype != SD_ATTN_F32) return SD_ATTN_ERR_UNSUPPORTED;
+    if (N == 0) return SD_ATTN_OK;
+    if (!x || !y) return SD_ATTN_ERR_INVALID_VALUE;
+    if ((long long)N * G > 2147483647ll) return SD_ATTN_ERR_INVALID_VALUE;
+    const size_t es = dtype == SD_ATTN_F16 ? 2 : 4;
+    if (((uintptr_t)x & 15u) || ((uintptr_t)y & 15u) || ((uintptr_t)gamma & (es - 1)) || ((uintptr_t)beta & (es - 1)))
+        return SD_ATTN_ERR_ALIGNMENT;
+    int dev = 0, major = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e == cudaSuccess) e = cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev);
+    if (e != cudaSuccess) return cuda_fail(nullptr, e);
+    if (major != 10) return SD_ATTN_ERR_ARCH;
+    if (dev < 0 || dev >= STATIC_MAX_DEVICES) return SD_ATTN_ERR_UNSUPPORTED;
+    {
+        std::lock_guard<std::mutex> lock(g_gn_mutex);
+        if (!g_gn_limits_raised[dev]) {
+            e = raise_smem_limit(groupnorm_staged_kernel<__half, 8>, GN_MAX_STAGED_BYTES);
+            if (e == cudaSuccess) e = raise_smem_limit(groupnorm_staged_kernel<float, 4>, GN_MAX_STAGED_BYTES);
+            if (e != cudaSuccess) return cuda_fail(nullptr, e);
+            g_gn_limits_raised[dev] = 1;
+        }
+    }
+    GroupNormArgs a;
+    a.x = x; a.gamma = gamma; a.beta = beta; a.y = y;
+    a.C = C; a.G = G; a.HW = HW; a.eps = eps;
+    cudaStream_t s = (cudaStream_t)stream;
+    const long long group_elems = (long long)(C / G) * HW;
+    const long long group_bytes = group_elems * (long long)es;
+    const int vec = (int)(16 / es);
+    const unsigned blocks = (unsigned)((long long)N * G);
+    // staged: the group fits shared memory and neither a channel nor the group ends inside a 16-byte piece
+    const bool staged = group_bytes <= GN_MAX_STAGED_BYTES && HW % vec == 0;
+    if (staged && dtype == SD_ATTN_F16)
+        groupnorm_staged_kernel<__half, 8><<<blocks, GN_THREADS, (size_t)group_bytes, s>>>(a);
+    else if (staged)
+        groupnorm_staged_kernel<float, 4><<<blocks, GN_THREADS, (size_t)group_bytes, s>>>(a);
+    else if (dtype == SD_ATTN_F16)
+        groupnorm_streaming_kernel<__half><<<blocks, GN_THREADS, 0, s>>>(a);
+    else
+        groupnorm_streaming_kernel<float><<<blocks, GN_THREADS, 0, s>>>(a);
     e = cudaGetLastError();
     return e == cudaSuccess ? SD_ATTN_OK : cuda_fail(nullptr, e);
 }
