@@ -921,11 +921,11 @@ extern "C" int sd_groupnorm_forward(const void* x, const void* gamma, const void
     const unsigned blocks = (unsigned)((long long)N * G);
     // staged: the group fits shared memory and neither a channel nor the group ends inside a 16-byte piece
     const bool staged = group_bytes <= GN_MAX_STAGED_BYTES && HW % vec == 0;
-    if (staged && dtype == SD_ATTN_F16)
+    if (staged && dtype == SD_ATTN_F16) {
         groupnorm_staged_kernel<__half, 8><<<blocks, GN_THREADS, (size_t)group_bytes, s>>>(a);
-    else if (staged)
+    } else if (staged) {
         groupnorm_staged_kernel<float, 4><<<blocks, GN_THREADS, (size_t)group_bytes, s>>>(a);
-    else if (dtype == SD_ATTN_F16)
+    } else if (dtype == SD_ATTN_F16)
         groupnorm_streaming_kernel<__half><<<blocks, GN_THREADS, 0, s>>>(a);
     else
         groupnorm_streaming_kernel<float><<<blocks, GN_THREADS, 0, s>>>(a);
