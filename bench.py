@@ -430,6 +430,16 @@ def extras(att, bd, device, stream, peaks):
                                           "frac_of_nominal_8000": gbs / 8000.0,
                                           "algorithmic_bytes": c.io_bytes(), "peak_source": peaks["source"]}
     att.check(stream)
+    # the same two measurements with the tensors read as token-major [B][N][H][d] (the head split and merge around
+    # the attention as views): the same buffers, so the same bytes and the same sizes
+    att_t = bd.Attention(layout=bd.LAYOUT_BNHD)
+    us_graph_t = time_calls(att_t, bd, tensors, stream, 20, graph=True)
+    us_cross_t = time_calls(att_t, bd, csets, stream, 10) / n_sets
+    att_t.check(stream)
+    att_t.close()
+    out["token_major_layout"] = {"unet_step_attention_set_us_cuda_graph": us_graph_t,
+                                 "cross_attention_9216x77_d40_us_per_call": us_cross_t,
+                                 "note": "sd_attn_set_layout(SD_ATTN_LAYOUT_BNHD); compare with the two entries above"}
     out["geglu_8192x1280_f16"] = geglu_numbers(bd, device, stream, peaks)
     out["groupnorm_2x320x64x64_f16"] = groupnorm_numbers(bd, device, stream, peaks)
     return out

@@ -56,6 +56,13 @@ typedef enum {
     SD_ATTN_MODE_SIMT = 4     /* CUDA-core kernel, F16 or F32 storage, fp32 arithmetic        */
 } sd_attn_mode;
 
+typedef enum {
+    SD_ATTN_LAYOUT_BHND = 0, /* head-major: q, out [B][H][Nq][d]; k, v [B][H][Nk][d] (the default)              */
+    SD_ATTN_LAYOUT_BNHD = 1  /* token-major: q, out [B][Nq][H][d]; k, v [B][Nk][H][d] -- what a projection to
+                                H*d channels leaves, so the head split before and the head merge after the
+                                attention (Sec. 3.2) are views, not copies                                      */
+} sd_attn_layout;
+
 /* Largest Nk the CROSS mode accepts (one key tile). */
 #define SD_ATTN_CROSS_MAX_NK 128
 /* Largest head dim any mode accepts; F16 tensor-core modes need d to be a multiple of 8. */
@@ -123,6 +130,15 @@ int sd_attn_destroy(sd_attn_handle *h);
 
 /* Choose the kernel family for later forwards (default AUTO). */
 int sd_attn_set_mode(sd_attn_handle *h, int mode);
+
+/*
+ * Choose where the heads of q, k, v and out lie for later forwards (sd_attn_layout; default BHND).  All four
+ * tensors of a call share the layout; each is dense in it.  BNHD is implemented by the kernels AUTO selects
+ * (FUSED, CROSS and SIMT modes, either dtype); TWOPASS mode, and FUSED under the environment switches that select
+ * its earlier kernels, answer UNSUPPORTED for it.  sd_attn_forward_host takes either layout (BNHD in one slice).
+ * Errors: INVALID_VALUE (null handle, unknown layout).
+ */
+int sd_attn_set_layout(sd_attn_handle *h, int layout);
 
 /*
  * Scratch the TWOPASS mode needs for a call of this shape: the score matrix

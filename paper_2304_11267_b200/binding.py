@@ -19,6 +19,7 @@ F16, F32 = 0, 1
 MODE_AUTO, MODE_FUSED, MODE_CROSS, MODE_TWOPASS, MODE_SIMT = range(5)
 MODE_NAMES = {MODE_AUTO: "auto", MODE_FUSED: "fused", MODE_CROSS: "cross", MODE_TWOPASS: "twopass",
               MODE_SIMT: "simt"}
+LAYOUT_BHND, LAYOUT_BNHD = 0, 1   # sd_attn_layout: head-major [B,H,N,d] / token-major [B,N,H,d]
 CROSS_MAX_NK = 128
 MAX_D = 160
 STATIC_MAX_SCRATCH = 34 * 1024 * 1024   # SD_ATTN_STATIC_MAX_SCRATCH: built-in scratch of the no-allocation entry point
@@ -27,7 +28,7 @@ EXPORTS = ["sd_attn_create", "sd_attn_forward", "sd_attn_destroy", "sd_attn_set_
            "sd_attn_workspace_bytes", "sd_attn_set_workspace", "sd_attn_twopass_buffers",
            "sd_attn_query_status", "sd_attn_last_mode", "sd_attn_launch_count", "sd_attn_status_string",
            "sd_attn_forward_host", "sd_attn_host_staging_bytes", "sd_attn_debug_dump_cross_scores",
-           "sd_attn_forward_twopass_static", "sd_geglu_forward", "sd_groupnorm_forward"]
+           "sd_attn_forward_twopass_static", "sd_geglu_forward", "sd_groupnorm_forward", "sd_attn_set_layout"]
 
 _lib = None
 
@@ -61,6 +62,8 @@ def load() -> ctypes.CDLL:
     lib.sd_attn_destroy.argtypes = [vp]
     lib.sd_attn_set_mode.restype = ci
     lib.sd_attn_set_mode.argtypes = [vp, ci]
+    lib.sd_attn_set_layout.restype = ci
+    lib.sd_attn_set_layout.argtypes = [vp, ci]
     lib.sd_attn_workspace_bytes.restype = sz
     lib.sd_attn_workspace_bytes.argtypes = [ci, ci, ci, ci, ci, ci, ci]
     lib.sd_attn_set_workspace.restype = ci
@@ -195,6 +198,10 @@ def sd_attn_set_mode(handle, mode: int) -> int:
     return load().sd_attn_set_mode(handle, mode)
 
 
+def sd_attn_set_layout(handle, layout: int) -> int:
+    return load().sd_attn_set_layout(handle, layout)
+
+
 def sd_attn_workspace_bytes(mode, B, H, Nq, Nk, d, dtype) -> int:
     return int(load().sd_attn_workspace_bytes(mode, B, H, Nq, Nk, d, dtype))
 
@@ -234,11 +241,21 @@ def sd_attn_debug_dump_cross_scores(handle, ptr) -> int:
 class Attention:
     """A handle plus torch-tensor marshalling: ``Attention().forward(q, k, v)``."""
 
-    def __init__(self, mode: int = MODE_AUTO):
+    def __init__(self, mode: int = MODE_AUTO, layout: int = LAYOUT_BHND):
         self.handle = sd_attn_create()
         self._workspace = None
+        self.layout = LAYOUT_BHND
         if mode != MODE_AUTO:
             self.set_mode(mode)
+        if layout != LAYOUT_BHND:
+            self.set_layout(layout)
+
+    def set_layout(self, layout: int) -> None:
+        """LAYOUT_BHND: q [B,H,Nq,d]; LAYOUT_BNHD: q [B,Nq,H,d] (k, v, out alike)."""
+        rc = sd_attn_set_layout(self.handle, layout)
+        if rc != OK:
+            raise SdAttnError(rc, "sd_attn_set_layout")
+        self.layout = layout
 
     def set_mode(self, mode: int) -> None:
         rc = sd_attn_set_mode(self.handle, mode)
@@ -250,15 +267,19 @@ class Attention:
         if not (q.is_cuda and k.is_cuda and v.is_cuda):
             raise ValueError("q, k, v must be CUDA tensors")
         if not (q.is_contiguous() and k.is_contiguous() and v.is_contiguous()):
-            raise ValueError("q, k, v must be contiguous [B,H,N,d] tensors")
+            raise ValueError("q, k, v must be contiguous [B,H,N,d] (or, token-major, [B,N,H,d]) tensors")
         if q.dtype == torch.float16:
             dtype = F16
         elif q.dtype == torch.float32:
             dtype = F32
         else:
             raise TypeError("float16 or float32 only")
-        B, H, Nq, d = q.shape
-        Nk = k.shape[2]
+        if self.layout == LAYOUT_BNHD:
+            B, Nq, H, d = q.shape
+            Nk = k.shape[1]
+        else:
+            B, H, Nq, d = q.shape
+            Nk = k.shape[2]
         if out is None:
             out = torch.empty_like(q)
         if scale is None:

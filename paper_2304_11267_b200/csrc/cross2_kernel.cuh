@@ -50,7 +50,8 @@ constexpr float X2_SUM_LIMIT = 4096.0f;    // no weight above 2^12 reaches the b
 
 struct Cross2Args {
     const __half* q;    // [BH][Nq][d]: the four-group variant fetches Q tiles with untiled bulk copies
-    __half* out;        // [BH][Nq][d]
+    __half* out;        // [BH][Nq][d], or as `lay` says (the four-group variant: head-major only)
+    HeadLayout lay;
     int Nq, Nk, d;
     int dpad, nch;
     int stages;         // depth of the Q ring
@@ -215,6 +216,7 @@ cross2_attention_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid
             for (int i = 0; i < n_local; ++i) {
                 const int item = item0 + i, bh = item / args.tiles_per_bh, tile = item - bh * args.tiles_per_bh;
                 const int s = i % stages, g = bh - bh0;
+                const int bz = bh / args.lay.heads, hz = bh - bz * args.lay.heads;
                 if (g != g_prev) {
                     // a new head: its K and V go into buffer g & 1 once the head two back has been consumed
                     if (g >= 2 && !mbar_wait(smem_u32(&bar_kv_empty[g & 1]), ((g >> 1) - 1) & 1, abort_p, args.status,
@@ -223,9 +225,9 @@ cross2_attention_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid
                     const uint32_t bar = smem_u32(&bar_kv_full[g & 1]), dst = kv_smem + (g & 1) * 2 * kv_bytes;
                     mbar_arrive_expect_tx(bar, 2 * kv_bytes);
                     for (int ch = 0; ch < nch; ++ch)
-                        tma_load_3d(dst + ch * X2_KN * CHUNK_ROW_BYTES, &tmap_k, bar, ch * CHUNK_COLS, 0, bh);
+                        tma_load_4d(dst + ch * X2_KN * CHUNK_ROW_BYTES, &tmap_k, bar, ch * CHUNK_COLS, 0, hz, bz);
                     for (int ch = 0; ch < nch; ++ch)
-                        tma_load_3d(dst + kv_bytes + ch * X2_KN * CHUNK_ROW_BYTES, &tmap_v, bar, ch * CHUNK_COLS, 0, bh);
+                        tma_load_4d(dst + kv_bytes + ch * X2_KN * CHUNK_ROW_BYTES, &tmap_v, bar, ch * CHUNK_COLS, 0, hz, bz);
                     g_prev = g;
                 }
                 if (i >= stages &&
@@ -243,7 +245,7 @@ cross2_attention_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid
                 }
                 mbar_arrive_expect_tx(bar, q_bytes);
                 for (int ch = 0; ch < nch; ++ch)
-                    tma_load_3d(dst + ch * TILE_M * CHUNK_ROW_BYTES, &tmap_q, bar, ch * CHUNK_COLS, tile * TILE_M, bh);
+                    tma_load_4d(dst + ch * TILE_M * CHUNK_ROW_BYTES, &tmap_q, bar, ch * CHUNK_COLS, tile * TILE_M, hz, bz);
             }
         }
     } else if (warp == S_ISSUER_WARP || warp == S2_ISSUER_WARP || warp == O_ISSUER_WARP) {
@@ -270,11 +272,12 @@ cross2_attention_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid
                 // K and V of the CTA's first head, while the producer thread fetches the first Q tiles: a copy
                 // instruction holds its thread for several hundred clocks, and the first scores wait for all three.
                 const uint32_t bar = smem_u32(&bar_kv_full[0]);
+                const int bz0 = bh0 / args.lay.heads, hz0 = bh0 - bz0 * args.lay.heads;
                 mbar_arrive_expect_tx(bar, 2 * kv_bytes);
                 for (int ch = 0; ch < nch; ++ch)
-                    tma_load_3d(kv_smem + ch * X2_KN * CHUNK_ROW_BYTES, &tmap_k, bar, ch * CHUNK_COLS, 0, bh0);
+                    tma_load_4d(kv_smem + ch * X2_KN * CHUNK_ROW_BYTES, &tmap_k, bar, ch * CHUNK_COLS, 0, hz0, bz0);
                 for (int ch = 0; ch < nch; ++ch)
-                    tma_load_3d(kv_smem + kv_bytes + ch * X2_KN * CHUNK_ROW_BYTES, &tmap_v, bar, ch * CHUNK_COLS, 0, bh0);
+                    tma_load_4d(kv_smem + kv_bytes + ch * X2_KN * CHUNK_ROW_BYTES, &tmap_v, bar, ch * CHUNK_COLS, 0, hz0, bz0);
             }
             if (warp != O_ISSUER_WARP) {
                 const int parity = warp == S_ISSUER_WARP ? 0 : 1;
@@ -419,16 +422,16 @@ cross2_attention_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid
                 const bool over = !(row_sum <= X2_SUM_LIMIT);
                 if (attempt == 1 || !__any_sync(0xffffffffu, over)) break;
                 // rare: the row maximum lies far above the first score.  Nothing has been stored yet: take L_i of
-                // Eq. 4 (to bf16 precision: it only anchors the exponent) from the scores and redo the row.
+                // Eq. 4 from the scores and redo the row.
                 float row_max;
                 {
                     uint32_t s[32];
                     tmem_ld32(tmem_s, &s[0]);
                     tmem_wait_ld();
-                    row_max = row_max_bf16<32>(s);
+                    row_max = row_max_masked<32>(s, 32);
                     tmem_ld32(tmem_s + 32, &s[0]);
                     tmem_wait_ld();
-                    row_max = fmaxf(row_max, row_max_bf16<32>(s));
+                    row_max = fmaxf(row_max, row_max_masked<32>(s, 32));
                     tmem_ld16(tmem_s + 64, *reinterpret_cast<uint32_t(*)[16]>(&s[0]));
                     tmem_wait_ld();
                     row_max = fmaxf(row_max, row_max_masked<16>(s, valid - 64));
@@ -468,7 +471,7 @@ cross2_attention_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid
             if (tracer) X2_TRACE(w, i, 3);
             const float inv = inv_sum[w][n & 1][r];
             const int row = tile * TILE_M + r;
-            __half* orow = args.out + ((size_t)bh * args.Nq + row) * args.d;
+            __half* orow = head_row(args.out, args.lay, bh, row);
             if (DENSE_Q) {
                 // The tile is one contiguous piece of global memory: rows go to a dense staging tile in shared memory
                 // (thread = row) and ONE bulk copy writes it out -- full lines instead of five strided 16-byte stores

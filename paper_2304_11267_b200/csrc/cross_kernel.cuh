@@ -24,7 +24,8 @@ constexpr int CHUNK_COLS = 64;       // fp16 elements per 128-byte swizzled row
 constexpr int CHUNK_ROW_BYTES = 128;
 
 struct CrossArgs {
-    __half* out;        // [BH][Nq][d]
+    __half* out;        // [BH][Nq][d], or as `lay` says
+    HeadLayout lay;
     int Nq, Nk, d;
     int kn;             // Nk rounded up to a multiple of 16 (the MMA N of S, the K of P.V)
     int dpad;           // d rounded up to a multiple of 16 (the MMA N of O)
@@ -91,14 +92,15 @@ cross_attention_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_
     bool ok = true;
 
     if (tid == 0) {
+        const int bz = bh / args.lay.heads, hz = bh - bz * args.lay.heads;
         mbar_arrive_expect_tx(bar_qk, (uint32_t)(nch * (TILE_M + kn) * CHUNK_ROW_BYTES));
         for (int ch = 0; ch < nch; ++ch)
-            tma_load_3d(q_smem + ch * TILE_M * CHUNK_ROW_BYTES, &tmap_q, bar_qk, ch * CHUNK_COLS, row0, bh);
+            tma_load_4d(q_smem + ch * TILE_M * CHUNK_ROW_BYTES, &tmap_q, bar_qk, ch * CHUNK_COLS, row0, hz, bz);
         for (int ch = 0; ch < nch; ++ch)
-            tma_load_3d(k_smem + ch * kn * CHUNK_ROW_BYTES, &tmap_k, bar_qk, ch * CHUNK_COLS, 0, bh);
+            tma_load_4d(k_smem + ch * kn * CHUNK_ROW_BYTES, &tmap_k, bar_qk, ch * CHUNK_COLS, 0, hz, bz);
         mbar_arrive_expect_tx(bar_v, (uint32_t)(nch * kn * CHUNK_ROW_BYTES));
         for (int ch = 0; ch < nch; ++ch)
-            tma_load_3d(v_smem + ch * kn * CHUNK_ROW_BYTES, &tmap_v, bar_v, ch * CHUNK_COLS, 0, bh);
+            tma_load_4d(v_smem + ch * kn * CHUNK_ROW_BYTES, &tmap_v, bar_v, ch * CHUNK_COLS, 0, hz, bz);
 
         // S = Q K^T: contraction over d in steps of 16 columns (32 bytes inside a swizzled row)
         if (mbar_wait(bar_qk, 0, abort_p, args.status, SITE_X_LOAD_QK, tile)) {
@@ -181,7 +183,7 @@ cross_attention_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_
         tc_fence_after_sync();
         const float inv = 1.f / row_sum;
         const int row = row0 + tid;
-        __half* orow = args.out + ((size_t)bh * args.Nq + row) * args.d;
+        __half* orow = head_row(args.out, args.lay, bh, row);
         for (int g = 0; g < (dpad >> 4); ++g) {
             uint32_t r[16];
             tmem_ld16(tmem_o + lane_off + g * 16, r);

@@ -38,7 +38,8 @@ constexpr int F4_STAGES = 8;
 constexpr int F4_MAX_D = 64;
 
 struct Fused4Args {
-    __half* out;  // [BH][Nq][d]
+    __half* out;  // [BH][Nq][d], or as `lay` says (spare-buffer kernel only)
+    HeadLayout lay;
     int Nq, Nk, d;
     int dpad;     // d rounded up to 16 (<= 64)
     int tiles_per_cta;   // spare-buffer kernel only: 1..4 query tiles per CTA (small problems spread over more SMs)
@@ -126,7 +127,7 @@ fused4_attention_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid
             for (int t = 0; t < n_qtiles; ++t) {
                 const uint32_t bar = smem_u32(&bar_q_full[t]);
                 mbar_arrive_expect_tx(bar, q_tile_bytes);
-                tma_load_3d(q_smem + t * q_tile_bytes, &tmap_q, bar, 0, row_base + t * TILE_M, bh);
+                tma_load_4d(q_smem + t * q_tile_bytes, &tmap_q, bar, 0, row_base + t * TILE_M, bh, 0);
             }
             for (int j = 0; j < n_kv; ++j) {
                 const int s = j % F4_STAGES;
@@ -136,8 +137,8 @@ fused4_attention_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid
                 const uint32_t k_dst = kv_smem + s * 2 * kv_tile_bytes, v_dst = k_dst + kv_tile_bytes;
                 const uint32_t bar = smem_u32(&bar_kv_full[s]);
                 mbar_arrive_expect_tx(bar, 2 * kv_tile_bytes);
-                tma_load_3d(k_dst, &tmap_k, bar, 0, j * BN, bh);
-                tma_load_3d(v_dst, &tmap_v, bar, 0, j * BN, bh);
+                tma_load_4d(k_dst, &tmap_k, bar, 0, j * BN, bh, 0);
+                tma_load_4d(v_dst, &tmap_v, bar, 0, j * BN, bh, 0);
             }
         }
     } else if (warp > 16) {
@@ -257,7 +258,8 @@ fused4_attention_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid
                     tmem_ld32(tmem_s, &s[0]);
                     tmem_ld32(tmem_s + 32, &s[32]);
                     tmem_wait_ld();
-                    const float row_max = ragged ? row_max_masked<BN>(s, valid) : row_max_bf16<BN>(s);
+                    // (the exact maximum: the truncated one may lie below it by more than the headroom)
+                    const float row_max = row_max_masked<BN>(s, ragged ? valid : BN);
                     const float m_new = row_max * c2 + FUSED_HEADROOM_LOG2;
                     const float alpha = over ? ex2_approx(m_run - m_new) : 1.f;
                     if (over) m_run = m_new;

@@ -167,12 +167,13 @@ fused4s_attention_kernel(const __grid_constant__ CUtensorMap tmap_q, const __gri
         if (elect_one()) {
             // In the order the issuers need them: Q_0 and the first key tile first (a tile of 80-byte rows costs the
             // TMA unit about 7 clocks per row, so the order decides when the first scores can start).
+            const int bz = bh / args.lay.heads, hz = bh - bz * args.lay.heads;
             auto load_q = [&](int t) {
                 const uint32_t bar = smem_u32(&bar_q_full[t]);
                 mbar_arrive_expect_tx(bar, q_tile_bytes);
                 for (int ch = 0; ch < nch; ++ch)
-                    tma_load_3d(q_smem + t * q_tile_bytes + ch * TILE_M * CHUNK_ROW_BYTES, &tmap_q, bar, ch * CHUNK_COLS,
-                                row_base + t * TILE_M, bh);
+                    tma_load_4d(q_smem + t * q_tile_bytes + ch * TILE_M * CHUNK_ROW_BYTES, &tmap_q, bar, ch * CHUNK_COLS,
+                                row_base + t * TILE_M, hz, bz);
             };
             load_q(0);
             int s = 0, pe = 1;   // stage of key tile j; parity of the kv_empty phase that frees it (from j = stages on)
@@ -184,9 +185,9 @@ fused4s_attention_kernel(const __grid_constant__ CUtensorMap tmap_q, const __gri
                 const uint32_t bar = smem_u32(&bar_kv_full[s]);
                 mbar_arrive_expect_tx(bar, 2 * kv_tile_bytes);
                 for (int ch = 0; ch < nch; ++ch)
-                    tma_load_3d(k_dst + ch * BN * CHUNK_ROW_BYTES, &tmap_k, bar, ch * CHUNK_COLS, j * BN, bh);
+                    tma_load_4d(k_dst + ch * BN * CHUNK_ROW_BYTES, &tmap_k, bar, ch * CHUNK_COLS, j * BN, hz, bz);
                 for (int ch = 0; ch < nch; ++ch)
-                    tma_load_3d(v_dst + ch * BN * CHUNK_ROW_BYTES, &tmap_v, bar, ch * CHUNK_COLS, j * BN, bh);
+                    tma_load_4d(v_dst + ch * BN * CHUNK_ROW_BYTES, &tmap_v, bar, ch * CHUNK_COLS, j * BN, hz, bz);
                 if (j == 0)
                     for (int t = 1; t < T; ++t) load_q(t);
             }
@@ -396,7 +397,8 @@ fused4s_attention_kernel(const __grid_constant__ CUtensorMap tmap_q, const __gri
                             if (!ok) break;
                             tc_fence_after_sync();
                         }
-                        const float row_max = ragged ? row_max_masked<BN>(s, valid) : row_max_bf16<BN>(s);
+                        // (the exact maximum: the truncated one may lie below it by more than the headroom)
+                        const float row_max = row_max_masked<BN>(s, ragged ? valid : BN);
                         const float m_new = row_max * c2 + FUSED_HEADROOM_LOG2;
                         const float alpha = over ? ex2_approx(m_run - m_new) : 1.f;
                         if (over) m_run = m_new;
@@ -454,7 +456,7 @@ fused4s_attention_kernel(const __grid_constant__ CUtensorMap tmap_q, const __gri
 #pragma unroll
                     for (int p2 = 0; p2 < SPLIT; ++p2) f[p2] *= inv;
                     const int row = row_base + r;
-                    __half* orow = args.out + ((size_t)bh * args.Nq + row) * args.d;
+                    __half* orow = head_row(args.out, args.lay, bh, row);
                     // the column groups of 16 are shared out among the parts; a thread reads its row of every O_p
                     for (int cg = g; cg < (dpad >> 4); cg += SPLIT) {
                         float acc[16];
@@ -546,7 +548,8 @@ fused4s_attention_kernel(const __grid_constant__ CUtensorMap tmap_q, const __gri
                     tmem_ld32(tmem_s, &s[0]);
                     tmem_ld32(tmem_s + 32, &s[32]);
                     tmem_wait_ld();
-                    const float row_max = ragged ? row_max_masked<BN>(s, valid) : row_max_bf16<BN>(s);
+                    // (the exact maximum: the truncated one may lie below it by more than the headroom)
+                    const float row_max = row_max_masked<BN>(s, ragged ? valid : BN);
                     const float m_new = row_max * c2 + FUSED_HEADROOM_LOG2;
                     const float alpha = over ? ex2_approx(m_run - m_new) : 1.f;
                     if (over) m_run = m_new;
@@ -593,7 +596,7 @@ fused4s_attention_kernel(const __grid_constant__ CUtensorMap tmap_q, const __gri
                 tc_fence_after_sync();
                 const float inv = 1.f / l_run;
                 const int row = row_base + t * TILE_M + r;
-                __half* orow = args.out + ((size_t)bh * args.Nq + row) * args.d;
+                __half* orow = head_row(args.out, args.lay, bh, row);
                 for (int g = 0; g < (dpad >> 4); ++g) {
                     uint32_t x[16];
                     tmem_ld16(tmem_o + g * 16, x);

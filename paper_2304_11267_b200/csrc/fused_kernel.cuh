@@ -176,8 +176,8 @@ fused_attention_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_
                 const uint32_t bar = smem_u32(&bar_q_full[t]);
                 mbar_arrive_expect_tx(bar, q_tile_bytes);
                 for (int ch = 0; ch < nch; ++ch)
-                    tma_load_3d(q_smem + t * q_tile_bytes + ch * TILE_M * CHUNK_ROW_BYTES, &tmap_q, bar,
-                                ch * CHUNK_COLS, row_base + t * TILE_M, bh);
+                    tma_load_4d(q_smem + t * q_tile_bytes + ch * TILE_M * CHUNK_ROW_BYTES, &tmap_q, bar,
+                                ch * CHUNK_COLS, row_base + t * TILE_M, bh, 0);
             }
             for (int j = 0; j < n_kv; ++j) {
                 const int s = j % stages;
@@ -188,9 +188,9 @@ fused_attention_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_
                 const uint32_t bar = smem_u32(&bar_kv_full[s]);
                 mbar_arrive_expect_tx(bar, 2 * kv_tile_bytes);
                 for (int ch = 0; ch < nch; ++ch)
-                    tma_load_3d(k_dst + ch * BN * CHUNK_ROW_BYTES, &tmap_k, bar, ch * CHUNK_COLS, j * BN, bh);
+                    tma_load_4d(k_dst + ch * BN * CHUNK_ROW_BYTES, &tmap_k, bar, ch * CHUNK_COLS, j * BN, bh, 0);
                 for (int ch = 0; ch < nch; ++ch)
-                    tma_load_3d(v_dst + ch * BN * CHUNK_ROW_BYTES, &tmap_v, bar, ch * CHUNK_COLS, j * BN, bh);
+                    tma_load_4d(v_dst + ch * BN * CHUNK_ROW_BYTES, &tmap_v, bar, ch * CHUNK_COLS, j * BN, bh, 0);
             }
         }
     } else if (warp >= 9) {
@@ -296,7 +296,7 @@ fused_attention_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_
                 if (lane == 0) mbar_arrive(b_sfree);
                 if (tracer) FUSED_TRACE(t, j, 2);
                 const bool ragged = valid < BN;   // only the last key tile can be
-                const float row_max = ragged ? row_max_masked<BN>(s, valid) : row_max_bf16<BN>(s);
+                const float row_max = row_max_masked<BN>(s, ragged ? valid : BN);   // exact: it decides the anchor alone
                 const float row_max2 = row_max * c2;   // in log2 units, as the exponent sees it
                 if (j == 0) {
                     m_run = row_max2 + FUSED_HEADROOM_LOG2;

@@ -37,6 +37,7 @@ typedef CUresult (*encode_tiled_fn)(CUtensorMap*, CUtensorMapDataType, cuuint32_
 struct TmapCacheEntry {
     const void* base;
     int BH, N, d, box_rows;
+    int heads;   // heads per batch entry of a token-major tensor, 0 for a head-major one
     CUtensorMap map;
 };
 constexpr int TMAP_CACHE_ENTRIES = 128;
@@ -48,6 +49,7 @@ struct sd_attn_handle {
     int tmap_cache_next;
     int device;
     int mode;
+    int layout;
     int last_mode;
     long long launches;
     int* dev_status;          // DEV_STATUS_INTS ints on the device
@@ -265,6 +267,12 @@ extern "C" int sd_attn_set_mode(sd_attn_handle* h, int mode) {
     return SD_ATTN_OK;
 }
 
+extern "C" int sd_attn_set_layout(sd_attn_handle* h, int layout) {
+    if (!h || (layout != SD_ATTN_LAYOUT_BHND && layout != SD_ATTN_LAYOUT_BNHD)) return SD_ATTN_ERR_INVALID_VALUE;
+    h->layout = layout;
+    return SD_ATTN_OK;
+}
+
 extern "C" size_t sd_attn_workspace_bytes(int mode, int B, int H, int Nq, int Nk, int d, int dtype) {
     (void)d;
     (void)dtype;
@@ -315,23 +323,41 @@ extern "C" int sd_attn_query_status(sd_attn_handle* h, void* stream, int* detail
     return SD_ATTN_OK;
 }
 
-// A [BH][N][d] fp16 tensor seen by the TMA as (x = d, y = N, z = BH); tiles are 64 columns wide
-// (one 128-byte swizzled row) by `box_rows` rows.  Columns >= d and rows >= N read as zero.
-static int make_tmap(sd_attn_handle* h, CUtensorMap* map, const void* base, int BH, int N, int d, int box_rows) {
+// The heads of a call's tensors: `heads` per batch entry when the tensors are token-major, 0 when head-major.
+static HeadLayout head_layout(int heads, int BH, int N, int d) {
+    HeadLayout l;
+    if (heads > 0) {
+        l.heads = heads; l.ld = heads * d; l.head_stride = d; l.batch_stride = (long long)N * heads * d;
+    } else {
+        l.heads = BH; l.ld = d; l.head_stride = (long long)N * d; l.batch_stride = (long long)BH * N * d;
+    }
+    return l;
+}
+
+static CUresult encode_tmap(encode_tiled_fn enc, CUtensorMap* map, const void* base, int heads, int BH, int N, int d,
+                            int box_rows) {
+    const HeadLayout l = head_layout(heads, BH, N, d);
+    cuuint64_t dims[4] = {(cuuint64_t)d, (cuuint64_t)N, (cuuint64_t)l.heads, (cuuint64_t)(BH / l.heads)};
+    cuuint64_t strides[3] = {(cuuint64_t)l.ld * 2, (cuuint64_t)l.head_stride * 2, (cuuint64_t)l.batch_stride * 2};
+    cuuint32_t box[4] = {(cuuint32_t)CHUNK_COLS, (cuuint32_t)box_rows, 1, 1};
+    cuuint32_t estr[4] = {1, 1, 1, 1};
+    return enc(map, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 4, const_cast<void*>(base), dims, strides, box, estr,
+               CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+}
+
+// An fp16 tensor of BH heads of N rows of d values seen by the TMA as (x = d, y = N, z = head, w = batch): tiles are
+// 64 columns wide (one 128-byte swizzled row) by `box_rows` rows.  Columns >= d and rows >= N read as zero.
+static int make_tmap(sd_attn_handle* h, CUtensorMap* map, const void* base, int BH, int N, int d, int box_rows,
+                     int heads = 0) {
     for (int i = 0; i < TMAP_CACHE_ENTRIES; ++i) {
         const TmapCacheEntry& e = h->tmap_cache[i];
-        if (e.base == base && e.BH == BH && e.N == N && e.d == d && e.box_rows == box_rows) {
+        if (e.base == base && e.BH == BH && e.N == N && e.d == d && e.box_rows == box_rows && e.heads == heads) {
             *map = e.map;
             return SD_ATTN_OK;
         }
     }
-    cuuint64_t dims[3] = {(cuuint64_t)d, (cuuint64_t)N, (cuuint64_t)BH};
-    cuuint64_t strides[2] = {(cuuint64_t)d * 2, (cuuint64_t)N * d * 2};
-    cuuint32_t box[3] = {(cuuint32_t)CHUNK_COLS, (cuuint32_t)box_rows, 1};
-    cuuint32_t estr[3] = {1, 1, 1};
-    CUresult r = h->encode_tiled(map, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 3, const_cast<void*>(base), dims, strides, box,
-                                 estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
-                                 CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    CUresult r = encode_tmap(h->encode_tiled, map, base, heads, BH, N, d, box_rows);
     if (r != CUDA_SUCCESS) {
         if (getenv("SD_ATTN_LOG")) fprintf(stderr, "[sd_attn] cuTensorMapEncodeTiled failed: %d\n", (int)r);
         h->last_cuda_error = cudaErrorInvalidValue;
@@ -339,7 +365,7 @@ static int make_tmap(sd_attn_handle* h, CUtensorMap* map, const void* base, int 
     }
     TmapCacheEntry& slot = h->tmap_cache[h->tmap_cache_next];
     h->tmap_cache_next = (h->tmap_cache_next + 1) % TMAP_CACHE_ENTRIES;
-    slot.base = base; slot.BH = BH; slot.N = N; slot.d = d; slot.box_rows = box_rows;
+    slot.base = base; slot.BH = BH; slot.N = N; slot.d = d; slot.box_rows = box_rows; slot.heads = heads;
     slot.map = *map;
     return SD_ATTN_OK;
 }
@@ -356,6 +382,7 @@ struct Problem {
     int BH, Nq, Nk, d;
     float scale;
     cudaStream_t stream;
+    int heads;   // token-major tensors: heads per batch entry; head-major: 0
 };
 
 template <typename T>
@@ -364,12 +391,13 @@ static int launch_simt(sd_attn_handle* h, const Problem& p) {
     const size_t smem = simt_smem_bytes(p.d);
     const T *q = (const T*)p.q, *k = (const T*)p.k, *v = (const T*)p.v;
     T* o = (T*)p.out;
+    const HeadLayout lq = head_layout(p.heads, p.BH, p.Nq, p.d), lk = head_layout(p.heads, p.BH, p.Nk, p.d);
     switch ((p.d + 31) / 32) {
-        case 1: simt_attention_kernel<T, 1><<<grid, block, smem, p.stream>>>(q, k, v, o, p.Nq, p.Nk, p.d, p.scale); break;
-        case 2: simt_attention_kernel<T, 2><<<grid, block, smem, p.stream>>>(q, k, v, o, p.Nq, p.Nk, p.d, p.scale); break;
-        case 3: simt_attention_kernel<T, 3><<<grid, block, smem, p.stream>>>(q, k, v, o, p.Nq, p.Nk, p.d, p.scale); break;
-        case 4: simt_attention_kernel<T, 4><<<grid, block, smem, p.stream>>>(q, k, v, o, p.Nq, p.Nk, p.d, p.scale); break;
-        default: simt_attention_kernel<T, 5><<<grid, block, smem, p.stream>>>(q, k, v, o, p.Nq, p.Nk, p.d, p.scale); break;
+        case 1: simt_attention_kernel<T, 1><<<grid, block, smem, p.stream>>>(q, k, v, o, p.Nq, p.Nk, p.d, p.scale, lq, lk); break;
+        case 2: simt_attention_kernel<T, 2><<<grid, block, smem, p.stream>>>(q, k, v, o, p.Nq, p.Nk, p.d, p.scale, lq, lk); break;
+        case 3: simt_attention_kernel<T, 3><<<grid, block, smem, p.stream>>>(q, k, v, o, p.Nq, p.Nk, p.d, p.scale, lq, lk); break;
+        case 4: simt_attention_kernel<T, 4><<<grid, block, smem, p.stream>>>(q, k, v, o, p.Nq, p.Nk, p.d, p.scale, lq, lk); break;
+        default: simt_attention_kernel<T, 5><<<grid, block, smem, p.stream>>>(q, k, v, o, p.Nq, p.Nk, p.d, p.scale, lq, lk); break;
     }
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) return cuda_fail(h, e);
@@ -382,6 +410,7 @@ static int launch_cross2(sd_attn_handle* h, const Problem& p) {
     Cross2Args a;
     a.q = (const __half*)p.q;
     a.out = (__half*)p.out;
+    a.lay = head_layout(p.heads, p.BH, p.Nq, p.d);
     a.Nq = p.Nq; a.Nk = p.Nk; a.d = p.d;
     a.dpad = (p.d + 15) / 16 * 16;
     a.nch = (p.d + CHUNK_COLS - 1) / CHUNK_COLS;
@@ -395,13 +424,14 @@ static int launch_cross2(sd_attn_handle* h, const Problem& p) {
     a.trace = (long long*)h->trace;
 #endif
     CUtensorMap tq, tk, tv;
-    int rc = make_tmap(h, &tq, p.q, p.BH, p.Nq, p.d, TILE_M);
-    if (rc == SD_ATTN_OK) rc = make_tmap(h, &tk, p.k, p.BH, p.Nk, p.d, X2_KN);
-    if (rc == SD_ATTN_OK) rc = make_tmap(h, &tv, p.v, p.BH, p.Nk, p.d, X2_KN);
+    int rc = make_tmap(h, &tq, p.q, p.BH, p.Nq, p.d, TILE_M, p.heads);
+    if (rc == SD_ATTN_OK) rc = make_tmap(h, &tk, p.k, p.BH, p.Nk, p.d, X2_KN, p.heads);
+    if (rc == SD_ATTN_OK) rc = make_tmap(h, &tv, p.v, p.BH, p.Nk, p.d, X2_KN, p.heads);
     if (rc != SD_ATTN_OK) return rc;
     const int grid = a.n_items < h->sm_count ? a.n_items : h->sm_count;
     int groups = cross2_groups(p.d);
-    if (groups >= 4 && !h->cross2_four_ok) groups = 3;
+    // (the four-group variant moves whole Q and output tiles as contiguous runs of memory: head-major tensors only)
+    if (groups >= 4 && (!h->cross2_four_ok || p.heads > 0)) groups = 3;
     size_t smem = cross2_smem_bytes(a.nch);
     if (groups >= 4) {   // d <= 48: Q tiles arrive as raw bulk copies and are rewritten in shared memory
         a.stages = cross2_dense_stages(p.d);
@@ -423,6 +453,7 @@ static int launch_cross(sd_attn_handle* h, const Problem& p) {
     if (cross2_supports(p.Nk, p.d) && !h->cross_one_tile_only && !h->dump_scores) return launch_cross2(h, p);
     CrossArgs a;
     a.out = (__half*)p.out;
+    a.lay = head_layout(p.heads, p.BH, p.Nq, p.d);
     a.Nq = p.Nq; a.Nk = p.Nk; a.d = p.d;
     a.kn = (p.Nk + 15) / 16 * 16;
     a.dpad = (p.d + 15) / 16 * 16;
@@ -433,9 +464,9 @@ static int launch_cross(sd_attn_handle* h, const Problem& p) {
     a.status = h->dev_status;
     a.dump_scores = h->dump_scores;
     CUtensorMap tq, tk, tv;
-    int rc = make_tmap(h, &tq, p.q, p.BH, p.Nq, p.d, TILE_M);
-    if (rc == SD_ATTN_OK) rc = make_tmap(h, &tk, p.k, p.BH, p.Nk, p.d, a.kn);
-    if (rc == SD_ATTN_OK) rc = make_tmap(h, &tv, p.v, p.BH, p.Nk, p.d, a.kn);
+    int rc = make_tmap(h, &tq, p.q, p.BH, p.Nq, p.d, TILE_M, p.heads);
+    if (rc == SD_ATTN_OK) rc = make_tmap(h, &tk, p.k, p.BH, p.Nk, p.d, a.kn, p.heads);
+    if (rc == SD_ATTN_OK) rc = make_tmap(h, &tv, p.v, p.BH, p.Nk, p.d, a.kn, p.heads);
     if (rc != SD_ATTN_OK) return rc;
     dim3 grid((p.Nq + TILE_M - 1) / TILE_M, p.BH), block(CROSS_THREADS);
     launch_overlapped(h, cross_attention_kernel, grid, block, cross_smem_bytes(a.nch, a.kn), p.stream, tq, tk, tv, a);
@@ -449,6 +480,7 @@ static int launch_cross(sd_attn_handle* h, const Problem& p) {
 static int launch_fused4(sd_attn_handle* h, const Problem& p) {
     Fused4Args a;
     a.out = (__half*)p.out;
+    a.lay = head_layout(0, p.BH, p.Nq, p.d);
     a.Nq = p.Nq; a.Nk = p.Nk; a.d = p.d;
     a.dpad = (p.d + 15) / 16 * 16;
     a.scale_log2e = fabsf(p.scale) * LOG2E;
@@ -477,6 +509,7 @@ static int launch_fused4(sd_attn_handle* h, const Problem& p) {
 static int launch_fused4s(sd_attn_handle* h, const Problem& p) {
     Fused4Args a;
     a.out = (__half*)p.out;
+    a.lay = head_layout(p.heads, p.BH, p.Nq, p.d);
     a.Nq = p.Nq; a.Nk = p.Nk; a.d = p.d;
     a.dpad = (p.d + 15) / 16 * 16;
     a.nch = (p.d + CHUNK_COLS - 1) / CHUNK_COLS;
@@ -511,9 +544,9 @@ static int launch_fused4s(sd_attn_handle* h, const Problem& p) {
     if (a.stages > F4_STAGES) a.stages = F4_STAGES;
     const size_t smem = (size_t)tile_slots * q_tile_bytes + (size_t)a.stages * stage_bytes + 1024;
     CUtensorMap tq, tk, tv;
-    int rc = make_tmap(h, &tq, p.q, p.BH, p.Nq, p.d, TILE_M);
-    if (rc == SD_ATTN_OK) rc = make_tmap(h, &tk, p.k, p.BH, p.Nk, p.d, F4_BN);
-    if (rc == SD_ATTN_OK) rc = make_tmap(h, &tv, p.v, p.BH, p.Nk, p.d, F4_BN);
+    int rc = make_tmap(h, &tq, p.q, p.BH, p.Nq, p.d, TILE_M, p.heads);
+    if (rc == SD_ATTN_OK) rc = make_tmap(h, &tk, p.k, p.BH, p.Nk, p.d, F4_BN, p.heads);
+    if (rc == SD_ATTN_OK) rc = make_tmap(h, &tv, p.v, p.BH, p.Nk, p.d, F4_BN, p.heads);
     if (rc != SD_ATTN_OK) return rc;
     dim3 grid((tiles_per_head + a.tiles_per_cta - 1) / a.tiles_per_cta, p.BH), block(F4_THREADS);
     // One tile per CTA: its key tiles are dealt out among 4 or 2 warpgroups (parts), each with an accumulator of its
@@ -552,6 +585,7 @@ static int launch_fused4s(sd_attn_handle* h, const Problem& p) {
 
 static int launch_fused(sd_attn_handle* h, const Problem& p) {
     if (h->fused4s_ok && !h->no_spare && !h->prefer_two_tile) return launch_fused4s(h, p);
+    if (p.heads > 0) return SD_ATTN_ERR_UNSUPPORTED;   // the earlier kernels take head-major tensors only
     if (p.d <= F4_MAX_D && !h->prefer_two_tile && h->fused4_ok) return launch_fused4(h, p);
     FusedArgs a;
     const int bn = fused_block_n(p.d);
@@ -580,6 +614,7 @@ static int launch_fused(sd_attn_handle* h, const Problem& p) {
 }
 
 static int launch_twopass(sd_attn_handle* h, const Problem& p) {
+    if (p.heads > 0) return SD_ATTN_ERR_UNSUPPORTED;   // the comparator takes head-major tensors only
     const size_t need = sd_attn_workspace_bytes(SD_ATTN_MODE_TWOPASS, p.BH, 1, p.Nq, p.Nk, p.d, SD_ATTN_F16);
     if (!h->workspace || h->workspace_bytes < need) return SD_ATTN_ERR_WORKSPACE;
     const size_t rows = (size_t)p.BH * p.Nq;
@@ -628,7 +663,8 @@ extern "C" int sd_attn_forward(sd_attn_handle* h, const void* q, const void* k, 
     if (mode != SD_ATTN_MODE_SIMT && !tensor_ok) return SD_ATTN_ERR_UNSUPPORTED;
     if (mode == SD_ATTN_MODE_CROSS && Nk > SD_ATTN_CROSS_MAX_NK) return SD_ATTN_ERR_UNSUPPORTED;
 
-    Problem p = {q, k, v, out, B * H, Nq, Nk, d, scale, (cudaStream_t)stream};
+    Problem p = {q, k, v, out, B * H, Nq, Nk, d, scale, (cudaStream_t)stream,
+                 h->layout == SD_ATTN_LAYOUT_BNHD ? H : 0};
     int rc;
     switch (mode) {
         case SD_ATTN_MODE_SIMT:
@@ -678,7 +714,7 @@ extern "C" int sd_attn_forward_host(sd_attn_handle* h, const void* q, const void
     // pointers sd_attn_twopass_buffers returns describe one whole call.)
     const int BH = B * H;
     const size_t q_head = (size_t)Nq * d * es, k_head = (size_t)Nk * d * es;
-    const bool sliceable = h->host_overlap && h->mode != SD_ATTN_MODE_TWOPASS &&
+    const bool sliceable = h->host_overlap && h->mode != SD_ATTN_MODE_TWOPASS && h->layout == SD_ATTN_LAYOUT_BHND &&
                            q_head % 16 == 0 && k_head % 16 == 0;   // every slice starts 16-byte aligned
     const int slices = sliceable ? (BH < HOST_SLICES ? BH : HOST_SLICES) : 1;
     if (slices > 1) {
@@ -781,14 +817,7 @@ static int static_setup(int dev, StaticDeviceState** out) {
 }
 
 static int static_tmap(encode_tiled_fn enc, CUtensorMap* map, const void* base, int BH, int N, int d, int box_rows) {
-    cuuint64_t dims[3] = {(cuuint64_t)d, (cuuint64_t)N, (cuuint64_t)BH};
-    cuuint64_t strides[2] = {(cuuint64_t)d * 2, (cuuint64_t)N * d * 2};
-    cuuint32_t box[3] = {(cuuint32_t)CHUNK_COLS, (cuuint32_t)box_rows, 1};
-    cuuint32_t estr[3] = {1, 1, 1};
-    CUresult r = enc(map, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 3, const_cast<void*>(base), dims, strides, box, estr,
-                     CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
-                     CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
-    return r == CUDA_SUCCESS ? SD_ATTN_OK : SD_ATTN_ERR_CUDA;
+    return encode_tmap(enc, map, base, 0, BH, N, d, box_rows) == CUDA_SUCCESS ? SD_ATTN_OK : SD_ATTN_ERR_CUDA;
 }
 
 extern "C" int sd_attn_forward_twopass_static(const void* q, const void* k, const void* v, void* out, int B, int H,

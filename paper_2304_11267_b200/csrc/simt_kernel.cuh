@@ -12,6 +12,8 @@
 #include <cuda_fp16.h>
 #include <cuda_runtime.h>
 
+#include "tc_common.cuh"
+
 namespace sd_attn {
 
 constexpr int SIMT_ROWS_PER_WARP = 4;
@@ -35,7 +37,7 @@ __device__ inline void from_f32(__half* p, float x) { *p = __float2half_rn(x); }
 template <typename T, int CC>  // CC = ceil(d / 32) output channels per lane
 __global__ void __launch_bounds__(SIMT_WARPS * 32)
 simt_attention_kernel(const T* __restrict__ q, const T* __restrict__ k, const T* __restrict__ v,
-                      T* __restrict__ out, int Nq, int Nk, int d, float scale) {
+                      T* __restrict__ out, int Nq, int Nk, int d, float scale, HeadLayout lq, HeadLayout lk) {
     extern __shared__ __align__(16) float simt_smem[];
     const int ks = simt_k_stride(d);
     const int vs = 32 * CC;
@@ -44,15 +46,16 @@ simt_attention_kernel(const T* __restrict__ q, const T* __restrict__ k, const T*
     float* Vs = Ks + SIMT_CHUNK * ks;             // [32][vs]
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    const long long bh = blockIdx.y;
+    const int bh = blockIdx.y;   // lq places the heads of q and out (Nq rows each), lk those of k and v (Nk rows)
     const int row0 = blockIdx.x * SIMT_BLOCK_ROWS;
-    const T* qb = q + (bh * Nq + row0) * (long long)d;
-    const T* kb = k + bh * (long long)Nk * d;
-    const T* vb = v + bh * (long long)Nk * d;
+    const T* qb = head_row(q, lq, bh, row0);
+    const T* kb = head_row(k, lk, bh, 0);
+    const T* vb = head_row(v, lk, bh, 0);
+    const long long ldq = lq.ld, ldk = lk.ld;
 
     for (int idx = tid; idx < SIMT_BLOCK_ROWS * ks; idx += blockDim.x) {
         const int r = idx / ks, c = idx - r * ks;
-        Qs[idx] = (c < d && row0 + r < Nq) ? to_f32(qb[(long long)r * d + c]) : 0.f;
+        Qs[idx] = (c < d && row0 + r < Nq) ? to_f32(qb[r * ldq + c]) : 0.f;
     }
 
     float m[SIMT_ROWS_PER_WARP], l[SIMT_ROWS_PER_WARP], o[SIMT_ROWS_PER_WARP][CC];
@@ -68,11 +71,11 @@ simt_attention_kernel(const T* __restrict__ q, const T* __restrict__ k, const T*
         __syncthreads();  // previous chunk fully consumed (and Qs written, first time round)
         for (int idx = tid; idx < SIMT_CHUNK * ks; idx += blockDim.x) {
             const int r = idx / ks, c = idx - r * ks;
-            Ks[idx] = (c < d && j0 + r < Nk) ? to_f32(kb[(long long)(j0 + r) * d + c]) : 0.f;
+            Ks[idx] = (c < d && j0 + r < Nk) ? to_f32(kb[(j0 + r) * ldk + c]) : 0.f;
         }
         for (int idx = tid; idx < SIMT_CHUNK * vs; idx += blockDim.x) {
             const int r = idx / vs, c = idx - r * vs;
-            Vs[idx] = (c < d && j0 + r < Nk) ? to_f32(vb[(long long)(j0 + r) * d + c]) : 0.f;
+            Vs[idx] = (c < d && j0 + r < Nk) ? to_f32(vb[(j0 + r) * ldk + c]) : 0.f;
         }
         __syncthreads();
 
@@ -131,7 +134,7 @@ simt_attention_kernel(const T* __restrict__ q, const T* __restrict__ k, const T*
         for (int sft = 16; sft > 0; sft >>= 1) s += __shfl_xor_sync(0xffffffffu, s, sft);
         const int row = row0 + warp * SIMT_ROWS_PER_WARP + r;
         if (row < Nq) {
-            T* orow = out + (bh * Nq + row) * (long long)d;
+            T* orow = head_row(out, lq, bh, row);
 #pragma unroll
             for (int cc = 0; cc < CC; ++cc) {
                 const int c = cc * 32 + lane;

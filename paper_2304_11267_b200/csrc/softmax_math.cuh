@@ -79,17 +79,35 @@ __device__ __forceinline__ uint64_t sub_f32x2(uint64_t a, uint64_t b) {
 }
 __host__ __device__ constexpr uint64_t dup_f32(uint32_t bits) { return ((uint64_t)bits << 32) | bits; }
 
-// 2^x for a PAIR of values on the FMA pipe (see ex2_poly in tc_common.cuh for the method): the
+__device__ __forceinline__ uint64_t fma_rm_f32x2(uint64_t a, uint64_t b, uint64_t c) {   // round toward -inf
+    uint64_t d;
+    asm("fma.rm.f32x2 %0, %1, %2, %3;" : "=l"(d) : "l"(a), "l"(b), "l"(c));
+    return d;
+}
+__device__ __forceinline__ float fma_sat(float a, float b, float c) {   // a * b + c clamped to [0, 1]
+    float d;
+    asm("fma.rn.sat.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(a), "f"(b), "f"(c));
+    return d;
+}
+
+// 2^(s*c2 + nm) for a PAIR of scores on the FMA pipe (see ex2_poly in tc_common.cuh for the method): the
 // special-function unit is the bound of the d = 40 kernel, so a share of the pairs goes this way.
-__device__ __forceinline__ void ex2_poly_pair(uint64_t x, float& p0, float& p1) {
-    constexpr uint64_t MAGIC = dup_f32(0x4B400000u);   // 1.5 * 2^23
+// The argument x = s*c2 + nm is clamped to [-126, 128] at both ends -- below, the exponent field would wrap; above,
+// the result must come out huge or non-finite (a score far above a stale anchor: the caller's sum test then
+// re-anchors the row), not wrap into garbage.  Both clamps and the scaling of the score are ONE saturating
+// multiply-add per value: y = sat(s * (c2/254) + (nm + 126)/254) in [0, 1], and the rest works on
+// x' = 254 y - 126 without ever forming it.  (x' differs from x by 1e-5 + 1e-7 |nm| at most: below the
+// polynomial's error for every anchor a finite softmax of binary16 data can have.)
+__device__ __forceinline__ void ex2_poly_pair(uint32_t s0, uint32_t s1, float c2_254, float nm_254, float& p0,
+                                              float& p1) {
+    constexpr uint64_t MAGIC_LO = dup_f32(0x4B3FFF82u);   // 1.5 * 2^23 - 126
+    constexpr uint64_t WIDTH = dup_f32(0x437E0000u);      // 254
     constexpr uint64_t C3 = dup_f32(0x3D9FCB52u), C2 = dup_f32(0x3E677E26u);   // 0.07802452, 0.22606716
     constexpr uint64_t C1 = dup_f32(0x3F322226u), C0 = dup_f32(0x3F7FFB19u);   // 0.69583356, 0.9999252
-    uint32_t x0, x1;
-    unpack_b64(x, x0, x1);
-    x = pack_b64(__float_as_uint(fmaxf(__uint_as_float(x0), -126.f)), __float_as_uint(fmaxf(__uint_as_float(x1), -126.f)));
-    const uint64_t t = add_rm_f32x2(x, MAGIC);           // low mantissa bits = floor(x)
-    const uint64_t f = sub_f32x2(x, sub_f32x2(t, MAGIC));   // x - floor(x), in [0, 1)
+    const uint64_t y = pack_b64(__float_as_uint(fma_sat(__uint_as_float(s0), c2_254, nm_254)),
+                                __float_as_uint(fma_sat(__uint_as_float(s1), c2_254, nm_254)));
+    const uint64_t t = fma_rm_f32x2(y, WIDTH, MAGIC_LO);              // low mantissa bits = floor(x')
+    const uint64_t f = fma_f32x2(y, WIDTH, sub_f32x2(MAGIC_LO, t));   // x' - floor(x'), in [0, 1]
     uint64_t p = fma_f32x2(f, C3, C2);
     p = fma_f32x2(p, f, C1);
     p = fma_f32x2(p, f, C0);
@@ -114,13 +132,16 @@ __device__ __forceinline__ constexpr bool pair_uses_poly(int k) {
 template <int POLY, int PAIRS = 16>
 __device__ __forceinline__ void exp2_pack_32(const uint32_t* s, uint64_t c2c2, uint64_t nmnm, uint32_t* packed,
                                              uint64_t* acc) {
+    // the polynomial's pairs take the score itself, with the constants of the clamped form (see ex2_poly_pair)
+    const float c2_254 = __uint_as_float((uint32_t)c2c2) * (1.f / 254.f);
+    const float nm_254 = fmaf(__uint_as_float((uint32_t)nmnm), 1.f / 254.f, 126.f / 254.f);
 #pragma unroll
     for (int k = 0; k < PAIRS; ++k) {
-        const uint64_t x = fma_f32x2(pack_b64(s[2 * k], s[2 * k + 1]), c2c2, nmnm);
         float p0, p1;
         if (pair_uses_poly<POLY>(k)) {
-            ex2_poly_pair(x, p0, p1);
+            ex2_poly_pair(s[2 * k], s[2 * k + 1], c2_254, nm_254, p0, p1);
         } else {
+            const uint64_t x = fma_f32x2(pack_b64(s[2 * k], s[2 * k + 1]), c2c2, nmnm);
             uint32_t x0, x1;
             unpack_b64(x, x0, x1);
             p0 = ex2_approx(__uint_as_float(x0));

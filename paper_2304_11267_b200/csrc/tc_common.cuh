@@ -153,6 +153,31 @@ __device__ __forceinline__ void tma_load_3d(uint32_t dst, const void* tmap, uint
         "l"(reinterpret_cast<uint64_t>(tmap)), "r"(bar), "r"(x), "r"(y), "r"(z)
         : "memory");
 }
+// Where the heads of a tensor lie.  A (batch, head) index bh splits into batch = bh / heads and head = bh % heads;
+// row r of that head starts batch * batch_stride + head * head_stride + r * ld elements into the tensor.
+// Head-major [B][H][N][d] is {heads = B*H, ld = d, head_stride = N*d} (the batch index is always 0); token-major
+// [B][N][H][d] -- the layout a projection to H*d channels leaves, so that the head split and merge around the
+// attention cost no copy -- is {heads = H, ld = H*d, head_stride = d, batch_stride = N*H*d}.
+struct HeadLayout {
+    int heads;
+    int ld;
+    long long head_stride;
+    long long batch_stride;
+};
+template <typename T>
+__device__ __forceinline__ T* head_row(T* base, const HeadLayout& lay, int bh, int row) {
+    const int batch = bh / lay.heads, head = bh - batch * lay.heads;
+    return base + batch * lay.batch_stride + head * lay.head_stride + (long long)row * lay.ld;
+}
+// 4-D tile load global -> shared: (x = innermost element, y = row, z = head, w = batch); x as for the 3-D load.
+__device__ __forceinline__ void tma_load_4d(uint32_t dst, const void* tmap, uint32_t bar, int x, int y, int z,
+                                            int w) {
+    asm volatile(
+        "cp.async.bulk.tensor.4d.shared::cluster.global.mbarrier::complete_tx::bytes"
+        " [%0], [%1, {%3, %4, %5, %6}], [%2];" ::"r"(dst),
+        "l"(reinterpret_cast<uint64_t>(tmap)), "r"(bar), "r"(x), "r"(y), "r"(z), "r"(w)
+        : "memory");
+}
 // Untiled bulk copy global -> shared, completion counted in bytes on `bar`.  Both addresses 16-byte aligned, the
 // size a multiple of 16 bytes.
 __device__ __forceinline__ void bulk_load(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar) {
@@ -342,9 +367,9 @@ __device__ __forceinline__ float ex2_approx(float x) {
 // clock per SM, so a share of them is computed here instead.  x = n + f with n = floor(x) taken from
 // the low mantissa bits of (x + 1.5*2^23) rounded down, 2^f by a degree-3 polynomial fitted to
 // [0, 1) (max relative error 7.5e-5, below the fp16 rounding of the weights), and n added into
-// the exponent field.  Inputs below -127 are clamped (the result is then a denormal ~ 0).
+// the exponent field.  Inputs are clamped to [-127, 127] (the exponent field would wrap outside).
 __device__ __forceinline__ float ex2_poly(float x) {
-    x = fmaxf(x, -127.f);
+    x = fminf(fmaxf(x, -127.f), 127.f);
     const float t = __fadd_rd(x, 12582912.f);
     const float f = x - (t - 12582912.f);
     float p = fmaf(f, 0.07802452f, 0.22606716f);

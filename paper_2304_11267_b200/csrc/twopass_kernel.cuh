@@ -107,8 +107,8 @@ twopass_scores_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_c
         const uint32_t bar = smem_u32(&bar_k[s]);
         mbar_arrive_expect_tx(bar, k_tile_bytes);
         for (int ch = 0; ch < nch; ++ch)
-            tma_load_3d(k_smem + s * k_tile_bytes + ch * TWOPASS_BN * CHUNK_ROW_BYTES, &tmap_k, bar, ch * CHUNK_COLS,
-                        j * TWOPASS_BN, bh);
+            tma_load_4d(k_smem + s * k_tile_bytes + ch * TWOPASS_BN * CHUNK_ROW_BYTES, &tmap_k, bar, ch * CHUNK_COLS,
+                        j * TWOPASS_BN, bh, 0);
     };
     auto issue_s = [&](int j) {   // S_(j&1) = Q K_j^T
         const int s = j & 1;
@@ -127,7 +127,7 @@ twopass_scores_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_c
         const uint32_t bq = smem_u32(&bar_q);
         mbar_arrive_expect_tx(bq, nch * TILE_M * CHUNK_ROW_BYTES);
         for (int ch = 0; ch < nch; ++ch)
-            tma_load_3d(q_smem + ch * TILE_M * CHUNK_ROW_BYTES, &tmap_q, bq, ch * CHUNK_COLS, row0, bh);
+            tma_load_4d(q_smem + ch * TILE_M * CHUNK_ROW_BYTES, &tmap_q, bq, ch * CHUNK_COLS, row0, bh, 0);
         load_k(0);
         if (n_kv > 1) load_k(1);
         ok = mbar_wait(bq, 0, abort_p, args.status, SITE_T_Q, tile) &&
@@ -289,8 +289,8 @@ twopass_pv_kernel(const __grid_constant__ CUtensorMap tmap_v, const TwoPassArgs 
         const uint32_t bar = smem_u32(&bar_v[s]);
         mbar_arrive_expect_tx(bar, v_tile_bytes);
         for (int ch = 0; ch < nch; ++ch)
-            tma_load_3d(v_smem + s * v_tile_bytes + ch * TWOPASS_BN * CHUNK_ROW_BYTES, &tmap_v, bar, ch * CHUNK_COLS,
-                        j * TWOPASS_BN, bh);
+            tma_load_4d(v_smem + s * v_tile_bytes + ch * TWOPASS_BN * CHUNK_ROW_BYTES, &tmap_v, bar, ch * CHUNK_COLS,
+                        j * TWOPASS_BN, bh, 0);
     };
     if (tid == 0) {
         tma_prefetch_desc(&tmap_v);

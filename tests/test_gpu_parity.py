@@ -635,3 +635,24 @@ def test_twopass_score_matrix_and_row_statistics(att, bd):
     np.testing.assert_allclose(A, a_ref, rtol=0, atol=1e-5 * np.abs(a_ref).max())
     np.testing.assert_allclose(LS[..., 0], L, rtol=0, atol=1e-5 * np.abs(L).max())   # L: exact to fp32 rounding
     np.testing.assert_allclose(LS[..., 1], S, rtol=1e-5)                              # S of Eq. 4
+
+
+# ------------------------------------------------------------------ scores of large magnitude
+
+@pytest.mark.parametrize("Nq,Nk,d", [(256, 256, 40), (1024, 1024, 40), (640, 640, 80), (256, 256, 160),
+                                     (512, 77, 40), (512, 77, 80), (256, 77, 160), (200, 50, 40)])
+@pytest.mark.parametrize("mult", [16.0, 30.0])
+def test_scores_of_large_magnitude(att, bd, Nq, Nk, d, mult):
+    """q and k scaled so that the scaled scores reach into the thousands: the softmax is all but one-hot and the
+    anchor of the exponent must sit within a few units of a row's true maximum.  (A maximum taken from truncated
+    scores lies below the true one by up to 1/128 of its size -- more than the headroom of the weights at this
+    magnitude; the kernels take the exact one whenever they re-anchor.)"""
+    B, H = 1, 4
+    q, k, v = rand_qkv(900 + Nq + d, B, H, Nq, Nk, d)
+    q = (q.astype(np.float32) * mult).astype(np.float16)
+    k = (k.astype(np.float32) * mult).astype(np.float16)
+    scale = d ** -0.5
+    ref, L, _ = oracle.forward(q, k, v, scale)
+    assert float(np.abs(L).max()) > 500.0          # the case is what it claims to be
+    got = run(att, bd, bd.MODE_AUTO, q, k, v, scale)
+    check(got, ref, v, what="large scores x%g %s" % (mult, (Nq, Nk, d)))
