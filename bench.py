@@ -361,14 +361,15 @@ def run_ours(args):
     return 0
 
 
-def time_calls(att, bd, tensors, stream, iters, graph=False):
+def time_calls(att, bd, tensors, stream, iters, graph=False, dtype=None):
     """Mean microseconds for one pass over `tensors` (a list of calls), rotating nothing: small extras."""
     import torch
+    dtype = bd.F16 if dtype is None else dtype
 
     def once():
         for c, tq, tk, tv, to in tensors:
             rc = bd.sd_attn_forward(att.handle, tq.data_ptr(), tk.data_ptr(), tv.data_ptr(), to.data_ptr(),
-                                    c.B, c.H, c.Nq, c.Nk, c.d, float(c.scale()), bd.F16, stream)
+                                    c.B, c.H, c.Nq, c.Nk, c.d, float(c.scale()), dtype, stream)
             if rc != bd.OK:
                 raise bd.SdAttnError(rc, "sd_attn_forward")
     start, end = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
@@ -382,7 +383,7 @@ def time_calls(att, bd, tensors, stream, iters, graph=False):
             with torch.cuda.graph(g, stream=s):
                 for c, tq, tk, tv, to in tensors:
                     bd.sd_attn_forward(att.handle, tq.data_ptr(), tk.data_ptr(), tv.data_ptr(), to.data_ptr(),
-                                       c.B, c.H, c.Nq, c.Nk, c.d, float(c.scale()), bd.F16, s.cuda_stream)
+                                       c.B, c.H, c.Nq, c.Nk, c.d, float(c.scale()), dtype, s.cuda_stream)
         g.replay()
         torch.cuda.synchronize()
         start.record()
@@ -440,6 +441,18 @@ def extras(att, bd, device, stream, peaks):
     out["token_major_layout"] = {"unet_step_attention_set_us_cuda_graph": us_graph_t,
                                  "cross_attention_9216x77_d40_us_per_call": us_cross_t,
                                  "note": "sd_attn_set_layout(SD_ATTN_LAYOUT_BNHD); compare with the two entries above"}
+    # the bench's own shape with bfloat16 tensors: the same kernel with the other operand format
+    c2 = workloads.config2()[0]
+    bsets = []
+    for r in range(8):     # 8 x 21 MB: larger than L2
+        tq, tk, tv = (torch.randn(c2.B, c2.H, n, c2.d, device=device, dtype=torch.float32).to(torch.bfloat16)
+                      for n in (c2.Nq, c2.Nk, c2.Nk))
+        bsets.append((c2, tq, tk, tv, torch.empty_like(tq)))
+    us_bf16 = time_calls(att, bd, bsets, stream, 5, dtype=bd.BF16) / len(bsets)
+    att.check(stream)
+    out["bf16_self_attention_4096_d40"] = {"us_per_call": us_bf16, "tflops": c2.flops / (us_bf16 * 1e-6) / 1e12,
+                                           "note": "dtype SD_ATTN_BF16, rotating through 8 sets (168 MB)"}
+    del bsets
     out["geglu_8192x1280_f16"] = geglu_numbers(bd, device, stream, peaks)
     out["groupnorm_2x320x64x64_f16"] = groupnorm_numbers(bd, device, stream, peaks)
     return out

@@ -45,7 +45,11 @@ typedef enum {
 
 typedef enum {
     SD_ATTN_F16 = 0, /* IEEE binary16 q/k/v/out, binary32 accumulation            */
-    SD_ATTN_F32 = 1  /* binary32 throughout (plain FMA arithmetic, no TF32)        */
+    SD_ATTN_F32 = 1, /* binary32 throughout (plain FMA arithmetic, no TF32)        */
+    SD_ATTN_BF16 = 2 /* bfloat16 q/k/v/out, binary32 accumulation; the softmax weights enter the second product
+                        rounded to bfloat16 (8 significant bits), so results are about 8x coarser than F16's.
+                        Implemented by the kernels AUTO selects (FUSED, CROSS, SIMT); TWOPASS mode and FUSED
+                        under the switches that select its earlier kernels answer UNSUPPORTED.               */
 } sd_attn_dtype;
 
 typedef enum {

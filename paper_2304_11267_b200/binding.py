@@ -15,7 +15,7 @@ LIB_PATH = os.path.join(_PKG, "libsd_attn.so")
 
 # status codes, dtypes and modes of include/sd_attn.h
 OK, ERR_INVALID_VALUE, ERR_UNSUPPORTED, ERR_ALIGNMENT, ERR_WORKSPACE, ERR_ARCH, ERR_CUDA, ERR_DEVICE_TIMEOUT = range(8)
-F16, F32 = 0, 1
+F16, F32, BF16 = 0, 1, 2
 MODE_AUTO, MODE_FUSED, MODE_CROSS, MODE_TWOPASS, MODE_SIMT = range(5)
 MODE_NAMES = {MODE_AUTO: "auto", MODE_FUSED: "fused", MODE_CROSS: "cross", MODE_TWOPASS: "twopass",
               MODE_SIMT: "simt"}
@@ -272,8 +272,10 @@ class Attention:
             dtype = F16
         elif q.dtype == torch.float32:
             dtype = F32
+        elif q.dtype == torch.bfloat16:
+            dtype = BF16
         else:
-            raise TypeError("float16 or float32 only")
+            raise TypeError("float16, bfloat16 or float32 only")
         if self.layout == LAYOUT_BNHD:
             B, Nq, H, d = q.shape
             Nk = k.shape[1]

@@ -117,7 +117,7 @@ __device__ __forceinline__ void issue_qk(uint32_t tmem_s, uint64_t q_desc, uint6
                    k_desc + (uint64_t)(((kk >> 2) * X2_KN * CHUNK_ROW_BYTES + (kk & 3) * 32) >> 4), idesc, kk > 0);
 }
 
-template <int NWG>
+template <int NWG, bool BF = false>   // BF: bfloat16 tensors
 __global__ void __launch_bounds__(NWG * 128 + 256, 1)
 cross2_attention_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__ CUtensorMap tmap_k,
                         const __grid_constant__ CUtensorMap tmap_v, const Cross2Args args) {
@@ -281,7 +281,7 @@ cross2_attention_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid
             }
             if (warp != O_ISSUER_WARP) {
                 const int parity = warp == S_ISSUER_WARP ? 0 : 1;
-                const uint32_t idesc_s = idesc_f16(TILE_M, X2_KN, false, false, args.negate != 0);
+                const uint32_t idesc_s = idesc_f16(TILE_M, X2_KN, false, false, args.negate != 0, BF);
                 const int ksteps_s = (args.d + 15) / 16;
                 const uint64_t q_desc0 = smem_desc_sw128(q_smem, 16, 1024);
                 const uint64_t k_desc0 = smem_desc_sw128(kv_smem, 16, 1024);
@@ -319,7 +319,7 @@ cross2_attention_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid
                     X2_TRACE(NWG, c.i, 4);
                 }
             } else {
-                const uint32_t idesc_o = idesc_f16(TILE_M, dpad, false, true, false);
+                const uint32_t idesc_o = idesc_f16(TILE_M, dpad, false, true, false, BF);
                 const uint64_t v_desc0 = smem_desc_sw128(kv_smem + kv_bytes, X2_KN * CHUNK_ROW_BYTES, 1024);
                 const uint32_t kv_buf_off = (2 * kv_bytes) >> 4;
                 for (; c.i < n_local && ok; advance(c)) {
@@ -405,8 +405,8 @@ cross2_attention_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid
                     const float neg_mc = -anchor;
                     const uint64_t c2c2 = pack_b64(__float_as_uint(c2), __float_as_uint(c2));
                     const uint64_t nmnm = pack_b64(__float_as_uint(neg_mc), __float_as_uint(neg_mc));
-                    exp2_pack_32<0>(&s[0], c2c2, nmnm, &packed[0], acc);
-                    exp2_pack_16<0>(&s[32], c2c2, nmnm, &packed[16], acc);
+                    exp2_pack_32<0, 16, BF>(&s[0], c2c2, nmnm, &packed[0], acc);
+                    exp2_pack_16<0, BF>(&s[32], c2c2, nmnm, &packed[16], acc);
                 }
                 {   // columns 48..79: the last 16 hold the keys past Nk (zero-filled) and are masked
                     uint32_t s[32];
@@ -415,8 +415,8 @@ cross2_attention_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid
                     const float neg_mc = -anchor;
                     const uint64_t c2c2 = pack_b64(__float_as_uint(c2), __float_as_uint(c2));
                     const uint64_t nmnm = pack_b64(__float_as_uint(neg_mc), __float_as_uint(neg_mc));
-                    exp2_pack_16<0>(&s[0], c2c2, nmnm, &packed[24], acc);
-                    exp2_pack_32_masked<8>(&s[16], c2, neg_mc, 64, valid, &packed[32], tail);
+                    exp2_pack_16<0, BF>(&s[0], c2c2, nmnm, &packed[24], acc);
+                    exp2_pack_32_masked<8, BF>(&s[16], c2, neg_mc, 64, valid, &packed[32], tail);
                 }
                 row_sum = sum_f32x2(acc[0], acc[1]) + tail;   // S_i of Eq. 4, relative to the anchor
                 const bool over = !(row_sum <= X2_SUM_LIMIT);
@@ -487,10 +487,10 @@ cross2_attention_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid
 #pragma unroll
                 for (int g = 0; g < 6; ++g) {
                     uint4 v8;
-                    v8.x = pack_half2(__uint_as_float(x[g * 8 + 0]) * inv, __uint_as_float(x[g * 8 + 1]) * inv);
-                    v8.y = pack_half2(__uint_as_float(x[g * 8 + 2]) * inv, __uint_as_float(x[g * 8 + 3]) * inv);
-                    v8.z = pack_half2(__uint_as_float(x[g * 8 + 4]) * inv, __uint_as_float(x[g * 8 + 5]) * inv);
-                    v8.w = pack_half2(__uint_as_float(x[g * 8 + 6]) * inv, __uint_as_float(x[g * 8 + 7]) * inv);
+                    v8.x = pack_16x2<BF>(__uint_as_float(x[g * 8 + 0]) * inv, __uint_as_float(x[g * 8 + 1]) * inv);
+                    v8.y = pack_16x2<BF>(__uint_as_float(x[g * 8 + 2]) * inv, __uint_as_float(x[g * 8 + 3]) * inv);
+                    v8.z = pack_16x2<BF>(__uint_as_float(x[g * 8 + 4]) * inv, __uint_as_float(x[g * 8 + 5]) * inv);
+                    v8.w = pack_16x2<BF>(__uint_as_float(x[g * 8 + 6]) * inv, __uint_as_float(x[g * 8 + 7]) * inv);
                     if (g * 8 + 8 <= args.d) st_shared_v4(dst + g * 16, v8);
                 }
                 fence_proxy_async_smem();   // generic-proxy stores before the bulk copy reads them
@@ -521,10 +521,10 @@ cross2_attention_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid
 #pragma unroll
                     for (int g = 0; g < 4; ++g) {
                         uint4 v8;
-                        v8.x = pack_half2(__uint_as_float(x[g * 8 + 0]) * inv, __uint_as_float(x[g * 8 + 1]) * inv);
-                        v8.y = pack_half2(__uint_as_float(x[g * 8 + 2]) * inv, __uint_as_float(x[g * 8 + 3]) * inv);
-                        v8.z = pack_half2(__uint_as_float(x[g * 8 + 4]) * inv, __uint_as_float(x[g * 8 + 5]) * inv);
-                        v8.w = pack_half2(__uint_as_float(x[g * 8 + 6]) * inv, __uint_as_float(x[g * 8 + 7]) * inv);
+                        v8.x = pack_16x2<BF>(__uint_as_float(x[g * 8 + 0]) * inv, __uint_as_float(x[g * 8 + 1]) * inv);
+                        v8.y = pack_16x2<BF>(__uint_as_float(x[g * 8 + 2]) * inv, __uint_as_float(x[g * 8 + 3]) * inv);
+                        v8.z = pack_16x2<BF>(__uint_as_float(x[g * 8 + 4]) * inv, __uint_as_float(x[g * 8 + 5]) * inv);
+                        v8.w = pack_16x2<BF>(__uint_as_float(x[g * 8 + 6]) * inv, __uint_as_float(x[g * 8 + 7]) * inv);
                         if (c0 + g * 8 + 8 <= args.d) *reinterpret_cast<uint4*>(orow + c0 + g * 8) = v8;
                     }
                 }

@@ -43,6 +43,7 @@ __host__ inline size_t cross_smem_bytes(int nch, int kn) {
 
 enum { SITE_X_LOAD_QK = 1, SITE_X_LOAD_V = 2, SITE_X_S = 3, SITE_X_O = 4 };
 
+template <bool BF = false>   // BF: bfloat16 tensors
 __global__ void __launch_bounds__(CROSS_THREADS)
 cross_attention_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__ CUtensorMap tmap_k,
                        const __grid_constant__ CUtensorMap tmap_v, const CrossArgs args) {
@@ -105,7 +106,7 @@ cross_attention_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_
         // S = Q K^T: contraction over d in steps of 16 columns (32 bytes inside a swizzled row)
         if (mbar_wait(bar_qk, 0, abort_p, args.status, SITE_X_LOAD_QK, tile)) {
             tc_fence_after_sync();
-            const uint32_t idesc = idesc_f16(TILE_M, kn, false, false, args.negate != 0);
+            const uint32_t idesc = idesc_f16(TILE_M, kn, false, false, args.negate != 0, BF);
             const int ksteps = (args.d + 15) / 16;
             for (int kk = 0; kk < ksteps; ++kk) {
                 const int ch = kk >> 2, within = (kk & 3) * 32;
@@ -154,7 +155,7 @@ cross_attention_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_
                 row_sum += p[c];
             }
 #pragma unroll
-            for (int c = 0; c < 8; ++c) packed[c] = pack_half2(p[2 * c], p[2 * c + 1]);
+            for (int c = 0; c < 8; ++c) packed[c] = pack_16x2<BF>(p[2 * c], p[2 * c + 1]);
             tmem_st8(tmem_s + lane_off + g * 8, packed);    // overwrites columns already consumed
         }
         tmem_wait_st();
@@ -166,7 +167,7 @@ cross_attention_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_
     if (tid == 0 && ok) {
         if (mbar_wait(bar_v, 0, abort_p, args.status, SITE_X_LOAD_V, tile)) {
             tc_fence_after_sync();
-            const uint32_t idesc = idesc_f16(TILE_M, dpad, false, true, false);
+            const uint32_t idesc = idesc_f16(TILE_M, dpad, false, true, false, BF);
             for (int kk = 0; kk < (kn >> 4); ++kk) {
                 const uint64_t b_desc = smem_desc_sw128(v_smem + kk * 16 * CHUNK_ROW_BYTES,
                                                         (uint32_t)(kn * CHUNK_ROW_BYTES), 1024);
@@ -189,14 +190,14 @@ cross_attention_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_
             tmem_ld16(tmem_o + lane_off + g * 16, r);
             tmem_wait_ld();
             uint4 lo, hi;
-            lo.x = pack_half2(__uint_as_float(r[0]) * inv, __uint_as_float(r[1]) * inv);
-            lo.y = pack_half2(__uint_as_float(r[2]) * inv, __uint_as_float(r[3]) * inv);
-            lo.z = pack_half2(__uint_as_float(r[4]) * inv, __uint_as_float(r[5]) * inv);
-            lo.w = pack_half2(__uint_as_float(r[6]) * inv, __uint_as_float(r[7]) * inv);
-            hi.x = pack_half2(__uint_as_float(r[8]) * inv, __uint_as_float(r[9]) * inv);
-            hi.y = pack_half2(__uint_as_float(r[10]) * inv, __uint_as_float(r[11]) * inv);
-            hi.z = pack_half2(__uint_as_float(r[12]) * inv, __uint_as_float(r[13]) * inv);
-            hi.w = pack_half2(__uint_as_float(r[14]) * inv, __uint_as_float(r[15]) * inv);
+            lo.x = pack_16x2<BF>(__uint_as_float(r[0]) * inv, __uint_as_float(r[1]) * inv);
+            lo.y = pack_16x2<BF>(__uint_as_float(r[2]) * inv, __uint_as_float(r[3]) * inv);
+            lo.z = pack_16x2<BF>(__uint_as_float(r[4]) * inv, __uint_as_float(r[5]) * inv);
+            lo.w = pack_16x2<BF>(__uint_as_float(r[6]) * inv, __uint_as_float(r[7]) * inv);
+            hi.x = pack_16x2<BF>(__uint_as_float(r[8]) * inv, __uint_as_float(r[9]) * inv);
+            hi.y = pack_16x2<BF>(__uint_as_float(r[10]) * inv, __uint_as_float(r[11]) * inv);
+            hi.z = pack_16x2<BF>(__uint_as_float(r[12]) * inv, __uint_as_float(r[13]) * inv);
+            hi.w = pack_16x2<BF>(__uint_as_float(r[14]) * inv, __uint_as_float(r[15]) * inv);
             if (row < args.Nq) {
                 if (g * 16 + 8 <= args.d) *reinterpret_cast<uint4*>(orow + g * 16) = lo;
                 if (g * 16 + 16 <= args.d) *reinterpret_cast<uint4*>(orow + g * 16 + 8) = hi;

@@ -75,7 +75,7 @@ static_assert(512 * F4S_SOFTMAX_REGS + 256 * F4S_CONTROL_REGS == 768 * 80, "setm
 // those of four query tiles do, and they need no agreement on an anchor because their products never share an
 // accumulator.  The score buffers run ahead of the products (NB of them, a multiple of SPLIT), and the MMAs come from
 // two threads: the products of key tile j from one, the scores of key tile j + NB from the other.
-template <int POLY, int NCH, int SPLIT = 1>   // NCH: 64-column chunks per row (head dim <= 64 * NCH)
+template <int POLY, int NCH, int SPLIT = 1, bool BF = false>   // NCH: 64-column chunks per row (head dim <= 64 * NCH); BF: bfloat16 tensors
 __global__ void __launch_bounds__(F4_THREADS, 1)
 fused4s_attention_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__ CUtensorMap tmap_k,
                          const __grid_constant__ CUtensorMap tmap_v, const Fused4Args args) {
@@ -201,8 +201,8 @@ fused4s_attention_kernel(const __grid_constant__ CUtensorMap tmap_q, const __gri
         // NEXT tile of the rotation.
         const int t = warp - 17;
         if ((t < T || (SPLIT > 1 && t == 1)) && elect_one()) {
-            const uint32_t idesc_s = idesc_f16(TILE_M, BN, false, false, args.negate != 0);
-            const uint32_t idesc_o = idesc_f16(TILE_M, dpad, false, true, false);
+            const uint32_t idesc_s = idesc_f16(TILE_M, BN, false, false, args.negate != 0, BF);
+            const uint32_t idesc_o = idesc_f16(TILE_M, dpad, false, true, false, BF);
             const int ksteps_s = (args.d + 15) / 16;   // 16 columns each; four to a swizzled 64-column chunk
             const int tn = (t + 1 == T) ? 0 : t + 1;   // the tile whose scores this thread requests
             const uint64_t q_desc = smem_desc_sw128(q_smem + tn * q_tile_bytes, 16, 1024);
@@ -378,13 +378,13 @@ fused4s_attention_kernel(const __grid_constant__ CUtensorMap tmap_q, const __gri
                             const uint64_t c2c2 = pack_b64(__float_as_uint(c2), __float_as_uint(c2));
                             const uint64_t nmnm = pack_b64(__float_as_uint(neg_mc), __float_as_uint(neg_mc));
                             uint64_t acc[2] = {0ull, 0ull};
-                            exp2_pack_32<POLY>(&s[0], c2c2, nmnm, &packed[0], acc);
-                            exp2_pack_32<POLY>(&s[32], c2c2, nmnm, &packed[16], acc);
+                            exp2_pack_32<POLY, 16, BF>(&s[0], c2c2, nmnm, &packed[0], acc);
+                            exp2_pack_32<POLY, 16, BF>(&s[32], c2c2, nmnm, &packed[16], acc);
                             tile_sum = sum_f32x2(acc[0], acc[1]);
                         } else {
                             tile_sum = 0.f;
-                            exp2_pack_32_masked(&s[0], c2, neg_mc, 0, valid, &packed[0], tile_sum);
-                            exp2_pack_32_masked(&s[32], c2, neg_mc, 32, valid, &packed[16], tile_sum);
+                            exp2_pack_32_masked<16, BF>(&s[0], c2, neg_mc, 0, valid, &packed[0], tile_sum);
+                            exp2_pack_32_masked<16, BF>(&s[32], c2, neg_mc, 32, valid, &packed[16], tile_sum);
                         }
                         const bool over = !(tile_sum <= FUSED_TILE_SUM_LIMIT);
                         if (attempt == 1 || !__any_sync(0xffffffffu, over)) break;
@@ -472,10 +472,10 @@ fused4s_attention_kernel(const __grid_constant__ CUtensorMap tmap_q, const __gri
                             for (int c = 0; c < 16; ++c) acc[c] = fmaf(__uint_as_float(x[c]), f[p2], acc[c]);
                         }
                         uint4 lo, hi;
-                        lo.x = pack_half2(acc[0], acc[1]);   lo.y = pack_half2(acc[2], acc[3]);
-                        lo.z = pack_half2(acc[4], acc[5]);   lo.w = pack_half2(acc[6], acc[7]);
-                        hi.x = pack_half2(acc[8], acc[9]);   hi.y = pack_half2(acc[10], acc[11]);
-                        hi.z = pack_half2(acc[12], acc[13]); hi.w = pack_half2(acc[14], acc[15]);
+                        lo.x = pack_16x2<BF>(acc[0], acc[1]);   lo.y = pack_16x2<BF>(acc[2], acc[3]);
+                        lo.z = pack_16x2<BF>(acc[4], acc[5]);   lo.w = pack_16x2<BF>(acc[6], acc[7]);
+                        hi.x = pack_16x2<BF>(acc[8], acc[9]);   hi.y = pack_16x2<BF>(acc[10], acc[11]);
+                        hi.z = pack_16x2<BF>(acc[12], acc[13]); hi.w = pack_16x2<BF>(acc[14], acc[15]);
                         if (row < args.Nq) {
                             if (cg * 16 + 8 <= args.d) *reinterpret_cast<uint4*>(orow + cg * 16) = lo;
                             if (cg * 16 + 16 <= args.d) *reinterpret_cast<uint4*>(orow + cg * 16 + 8) = hi;
@@ -525,13 +525,13 @@ fused4s_attention_kernel(const __grid_constant__ CUtensorMap tmap_q, const __gri
                         const uint64_t c2c2 = pack_b64(__float_as_uint(c2), __float_as_uint(c2));
                         const uint64_t nmnm = pack_b64(__float_as_uint(neg_mc), __float_as_uint(neg_mc));
                         uint64_t acc[2] = {0ull, 0ull};
-                        exp2_pack_32<POLY>(&s[0], c2c2, nmnm, &packed[0], acc);
-                        exp2_pack_32<POLY>(&s[32], c2c2, nmnm, &packed[16], acc);
+                        exp2_pack_32<POLY, 16, BF>(&s[0], c2c2, nmnm, &packed[0], acc);
+                        exp2_pack_32<POLY, 16, BF>(&s[32], c2c2, nmnm, &packed[16], acc);
                         tile_sum = sum_f32x2(acc[0], acc[1]);
                     } else {
                         tile_sum = 0.f;
-                        exp2_pack_32_masked(&s[0], c2, neg_mc, 0, valid, &packed[0], tile_sum);
-                        exp2_pack_32_masked(&s[32], c2, neg_mc, 32, valid, &packed[16], tile_sum);
+                        exp2_pack_32_masked<16, BF>(&s[0], c2, neg_mc, 0, valid, &packed[0], tile_sum);
+                        exp2_pack_32_masked<16, BF>(&s[32], c2, neg_mc, 32, valid, &packed[16], tile_sum);
                     }
                     const bool over = !(tile_sum <= FUSED_TILE_SUM_LIMIT);
                     if (attempt == 1 || !__any_sync(0xffffffffu, over)) break;
@@ -602,14 +602,14 @@ fused4s_attention_kernel(const __grid_constant__ CUtensorMap tmap_q, const __gri
                     tmem_ld16(tmem_o + g * 16, x);
                     tmem_wait_ld();
                     uint4 lo, hi;
-                    lo.x = pack_half2(__uint_as_float(x[0]) * inv, __uint_as_float(x[1]) * inv);
-                    lo.y = pack_half2(__uint_as_float(x[2]) * inv, __uint_as_float(x[3]) * inv);
-                    lo.z = pack_half2(__uint_as_float(x[4]) * inv, __uint_as_float(x[5]) * inv);
-                    lo.w = pack_half2(__uint_as_float(x[6]) * inv, __uint_as_float(x[7]) * inv);
-                    hi.x = pack_half2(__uint_as_float(x[8]) * inv, __uint_as_float(x[9]) * inv);
-                    hi.y = pack_half2(__uint_as_float(x[10]) * inv, __uint_as_float(x[11]) * inv);
-                    hi.z = pack_half2(__uint_as_float(x[12]) * inv, __uint_as_float(x[13]) * inv);
-                    hi.w = pack_half2(__uint_as_float(x[14]) * inv, __uint_as_float(x[15]) * inv);
+                    lo.x = pack_16x2<BF>(__uint_as_float(x[0]) * inv, __uint_as_float(x[1]) * inv);
+                    lo.y = pack_16x2<BF>(__uint_as_float(x[2]) * inv, __uint_as_float(x[3]) * inv);
+                    lo.z = pack_16x2<BF>(__uint_as_float(x[4]) * inv, __uint_as_float(x[5]) * inv);
+                    lo.w = pack_16x2<BF>(__uint_as_float(x[6]) * inv, __uint_as_float(x[7]) * inv);
+                    hi.x = pack_16x2<BF>(__uint_as_float(x[8]) * inv, __uint_as_float(x[9]) * inv);
+                    hi.y = pack_16x2<BF>(__uint_as_float(x[10]) * inv, __uint_as_float(x[11]) * inv);
+                    hi.z = pack_16x2<BF>(__uint_as_float(x[12]) * inv, __uint_as_float(x[13]) * inv);
+                    hi.w = pack_16x2<BF>(__uint_as_float(x[14]) * inv, __uint_as_float(x[15]) * inv);
                     if (row < args.Nq) {
                         if (g * 16 + 8 <= args.d) *reinterpret_cast<uint4*>(orow + g * 16) = lo;
                         if (g * 16 + 16 <= args.d) *reinterpret_cast<uint4*>(orow + g * 16 + 8) = hi;

@@ -38,6 +38,7 @@ struct TmapCacheEntry {
     const void* base;
     int BH, N, d, box_rows;
     int heads;   // heads per batch entry of a token-major tensor, 0 for a head-major one
+    int bf16;    // bfloat16 elements (binary16 otherwise)
     CUtensorMap map;
 };
 constexpr int TMAP_CACHE_ENTRIES = 128;
@@ -151,6 +152,44 @@ static void destroy_host_overlap(sd_attn_handle* h) {   // the handle was calloc
     h->host_overlap = 0;
 }
 
+// The kernels AUTO selects exist for binary16 and for bfloat16 tensors (BF); each needs its shared-memory limit raised.
+template <bool BF>
+static cudaError_t raise_layout_kernels() {
+    cudaError_t e = raise_smem_limit(cross_attention_kernel<BF>, cross_smem_bytes(3, 128));
+    if (e == cudaSuccess) e = raise_smem_limit(cross2_attention_kernel<2, BF>, X2_SMEM_BUDGET + 1024);
+    if (e == cudaSuccess) e = raise_smem_limit(cross2_attention_kernel<3, BF>, X2_SMEM_BUDGET + 1024);
+    if (e == cudaSuccess) e = raise_smem_limit(cross2_attention_kernel<4, BF>, X2_SMEM_BUDGET + 1024);
+    if (e == cudaSuccess) e = raise_smem_limit(fused4s_attention_kernel<F4S_POLY_PER8, 1, 1, BF>, F4S_SMEM_BUDGET + 1024);
+    if (e == cudaSuccess) e = raise_smem_limit(fused4s_attention_kernel<0, 1, 1, BF>, F4S_SMEM_BUDGET + 1024);
+    if (e == cudaSuccess) e = raise_smem_limit(fused4s_attention_kernel<0, 2, 1, BF>, F4S_SMEM_BUDGET + 1024);
+    if (e == cudaSuccess) e = raise_smem_limit(fused4s_attention_kernel<0, 3, 1, BF>, F4S_SMEM_BUDGET + 1024);
+    if (e == cudaSuccess) e = raise_smem_limit(fused4s_attention_kernel<F4S_POLY_PER8, 1, 4, BF>, F4S_SMEM_BUDGET + 1024);
+    if (e == cudaSuccess) e = raise_smem_limit(fused4s_attention_kernel<F4S_POLY_PER8, 1, 2, BF>, F4S_SMEM_BUDGET + 1024);
+    if (e == cudaSuccess) e = raise_smem_limit(fused4s_attention_kernel<F4S_POLY_PER8, 2, 2, BF>, F4S_SMEM_BUDGET + 1024);
+    if (e == cudaSuccess) e = raise_smem_limit(fused4s_attention_kernel<F4S_POLY_PER8, 3, 2, BF>, F4S_SMEM_BUDGET + 1024);
+    return e;
+}
+
+// Register budgets of the warp-specialised kernels (setmaxnreg pools must fit the launch allocation).
+template <bool BF>
+static cudaError_t check_register_pools(sd_attn_handle* h) {
+    cudaFuncAttributes fa;
+    cudaError_t e = cudaSuccess;
+    const void* f4s[8] = {(const void*)fused4s_attention_kernel<F4S_POLY_PER8, 1, 1, BF>, (const void*)fused4s_attention_kernel<0, 1, 1, BF>,
+                          (const void*)fused4s_attention_kernel<0, 2, 1, BF>, (const void*)fused4s_attention_kernel<0, 3, 1, BF>,
+                          (const void*)fused4s_attention_kernel<F4S_POLY_PER8, 1, 4, BF>, (const void*)fused4s_attention_kernel<F4S_POLY_PER8, 1, 2, BF>,
+                          (const void*)fused4s_attention_kernel<F4S_POLY_PER8, 2, 2, BF>,
+                          (const void*)fused4s_attention_kernel<F4S_POLY_PER8, 3, 2, BF>};
+    for (int i = 0; i < 8 && e == cudaSuccess; ++i) {
+        e = cudaFuncGetAttributes(&fa, f4s[i]);
+        if (e == cudaSuccess && F4_THREADS * fa.numRegs < 512 * F4S_SOFTMAX_REGS + 256 * F4S_CONTROL_REGS) h->fused4s_ok = 0;
+    }
+    if (e == cudaSuccess) e = cudaFuncGetAttributes(&fa, cross2_attention_kernel<4, BF>);
+    if (e == cudaSuccess && cross2_threads(4) * fa.numRegs < 512 * X2_SOFTMAX_REGS + 128 * X2_EPILOGUE_REGS + 128 * X2_CONTROL_REGS)
+        h->cross2_four_ok = 0;
+    return e;
+}
+
 extern "C" int sd_attn_create(sd_attn_handle** out) {
     if (!out) return SD_ATTN_ERR_INVALID_VALUE;
     *out = nullptr;
@@ -198,27 +237,19 @@ extern "C" int sd_attn_create(sd_attn_handle** out) {
     h->prefer_two_tile = (two && two[0] == '1') ? 1 : 0;
 
     // dynamic shared memory ceilings of every kernel, once
-    e = raise_smem_limit(cross_attention_kernel, cross_smem_bytes(3, 128));
-    if (e == cudaSuccess) e = raise_smem_limit(cross2_attention_kernel<2>, X2_SMEM_BUDGET + 1024);
-    if (e == cudaSuccess) e = raise_smem_limit(cross2_attention_kernel<3>, X2_SMEM_BUDGET + 1024);
-    if (e == cudaSuccess) e = raise_smem_limit(cross2_attention_kernel<4>, X2_SMEM_BUDGET + 1024);
+    e = raise_layout_kernels<false>();
+    if (e == cudaSuccess) e = raise_layout_kernels<true>();
     if (e == cudaSuccess) e = raise_smem_limit(fused_attention_kernel<128>, fused_smem_bytes_max());
     if (e == cudaSuccess) e = raise_smem_limit(fused_attention_kernel<64>, fused_smem_bytes_max());
     if (e == cudaSuccess) e = raise_smem_limit(fused4_attention_kernel, fused4_smem_bytes());
-    if (e == cudaSuccess) e = raise_smem_limit(fused4s_attention_kernel<F4S_POLY_PER8, 1>, F4S_SMEM_BUDGET + 1024);
-    if (e == cudaSuccess) e = raise_smem_limit(fused4s_attention_kernel<0, 1>, F4S_SMEM_BUDGET + 1024);
-    if (e == cudaSuccess) e = raise_smem_limit(fused4s_attention_kernel<0, 2>, F4S_SMEM_BUDGET + 1024);
-    if (e == cudaSuccess) e = raise_smem_limit(fused4s_attention_kernel<0, 3>, F4S_SMEM_BUDGET + 1024);
-    if (e == cudaSuccess) e = raise_smem_limit(fused4s_attention_kernel<F4S_POLY_PER8, 1, 4>, F4S_SMEM_BUDGET + 1024);
-    if (e == cudaSuccess) e = raise_smem_limit(fused4s_attention_kernel<F4S_POLY_PER8, 1, 2>, F4S_SMEM_BUDGET + 1024);
-    if (e == cudaSuccess) e = raise_smem_limit(fused4s_attention_kernel<F4S_POLY_PER8, 2, 2>, F4S_SMEM_BUDGET + 1024);
-    if (e == cudaSuccess) e = raise_smem_limit(fused4s_attention_kernel<F4S_POLY_PER8, 3, 2>, F4S_SMEM_BUDGET + 1024);
     if (e == cudaSuccess) e = raise_smem_limit(twopass_scores_kernel, twopass_scores_smem_bytes(3));
     if (e == cudaSuccess) e = raise_smem_limit(twopass_pv_kernel, twopass_pv_smem_bytes(3));
     if (e == cudaSuccess) e = raise_smem_limit(simt_attention_kernel<float, 5>, simt_smem_bytes(160));
     if (e == cudaSuccess) e = raise_smem_limit(simt_attention_kernel<__half, 5>, simt_smem_bytes(160));
     if (e == cudaSuccess) e = raise_smem_limit(simt_attention_kernel<float, 4>, simt_smem_bytes(128));
     if (e == cudaSuccess) e = raise_smem_limit(simt_attention_kernel<__half, 4>, simt_smem_bytes(128));
+    if (e == cudaSuccess) e = raise_smem_limit(simt_attention_kernel<__nv_bfloat16, 5>, simt_smem_bytes(160));
+    if (e == cudaSuccess) e = raise_smem_limit(simt_attention_kernel<__nv_bfloat16, 4>, simt_smem_bytes(128));
     // setmaxnreg budgets (see the kernels): only use a variant whose increases are covered by its decreases
     if (e == cudaSuccess) {
         cudaFuncAttributes fa;
@@ -226,18 +257,9 @@ extern "C" int sd_attn_create(sd_attn_handle** out) {
         if (e == cudaSuccess)
             h->fused4_ok = F4_THREADS * fa.numRegs >= 512 * F4_SOFTMAX_REGS + 256 * F4_CONTROL_REGS;
         h->fused4s_ok = 1;
-        const void* f4s[8] = {(const void*)fused4s_attention_kernel<F4S_POLY_PER8, 1>, (const void*)fused4s_attention_kernel<0, 1>,
-                              (const void*)fused4s_attention_kernel<0, 2>, (const void*)fused4s_attention_kernel<0, 3>,
-                              (const void*)fused4s_attention_kernel<F4S_POLY_PER8, 1, 4>, (const void*)fused4s_attention_kernel<F4S_POLY_PER8, 1, 2>,
-                              (const void*)fused4s_attention_kernel<F4S_POLY_PER8, 2, 2>,
-                              (const void*)fused4s_attention_kernel<F4S_POLY_PER8, 3, 2>};
-        for (int i = 0; i < 8 && e == cudaSuccess; ++i) {
-            e = cudaFuncGetAttributes(&fa, f4s[i]);
-            if (e == cudaSuccess && F4_THREADS * fa.numRegs < 512 * F4S_SOFTMAX_REGS + 256 * F4S_CONTROL_REGS) h->fused4s_ok = 0;
-        }
-        if (e == cudaSuccess) e = cudaFuncGetAttributes(&fa, cross2_attention_kernel<4>);
-        if (e == cudaSuccess)
-            h->cross2_four_ok = cross2_threads(4) * fa.numRegs >= 512 * X2_SOFTMAX_REGS + 128 * X2_EPILOGUE_REGS + 128 * X2_CONTROL_REGS;
+        h->cross2_four_ok = 1;
+        if (e == cudaSuccess) e = check_register_pools<false>(h);
+        if (e == cudaSuccess) e = check_register_pools<true>(h);
     }
     if (e == cudaSuccess) e = cudaMalloc((void**)&h->dev_status, sizeof(int) * DEV_STATUS_INTS);
     if (e == cudaSuccess) e = cudaMemset(h->dev_status, 0, sizeof(int) * DEV_STATUS_INTS);
@@ -335,13 +357,14 @@ static HeadLayout head_layout(int heads, int BH, int N, int d) {
 }
 
 static CUresult encode_tmap(encode_tiled_fn enc, CUtensorMap* map, const void* base, int heads, int BH, int N, int d,
-                            int box_rows) {
+                            int box_rows, int bf16 = 0) {
     const HeadLayout l = head_layout(heads, BH, N, d);
     cuuint64_t dims[4] = {(cuuint64_t)d, (cuuint64_t)N, (cuuint64_t)l.heads, (cuuint64_t)(BH / l.heads)};
     cuuint64_t strides[3] = {(cuuint64_t)l.ld * 2, (cuuint64_t)l.head_stride * 2, (cuuint64_t)l.batch_stride * 2};
     cuuint32_t box[4] = {(cuuint32_t)CHUNK_COLS, (cuuint32_t)box_rows, 1, 1};
     cuuint32_t estr[4] = {1, 1, 1, 1};
-    return enc(map, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 4, const_cast<void*>(base), dims, strides, box, estr,
+    return enc(map, bf16 ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 4,
+               const_cast<void*>(base), dims, strides, box, estr,
                CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
                CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
 }
@@ -349,15 +372,15 @@ static CUresult encode_tmap(encode_tiled_fn enc, CUtensorMap* map, const void* b
 // An fp16 tensor of BH heads of N rows of d values seen by the TMA as (x = d, y = N, z = head, w = batch): tiles are
 // 64 columns wide (one 128-byte swizzled row) by `box_rows` rows.  Columns >= d and rows >= N read as zero.
 static int make_tmap(sd_attn_handle* h, CUtensorMap* map, const void* base, int BH, int N, int d, int box_rows,
-                     int heads = 0) {
+                     int heads = 0, int bf16 = 0) {
     for (int i = 0; i < TMAP_CACHE_ENTRIES; ++i) {
         const TmapCacheEntry& e = h->tmap_cache[i];
-        if (e.base == base && e.BH == BH && e.N == N && e.d == d && e.box_rows == box_rows && e.heads == heads) {
+        if (e.base == base && e.BH == BH && e.N == N && e.d == d && e.box_rows == box_rows && e.heads == heads && e.bf16 == bf16) {
             *map = e.map;
             return SD_ATTN_OK;
         }
     }
-    CUresult r = encode_tmap(h->encode_tiled, map, base, heads, BH, N, d, box_rows);
+    CUresult r = encode_tmap(h->encode_tiled, map, base, heads, BH, N, d, box_rows, bf16);
     if (r != CUDA_SUCCESS) {
         if (getenv("SD_ATTN_LOG")) fprintf(stderr, "[sd_attn] cuTensorMapEncodeTiled failed: %d\n", (int)r);
         h->last_cuda_error = cudaErrorInvalidValue;
@@ -365,7 +388,7 @@ static int make_tmap(sd_attn_handle* h, CUtensorMap* map, const void* base, int 
     }
     TmapCacheEntry& slot = h->tmap_cache[h->tmap_cache_next];
     h->tmap_cache_next = (h->tmap_cache_next + 1) % TMAP_CACHE_ENTRIES;
-    slot.base = base; slot.BH = BH; slot.N = N; slot.d = d; slot.box_rows = box_rows; slot.heads = heads;
+    slot.base = base; slot.BH = BH; slot.N = N; slot.d = d; slot.box_rows = box_rows; slot.heads = heads; slot.bf16 = bf16;
     slot.map = *map;
     return SD_ATTN_OK;
 }
@@ -383,6 +406,7 @@ struct Problem {
     float scale;
     cudaStream_t stream;
     int heads;   // token-major tensors: heads per batch entry; head-major: 0
+    int bf16;    // bfloat16 tensors (binary16 otherwise); tensor-core kernels only
 };
 
 template <typename T>
@@ -424,9 +448,9 @@ static int launch_cross2(sd_attn_handle* h, const Problem& p) {
     a.trace = (long long*)h->trace;
 #endif
     CUtensorMap tq, tk, tv;
-    int rc = make_tmap(h, &tq, p.q, p.BH, p.Nq, p.d, TILE_M, p.heads);
-    if (rc == SD_ATTN_OK) rc = make_tmap(h, &tk, p.k, p.BH, p.Nk, p.d, X2_KN, p.heads);
-    if (rc == SD_ATTN_OK) rc = make_tmap(h, &tv, p.v, p.BH, p.Nk, p.d, X2_KN, p.heads);
+    int rc = make_tmap(h, &tq, p.q, p.BH, p.Nq, p.d, TILE_M, p.heads, p.bf16);
+    if (rc == SD_ATTN_OK) rc = make_tmap(h, &tk, p.k, p.BH, p.Nk, p.d, X2_KN, p.heads, p.bf16);
+    if (rc == SD_ATTN_OK) rc = make_tmap(h, &tv, p.v, p.BH, p.Nk, p.d, X2_KN, p.heads, p.bf16);
     if (rc != SD_ATTN_OK) return rc;
     const int grid = a.n_items < h->sm_count ? a.n_items : h->sm_count;
     int groups = cross2_groups(p.d);
@@ -437,12 +461,16 @@ static int launch_cross2(sd_attn_handle* h, const Problem& p) {
         a.stages = cross2_dense_stages(p.d);
         smem = cross2_dense_smem_bytes(p.d);
     }
-    if (groups >= 4)
-        launch_overlapped(h, cross2_attention_kernel<4>, dim3(grid), dim3(cross2_threads(4)), smem, p.stream, tq, tk, tv, a);
-    else if (groups == 3)
-        launch_overlapped(h, cross2_attention_kernel<3>, dim3(grid), dim3(cross2_threads(3)), smem, p.stream, tq, tk, tv, a);
-    else
-        launch_overlapped(h, cross2_attention_kernel<2>, dim3(grid), dim3(cross2_threads(2)), smem, p.stream, tq, tk, tv, a);
+    const dim3 g(grid);
+    if (p.bf16) {
+        if (groups >= 4) launch_overlapped(h, cross2_attention_kernel<4, true>, g, dim3(cross2_threads(4)), smem, p.stream, tq, tk, tv, a);
+        else if (groups == 3) launch_overlapped(h, cross2_attention_kernel<3, true>, g, dim3(cross2_threads(3)), smem, p.stream, tq, tk, tv, a);
+        else launch_overlapped(h, cross2_attention_kernel<2, true>, g, dim3(cross2_threads(2)), smem, p.stream, tq, tk, tv, a);
+    } else {
+        if (groups >= 4) launch_overlapped(h, cross2_attention_kernel<4>, g, dim3(cross2_threads(4)), smem, p.stream, tq, tk, tv, a);
+        else if (groups == 3) launch_overlapped(h, cross2_attention_kernel<3>, g, dim3(cross2_threads(3)), smem, p.stream, tq, tk, tv, a);
+        else launch_overlapped(h, cross2_attention_kernel<2>, g, dim3(cross2_threads(2)), smem, p.stream, tq, tk, tv, a);
+    }
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) return cuda_fail(h, e);
     h->launches += 1;
@@ -464,12 +492,15 @@ static int launch_cross(sd_attn_handle* h, const Problem& p) {
     a.status = h->dev_status;
     a.dump_scores = h->dump_scores;
     CUtensorMap tq, tk, tv;
-    int rc = make_tmap(h, &tq, p.q, p.BH, p.Nq, p.d, TILE_M, p.heads);
-    if (rc == SD_ATTN_OK) rc = make_tmap(h, &tk, p.k, p.BH, p.Nk, p.d, a.kn, p.heads);
-    if (rc == SD_ATTN_OK) rc = make_tmap(h, &tv, p.v, p.BH, p.Nk, p.d, a.kn, p.heads);
+    int rc = make_tmap(h, &tq, p.q, p.BH, p.Nq, p.d, TILE_M, p.heads, p.bf16);
+    if (rc == SD_ATTN_OK) rc = make_tmap(h, &tk, p.k, p.BH, p.Nk, p.d, a.kn, p.heads, p.bf16);
+    if (rc == SD_ATTN_OK) rc = make_tmap(h, &tv, p.v, p.BH, p.Nk, p.d, a.kn, p.heads, p.bf16);
     if (rc != SD_ATTN_OK) return rc;
     dim3 grid((p.Nq + TILE_M - 1) / TILE_M, p.BH), block(CROSS_THREADS);
-    launch_overlapped(h, cross_attention_kernel, grid, block, cross_smem_bytes(a.nch, a.kn), p.stream, tq, tk, tv, a);
+    if (p.bf16)
+        launch_overlapped(h, cross_attention_kernel<true>, grid, block, cross_smem_bytes(a.nch, a.kn), p.stream, tq, tk, tv, a);
+    else
+        launch_overlapped(h, cross_attention_kernel<false>, grid, block, cross_smem_bytes(a.nch, a.kn), p.stream, tq, tk, tv, a);
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) return cuda_fail(h, e);
     h->launches += 1;
@@ -503,6 +534,28 @@ static int launch_fused4(sd_attn_handle* h, const Problem& p) {
     if (e != cudaSuccess) return cuda_fail(h, e);
     h->launches += 1;
     return SD_ATTN_OK;
+}
+
+template <bool BF>
+static void dispatch_fused4s(sd_attn_handle* h, int split, const Fused4Args& a, dim3 grid, dim3 block, size_t smem,
+                             cudaStream_t stream, const CUtensorMap& tq, const CUtensorMap& tk, const CUtensorMap& tv) {
+    if (split == 4 && a.nch == 1)
+        launch_overlapped(h, fused4s_attention_kernel<F4S_POLY_PER8, 1, 4, BF>, grid, block, smem, stream, tq, tk, tv, a);
+    else if (split == 2 && a.nch == 1)
+        launch_overlapped(h, fused4s_attention_kernel<F4S_POLY_PER8, 1, 2, BF>, grid, block, smem, stream, tq, tk, tv, a);
+    else if (split == 2 && a.nch == 2)
+        launch_overlapped(h, fused4s_attention_kernel<F4S_POLY_PER8, 2, 2, BF>, grid, block, smem, stream, tq, tk, tv, a);
+    else if (split == 2 && a.nch == 3)
+        launch_overlapped(h, fused4s_attention_kernel<F4S_POLY_PER8, 3, 2, BF>, grid, block, smem, stream, tq, tk, tv, a);
+    // the polynomial share of the exponentials only pays where four tiles saturate the special function unit
+    else if (a.dpad <= 48)
+        launch_overlapped(h, fused4s_attention_kernel<F4S_POLY_PER8, 1, 1, BF>, grid, block, smem, stream, tq, tk, tv, a);
+    else if (a.nch == 1)
+        launch_overlapped(h, fused4s_attention_kernel<0, 1, 1, BF>, grid, block, smem, stream, tq, tk, tv, a);
+    else if (a.nch == 2)
+        launch_overlapped(h, fused4s_attention_kernel<0, 2, 1, BF>, grid, block, smem, stream, tq, tk, tv, a);
+    else
+        launch_overlapped(h, fused4s_attention_kernel<0, 3, 1, BF>, grid, block, smem, stream, tq, tk, tv, a);
 }
 
 // The spare-buffer kernel: any head dim up to 160, 1..4 query tiles per CTA.
@@ -544,9 +597,9 @@ static int launch_fused4s(sd_attn_handle* h, const Problem& p) {
     if (a.stages > F4_STAGES) a.stages = F4_STAGES;
     const size_t smem = (size_t)tile_slots * q_tile_bytes + (size_t)a.stages * stage_bytes + 1024;
     CUtensorMap tq, tk, tv;
-    int rc = make_tmap(h, &tq, p.q, p.BH, p.Nq, p.d, TILE_M, p.heads);
-    if (rc == SD_ATTN_OK) rc = make_tmap(h, &tk, p.k, p.BH, p.Nk, p.d, F4_BN, p.heads);
-    if (rc == SD_ATTN_OK) rc = make_tmap(h, &tv, p.v, p.BH, p.Nk, p.d, F4_BN, p.heads);
+    int rc = make_tmap(h, &tq, p.q, p.BH, p.Nq, p.d, TILE_M, p.heads, p.bf16);
+    if (rc == SD_ATTN_OK) rc = make_tmap(h, &tk, p.k, p.BH, p.Nk, p.d, F4_BN, p.heads, p.bf16);
+    if (rc == SD_ATTN_OK) rc = make_tmap(h, &tv, p.v, p.BH, p.Nk, p.d, F4_BN, p.heads, p.bf16);
     if (rc != SD_ATTN_OK) return rc;
     dim3 grid((tiles_per_head + a.tiles_per_cta - 1) / a.tiles_per_cta, p.BH), block(F4_THREADS);
     // One tile per CTA: its key tiles are dealt out among 4 or 2 warpgroups (parts), each with an accumulator of its
@@ -560,23 +613,10 @@ static int launch_fused4s(sd_attn_handle* h, const Problem& p) {
         a.split_buffers = (4 * F4_BN + split * a.dpad <= 512 && a.stages >= 5) ? 4 : 2;
         if (a.split_buffers < split || 2 * F4_BN + 2 * a.dpad > 512) split = 1;   // (no room: d > 192)
     }
-    if (split == 4 && a.nch == 1)
-        launch_overlapped(h, fused4s_attention_kernel<F4S_POLY_PER8, 1, 4>, grid, block, smem, p.stream, tq, tk, tv, a);
-    else if (split == 2 && a.nch == 1)
-        launch_overlapped(h, fused4s_attention_kernel<F4S_POLY_PER8, 1, 2>, grid, block, smem, p.stream, tq, tk, tv, a);
-    else if (split == 2 && a.nch == 2)
-        launch_overlapped(h, fused4s_attention_kernel<F4S_POLY_PER8, 2, 2>, grid, block, smem, p.stream, tq, tk, tv, a);
-    else if (split == 2 && a.nch == 3)
-        launch_overlapped(h, fused4s_attention_kernel<F4S_POLY_PER8, 3, 2>, grid, block, smem, p.stream, tq, tk, tv, a);
-    // the polynomial share of the exponentials only pays where four tiles saturate the special function unit
-    else if (a.dpad <= 48)
-        launch_overlapped(h, fused4s_attention_kernel<F4S_POLY_PER8, 1>, grid, block, smem, p.stream, tq, tk, tv, a);
-    else if (a.nch == 1)
-        launch_overlapped(h, fused4s_attention_kernel<0, 1>, grid, block, smem, p.stream, tq, tk, tv, a);
-    else if (a.nch == 2)
-        launch_overlapped(h, fused4s_attention_kernel<0, 2>, grid, block, smem, p.stream, tq, tk, tv, a);
+    if (p.bf16)
+        dispatch_fused4s<true>(h, split, a, grid, block, smem, p.stream, tq, tk, tv);
     else
-        launch_overlapped(h, fused4s_attention_kernel<0, 3>, grid, block, smem, p.stream, tq, tk, tv, a);
+        dispatch_fused4s<false>(h, split, a, grid, block, smem, p.stream, tq, tk, tv);
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) return cuda_fail(h, e);
     h->launches += 1;
@@ -585,7 +625,7 @@ static int launch_fused4s(sd_attn_handle* h, const Problem& p) {
 
 static int launch_fused(sd_attn_handle* h, const Problem& p) {
     if (h->fused4s_ok && !h->no_spare && !h->prefer_two_tile) return launch_fused4s(h, p);
-    if (p.heads > 0) return SD_ATTN_ERR_UNSUPPORTED;   // the earlier kernels take head-major tensors only
+    if (p.heads > 0 || p.bf16) return SD_ATTN_ERR_UNSUPPORTED;   // the earlier kernels: head-major binary16 only
     if (p.d <= F4_MAX_D && !h->prefer_two_tile && h->fused4_ok) return launch_fused4(h, p);
     FusedArgs a;
     const int bn = fused_block_n(p.d);
@@ -614,7 +654,7 @@ static int launch_fused(sd_attn_handle* h, const Problem& p) {
 }
 
 static int launch_twopass(sd_attn_handle* h, const Problem& p) {
-    if (p.heads > 0) return SD_ATTN_ERR_UNSUPPORTED;   // the comparator takes head-major tensors only
+    if (p.heads > 0 || p.bf16) return SD_ATTN_ERR_UNSUPPORTED;   // the comparator: head-major binary16 only
     const size_t need = sd_attn_workspace_bytes(SD_ATTN_MODE_TWOPASS, p.BH, 1, p.Nq, p.Nk, p.d, SD_ATTN_F16);
     if (!h->workspace || h->workspace_bytes < need) return SD_ATTN_ERR_WORKSPACE;
     const size_t rows = (size_t)p.BH * p.Nq;
@@ -647,7 +687,7 @@ extern "C" int sd_attn_forward(sd_attn_handle* h, const void* q, const void* k, 
     if (!h) return SD_ATTN_ERR_INVALID_VALUE;
     if (B <= 0 || H <= 0 || Nq < 0 || Nk <= 0 || d <= 0) return SD_ATTN_ERR_INVALID_VALUE;
     if (!isfinite(scale)) return SD_ATTN_ERR_INVALID_VALUE;
-    if (dtype != SD_ATTN_F16 && dtype != SD_ATTN_F32) return SD_ATTN_ERR_UNSUPPORTED;
+    if (dtype != SD_ATTN_F16 && dtype != SD_ATTN_F32 && dtype != SD_ATTN_BF16) return SD_ATTN_ERR_UNSUPPORTED;
     if (d > SD_ATTN_MAX_D) return SD_ATTN_ERR_UNSUPPORTED;
     if ((long long)B * H > 65535) return SD_ATTN_ERR_UNSUPPORTED;
     if (Nq == 0) return SD_ATTN_OK;
@@ -655,7 +695,7 @@ extern "C" int sd_attn_forward(sd_attn_handle* h, const void* q, const void* k, 
     if ((((uintptr_t)q | (uintptr_t)k | (uintptr_t)v | (uintptr_t)out) & 15u) != 0) return SD_ATTN_ERR_ALIGNMENT;
 
     int mode = h->mode;
-    const bool tensor_ok = (dtype == SD_ATTN_F16) && (d % 8 == 0);
+    const bool tensor_ok = (dtype == SD_ATTN_F16 || dtype == SD_ATTN_BF16) && (d % 8 == 0);
     if (mode == SD_ATTN_MODE_AUTO) {
         if (!tensor_ok) mode = SD_ATTN_MODE_SIMT;
         else mode = (Nk <= SD_ATTN_CROSS_MAX_NK) ? SD_ATTN_MODE_CROSS : SD_ATTN_MODE_FUSED;
@@ -664,11 +704,13 @@ extern "C" int sd_attn_forward(sd_attn_handle* h, const void* q, const void* k, 
     if (mode == SD_ATTN_MODE_CROSS && Nk > SD_ATTN_CROSS_MAX_NK) return SD_ATTN_ERR_UNSUPPORTED;
 
     Problem p = {q, k, v, out, B * H, Nq, Nk, d, scale, (cudaStream_t)stream,
-                 h->layout == SD_ATTN_LAYOUT_BNHD ? H : 0};
+                 h->layout == SD_ATTN_LAYOUT_BNHD ? H : 0, dtype == SD_ATTN_BF16 ? 1 : 0};
     int rc;
     switch (mode) {
         case SD_ATTN_MODE_SIMT:
-            rc = (dtype == SD_ATTN_F16) ? launch_simt<__half>(h, p) : launch_simt<float>(h, p);
+            rc = dtype == SD_ATTN_F16    ? launch_simt<__half>(h, p)
+                 : dtype == SD_ATTN_BF16 ? launch_simt<__nv_bfloat16>(h, p)
+                                         : launch_simt<float>(h, p);
             break;
         case SD_ATTN_MODE_CROSS: rc = launch_cross(h, p); break;
         case SD_ATTN_MODE_FUSED: rc = launch_fused(h, p); break;
@@ -695,7 +737,7 @@ extern "C" int sd_attn_forward_host(sd_attn_handle* h, const void* q, const void
                                     float scale, int dtype, void* stream) {
     if (!h) return SD_ATTN_ERR_INVALID_VALUE;
     if (B <= 0 || H <= 0 || Nq < 0 || Nk <= 0 || d <= 0) return SD_ATTN_ERR_INVALID_VALUE;
-    if (dtype != SD_ATTN_F16 && dtype != SD_ATTN_F32) return SD_ATTN_ERR_UNSUPPORTED;
+    if (dtype != SD_ATTN_F16 && dtype != SD_ATTN_F32 && dtype != SD_ATTN_BF16) return SD_ATTN_ERR_UNSUPPORTED;
     if (Nq == 0) return SD_ATTN_OK;
     if (!q || !k || !v || !out) return SD_ATTN_ERR_INVALID_VALUE;
     const size_t need = sd_attn_host_staging_bytes(B, H, Nq, Nk, d, dtype);

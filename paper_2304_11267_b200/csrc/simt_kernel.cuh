@@ -31,8 +31,10 @@ __host__ inline size_t simt_smem_bytes(int d) {
 
 __device__ inline float to_f32(float x) { return x; }
 __device__ inline float to_f32(__half x) { return __half2float(x); }
+__device__ inline float to_f32(__nv_bfloat16 x) { return __bfloat162float(x); }
 __device__ inline void from_f32(float* p, float x) { *p = x; }
 __device__ inline void from_f32(__half* p, float x) { *p = __float2half_rn(x); }
+__device__ inline void from_f32(__nv_bfloat16* p, float x) { *p = __float2bfloat16_rn(x); }
 
 template <typename T, int CC>  // CC = ceil(d / 32) output channels per lane
 __global__ void __launch_bounds__(SIMT_WARPS * 32)

@@ -128,8 +128,9 @@ __device__ __forceinline__ constexpr bool pair_uses_poly(int k) {
                      : (k & 1) == 0;
 }
 
-// p = exp2(s*c2 + neg_mc) for 32 scores -> 16 packed fp16 pairs; adds the 32 weights into acc[0..1].
-template <int POLY, int PAIRS = 16>
+// p = exp2(s*c2 + neg_mc) for 32 scores -> 16 packed pairs of 16-bit weights (binary16, or bfloat16 when BF);
+// adds the 32 weights into acc[0..1].
+template <int POLY, int PAIRS = 16, bool BF = false>
 __device__ __forceinline__ void exp2_pack_32(const uint32_t* s, uint64_t c2c2, uint64_t nmnm, uint32_t* packed,
                                              uint64_t* acc) {
     // the polynomial's pairs take the score itself, with the constants of the clamped form (see ex2_poly_pair)
@@ -148,19 +149,19 @@ __device__ __forceinline__ void exp2_pack_32(const uint32_t* s, uint64_t c2c2, u
             p1 = ex2_approx(__uint_as_float(x1));
         }
         acc[k & 1] = add_f32x2(acc[k & 1], pack_b64(__float_as_uint(p0), __float_as_uint(p1)));
-        packed[k] = pack_half2(p0, p1);
+        packed[k] = pack_16x2<BF>(p0, p1);
     }
 }
 
 // 16 scores -> 8 packed pairs.
-template <int POLY>
+template <int POLY, bool BF = false>
 __device__ __forceinline__ void exp2_pack_16(const uint32_t* s, uint64_t c2c2, uint64_t nmnm, uint32_t* packed,
                                              uint64_t* acc) {
-    exp2_pack_32<POLY, 8>(s, c2c2, nmnm, packed, acc);
+    exp2_pack_32<POLY, 8, BF>(s, c2c2, nmnm, packed, acc);
 }
 
 // The same for a ragged tile: scores at column >= valid get weight zero (also when the scale is zero).
-template <int PAIRS = 16>
+template <int PAIRS = 16, bool BF = false>
 __device__ __forceinline__ void exp2_pack_32_masked(const uint32_t* s, float c2, float neg_mc, int first_col, int valid,
                                                     uint32_t* packed, float& sum) {
 #pragma unroll
@@ -170,7 +171,7 @@ __device__ __forceinline__ void exp2_pack_32_masked(const uint32_t* s, float c2,
         if (first_col + 2 * k >= valid) p0 = 0.f;
         if (first_col + 2 * k + 1 >= valid) p1 = 0.f;
         sum += p0 + p1;
-        packed[k] = pack_half2(p0, p1);
+        packed[k] = pack_16x2<BF>(p0, p1);
     }
 }
 

@@ -5,6 +5,7 @@
 // Every wait in this file gives up after a fixed number of polls and reports through a status
 // block instead of spinning for ever; callers then drain and return normally.
 #pragma once
+#include <cuda_bf16.h>
 #include <cuda_fp16.h>
 #include <cuda_runtime.h>
 #include <stdint.h>
@@ -347,13 +348,13 @@ __host__ __device__ constexpr uint64_t smem_desc_sw128(uint32_t byte_addr, uint3
            ((uint64_t)((sbo_bytes >> 4) & 0x3FFFu) << 32) | (1ull << 46) | (2ull << 61);
 }
 
-// Instruction descriptor for kind::f16 with fp16 A/B and fp32 D.
-//   bits 4..5 D format (1 = f32)   bits 7..9 A format (0 = f16)   bits 10..12 B format (0 = f16)
+// Instruction descriptor for kind::f16 with fp16 (or bf16) A/B and fp32 D.
+//   bits 4..5 D format (1 = f32)   bits 7..9 A format (0 = f16, 1 = bf16)   bits 10..12 B format (likewise)
 //   bit 13 negate A   bit 14 negate B   bit 15 A is MN-major   bit 16 B is MN-major
 //   bits 17..22 N >> 3   bits 24..28 M >> 4
 __host__ __device__ constexpr uint32_t idesc_f16(int m, int n, bool a_mn_major, bool b_mn_major,
-                                                 bool negate_a) {
-    return (1u << 4) | (negate_a ? (1u << 13) : 0u) | (a_mn_major ? (1u << 15) : 0u) |
+                                                 bool negate_a, bool bf16 = false) {
+    return (1u << 4) | (bf16 ? ((1u << 7) | (1u << 10)) : 0u) | (negate_a ? (1u << 13) : 0u) | (a_mn_major ? (1u << 15) : 0u) |
            (b_mn_major ? (1u << 16) : 0u) | ((uint32_t)(n >> 3) << 17) | ((uint32_t)(m >> 4) << 24);
 }
 
@@ -380,6 +381,16 @@ __device__ __forceinline__ float ex2_poly(float x) {
 __device__ __forceinline__ uint32_t pack_half2(float lo, float hi) {
     __half2 h = __floats2half2_rn(lo, hi);  // .x (low 16 bits) = lo
     return *reinterpret_cast<uint32_t*>(&h);
+}
+// Two values rounded to the storage type of the call -- binary16, or bfloat16 when BF -- low 16 bits = lo.
+template <bool BF>
+__device__ __forceinline__ uint32_t pack_16x2(float lo, float hi) {
+    if (BF) {
+        uint32_t r;
+        asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(r) : "f"(hi), "f"(lo));
+        return r;
+    }
+    return pack_half2(lo, hi);
 }
 
 }  // namespace sd_attn
