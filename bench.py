@@ -399,6 +399,41 @@ def time_calls(att, bd, tensors, stream, iters, graph=False, dtype=None):
     return 1e3 * start.elapsed_time(end) / iters
 
 
+def time_batch(att, bd, tensors, stream, iters):
+    """Mean microseconds of one sd_attn_forward_batch call over `tensors`: plain, and replayed as a CUDA graph."""
+    import torch
+    probs = bd.make_problems([(tq.data_ptr(), tk.data_ptr(), tv.data_ptr(), to.data_ptr(), c.B, c.H, c.Nq, c.Nk, c.d,
+                               float(c.scale())) for c, tq, tk, tv, to in tensors])
+
+    def once(s):
+        rc = bd.sd_attn_forward_batch(att.handle, probs, bd.F16, s)
+        if rc != bd.OK:
+            raise bd.SdAttnError(rc, "sd_attn_forward_batch")
+    start, end = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    for _ in range(3):
+        once(stream)
+    torch.cuda.synchronize()
+    start.record()
+    for _ in range(iters):
+        once(stream)
+    end.record()
+    torch.cuda.synchronize()
+    plain = 1e3 * start.elapsed_time(end) / iters
+    side = torch.cuda.Stream()
+    g = torch.cuda.CUDAGraph()
+    with torch.cuda.stream(side):
+        with torch.cuda.graph(g, stream=side):
+            once(side.cuda_stream)
+    g.replay()
+    torch.cuda.synchronize()
+    start.record()
+    for _ in range(iters):
+        g.replay()
+    end.record()
+    torch.cuda.synchronize()
+    return plain, 1e3 * start.elapsed_time(end) / iters
+
+
 def extras(att, bd, device, stream, peaks):
     """Secondary numbers: the UNet-step attention set (32 calls) and the memory-bound cross-attention."""
     import torch
@@ -412,8 +447,13 @@ def extras(att, bd, device, stream, peaks):
     flops = sum(c.flops for c in calls)
     us = time_calls(att, bd, tensors, stream, 20)
     us_graph = time_calls(att, bd, tensors, stream, 20, graph=True)
+    us_batch, us_batch_graph = time_batch(att, bd, tensors, stream, 20)
     out["unet_step_attention_set"] = {"calls": len(calls), "us_plain_launches": us, "us_cuda_graph": us_graph,
                                       "tflops_cuda_graph": flops / (us_graph * 1e-6) / 1e12,
+                                      "us_batch_call": us_batch, "us_batch_call_cuda_graph": us_batch_graph,
+                                      "tflops_batch_call_cuda_graph": flops / (us_batch_graph * 1e-6) / 1e12,
+                                      "batch_note": "the same 32 calls as independent problems of one "
+                                                    "sd_attn_forward_batch call (spread over four streams)",
                                       "note": "512x512, B=2, H=8: 16 self + 16 cross calls (L2-warm: 285 MB of tensors)"}
     # cross-attention at the large-latent size, rotating sets so that Q/O stream from HBM
     c = workloads.config5()[2]

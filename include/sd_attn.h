@@ -76,7 +76,8 @@ typedef enum {
  * Create a handle on the CURRENT CUDA device.  Checks the architecture (ERR_ARCH unless
  * compute capability 10.x), resolves the driver's tensor-map encoder, raises the kernels'
  * dynamic shared-memory limits, allocates one 64-byte device status block and creates the two
- * copy streams and ten events sd_attn_forward_host uses.  No stream work.  *out receives the
+ * copy streams and ten events sd_attn_forward_host uses, and the three streams and four events of
+ * sd_attn_forward_batch.  No stream work.  *out receives the
  * handle (NULL on failure).
  *
  * Switches read from the environment at this call (all default off; they select slower variants that exist
@@ -92,6 +93,7 @@ typedef enum {
  *   SD_ATTN_FUSED_TWO_TILE=1    FUSED: the two-tile kernel
  *   SD_ATTN_CROSS_ONE_TILE=1    CROSS: one tile per CTA also for 65..80 keys
  *   SD_ATTN_HOST_ONE_SLICE=1    sd_attn_forward_host: one slice, copies and kernel all on the caller's stream
+ *   SD_ATTN_BATCH_ONE_LANE=1    sd_attn_forward_batch: every problem on the caller's stream, one after another
  */
 int sd_attn_create(sd_attn_handle **out);
 
@@ -108,6 +110,29 @@ int sd_attn_create(sd_attn_handle **out);
  */
 int sd_attn_forward(sd_attn_handle *h, const void *q, const void *k, const void *v, void *out,
                     int B, int H, int Nq, int Nk, int d, float scale, int dtype, void *stream);
+
+/* One problem of a batch: the arguments of sd_attn_forward. */
+typedef struct {
+    const void *q, *k, *v; /* device pointers, 16-byte aligned, in the handle's layout */
+    void *out;
+    int B, H, Nq, Nk, d;
+    float scale;
+} sd_attn_problem;
+
+/*
+ * `count` INDEPENDENT problems of Eq. 3 -- e.g. the attention calls of several UNet blocks evaluated side by side,
+ * or of several requests -- as one piece of stream-ordered work on `stream`: no problem's output may be another's
+ * input or output.  The library is free to run them at the same time: it forks three streams of its own from
+ * `stream`, gives each problem (in the order given) to the stream with the least estimated work so far and joins
+ * them back, so small problems run in the SMs that large ones leave idle.  Capturable into a CUDA graph through
+ * `stream`.  All problems share `dtype`, the handle's mode and layout; each is validated as by sd_attn_forward
+ * and the first error is returned (problems before it have been enqueued; the streams are joined in every case).
+ * In TWOPASS mode (one workspace) and with SD_ATTN_BATCH_ONE_LANE=1 in the environment at sd_attn_create the
+ * problems run one after another on `stream`.  `problems` is a HOST array, read during the call only.
+ * Errors: INVALID_VALUE (null handle, negative count, null array), then as sd_attn_forward.
+ */
+int sd_attn_forward_batch(sd_attn_handle *h, const sd_attn_problem *problems, int count, int dtype,
+                          void *stream);
 
 /*
  * The same operation (Eq. 3) for callers whose tensors live in HOST memory: q, k, v, out are HOST

@@ -28,9 +28,16 @@ EXPORTS = ["sd_attn_create", "sd_attn_forward", "sd_attn_destroy", "sd_attn_set_
            "sd_attn_workspace_bytes", "sd_attn_set_workspace", "sd_attn_twopass_buffers",
            "sd_attn_query_status", "sd_attn_last_mode", "sd_attn_launch_count", "sd_attn_status_string",
            "sd_attn_forward_host", "sd_attn_host_staging_bytes", "sd_attn_debug_dump_cross_scores",
-           "sd_attn_forward_twopass_static", "sd_geglu_forward", "sd_groupnorm_forward", "sd_attn_set_layout"]
+           "sd_attn_forward_twopass_static", "sd_geglu_forward", "sd_groupnorm_forward", "sd_attn_set_layout", "sd_attn_forward_batch"]
 
 _lib = None
+
+
+class Problem(ctypes.Structure):
+    """sd_attn_problem: one problem of sd_attn_forward_batch."""
+    _fields_ = [("q", ctypes.c_void_p), ("k", ctypes.c_void_p), ("v", ctypes.c_void_p), ("out", ctypes.c_void_p),
+                ("B", ctypes.c_int), ("H", ctypes.c_int), ("Nq", ctypes.c_int), ("Nk", ctypes.c_int),
+                ("d", ctypes.c_int), ("scale", ctypes.c_float)]
 
 
 class SdAttnError(RuntimeError):
@@ -62,6 +69,8 @@ def load() -> ctypes.CDLL:
     lib.sd_attn_destroy.argtypes = [vp]
     lib.sd_attn_set_mode.restype = ci
     lib.sd_attn_set_mode.argtypes = [vp, ci]
+    lib.sd_attn_forward_batch.restype = ci
+    lib.sd_attn_forward_batch.argtypes = [vp, ctypes.POINTER(Problem), ci, ci, vp]
     lib.sd_attn_set_layout.restype = ci
     lib.sd_attn_set_layout.argtypes = [vp, ci]
     lib.sd_attn_workspace_bytes.restype = sz
@@ -196,6 +205,21 @@ def groupnorm(x, groups: int, eps: float = 1e-5, gamma=None, beta=None, out=None
 
 def sd_attn_set_mode(handle, mode: int) -> int:
     return load().sd_attn_set_mode(handle, mode)
+
+
+def sd_attn_forward_batch(handle, problems, dtype: int, stream) -> int:
+    """problems: a ctypes array of Problem (see make_problems) or a sequence of Problem."""
+    if not isinstance(problems, ctypes.Array):
+        problems = (Problem * len(problems))(*problems)
+    return load().sd_attn_forward_batch(handle, problems, len(problems), dtype, stream or None)
+
+
+def make_problems(items):
+    """items: (q_ptr, k_ptr, v_ptr, out_ptr, B, H, Nq, Nk, d, scale) tuples -> a ctypes array of Problem."""
+    arr = (Problem * len(items))()
+    for p, it in zip(arr, items):
+        p.q, p.k, p.v, p.out, p.B, p.H, p.Nq, p.Nk, p.d, p.scale = it
+    return arr
 
 
 def sd_attn_set_layout(handle, layout: int) -> int:

@@ -43,6 +43,11 @@ struct TmapCacheEntry {
 };
 constexpr int TMAP_CACHE_ENTRIES = 128;
 
+#ifndef SD_ATTN_BATCH_LANES
+#define SD_ATTN_BATCH_LANES 3
+#endif
+constexpr int BATCH_LANES = SD_ATTN_BATCH_LANES;   // sd_attn_forward_batch spreads independent problems over the caller's stream and these
+
 constexpr int HOST_SLICES = 4;   // sd_attn_forward_host cuts the (batch, head) range into at most this many slices
 
 struct sd_attn_handle {
@@ -52,6 +57,9 @@ struct sd_attn_handle {
     int mode;
     int layout;
     int last_mode;
+    cudaStream_t batch_lane[BATCH_LANES];   // sd_attn_forward_batch: lanes beside the caller's stream
+    cudaEvent_t ev_batch_fork, ev_batch_join[BATCH_LANES];
+    int batch_lanes_ok;
     long long launches;
     int* dev_status;          // DEV_STATUS_INTS ints on the device
     void* workspace;          // caller-owned
@@ -137,6 +145,14 @@ static cudaError_t create_host_overlap(sd_attn_handle* h) {
     }
     const char* one = getenv("SD_ATTN_HOST_ONE_SLICE");
     h->host_overlap = e == cudaSuccess && !(one && one[0] == '1');
+    // the lanes of sd_attn_forward_batch
+    if (e == cudaSuccess) e = cudaEventCreateWithFlags(&h->ev_batch_fork, cudaEventDisableTiming);
+    for (int l = 0; l < BATCH_LANES && e == cudaSuccess; ++l) {
+        e = cudaStreamCreateWithFlags(&h->batch_lane[l], cudaStreamNonBlocking);
+        if (e == cudaSuccess) e = cudaEventCreateWithFlags(&h->ev_batch_join[l], cudaEventDisableTiming);
+    }
+    const char* lane = getenv("SD_ATTN_BATCH_ONE_LANE");
+    h->batch_lanes_ok = e == cudaSuccess && !(lane && lane[0] == '1');
     return e;
 }
 
@@ -150,6 +166,12 @@ static void destroy_host_overlap(sd_attn_handle* h) {   // the handle was calloc
     if (h->copy_in) cudaStreamDestroy(h->copy_in);
     if (h->copy_out) cudaStreamDestroy(h->copy_out);
     h->host_overlap = 0;
+    for (int l = 0; l < BATCH_LANES; ++l) {
+        if (h->ev_batch_join[l]) cudaEventDestroy(h->ev_batch_join[l]);
+        if (h->batch_lane[l]) cudaStreamDestroy(h->batch_lane[l]);
+    }
+    if (h->ev_batch_fork) cudaEventDestroy(h->ev_batch_fork);
+    h->batch_lanes_ok = 0;
 }
 
 // The kernels AUTO selects exist for binary16 and for bfloat16 tensors (BF); each needs its shared-memory limit raised.
@@ -721,6 +743,58 @@ extern "C" int sd_attn_forward(sd_attn_handle* h, const void* q, const void* k, 
     if (rc == SD_ATTN_OK && getenv("SD_ATTN_LOG"))
         fprintf(stderr, "[sd_attn] forward BH=%d Nq=%d Nk=%d d=%d dtype=%d -> mode %d\n", B * H, Nq, Nk, d, dtype, mode);
     return rc;
+}
+
+// A rough cost of one problem in microseconds, only to balance the lanes of a batch: a floor for the fixed part of
+// a call, tensor time at the rate the single-pass kernel reaches, memory time at the rate the cross kernel reaches.
+static double problem_cost_us(const sd_attn_problem& p, int dtype) {
+    const double bh = (double)p.B * p.H, es = dtype == SD_ATTN_F32 ? 4.0 : 2.0;
+    const double flops = 4.0 * bh * p.Nq * (double)p.Nk * p.d;
+    const double bytes = es * bh * p.d * (2.0 * p.Nq + 2.0 * p.Nk);
+    const double t = flops / 450e6, m = bytes / 2.5e6;
+    const double c = t > m ? t : m;
+    return c > 8.0 ? c : 8.0;
+}
+
+extern "C" int sd_attn_forward_batch(sd_attn_handle* h, const sd_attn_problem* problems, int count, int dtype,
+                                     void* stream) {
+    if (!h || count < 0 || (count > 0 && !problems)) return SD_ATTN_ERR_INVALID_VALUE;
+    if (count == 0) return SD_ATTN_OK;
+    cudaStream_t s = (cudaStream_t)stream;
+    // TWOPASS mode lends ONE workspace to every call: its problems run one after another
+    const bool spread = h->batch_lanes_ok && count > 1 && h->mode != SD_ATTN_MODE_TWOPASS;
+    if (!spread) {
+        for (int i = 0; i < count; ++i) {
+            const sd_attn_problem& p = problems[i];
+            const int rc = sd_attn_forward(h, p.q, p.k, p.v, p.out, p.B, p.H, p.Nq, p.Nk, p.d, p.scale, dtype, stream);
+            if (rc != SD_ATTN_OK) return rc;
+        }
+        return SD_ATTN_OK;
+    }
+    // Fork the lanes from the caller's stream, give every problem to the lane with the least work so far (in the
+    // order given), join the lanes back: for the caller one piece of stream-ordered work, capturable in a graph.
+    cudaError_t e = cudaEventRecord(h->ev_batch_fork, s);
+    for (int l = 0; l < BATCH_LANES && e == cudaSuccess; ++l) e = cudaStreamWaitEvent(h->batch_lane[l], h->ev_batch_fork, 0);
+    if (e != cudaSuccess) return cuda_fail(h, e);
+    double load[BATCH_LANES + 1] = {0};
+    int rc = SD_ATTN_OK;
+    for (int i = 0; i < count && rc == SD_ATTN_OK; ++i) {
+        const sd_attn_problem& p = problems[i];
+        int best = 0;
+        for (int l = 1; l <= BATCH_LANES; ++l)
+            if (load[l] < load[best]) best = l;
+        if (p.B > 0 && p.H > 0 && p.Nq > 0 && p.Nk > 0 && p.d > 0) load[best] += problem_cost_us(p, dtype);
+        cudaStream_t target = best == 0 ? s : h->batch_lane[best - 1];
+        rc = sd_attn_forward(h, p.q, p.k, p.v, p.out, p.B, p.H, p.Nq, p.Nk, p.d, p.scale, dtype, (void*)target);
+    }
+    // join in every case: the caller's stream must not run ahead of work that was enqueued
+    for (int l = 0; l < BATCH_LANES; ++l) {
+        cudaError_t ej = cudaEventRecord(h->ev_batch_join[l], h->batch_lane[l]);
+        if (ej == cudaSuccess) ej = cudaStreamWaitEvent(s, h->ev_batch_join[l], 0);
+        if (ej != cudaSuccess && e == cudaSuccess) e = ej;
+    }
+    if (rc != SD_ATTN_OK) return rc;
+    return e == cudaSuccess ? SD_ATTN_OK : cuda_fail(h, e);
 }
 
 static size_t round256(size_t x) { return (x + 255) & ~(size_t)255; }
