@@ -233,3 +233,66 @@ def groupnorm_forward(x: np.ndarray, groups: int, eps: float, gamma=None, beta=N
     if rc != 0:
         raise ValueError("sd_groupnorm_oracle_forward rejected its arguments")
     return y, mean, rstd
+
+
+# ---------------------------------------------------------------------------------------------------------------
+# The 3x3 convolution behind the Winograd step (Sec. 3.3).  The arithmetic lives in sd_conv_oracle.c; the cost model
+# of Table 2 is three ratios, written out below.
+
+_CONV_SRC = os.path.join(_HERE, "sd_conv_oracle.c")
+_CONV_LIB = os.path.join(_HERE, "libsd_conv_oracle.so")
+_conv_lib = None
+
+
+def build_conv(force: bool = False) -> str:
+    stale = (not os.path.exists(_CONV_LIB)) or os.path.getmtime(_CONV_LIB) < os.path.getmtime(_CONV_SRC)
+    if force or stale:
+        tmp = _CONV_LIB + ".tmp.%d" % os.getpid()
+        cmd = ["gcc", "-O2", "-std=c11", "-fopenmp", "-ffp-contract=off", "-fPIC", "-shared", "-o", tmp, _CONV_SRC, "-lm"]
+        subprocess.run(cmd, check=True, capture_output=True)
+        os.replace(tmp, _CONV_LIB)
+    return _CONV_LIB
+
+
+def _load_conv():
+    global _conv_lib
+    with _lock:
+        if _conv_lib is None:
+            lib = ctypes.CDLL(build_conv())
+            lib.sd_conv3x3_oracle_forward.restype = ctypes.c_int
+            lib.sd_conv3x3_oracle_forward.argtypes = [ctypes.c_void_p] * 4 + [ctypes.c_int64] * 5 + [ctypes.c_int]
+            _conv_lib = lib
+    return _conv_lib
+
+
+def conv3x3_forward(x: np.ndarray, w: np.ndarray, bias=None) -> np.ndarray:
+    """x: [N, H, W, C], w: [K, 3, 3, C], bias: [K] or None, all float16 or all float32 -> y [N, H, W, K] float64:
+    stride 1, zero padding 1, the filter not flipped (Sec. 3.3's convolution, by its definition)."""
+    if x.dtype == np.float16:
+        dtype = F16
+    elif x.dtype == np.float32:
+        dtype = F32
+    else:
+        raise TypeError("x must be float16 or float32")
+    if x.ndim != 4 or w.ndim != 4 or w.shape[1:3] != (3, 3) or w.shape[3] != x.shape[3] or w.dtype != x.dtype:
+        raise ValueError("x must be [N,H,W,C] and w [K,3,3,C] in the same dtype")
+    if bias is not None and (bias.dtype != x.dtype or bias.shape != (w.shape[0],)):
+        raise ValueError("bias must be [K] in x's dtype")
+    x, w = np.ascontiguousarray(x), np.ascontiguousarray(w)
+    b = np.ascontiguousarray(bias) if bias is not None else None
+    N, H, W, C = x.shape
+    K = w.shape[0]
+    y = np.empty((N, H, W, K), dtype=np.float64)
+    rc = _load_conv().sd_conv3x3_oracle_forward(x.ctypes.data, w.ctypes.data, b.ctypes.data if b is not None else None,
+                                                y.ctypes.data, N, H, W, C, K, dtype)
+    if rc != 0:
+        raise ValueError("sd_conv3x3_oracle_forward rejected its arguments")
+    return y
+
+
+def winograd_cost_model(m: int):
+    """Table 2 for an m x m output tile of a 3 x 3 filter, from the definitions: a tile of m*m outputs costs 9 m^2
+    multiplications directly and (m + 2)^2 in the transformed domain ("Flops Saving" = their ratio); the transformed
+    input holds (m + 2)^2 values per m^2 of the tensor ("Tensor"), the transformed filter (m + 2)^2 per 9 ("Weight")."""
+    t = (m + 2) ** 2
+    return 9.0 * m * m / t, t / float(m * m), t / 9.0
