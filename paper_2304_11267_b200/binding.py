@@ -28,7 +28,9 @@ EXPORTS = ["sd_attn_create", "sd_attn_forward", "sd_attn_destroy", "sd_attn_set_
            "sd_attn_workspace_bytes", "sd_attn_set_workspace", "sd_attn_twopass_buffers",
            "sd_attn_query_status", "sd_attn_last_mode", "sd_attn_launch_count", "sd_attn_status_string",
            "sd_attn_forward_host", "sd_attn_host_staging_bytes", "sd_attn_debug_dump_cross_scores",
-           "sd_attn_forward_twopass_static", "sd_geglu_forward", "sd_groupnorm_forward", "sd_attn_set_layout", "sd_attn_forward_batch"]
+           "sd_attn_forward_twopass_static", "sd_geglu_forward", "sd_groupnorm_forward", "sd_attn_set_layout", "sd_attn_forward_batch",
+           "sd_winograd_filter_elems", "sd_winograd_transform_filter", "sd_winograd_workspace_bytes",
+           "sd_winograd_conv3x3_forward", "sd_winograd_query_status"]
 
 _lib = None
 
@@ -71,6 +73,16 @@ def load() -> ctypes.CDLL:
     lib.sd_attn_set_mode.argtypes = [vp, ci]
     lib.sd_attn_forward_batch.restype = ci
     lib.sd_attn_forward_batch.argtypes = [vp, ctypes.POINTER(Problem), ci, ci, vp]
+    lib.sd_winograd_filter_elems.restype = sz
+    lib.sd_winograd_filter_elems.argtypes = [ci, ci]
+    lib.sd_winograd_transform_filter.restype = ci
+    lib.sd_winograd_transform_filter.argtypes = [vp, vp, ci, ci, vp]
+    lib.sd_winograd_workspace_bytes.restype = sz
+    lib.sd_winograd_workspace_bytes.argtypes = [ci, ci, ci, ci, ci]
+    lib.sd_winograd_conv3x3_forward.restype = ci
+    lib.sd_winograd_conv3x3_forward.argtypes = [vp, vp, vp, vp, vp, sz, ci, ci, ci, ci, ci, vp]
+    lib.sd_winograd_query_status.restype = ci
+    lib.sd_winograd_query_status.argtypes = [vp, ctypes.POINTER(ci)]
     lib.sd_attn_set_layout.restype = ci
     lib.sd_attn_set_layout.argtypes = [vp, ci]
     lib.sd_attn_workspace_bytes.restype = sz
@@ -201,6 +213,65 @@ def groupnorm(x, groups: int, eps: float = 1e-5, gamma=None, beta=None, out=None
     if rc != OK:
         raise SdAttnError(rc, "sd_groupnorm_forward")
     return out
+
+
+def sd_winograd_filter_elems(K: int, C: int) -> int:
+    return int(load().sd_winograd_filter_elems(K, C))
+
+
+def sd_winograd_transform_filter(w, U, K, C, stream) -> int:
+    return load().sd_winograd_transform_filter(w or None, U or None, K, C, stream or None)
+
+
+def sd_winograd_workspace_bytes(N, H, W, C, K) -> int:
+    return int(load().sd_winograd_workspace_bytes(N, H, W, C, K))
+
+
+def sd_winograd_conv3x3_forward(x, U, bias, y, workspace, workspace_bytes, N, H, W, C, K, stream) -> int:
+    return load().sd_winograd_conv3x3_forward(x or None, U or None, bias or None, y or None, workspace or None,
+                                              workspace_bytes, N, H, W, C, K, stream or None)
+
+
+def sd_winograd_query_status(stream=0):
+    detail = (ctypes.c_int * 4)()
+    rc = load().sd_winograd_query_status(stream or None, detail)
+    return rc, list(detail)
+
+
+class WinogradConv3x3:
+    """A layer's transformed filter plus torch-tensor marshalling: ``WinogradConv3x3(w, bias)(x)`` with
+    w [K,3,3,C], bias [K] or None, x [N,H,W,C] float16 CUDA tensors (channels-last memory) -> y [N,H,W,K]."""
+
+    def __init__(self, w, bias=None, stream: Optional[int] = None):
+        import torch
+        if not (w.is_cuda and w.dtype == torch.float16 and w.is_contiguous() and w.dim() == 4 and w.shape[1:3] == (3, 3)):
+            raise ValueError("w must be a contiguous float16 CUDA tensor [K,3,3,C]")
+        self.K, self.C = int(w.shape[0]), int(w.shape[3])
+        self.bias = bias.contiguous() if bias is not None else None
+        self.U = torch.empty(sd_winograd_filter_elems(self.K, self.C), dtype=torch.float16, device=w.device)
+        s = stream if stream is not None else torch.cuda.current_stream(w.device).cuda_stream
+        rc = sd_winograd_transform_filter(w.data_ptr(), self.U.data_ptr(), self.K, self.C, s)
+        if rc != OK:
+            raise SdAttnError(rc, "sd_winograd_transform_filter")
+        self._workspace = None
+
+    def __call__(self, x, out=None, stream: Optional[int] = None):
+        import torch
+        if not (x.is_cuda and x.dtype == torch.float16 and x.is_contiguous() and x.dim() == 4 and x.shape[3] == self.C):
+            raise ValueError("x must be a contiguous float16 CUDA tensor [N,H,W,%d]" % self.C)
+        N, H, W, _ = (int(v) for v in x.shape)
+        need = sd_winograd_workspace_bytes(N, H, W, self.C, self.K)
+        if self._workspace is None or self._workspace.numel() < need:
+            self._workspace = torch.empty(max(need, 256), dtype=torch.uint8, device=x.device)
+        if out is None:
+            out = torch.empty(N, H, W, self.K, dtype=torch.float16, device=x.device)
+        s = stream if stream is not None else torch.cuda.current_stream(x.device).cuda_stream
+        rc = sd_winograd_conv3x3_forward(x.data_ptr(), self.U.data_ptr(),
+                                         self.bias.data_ptr() if self.bias is not None else 0, out.data_ptr(),
+                                         self._workspace.data_ptr(), self._workspace.numel(), N, H, W, self.C, self.K, s)
+        if rc != OK:
+            raise SdAttnError(rc, "sd_winograd_conv3x3_forward")
+        return out
 
 
 def sd_attn_set_mode(handle, mode: int) -> int:

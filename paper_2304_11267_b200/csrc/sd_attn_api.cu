@@ -15,10 +15,12 @@
 #include "../../include/sd_attn_debug.h"
 #include "../../include/sd_geglu.h"
 #include "../../include/sd_groupnorm.h"
+#include "../../include/sd_winograd.h"
 #include "cross_kernel.cuh"
 #include "cross2_kernel.cuh"
 #include "geglu_kernel.cuh"
 #include "groupnorm_kernel.cuh"
+#include "winograd_kernel.cuh"
 #include "fused_kernel.cuh"
 #include "fused4_kernel.cuh"
 #include "fused4s_kernel.cuh"
@@ -1076,4 +1078,147 @@ extern "C" int sd_groupnorm_forward(const void* x, const void* gamma, const void
         groupnorm_streaming_kernel<float><<<blocks, GN_THREADS, 0, s>>>(a);
     e = cudaGetLastError();
     return e == cudaSuccess ? SD_ATTN_OK : cuda_fail(nullptr, e);
+}
+
+// ------------------------------------------------------------------------------------------------
+// Winograd F(4x4, 3x3) convolution (Sec. 3.3): stateless; filter transform once, then input transform, 36 GEMMs on
+// the tensor cores and output transform per call.
+static __device__ __align__(256) int g_winograd_status[DEV_STATUS_INTS];
+static std::mutex g_wg_mutex;
+struct WinogradDeviceState {
+    int ready;
+    int* status;
+    encode_tiled_fn encode_tiled;
+};
+static WinogradDeviceState g_wg_state[STATIC_MAX_DEVICES];
+
+static int winograd_setup(WinogradDeviceState** out) {
+    int dev = 0, major = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e == cudaSuccess) e = cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev);
+    if (e != cudaSuccess) return cuda_fail(nullptr, e);
+    if (major != 10) return SD_ATTN_ERR_ARCH;
+    if (dev < 0 || dev >= STATIC_MAX_DEVICES) return SD_ATTN_ERR_UNSUPPORTED;
+    WinogradDeviceState* st = &g_wg_state[dev];
+    std::lock_guard<std::mutex> lock(g_wg_mutex);
+    if (!st->ready) {
+        void* status = nullptr;
+        e = cudaGetSymbolAddress(&status, g_winograd_status);
+        if (e != cudaSuccess || !status) return cuda_fail(nullptr, e != cudaSuccess ? e : cudaErrorUnknown);
+        void* fn = nullptr;
+        cudaDriverEntryPointQueryResult qres;
+        e = cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres);
+        if (e != cudaSuccess || qres != cudaDriverEntryPointSuccess || !fn)
+            return cuda_fail(nullptr, e != cudaSuccess ? e : cudaErrorUnknown);
+        e = raise_smem_limit(winograd_gemm_kernel, winograd_gemm_smem_bytes(256, WG_MAX_STAGES));
+        if (e == cudaSuccess) e = cudaMemset(status, 0, sizeof(int) * DEV_STATUS_INTS);
+        if (e != cudaSuccess) return cuda_fail(nullptr, e);
+        st->status = (int*)status;
+        st->encode_tiled = (encode_tiled_fn)fn;
+        st->ready = 1;
+    }
+    *out = st;
+    return SD_ATTN_OK;
+}
+
+extern "C" size_t sd_winograd_filter_elems(int K, int C) {
+    return (K > 0 && C > 0) ? (size_t)WG_XI * (size_t)K * (size_t)C : 0;
+}
+
+static long long winograd_tiles(int N, int H, int W) {
+    return (long long)N * ((H + WG_TILE - 1) / WG_TILE) * ((W + WG_TILE - 1) / WG_TILE);
+}
+
+extern "C" size_t sd_winograd_workspace_bytes(int N, int H, int W, int C, int K) {
+    if (N <= 0 || H <= 0 || W <= 0 || C <= 0 || K <= 0) return 0;
+    const size_t T = (size_t)winograd_tiles(N, H, W);
+    return round256((size_t)WG_XI * T * C * sizeof(__half)) + round256((size_t)WG_XI * T * K * sizeof(float));
+}
+
+extern "C" int sd_winograd_transform_filter(const void* w, void* U, int K, int C, void* stream) {
+    if (!w || !U || K <= 0 || C <= 0) return SD_ATTN_ERR_INVALID_VALUE;
+    if (K % 8 != 0 || C % 8 != 0) return SD_ATTN_ERR_UNSUPPORTED;
+    if (((uintptr_t)w & 15u) || ((uintptr_t)U & 15u)) return SD_ATTN_ERR_ALIGNMENT;
+    WinogradDeviceState* st = nullptr;
+    const int rc = winograd_setup(&st);
+    if (rc != SD_ATTN_OK) return rc;
+    const long long n = (long long)K * C;
+    winograd_filter_kernel<<<(unsigned)((n + 255) / 256), 256, 0, (cudaStream_t)stream>>>((const __half*)w, (__half*)U, K, C);
+    const cudaError_t e = cudaGetLastError();
+    return e == cudaSuccess ? SD_ATTN_OK : cuda_fail(nullptr, e);
+}
+
+// A [36][rows][C] fp16 scratch plane seen by the TMA as (x = C, y = rows, z = 36): tiles of 64 columns by box_rows.
+static CUresult winograd_tmap(encode_tiled_fn enc, CUtensorMap* map, const void* base, long long rows, int C, int box_rows) {
+    cuuint64_t dims[3] = {(cuuint64_t)C, (cuuint64_t)rows, (cuuint64_t)WG_XI};
+    cuuint64_t strides[2] = {(cuuint64_t)C * 2, (cuuint64_t)rows * C * 2};
+    cuuint32_t box[3] = {(cuuint32_t)CHUNK_COLS, (cuuint32_t)box_rows, 1};
+    cuuint32_t estr[3] = {1, 1, 1};
+    return enc(map, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 3, const_cast<void*>(base), dims, strides, box, estr,
+               CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+}
+
+extern "C" int sd_winograd_conv3x3_forward(const void* x, const void* U, const void* bias, void* y, void* workspace,
+                                           size_t workspace_bytes, int N, int H, int W, int C, int K, void* stream) {
+    if (N < 0 || H <= 0 || W <= 0 || C <= 0 || K <= 0) return SD_ATTN_ERR_INVALID_VALUE;
+    if (C % 8 != 0 || K % 8 != 0) return SD_ATTN_ERR_UNSUPPORTED;
+    if (N == 0) return SD_ATTN_OK;
+    if (!x || !U || !y) return SD_ATTN_ERR_INVALID_VALUE;
+    if (((uintptr_t)x & 15u) || ((uintptr_t)U & 15u) || ((uintptr_t)y & 15u) || ((uintptr_t)bias & 3u))
+        return SD_ATTN_ERR_ALIGNMENT;
+    const long long T = winograd_tiles(N, H, W);
+    // (tile indices are ints; the transform grids are T * C / 256 and T * K / 256 blocks)
+    if (T > 2147483647ll || T * (C > K ? C : K) / 256 > 2147483647ll) return SD_ATTN_ERR_UNSUPPORTED;
+    const size_t need = sd_winograd_workspace_bytes(N, H, W, C, K);
+    if (!workspace || workspace_bytes < need || ((uintptr_t)workspace & 255u)) return SD_ATTN_ERR_WORKSPACE;
+    WinogradDeviceState* st = nullptr;
+    int rc = winograd_setup(&st);
+    if (rc != SD_ATTN_OK) return rc;
+
+    WinogradArgs a;
+    a.N = N; a.H = H; a.W = W; a.C = C; a.K = K;
+    a.tiles_y = (H + WG_TILE - 1) / WG_TILE;
+    a.tiles_x = (W + WG_TILE - 1) / WG_TILE;
+    a.T = (int)T;
+    const int chunks = (K + 255) / 256;
+    a.n_chunk = ((K + chunks - 1) / chunks + 15) / 16 * 16;
+    a.tmem_cols = next_pow2_cols(a.n_chunk);
+    a.stages = WG_MAX_STAGES;
+    a.status = st->status;
+    __half* V = (__half*)workspace;
+    float* M = (float*)((char*)workspace + round256((size_t)WG_XI * T * C * sizeof(__half)));
+    CUtensorMap tv, tu;
+    if (winograd_tmap(st->encode_tiled, &tv, V, T, C, TILE_M) != CUDA_SUCCESS ||
+        winograd_tmap(st->encode_tiled, &tu, U, K, C, a.n_chunk) != CUDA_SUCCESS)
+        return SD_ATTN_ERR_CUDA;
+    cudaStream_t s = (cudaStream_t)stream;
+    const long long in_threads = T * (C / 2), out_threads = T * (K / 2);
+    winograd_input_kernel<<<(unsigned)((in_threads + 127) / 128), 128, 0, s>>>((const __half*)x, V, a);
+    cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess) return cuda_fail(nullptr, e);
+    dim3 grid((unsigned)((T + TILE_M - 1) / TILE_M), (unsigned)chunks, WG_XI);
+    winograd_gemm_kernel<<<grid, WG_THREADS, winograd_gemm_smem_bytes(a.n_chunk, a.stages), s>>>(tv, tu, M, a);
+    e = cudaGetLastError();
+    if (e != cudaSuccess) return cuda_fail(nullptr, e);
+    winograd_output_kernel<<<(unsigned)((out_threads + 127) / 128), 128, 0, s>>>(M, (const __half*)bias, (__half*)y, a);
+    e = cudaGetLastError();
+    return e == cudaSuccess ? SD_ATTN_OK : cuda_fail(nullptr, e);
+}
+
+extern "C" int sd_winograd_query_status(void* stream, int* detail) {
+    WinogradDeviceState* st = nullptr;
+    const int rc = winograd_setup(&st);
+    if (rc != SD_ATTN_OK) return rc;
+    int host[DEV_STATUS_INTS];
+    cudaError_t e = cudaStreamSynchronize((cudaStream_t)stream);
+    if (e == cudaSuccess) e = cudaMemcpy(host, st->status, sizeof(host), cudaMemcpyDeviceToHost);
+    if (e != cudaSuccess) return cuda_fail(nullptr, e);
+    if (detail) memcpy(detail, host, 4 * sizeof(int));
+    if (host[0] != 0) {
+        e = cudaMemset(st->status, 0, sizeof(host));
+        if (e != cudaSuccess) return cuda_fail(nullptr, e);
+        return SD_ATTN_ERR_DEVICE_TIMEOUT;
+    }
+    return SD_ATTN_OK;
 }

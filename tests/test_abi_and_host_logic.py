@@ -26,7 +26,7 @@ def declared_functions():
     for header in sorted(glob.glob(os.path.join(ROOT, "include", "*.h"))):
         text = open(header).read()
         text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
-        names += re.findall(r"\b(sd_(?:attn|geglu|groupnorm)_[a-z_0-9]+)\s*\(", text)
+        names += re.findall(r"\b(sd_(?:attn|geglu|groupnorm|winograd)_[a-z_0-9]+)\s*\(", text)
     return sorted(set(names))
 
 
