@@ -220,6 +220,18 @@ def run_ours(args):
         torch.cuda.synchronize()
         print(json.dumps({"kernel_loop_only": True, "workload": "groupnorm", "launches": max(args.warmup, 3) + args.steps}))
         return 0
+    if args.workload == "winograd":
+        N, H, W, C, K = WG_SHAPE
+        g = torch.Generator(device=device).manual_seed(11)
+        w = (torch.randn(K, 3, 3, C, device=device, generator=g) / (9.0 * C) ** 0.5).to(torch.float16)
+        layer = bd.WinogradConv3x3(w, None, stream)
+        xs = [torch.randn(N, H, W, C, device=device, generator=g).to(torch.float16) for _ in range(4)]
+        y = torch.empty(N, H, W, K, device=device, dtype=torch.float16)
+        for i in range(max(args.warmup, 3) + args.steps):
+            layer(xs[i % 4], out=y, stream=stream)
+        torch.cuda.synchronize()
+        print(json.dumps({"kernel_loop_only": True, "workload": "winograd", "launches": 3 * (max(args.warmup, 3) + args.steps)}))
+        return 0
     if args.workload == "geglu":
         sets = geglu_sets(device, 4)
         for i in range(max(args.warmup, 3) + args.steps):
@@ -493,9 +505,64 @@ def extras(att, bd, device, stream, peaks):
     out["bf16_self_attention_4096_d40"] = {"us_per_call": us_bf16, "tflops": c2.flops / (us_bf16 * 1e-6) / 1e12,
                                            "note": "dtype SD_ATTN_BF16, rotating through 8 sets (168 MB)"}
     del bsets
+    out["winograd_conv3x3_2x64x64x320_f16"] = winograd_numbers(bd, device, stream, peaks)
     out["geglu_8192x1280_f16"] = geglu_numbers(bd, device, stream, peaks)
     out["groupnorm_2x320x64x64_f16"] = groupnorm_numbers(bd, device, stream, peaks)
     return out
+
+
+WG_SHAPE = (2, 64, 64, 320, 320)      # N, H, W, C, K: a 3x3 convolution of the UNet's 64 x 64 level at 512 x 512, batch 2
+
+
+def winograd_numbers(bd, device, stream, peaks):
+    """The Winograd 3x3 convolution (Sec. 3.3) on one UNet layer shape: microseconds per call (input transform, 36
+    GEMMs, output transform), the rate in terms of the direct convolution's FLOPs, and the oracle on a sample."""
+    import torch
+    import oracle
+    N, H, W, C, K = WG_SHAPE
+    g = torch.Generator(device=device).manual_seed(11)
+    w = (torch.randn(K, 3, 3, C, device=device, generator=g) / (9.0 * C) ** 0.5).to(torch.float16)
+    b = (0.1 * torch.randn(K, device=device, generator=g)).to(torch.float16)
+    layer = bd.WinogradConv3x3(w, b, stream)
+    n_sets = 16       # 16 x (5.2 MB in + 5.2 MB out): with the 7.4 MB filter and 35 MB of scratch, more than the L2
+    xs = [torch.randn(N, H, W, C, device=device, generator=g).to(torch.float16) for _ in range(n_sets)]
+    ys = [torch.empty(N, H, W, K, device=device, dtype=torch.float16) for _ in range(n_sets)]
+    for i in range(4):
+        layer(xs[i], out=ys[i], stream=stream)
+    torch.cuda.synchronize()
+    start, end = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    iters = 48
+    start.record()
+    for i in range(iters):
+        layer(xs[i % n_sets], out=ys[i % n_sets], stream=stream)
+    end.record()
+    torch.cuda.synchronize()
+    rc, detail = bd.sd_winograd_query_status(stream)
+    if rc != bd.OK:
+        raise bd.SdAttnError(rc, "winograd device status %s" % detail)
+    us = 1e3 * start.elapsed_time(end) / iters
+    direct_flops = 2.0 * N * H * W * K * C * 9
+    tiles = N * ((H + 3) // 4) * ((W + 3) // 4)
+    gemm_flops = 2.0 * 36 * tiles * K * C
+    io_bytes = 2.0 * (N * H * W * C + N * H * W * K + 36 * K * C)
+    # the oracle, timed on the first rows of the first image (a few seconds of CPU work)
+    hs, ws_ = 9, 64
+    x0 = xs[0][:1, :hs + 1].cpu().numpy()
+    t0 = time.perf_counter()
+    ref = oracle.conv3x3_forward(x0, w.cpu().numpy(), b.cpu().numpy())[:, :hs]
+    cpu_s = time.perf_counter() - t0
+    got = ys[0][:1, :hs].cpu().numpy().astype("float64")
+    rel = float(((got - ref) ** 2).sum() ** 0.5 / ((ref ** 2).sum() ** 0.5))
+    return {"us_per_call": us, "launches_per_call": 3,
+            "direct_conv_tflops_equivalent": direct_flops / (us * 1e-6) / 1e12,
+            "gemm_tflops": gemm_flops / (us * 1e-6) / 1e12,
+            "bound": "hbm", "algorithmic_bytes": io_bytes, "achieved_gbs": io_bytes / (us * 1e-6) / 1e9,
+            "peak_gbs": peaks["hbm_gbs"], "frac": io_bytes / (us * 1e-6) / 1e9 / peaks["hbm_gbs"],
+            "peak_source": peaks["source"],
+            "note": "x + y + transformed filter are the algorithmic bytes; V and M (35 MB) go through the L2",
+            "rel_l2_vs_oracle_on_sample": rel,
+            "cpu_oracle_gflops": 2.0 * 1 * (hs + 1) * ws_ * K * C * 9 / cpu_s / 1e9,
+            "cpu_oracle_sample": "%d of %d rows of one image" % (hs + 1, H)}
 
 
 GN_SHAPE, GN_GROUPS, GN_EPS = (2, 320, 64, 64), 32, 1e-5      # the 64 x 64 level of the UNet at 512 x 512, batch 2
@@ -649,7 +716,7 @@ def main():
     ap.add_argument("--steps", type=int, default=200)
     ap.add_argument("--warmup", type=int, default=10)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--workload", default="c2", choices=["c2", "c5-cross", "c3-cross", "c4", "c4-d80", "c1", "c1-twopass", "geglu", "groupnorm"],
+    ap.add_argument("--workload", default="c2", choices=["c2", "c5-cross", "c3-cross", "c4", "c4-d80", "c1", "c1-twopass", "geglu", "groupnorm", "winograd"],
                     help="with --kernel-loop-only: which calls the loop runs (the bench line is always c2)")
     ap.add_argument("--kernel-loop-only", action="store_true",
                     help="run only the warm-up and the timed loop (for ncu captures)")

@@ -115,8 +115,8 @@ static int cuda_fail(sd_attn_handle* h, cudaError_t e) {
 // kernel of the stream is still running and waits for it (griddepcontrol.wait) before it touches global memory.
 // Only the kernels that contain that wait are launched this way.
 template <typename... KArgs, typename... Args>
-static cudaError_t launch_overlapped(const sd_attn_handle* h, void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem,
-                                     cudaStream_t stream, Args&&... args) {
+static cudaError_t launch_overlapped_if(bool overlap, void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem,
+                                        cudaStream_t stream, Args&&... args) {
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = grid;
     cfg.blockDim = block;
@@ -126,8 +126,13 @@ static cudaError_t launch_overlapped(const sd_attn_handle* h, void (*kernel)(KAr
     attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
-    cfg.numAttrs = h->no_pdl ? 0 : 1;
+    cfg.numAttrs = overlap ? 1 : 0;
     return cudaLaunchKernelEx(&cfg, kernel, KArgs(args)...);
+}
+template <typename... KArgs, typename... Args>
+static cudaError_t launch_overlapped(const sd_attn_handle* h, void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem,
+                                     cudaStream_t stream, Args&&... args) {
+    return launch_overlapped_if(!h->no_pdl, kernel, grid, block, smem, stream, static_cast<Args&&>(args)...);
 }
 
 template <typename K>
@@ -1184,7 +1189,8 @@ extern "C" int sd_winograd_conv3x3_forward(const void* x, const void* U, const v
     const int chunks = (K + 255) / 256;
     a.n_chunk = ((K + chunks - 1) / chunks + 15) / 16 * 16;
     a.tmem_cols = next_pow2_cols(a.n_chunk);
-    a.stages = WG_MAX_STAGES;
+    // two CTAs per SM (shared memory and the 512 columns of tensor memory allow it): one's epilogue under the other's loads
+    a.stages = wg_stage_bytes(a.n_chunk) > 37 * 1024 ? 2 : 3;
     a.status = st->status;
     __half* V = (__half*)workspace;
     float* M = (float*)((char*)workspace + round256((size_t)WG_XI * T * C * sizeof(__half)));
@@ -1193,16 +1199,20 @@ extern "C" int sd_winograd_conv3x3_forward(const void* x, const void* U, const v
         winograd_tmap(st->encode_tiled, &tu, U, K, C, a.n_chunk) != CUDA_SUCCESS)
         return SD_ATTN_ERR_CUDA;
     cudaStream_t s = (cudaStream_t)stream;
-    const long long in_threads = T * (C / 2), out_threads = T * (K / 2);
-    winograd_input_kernel<<<(unsigned)((in_threads + 127) / 128), 128, 0, s>>>((const __half*)x, V, a);
-    cudaError_t e = cudaGetLastError();
+    const long long in_threads = T * (C / 4), out_threads = T * (K / 2);
+    // Each of the three kernels lets the next one of the stream start its set-up early and waits for its
+    // predecessor to complete before it touches global memory (SD_ATTN_NO_PDL=1: ordinary launches).
+    const char* npd = getenv("SD_ATTN_NO_PDL");
+    const bool overlap = !(npd && npd[0] == '1');
+    cudaError_t e = launch_overlapped_if(overlap, winograd_input_kernel, dim3((unsigned)((in_threads + 127) / 128)), dim3(128), 0, s,
+                                         (const __half*)x, V, a);
     if (e != cudaSuccess) return cuda_fail(nullptr, e);
     dim3 grid((unsigned)((T + TILE_M - 1) / TILE_M), (unsigned)chunks, WG_XI);
-    winograd_gemm_kernel<<<grid, WG_THREADS, winograd_gemm_smem_bytes(a.n_chunk, a.stages), s>>>(tv, tu, M, a);
-    e = cudaGetLastError();
+    e = launch_overlapped_if(overlap, winograd_gemm_kernel, grid, dim3(WG_THREADS), winograd_gemm_smem_bytes(a.n_chunk, a.stages), s,
+                             tv, tu, M, a);
     if (e != cudaSuccess) return cuda_fail(nullptr, e);
-    winograd_output_kernel<<<(unsigned)((out_threads + 127) / 128), 128, 0, s>>>(M, (const __half*)bias, (__half*)y, a);
-    e = cudaGetLastError();
+    e = launch_overlapped_if(overlap, winograd_output_kernel, dim3((unsigned)((out_threads + 127) / 128)), dim3(128), 0, s,
+                             (const float*)M, (const __half*)bias, (__half*)y, a);
     return e == cudaSuccess ? SD_ATTN_OK : cuda_fail(nullptr, e);
 }
 

@@ -95,52 +95,66 @@ struct WinogradArgs {
     int* status;
 };
 
-// x [N][H][W][C] fp16 -> V [36][T][C] fp16; one thread per (tile, channel pair).
+// x [N][H][W][C] fp16 -> V [36][T][C] fp16; one thread per (tile, four channels): 8-byte loads and stores.
 __global__ void __launch_bounds__(128) winograd_input_kernel(const __half* __restrict__ x, __half* __restrict__ V,
                                                              const WinogradArgs a) {
-    const int cp = a.C >> 1;
+    pdl_launch_dependents();   // the next kernel of the stream may start its set-up
+    pdl_wait();                // x may come from the previous kernel of the stream; V may still be read by it
+    const int cq = a.C >> 2;
     const long long idx = (long long)blockIdx.x * blockDim.x + threadIdx.x;
-    if (idx >= (long long)a.T * cp) return;
-    const int t = (int)(idx / cp), c = (int)(idx - (long long)t * cp) * 2;
+    if (idx >= (long long)a.T * cq) return;
+    const int t = (int)(idx / cq), c = (int)(idx - (long long)t * cq) * 4;
     const int n = t / (a.tiles_y * a.tiles_x), ty = (t / a.tiles_x) % a.tiles_y, tx = t % a.tiles_x;
     const int i0 = ty * WG_TILE - 1, j0 = tx * WG_TILE - 1;
-    float2 d[6][6];
+    float d[6][6][4];
 #pragma unroll
     for (int r = 0; r < 6; ++r)
 #pragma unroll
         for (int s = 0; s < 6; ++s) {
             const int i = i0 + r, j = j0 + s;
-            float2 v = make_float2(0.f, 0.f);
+            uint2 raw = make_uint2(0u, 0u);
             if (i >= 0 && i < a.H && j >= 0 && j < a.W)
-                v = __half22float2(*reinterpret_cast<const __half2*>(x + (((long long)n * a.H + i) * a.W + j) * a.C + c));
-            d[r][s] = v;
+                raw = __ldg(reinterpret_cast<const uint2*>(x + (((long long)n * a.H + i) * a.W + j) * a.C + c));
+            const float2 lo = __half22float2(*reinterpret_cast<const __half2*>(&raw.x));
+            const float2 hi = __half22float2(*reinterpret_cast<const __half2*>(&raw.y));
+            d[r][s][0] = lo.x; d[r][s][1] = lo.y; d[r][s][2] = hi.x; d[r][s][3] = hi.y;
         }
 #pragma unroll
-    for (int s = 0; s < 6; ++s) {   // B^T d: down the columns
-        const float cx[6] = {d[0][s].x, d[1][s].x, d[2][s].x, d[3][s].x, d[4][s].x, d[5][s].x};
-        const float cy[6] = {d[0][s].y, d[1][s].y, d[2][s].y, d[3][s].y, d[4][s].y, d[5][s].y};
-        float ox[6], oy[6];
-        wg_bt(cx, ox);
-        wg_bt(cy, oy);
+    for (int e = 0; e < 4; ++e) {
 #pragma unroll
-        for (int r = 0; r < 6; ++r) d[r][s] = make_float2(ox[r], oy[r]);
+        for (int s = 0; s < 6; ++s) {   // B^T d: down the columns
+            const float col[6] = {d[0][s][e], d[1][s][e], d[2][s][e], d[3][s][e], d[4][s][e], d[5][s][e]};
+            float o[6];
+            wg_bt(col, o);
+#pragma unroll
+            for (int r = 0; r < 6; ++r) d[r][s][e] = o[r];
+        }
+#pragma unroll
+        for (int r = 0; r < 6; ++r) {   // (B^T d) B: along the rows
+            const float row[6] = {d[r][0][e], d[r][1][e], d[r][2][e], d[r][3][e], d[r][4][e], d[r][5][e]};
+            float o[6];
+            wg_bt(row, o);
+#pragma unroll
+            for (int s = 0; s < 6; ++s) d[r][s][e] = o[s];
+        }
     }
 #pragma unroll
-    for (int r = 0; r < 6; ++r) {   // (B^T d) B: along the rows
-        const float rx[6] = {d[r][0].x, d[r][1].x, d[r][2].x, d[r][3].x, d[r][4].x, d[r][5].x};
-        const float ry[6] = {d[r][0].y, d[r][1].y, d[r][2].y, d[r][3].y, d[r][4].y, d[r][5].y};
-        float ox[6], oy[6];
-        wg_bt(rx, ox);
-        wg_bt(ry, oy);
+    for (int r = 0; r < 6; ++r)
 #pragma unroll
-        for (int s = 0; s < 6; ++s)
-            *reinterpret_cast<__half2*>(V + ((long long)(r * 6 + s) * a.T + t) * a.C + c) = __floats2half2_rn(ox[s], oy[s]);
-    }
+        for (int s = 0; s < 6; ++s) {
+            const __half2 lo = __floats2half2_rn(d[r][s][0], d[r][s][1]), hi = __floats2half2_rn(d[r][s][2], d[r][s][3]);
+            uint2 raw;
+            raw.x = *reinterpret_cast<const uint32_t*>(&lo);
+            raw.y = *reinterpret_cast<const uint32_t*>(&hi);
+            *reinterpret_cast<uint2*>(V + ((long long)(r * 6 + s) * a.T + t) * a.C + c) = raw;
+        }
 }
 
 // M [36][T][K] fp32 -> y [N][H][W][K] fp16 (+ bias); one thread per (tile, output channel pair).
 __global__ void __launch_bounds__(128) winograd_output_kernel(const float* __restrict__ M, const __half* __restrict__ bias,
                                                               __half* __restrict__ y, const WinogradArgs a) {
+    pdl_launch_dependents();
+    pdl_wait();                // M is complete once the GEMM kernel has finished
     const int kp = a.K >> 1;
     const long long idx = (long long)blockIdx.x * blockDim.x + threadIdx.x;
     if (idx >= (long long)a.T * kp) return;
@@ -206,6 +220,7 @@ winograd_gemm_kernel(const __grid_constant__ CUtensorMap tmap_v, const __grid_co
     __shared__ int abort_flag;
 
     const int tid = threadIdx.x, warp = tid >> 5;
+    if (tid == 0) pdl_launch_dependents();
     const int t0 = blockIdx.x * TILE_M, k0 = blockIdx.y * args.n_chunk, xi = blockIdx.z;
     const int n_chunk = args.n_chunk, stages = args.stages;
     const int c_steps = (args.C + CHUNK_COLS - 1) / CHUNK_COLS;
@@ -230,6 +245,9 @@ winograd_gemm_kernel(const __grid_constant__ CUtensorMap tmap_v, const __grid_co
     tc_fence_before_sync();
     __syncthreads();
     tc_fence_after_sync();
+    // Set-up (barriers, tensor memory) overlapped the tail of the input transform; V is complete, and M free to be
+    // overwritten, once that kernel -- which itself waited for the previous call's output transform -- has finished.
+    pdl_wait();
     const uint32_t tmem_d = tmem_base_slot;
     volatile int* abort_p = &abort_flag;
 
