@@ -1115,7 +1115,7 @@ static int winograd_setup(WinogradDeviceState** out) {
         e = cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres);
         if (e != cudaSuccess || qres != cudaDriverEntryPointSuccess || !fn)
             return cuda_fail(nullptr, e != cudaSuccess ? e : cudaErrorUnknown);
-        e = raise_smem_limit(winograd_gemm_kernel, winograd_gemm_smem_bytes(256, WG_MAX_STAGES));
+        e = raise_smem_limit(winograd_gemm_kernel, winograd_gemm_smem_bytes(WG_MAX_N_CHUNK, WG_MAX_STAGES));
         if (e == cudaSuccess) e = cudaMemset(status, 0, sizeof(int) * DEV_STATUS_INTS);
         if (e != cudaSuccess) return cuda_fail(nullptr, e);
         st->status = (int*)status;
@@ -1186,11 +1186,11 @@ extern "C" int sd_winograd_conv3x3_forward(const void* x, const void* U, const v
     a.tiles_y = (H + WG_TILE - 1) / WG_TILE;
     a.tiles_x = (W + WG_TILE - 1) / WG_TILE;
     a.T = (int)T;
-    const int chunks = (K + 255) / 256;
+    const int chunks = (K + WG_MAX_N_CHUNK - 1) / WG_MAX_N_CHUNK;
     a.n_chunk = ((K + chunks - 1) / chunks + 15) / 16 * 16;
     a.tmem_cols = next_pow2_cols(a.n_chunk);
     // two CTAs per SM (shared memory and the 512 columns of tensor memory allow it): one's epilogue under the other's loads
-    a.stages = wg_stage_bytes(a.n_chunk) > 37 * 1024 ? 2 : 3;
+    a.stages = 3;
     a.status = st->status;
     __half* V = (__half*)workspace;
     float* M = (float*)((char*)workspace + round256((size_t)WG_XI * T * C * sizeof(__half)));

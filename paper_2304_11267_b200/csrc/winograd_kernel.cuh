@@ -89,7 +89,7 @@ struct WinogradArgs {
     int N, H, W, C, K;
     int tiles_y, tiles_x;   // ceil(H / 4), ceil(W / 4)
     int T;                  // N * tiles_y * tiles_x
-    int n_chunk;            // output channels per GEMM CTA (multiple of 16, <= 256)
+    int n_chunk;            // output channels per GEMM CTA (multiple of 16, <= WG_MAX_N_CHUNK)
     int tmem_cols;          // power of two >= n_chunk
     int stages;             // ring depth of the GEMM's operand tiles
     int* status;
@@ -207,8 +207,11 @@ constexpr int WG_MAX_STAGES = 4;
 enum { SITE_W_EMPTY = 50, SITE_W_FULL = 51, SITE_W_DONE = 52 };
 
 __host__ __device__ inline int wg_stage_bytes(int n_chunk) { return (TILE_M + n_chunk) * CHUNK_ROW_BYTES; }
+constexpr int WG_MAX_N_CHUNK = 176;   // ring of three stages and the epilogue's staging tile both fit twice per SM
 __host__ inline size_t winograd_gemm_smem_bytes(int n_chunk, int stages) {
-    return (size_t)stages * (size_t)((wg_stage_bytes(n_chunk) + 1023) & ~1023) + 1024;
+    const size_t ring = (size_t)stages * (size_t)((wg_stage_bytes(n_chunk) + 1023) & ~1023);
+    const size_t staging = (size_t)TILE_M * (n_chunk + 4) * sizeof(float);   // the epilogue reuses the ring
+    return (ring > staging ? ring : staging) + 1024;
 }
 
 __global__ void __launch_bounds__(WG_THREADS, 1)
@@ -288,29 +291,34 @@ winograd_gemm_kernel(const __grid_constant__ CUtensorMap tmap_v, const __grid_co
             if (ok) tc_commit(smem_u32(&bar_done));
         }
     } else {
-        // -------------------------------------------------------------------- epilogue: thread = row of the tile
+        // -------------------------------------------------------------------- epilogue
+        // Thread = row of the tile when it reads the accumulator; a row of M is n_chunk consecutive floats, so the
+        // tile goes through shared memory (the operand ring is idle by now: every MMA has completed) and leaves as
+        // whole rows, a warp writing 512 contiguous bytes at a time.  Each warp stages and writes its own 32 rows.
         bool ok = mbar_wait(smem_u32(&bar_done), 0, abort_p, args.status, SITE_W_DONE, blockIdx.x);
         ok = __all_sync(0xffffffffu, ok);
         if (ok) {
             tc_fence_after_sync();
-            const int q = warp & 3;                        // a warp reads the 32 lanes of its quarter (warp id mod 4)
+            const int q = warp & 3, lane = tid & 31;       // a warp reads the 32 lanes of its quarter (warp id mod 4)
             const uint32_t lane_off = (uint32_t)(q * 32) << 16;
-            const int row = t0 + q * 32 + (tid & 31);
-            float* mrow = M + ((long long)xi * args.T + row) * args.K + k0;
+            const int pitch = n_chunk + 4;                 // floats; + 4 keeps the 16-byte row writes off each other's banks
+            float* stage = reinterpret_cast<float*>(wg_smem_raw + (smem_base - smem_u32(wg_smem_raw))) + q * 32 * pitch;
             for (int g = 0; g < (n_chunk >> 4); ++g) {
                 uint32_t r[16];
                 tmem_ld16(tmem_d + lane_off + g * 16, r);
                 tmem_wait_ld();
-                if (row < args.T) {
 #pragma unroll
-                    for (int c = 0; c < 16; c += 4) {
-                        if (k0 + g * 16 + c + 4 <= args.K)
-                            *reinterpret_cast<uint4*>(mrow + g * 16 + c) = make_uint4(r[c], r[c + 1], r[c + 2], r[c + 3]);
-                        else
-                            for (int e = 0; e < 4; ++e)
-                                if (k0 + g * 16 + c + e < args.K) mrow[g * 16 + c + e] = __uint_as_float(r[c + e]);
-                    }
-                }
+                for (int c = 0; c < 16; c += 4)
+                    *reinterpret_cast<uint4*>(stage + lane * pitch + g * 16 + c) = make_uint4(r[c], r[c + 1], r[c + 2], r[c + 3]);
+            }
+            __syncwarp();
+            const int cols = min(n_chunk, args.K - k0);    // a multiple of 8: K and k0 are
+            for (int rr = 0; rr < 32; ++rr) {
+                const int row = t0 + q * 32 + rr;
+                if (row >= args.T) break;
+                float* mrow = M + ((long long)xi * args.T + row) * args.K + k0;
+                for (int c = lane * 4; c < cols; c += 128)
+                    *reinterpret_cast<uint4*>(mrow + c) = *reinterpret_cast<const uint4*>(stage + rr * pitch + c);
             }
         }
     }
