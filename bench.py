@@ -553,7 +553,24 @@ def winograd_numbers(bd, device, stream, peaks):
     cpu_s = time.perf_counter() - t0
     got = ys[0][:1, :hs].cpu().numpy().astype("float64")
     rel = float(((got - ref) ** 2).sum() ** 0.5 / ((ref ** 2).sum() ** 0.5))
+    # the same layer at 16 times the batch: enough tiles for many waves of GEMM CTAs (the rate of the kernels
+    # themselves, where the UNet's own shape is a chain of three short kernels)
+    NB = 16 * N
+    xb = torch.randn(NB, H, W, C, device=device, generator=g).to(torch.float16)
+    yb = torch.empty(NB, H, W, K, device=device, dtype=torch.float16)
+    for _ in range(2):
+        layer(xb, out=yb, stream=stream)
+    torch.cuda.synchronize()
+    start.record()
+    for _ in range(5):
+        layer(xb, out=yb, stream=stream)
+    end.record()
+    torch.cuda.synchronize()
+    us_b = 1e3 * start.elapsed_time(end) / 5
+    del xb, yb
     return {"us_per_call": us, "launches_per_call": 3,
+            "at_16x_batch": {"us_per_call": us_b, "direct_conv_tflops_equivalent": 16 * direct_flops / (us_b * 1e-6) / 1e12,
+                             "gemm_tflops": 16 * gemm_flops / (us_b * 1e-6) / 1e12},
             "direct_conv_tflops_equivalent": direct_flops / (us * 1e-6) / 1e12,
             "gemm_tflops": gemm_flops / (us * 1e-6) / 1e12,
             "bound": "hbm", "algorithmic_bytes": io_bytes, "achieved_gbs": io_bytes / (us * 1e-6) / 1e9,
