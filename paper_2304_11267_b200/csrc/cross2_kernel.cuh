@@ -54,6 +54,8 @@ struct Cross2Args {
     HeadLayout lay;
     int Nq, Nk, d;
     int dpad, nch;
+    int strided_rows;   // four-group variant: a tile's rows are not one contiguous run (token-major tensors): Q and the
+                        // output move as unswizzled tiles of d columns through tmap_q_rows / tmap_out_rows
     int stages;         // depth of the Q ring
     int tiles_per_bh;   // ceil(Nq / 128)
     int n_items;        // BH * tiles_per_bh
@@ -120,7 +122,8 @@ __device__ __forceinline__ void issue_qk(uint32_t tmem_s, uint64_t q_desc, uint6
 template <int NWG, bool BF = false>   // BF: bfloat16 tensors
 __global__ void __launch_bounds__(NWG * 128 + 256, 1)
 cross2_attention_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__ CUtensorMap tmap_k,
-                        const __grid_constant__ CUtensorMap tmap_v, const Cross2Args args) {
+                        const __grid_constant__ CUtensorMap tmap_v, const __grid_constant__ CUtensorMap tmap_q_rows,
+                        const __grid_constant__ CUtensorMap tmap_out_rows, const Cross2Args args) {
     extern __shared__ uint8_t x2_smem_raw[];
     __shared__ __align__(8) uint64_t bar_full[X2_MAX_STAGES], bar_empty[X2_MAX_STAGES];
     __shared__ __align__(8) uint64_t bar_kv_full[2], bar_kv_empty[2];
@@ -147,6 +150,10 @@ cross2_attention_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid
         tma_prefetch_desc(&tmap_q);
         tma_prefetch_desc(&tmap_k);
         tma_prefetch_desc(&tmap_v);
+        if (NWG == 4 && args.strided_rows) {
+            tma_prefetch_desc(&tmap_q_rows);
+            tma_prefetch_desc(&tmap_out_rows);
+        }
     }
     const int nch = args.nch, dpad = args.dpad, stages = args.stages;
     // contiguous range of items for this CTA: consecutive items share a head, so K and V are fetched rarely
@@ -239,6 +246,11 @@ cross2_attention_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid
                     int rows = args.Nq - tile * TILE_M;
                     if (rows > TILE_M) rows = TILE_M;
                     const uint32_t bytes = (uint32_t)rows * args.d * 2;   // d % 8 == 0: a multiple of 16
+                    if (args.strided_rows) {   // the same dense tile, row by row (rows past Nq arrive as zeros)
+                        mbar_arrive_expect_tx(bar, raw_bytes);
+                        tma_load_4d(raw_smem + s * raw_bytes, &tmap_q_rows, bar, 0, tile * TILE_M, hz, bz);
+                        continue;
+                    }
                     mbar_arrive_expect_tx(bar, bytes);
                     bulk_load(raw_smem + s * raw_bytes, args.q + ((size_t)bh * args.Nq + (size_t)tile * TILE_M) * args.d, bytes, bar);
                     continue;
@@ -498,8 +510,13 @@ cross2_attention_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid
                 if (tid == EPILOGUE_WARP0 * 32) {
                     int rows = args.Nq - tile * TILE_M;
                     if (rows > TILE_M) rows = TILE_M;
-                    bulk_store(args.out + ((size_t)bh * args.Nq + (size_t)tile * TILE_M) * args.d, stage,
-                               (uint32_t)rows * args.d * 2);
+                    if (args.strided_rows) {   // rows past Nq are clipped by the hardware
+                        const int bz = bh / args.lay.heads, hz = bh - bz * args.lay.heads;
+                        tma_store_4d(&tmap_out_rows, stage, 0, tile * TILE_M, hz, bz);
+                    } else {
+                        bulk_store(args.out + ((size_t)bh * args.Nq + (size_t)tile * TILE_M) * args.d, stage,
+                                   (uint32_t)rows * args.d * 2);
+                    }
                     bulk_commit();
                 }
                 if (tracer) X2_TRACE(w, i, 4);

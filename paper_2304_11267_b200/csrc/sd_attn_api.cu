@@ -398,6 +398,21 @@ static CUresult encode_tmap(encode_tiled_fn enc, CUtensorMap* map, const void* b
                CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
 }
 
+// The same tensor as unswizzled tiles of exactly d columns by 128 rows: a tile lands in (or leaves) shared memory as
+// dense rows of 2d bytes.  For the 77-key kernel's raw Q ring and output staging when a head's rows are not one
+// contiguous run of memory (token-major tensors).
+static CUresult encode_row_tmap(encode_tiled_fn enc, CUtensorMap* map, const void* base, int heads, int BH, int N, int d,
+                                int bf16) {
+    const HeadLayout l = head_layout(heads, BH, N, d);
+    cuuint64_t dims[4] = {(cuuint64_t)d, (cuuint64_t)N, (cuuint64_t)l.heads, (cuuint64_t)(BH / l.heads)};
+    cuuint64_t strides[3] = {(cuuint64_t)l.ld * 2, (cuuint64_t)l.head_stride * 2, (cuuint64_t)l.batch_stride * 2};
+    cuuint32_t box[4] = {(cuuint32_t)d, (cuuint32_t)TILE_M, 1, 1};
+    cuuint32_t estr[4] = {1, 1, 1, 1};
+    return enc(map, bf16 ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 4,
+               const_cast<void*>(base), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+               CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+}
+
 // An fp16 tensor of BH heads of N rows of d values seen by the TMA as (x = d, y = N, z = head, w = batch): tiles are
 // 64 columns wide (one 128-byte swizzled row) by `box_rows` rows.  Columns >= d and rows >= N read as zero.
 static int make_tmap(sd_attn_handle* h, CUtensorMap* map, const void* base, int BH, int N, int d, int box_rows,
@@ -483,8 +498,18 @@ static int launch_cross2(sd_attn_handle* h, const Problem& p) {
     if (rc != SD_ATTN_OK) return rc;
     const int grid = a.n_items < h->sm_count ? a.n_items : h->sm_count;
     int groups = cross2_groups(p.d);
-    // (the four-group variant moves whole Q and output tiles as contiguous runs of memory: head-major tensors only)
-    if (groups >= 4 && (!h->cross2_four_ok || p.heads > 0)) groups = 3;
+    if (groups >= 4 && !h->cross2_four_ok) groups = 3;
+    // The four-group variant moves whole Q and output tiles: as single contiguous runs when the tensors are
+    // head-major, as unswizzled tiles of d columns (two more tensor maps) when they are token-major.
+    a.strided_rows = (groups >= 4 && p.heads > 0) ? 1 : 0;
+    CUtensorMap tqr = tq, tor = tq;
+    if (a.strided_rows) {
+        if (encode_row_tmap(h->encode_tiled, &tqr, p.q, p.heads, p.BH, p.Nq, p.d, p.bf16) != CUDA_SUCCESS ||
+            encode_row_tmap(h->encode_tiled, &tor, p.out, p.heads, p.BH, p.Nq, p.d, p.bf16) != CUDA_SUCCESS) {
+            h->last_cuda_error = cudaErrorInvalidValue;
+            return SD_ATTN_ERR_CUDA;
+        }
+    }
     size_t smem = cross2_smem_bytes(a.nch);
     if (groups >= 4) {   // d <= 48: Q tiles arrive as raw bulk copies and are rewritten in shared memory
         a.stages = cross2_dense_stages(p.d);
@@ -492,13 +517,13 @@ static int launch_cross2(sd_attn_handle* h, const Problem& p) {
     }
     const dim3 g(grid);
     if (p.bf16) {
-        if (groups >= 4) launch_overlapped(h, cross2_attention_kernel<4, true>, g, dim3(cross2_threads(4)), smem, p.stream, tq, tk, tv, a);
-        else if (groups == 3) launch_overlapped(h, cross2_attention_kernel<3, true>, g, dim3(cross2_threads(3)), smem, p.stream, tq, tk, tv, a);
-        else launch_overlapped(h, cross2_attention_kernel<2, true>, g, dim3(cross2_threads(2)), smem, p.stream, tq, tk, tv, a);
+        if (groups >= 4) launch_overlapped(h, cross2_attention_kernel<4, true>, g, dim3(cross2_threads(4)), smem, p.stream, tq, tk, tv, tqr, tor, a);
+        else if (groups == 3) launch_overlapped(h, cross2_attention_kernel<3, true>, g, dim3(cross2_threads(3)), smem, p.stream, tq, tk, tv, tqr, tor, a);
+        else launch_overlapped(h, cross2_attention_kernel<2, true>, g, dim3(cross2_threads(2)), smem, p.stream, tq, tk, tv, tqr, tor, a);
     } else {
-        if (groups >= 4) launch_overlapped(h, cross2_attention_kernel<4>, g, dim3(cross2_threads(4)), smem, p.stream, tq, tk, tv, a);
-        else if (groups == 3) launch_overlapped(h, cross2_attention_kernel<3>, g, dim3(cross2_threads(3)), smem, p.stream, tq, tk, tv, a);
-        else launch_overlapped(h, cross2_attention_kernel<2>, g, dim3(cross2_threads(2)), smem, p.stream, tq, tk, tv, a);
+        if (groups >= 4) launch_overlapped(h, cross2_attention_kernel<4>, g, dim3(cross2_threads(4)), smem, p.stream, tq, tk, tv, tqr, tor, a);
+        else if (groups == 3) launch_overlapped(h, cross2_attention_kernel<3>, g, dim3(cross2_threads(3)), smem, p.stream, tq, tk, tv, tqr, tor, a);
+        else launch_overlapped(h, cross2_attention_kernel<2>, g, dim3(cross2_threads(2)), smem, p.stream, tq, tk, tv, tqr, tor, a);
     }
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) return cuda_fail(h, e);

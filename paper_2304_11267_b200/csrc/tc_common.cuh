@@ -222,6 +222,13 @@ __device__ __forceinline__ void tma_store_3d(const void* tmap, uint32_t src, int
                  "r"(src), "r"(x), "r"(y), "r"(z)
                  : "memory");
 }
+// 4-D tile store shared -> global, coordinates as for the 4-D load.
+__device__ __forceinline__ void tma_store_4d(const void* tmap, uint32_t src, int x, int y, int z, int w) {
+    asm volatile("cp.async.bulk.tensor.4d.global.shared::cta.bulk_group [%0, {%2, %3, %4, %5}], [%1];" ::"l"(
+                     reinterpret_cast<uint64_t>(tmap)),
+                 "r"(src), "r"(x), "r"(y), "r"(z), "r"(w)
+                 : "memory");
+}
 __device__ __forceinline__ void tma_store_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
 // Wait until the committed stores have finished READING shared memory (it may then be reused).
 __device__ __forceinline__ void tma_store_wait_read() {

@@ -95,7 +95,7 @@ def test_small_weights_stay_out_of_the_subnormals(bd):
     w = (w.astype(np.float32) * 0.02).astype(np.float16)
     ref = oracle.conv3x3_forward(x, w, b)
     got = run(bd, x, w, b).astype(np.float64)
-    ref0 = oracle.conv3x3_forward(x, w)            # the bias is exact: judge the convolution part on its own scale
+    ref0 = oracle.conv3x3_forward(x, w)            # the bias is exact: measure the convolution part against its own scale
     err = np.abs((got - ref))
     rms = float(np.sqrt(np.mean(ref0 ** 2)))
     assert np.all(err <= MAX_ABS_OF_RMS * rms + 2.0 ** -10 * np.abs(ref)), (float(err.max()), rms)
