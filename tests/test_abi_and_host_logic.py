@@ -69,6 +69,35 @@ def test_workspace_and_staging_sizes(lib):
     assert bd.sd_attn_host_staging_bytes(0, 8, 4096, 77, 40, bd.F16) == 0
 
 
+def test_newer_entry_points_reject_bad_arguments_before_touching_a_device(lib):
+    """Argument checks come before any CUDA call, so they answer on a machine without a GPU."""
+    assert bd.sd_attn_set_layout(None, bd.LAYOUT_BNHD) == bd.ERR_INVALID_VALUE
+    assert lib.sd_attn_forward_batch(None, None, 0, bd.F16, None) == bd.ERR_INVALID_VALUE
+    # the Winograd convolution: sizes are host arithmetic
+    assert bd.sd_winograd_filter_elems(320, 320) == 36 * 320 * 320
+    assert bd.sd_winograd_filter_elems(0, 320) == 0
+    T = 2 * 16 * 16                                                  # 64 x 64 image, batch 2: 4 x 4 output tiles
+    assert bd.sd_winograd_workspace_bytes(2, 64, 64, 320, 320) == 36 * T * 320 * 2 + 36 * T * 320 * 4
+    r256 = lambda n: (n + 255) // 256 * 256                        # each plane starts 256-byte aligned
+    assert bd.sd_winograd_workspace_bytes(1, 5, 9, 8, 16) == r256(36 * 6 * 8 * 2) + r256(36 * 6 * 16 * 4)   # ragged: 2 x 3 tiles
+    assert bd.sd_winograd_workspace_bytes(1, 1, 1, 8, 8) == r256(36 * 8 * 2) + r256(36 * 8 * 4)
+    assert bd.sd_winograd_workspace_bytes(1, 0, 8, 8, 8) == 0
+    f = bd.sd_winograd_conv3x3_forward
+    assert f(256, 256, 0, 256, 256, 1 << 30, 1, 8, 8, 0, 16, 0) == bd.ERR_INVALID_VALUE     # C = 0
+    assert f(256, 256, 0, 256, 256, 1 << 30, 1, 8, 8, 12, 16, 0) == bd.ERR_UNSUPPORTED      # C % 8 != 0
+    assert f(256, 256, 0, 256, 256, 1 << 30, 0, 8, 8, 16, 16, 0) == bd.OK                   # N = 0: nothing to do
+    assert f(0, 256, 0, 256, 256, 1 << 30, 1, 8, 8, 16, 16, 0) == bd.ERR_INVALID_VALUE      # null x
+    assert f(264, 256, 0, 256, 256, 1 << 30, 1, 8, 8, 16, 16, 0) == bd.ERR_ALIGNMENT
+    assert f(256, 256, 0, 256, 256, 100, 1, 8, 8, 16, 16, 0) == bd.ERR_WORKSPACE            # scratch too small
+    assert f(256, 256, 0, 256, 384, 1 << 30, 1, 8, 8, 16, 16, 0) == bd.ERR_WORKSPACE        # scratch not 256-aligned
+    assert bd.sd_winograd_transform_filter(0, 256, 16, 16, 0) == bd.ERR_INVALID_VALUE
+    assert bd.sd_winograd_transform_filter(256, 256, 12, 16, 0) == bd.ERR_UNSUPPORTED
+    # the element-wise and normalisation steps
+    assert bd.load().sd_geglu_forward(None, None, 4, 8, bd.F16, None) == bd.ERR_INVALID_VALUE
+    assert bd.load().sd_geglu_forward(None, None, 0, 8, bd.F16, None) == bd.OK
+    assert bd.load().sd_groupnorm_forward(None, None, None, None, 1, 30, 4, 4, ctypes.c_float(1e-5), bd.F16, None) == bd.ERR_INVALID_VALUE
+
+
 def test_create_without_a_device_fails_cleanly(lib):
     import torch
     if torch.cuda.is_available():

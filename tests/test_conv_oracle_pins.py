@@ -118,3 +118,43 @@ def test_cost_model_reproduces_table_2():
             digits = len(cell.split(".")[1]) if "." in cell else 0
             assert abs(value - float(cell)) <= 10.0 ** -digits * 1.0001 + 1e-12, (m, cell, value)
     assert oracle.winograd_cost_model(4) == (4.0, 2.25, 4.0)     # the tile the paper selects
+
+
+def test_error_level_of_the_transformed_domain_in_binary16():
+    """Where the GPU test's tolerance comes from.  The algorithm for the points 0, +-1, +-2, inf, written here in double
+    precision, (a) reproduces the oracle to rounding when nothing is rounded -- so the oracle is also pinned to the
+    very identity the CUDA path relies on -- and (b) with the transformed filter and input rounded to binary16, as the
+    tensor cores take them, lands at about 3e-3 relative L2 with its largest errors in the tile's last row and column:
+    the bounds of the GPU test (6e-3, 0.08 of the output's r.m.s.) are twice that and nine sigma of the worst position."""
+    BT = np.array([[4, 0, -5, 0, 1, 0], [0, -4, -4, 1, 1, 0], [0, 4, -4, -1, 1, 0],
+                   [0, -2, -1, 2, 1, 0], [0, 2, -1, -2, 1, 0], [0, 4, 0, -5, 0, 1]], float)
+    G = np.array([[1 / 4, 0, 0], [-1 / 6, -1 / 6, -1 / 6], [-1 / 6, 1 / 6, -1 / 6],
+                  [1 / 24, 1 / 12, 1 / 6], [1 / 24, -1 / 12, 1 / 6], [0, 0, 1]], float)
+    AT = np.array([[1, 1, 1, 1, 1, 0], [0, 1, -1, 2, -2, 0], [0, 1, 1, 4, 4, 0], [0, 1, -1, 8, -8, 1]], float)
+    N, H, W, C, K = 1, 16, 16, 320, 24
+    x = rand(31, (N, H, W, C))
+    w = (np.random.default_rng(32).standard_normal((K, 3, 3, C), dtype=np.float32) / np.sqrt(9.0 * C)).astype(np.float16)
+    ref = oracle.conv3x3_forward(x, w)[0]
+    xp = np.zeros((H + 2, W + 2, C))
+    xp[1:-1, 1:-1] = x[0].astype(np.float64)
+    patches = np.stack([xp[4 * ty:4 * ty + 6, 4 * tx:4 * tx + 6] for ty in range(H // 4) for tx in range(W // 4)])
+    U = np.einsum("ar,krsc,bs->kabc", G, w.astype(np.float64), G)
+    V = np.einsum("ar,trsc,bs->tabc", BT, patches, BT)
+
+    def finish(U_, V_):
+        M = np.einsum("kabc,tabc->tkab", U_, V_)
+        Y = np.einsum("ia,tkab,jb->tijk", AT, M, AT)
+        return Y.reshape(H // 4, W // 4, 4, 4, K).transpose(0, 2, 1, 3, 4).reshape(H, W, K)
+
+    np.testing.assert_allclose(finish(U, V), ref, rtol=0, atol=1e-12)                      # (a)
+    to16 = lambda t: t.astype(np.float16).astype(np.float64)
+    got = finish(to16(U * 128.0) / 128.0, to16(V))                                         # (b)
+    rms = float(np.sqrt(np.mean(ref ** 2)))
+    rel = float(np.linalg.norm(got - ref) / np.linalg.norm(ref))
+    assert 1.5e-3 < rel < 4.5e-3, rel
+    err = np.abs(got - ref).reshape(H // 4, 4, W // 4, 4, K)
+    per_pos = np.sqrt((err ** 2).mean(axis=(0, 2, 4))) / rms
+    assert per_pos[3, 3] == per_pos.max() and 4e-3 < per_pos[3, 3] < 1.4e-2, per_pos
+    assert per_pos[0, 0] < 2e-3
+    assert float(np.abs(got - ref).max()) < 0.08 * rms
+    assert float(np.abs(V).max()) < 400 and float(np.abs(U).max() * 128.0) < 64             # binary16's range is far
