@@ -14,12 +14,14 @@
  *     library never allocates, frees or keeps them.  `stream` is a cudaStream_t passed as
  *     void* (NULL = the legacy default stream).  Handles and status words are HOST objects.
  *   - Layout: q and out are dense [B][H][Nq][d], k and v dense [B][H][Nk][d], d innermost,
- *     no strides; `d` is the true head dim (padding to tensor-core widths is internal).
+ *     no strides -- or, after sd_attn_set_layout(SD_ATTN_LAYOUT_BNHD), dense [B][Nq][H][d] and
+ *     [B][Nk][H][d]; `d` is the true head dim (padding to tensor-core widths is internal).
  *     `out` must not overlap any input.
  *   - Every function returns an sd_attn_status.  Validation happens before any launch: a
  *     non-OK return means nothing was enqueued.  No function throws, aborts or exits.
  *   - sd_attn_forward is asynchronous and stream-ordered: it does not synchronise, allocate
- *     or read back.  One handle serves one host thread at a time.
+ *     or read back.  One handle serves one host thread and one stream at a time (its status
+ *     block and the streams of the host and batch entry points are per handle).
  */
 #ifndef SD_ATTN_H_
 #define SD_ATTN_H_
