@@ -12,13 +12,20 @@
  * Conventions that hold for every entry point
  *   - Pointers named q, k, v, out, workspace are DEVICE pointers owned by the caller; the
  *     library never allocates, frees or keeps them.  `stream` is a cudaStream_t passed as
- *     void* (NULL = the legacy default stream).  Handles and status words are HOST objects.
+ *     void* (NULL = the legacy default stream).  Handles are HOST objects; the status block a
+ *     handle owns is DEVICE memory, read back only by sd_attn_query_status.
  *   - Layout: q and out are dense [B][H][Nq][d], k and v dense [B][H][Nk][d], d innermost,
  *     no strides -- or, after sd_attn_set_layout(SD_ATTN_LAYOUT_BNHD), dense [B][Nq][H][d] and
  *     [B][Nk][H][d]; `d` is the true head dim (padding to tensor-core widths is internal).
  *     `out` must not overlap any input.
- *   - Every function returns an sd_attn_status.  Validation happens before any launch: a
- *     non-OK return means nothing was enqueued.  No function throws, aborts or exits.
+ *   - Every function returns an sd_attn_status.  No function throws, aborts or exits.
+ *     sd_attn_forward and sd_attn_forward_twopass_static validate before any launch: an argument
+ *     error from them means nothing was enqueued (ERR_CUDA can come from a launch itself, in
+ *     TWOPASS mode from the second of its two).  sd_attn_forward_batch and sd_attn_forward_host
+ *     enqueue piece by piece: when they return an error, earlier problems or slices may already
+ *     be enqueued, and the library's own streams have been joined back into `stream` in every case.
+ *   - A handle belongs to the device that was current at sd_attn_create; every call that takes a
+ *     handle returns INVALID_VALUE when another device is current.
  *   - sd_attn_forward is asynchronous and stream-ordered: it does not synchronise, allocate
  *     or read back.  One handle serves one host thread and one stream at a time (its status
  *     block and the streams of the host and batch entry points are per handle).
@@ -50,8 +57,7 @@ typedef enum {
     SD_ATTN_F32 = 1, /* binary32 throughout (plain FMA arithmetic, no TF32)        */
     SD_ATTN_BF16 = 2 /* bfloat16 q/k/v/out, binary32 accumulation; the softmax weights enter the second product
                         rounded to bfloat16 (8 significant bits), so results are about 8x coarser than F16's.
-                        Implemented by the kernels AUTO selects (FUSED, CROSS, SIMT); TWOPASS mode and FUSED
-                        under the switches that select its earlier kernels answer UNSUPPORTED.               */
+                        Implemented by FUSED, CROSS and SIMT; TWOPASS mode answers UNSUPPORTED.              */
 } sd_attn_dtype;
 
 typedef enum {
@@ -75,29 +81,41 @@ typedef enum {
 #define SD_ATTN_MAX_D 160
 
 /*
- * Create a handle on the CURRENT CUDA device.  Checks the architecture (ERR_ARCH unless
- * compute capability 10.x), resolves the driver's tensor-map encoder, raises the kernels'
- * dynamic shared-memory limits, allocates one 64-byte device status block and creates the two
- * copy streams and ten events sd_attn_forward_host uses, and the three streams and four events of
- * sd_attn_forward_batch.  No stream work.  *out receives the
- * handle (NULL on failure).
- *
- * Switches read from the environment at this call (all default off; they select slower variants that exist
- * for comparison and testing, results are the same within the tolerance):
- *   SD_ATTN_NO_PDL=1            launch every kernel the ordinary way.  By default the tensor-core kernels are
- *                               launched with programmatic stream serialization: a kernel may run its set-up
- *                               while the previous kernel of the stream finishes, and waits for that kernel to
- *                               complete before it reads or writes global memory, so stream order is kept.
- *   SD_ATTN_FUSED_TILES=1..4    fixed number of query tiles per CTA of the FUSED kernel (default: by problem size)
- *   SD_ATTN_FUSED_NO_SPLIT=1    FUSED, one query tile per CTA: the tile's score columns stay with one warpgroup
- *   SD_ATTN_FUSED_SPLIT=2|4     FUSED, one query tile per CTA: that many warpgroups share them (default: by head dim)
- *   SD_ATTN_FUSED_NO_SPARE=1    FUSED: the four-tile kernel without the spare score buffer (d <= 64)
- *   SD_ATTN_FUSED_TWO_TILE=1    FUSED: the two-tile kernel
- *   SD_ATTN_CROSS_ONE_TILE=1    CROSS: one tile per CTA also for 65..80 keys
- *   SD_ATTN_HOST_ONE_SLICE=1    sd_attn_forward_host: one slice, copies and kernel all on the caller's stream
- *   SD_ATTN_BATCH_ONE_LANE=1    sd_attn_forward_batch: every problem on the caller's stream, one after another
+ * Choices a caller (or a test) can make when a handle is created.  All zero = the defaults; every non-default
+ * choice selects a slower variant that exists for comparison and testing, with the same results within the
+ * tolerance.  Nothing in the library's kernel selection depends on the process environment.
+ */
+typedef struct {
+    size_t struct_size;    /* sizeof(sd_attn_options): lets the struct grow without breaking callers       */
+    int no_pdl;            /* 1: launch every kernel the ordinary way.  By default the tensor-core kernels are
+                              launched with programmatic stream serialization: a kernel may run its set-up
+                              while the previous kernel of the stream finishes, and waits for that kernel to
+                              complete before it reads or writes global memory, so stream order is kept      */
+    int fused_tiles;       /* 1..4: fixed number of query tiles per CTA of the FUSED kernel (0: by problem size) */
+    int fused_split;       /* FUSED with one query tile per CTA: 2 or 4 warpgroups share its key tiles, 1 none
+                              (0: by head dim)                                                                */
+    int fused_shares;      /* FUSED: a problem of more groups of query tiles than SMs has the key range of a group
+                              cut between CTAs, so that every SM gets an equal share; partial results are combined
+                              through the handle's scratch.  0: where the cost model says it pays; 1: never (the
+                              scratch is not even allocated); 2: wherever the kernel allows it (tests)             */
+    int cross_one_tile;    /* 1: CROSS runs one tile per CTA also for 65..80 keys                             */
+    int host_one_slice;    /* 1: sd_attn_forward_host uses one slice, copies and kernel all on the caller's stream */
+    int batch_serial;      /* 1: sd_attn_forward_batch runs its problems one after another on the caller's stream */
+} sd_attn_options;
+
+/*
+ * Create a handle on the CURRENT CUDA device.  Checks the architecture (ERR_ARCH unless compute capability
+ * 10.x), resolves the driver's tensor-map encoder, raises the kernels' dynamic shared-memory limits, allocates
+ * the handle's device memory -- one 64-byte status block and the scratch through which the FUSED kernel combines
+ * partial results of a group of query tiles whose keys were shared out among CTAs (about 50 MB) -- and creates
+ * the two copy streams and ten events sd_attn_forward_host uses, and the three streams and four events of
+ * sd_attn_forward_batch.  No stream work.  *out receives the handle (NULL on failure).
+ * sd_attn_create(out) is sd_attn_create_ex(NULL, out): the defaults.  `options` may be NULL; it is read during
+ * the call only.  Errors: INVALID_VALUE (null `out`, an option out of range, struct_size not that of a known
+ * version), ARCH, CUDA.
  */
 int sd_attn_create(sd_attn_handle **out);
+int sd_attn_create_ex(const sd_attn_options *options, sd_attn_handle **out);
 
 /*
  * out = softmax(q k^T * scale) v, Eq. 3, for every (b, h); see the conventions above.
@@ -124,13 +142,16 @@ typedef struct {
 /*
  * `count` INDEPENDENT problems of Eq. 3 -- e.g. the attention calls of several UNet blocks evaluated side by side,
  * or of several requests -- as one piece of stream-ordered work on `stream`: no problem's output may be another's
- * input or output.  The library is free to run them at the same time: it forks three streams of its own from
- * `stream`, gives each problem (in the order given) to the stream with the least estimated work so far and joins
- * them back, so small problems run in the SMs that large ones leave idle.  Capturable into a CUDA graph through
- * `stream`.  All problems share `dtype`, the handle's mode and layout; each is validated as by sd_attn_forward
- * and the first error is returned (problems before it have been enqueued; the streams are joined in every case).
- * In TWOPASS mode (one workspace) and with SD_ATTN_BATCH_ONE_LANE=1 in the environment at sd_attn_create the
- * problems run one after another on `stream`.  `problems` is a HOST array, read during the call only.
+ * input or output.  Problems of the same shape (B, H, Nq, Nk, d) that the same kernel serves become ONE launch of
+ * that kernel over all of them (up to eight per launch for FUSED, five for the 77-key CROSS kernel; the 32 calls
+ * of a UNet step are seven launches); the launches of different shapes are spread over `stream` and three streams
+ * of the handle, forked from `stream` and joined back by events, so small shapes run in the SMs that large ones
+ * leave idle.  Capturable into a CUDA graph through `stream`.  All problems share `dtype`, the handle's mode and
+ * layout; every problem is validated as by sd_attn_forward BEFORE anything is enqueued, and the first error is
+ * returned with nothing enqueued (an error of a launch itself, ERR_CUDA, can leave earlier launches enqueued; the
+ * streams are joined in every case).  Results are bitwise those of the same problems run one by one.
+ * In TWOPASS mode (one workspace), in SIMT mode and with `batch_serial` set at creation the problems run one
+ * after another on `stream`.  `problems` is a HOST array, read during the call only.
  * Errors: INVALID_VALUE (null handle, negative count, null array), then as sd_attn_forward.
  */
 int sd_attn_forward_batch(sd_attn_handle *h, const sd_attn_problem *problems, int count, int dtype,
@@ -164,9 +185,9 @@ int sd_attn_set_mode(sd_attn_handle *h, int mode);
 
 /*
  * Choose where the heads of q, k, v and out lie for later forwards (sd_attn_layout; default BHND).  All four
- * tensors of a call share the layout; each is dense in it.  BNHD is implemented by the kernels AUTO selects
- * (FUSED, CROSS and SIMT modes, either dtype); TWOPASS mode, and FUSED under the environment switches that select
- * its earlier kernels, answer UNSUPPORTED for it.  sd_attn_forward_host takes either layout (BNHD in one slice).
+ * tensors of a call share the layout; each is dense in it.  BNHD is implemented by FUSED, CROSS and SIMT modes
+ * (every dtype); TWOPASS mode answers UNSUPPORTED for it.  sd_attn_forward_host takes either layout (BNHD in
+ * one slice).
  * Errors: INVALID_VALUE (null handle, unknown layout).
  */
 int sd_attn_set_layout(sd_attn_handle *h, int layout);
@@ -191,9 +212,22 @@ int sd_attn_twopass_buffers(sd_attn_handle *h, const float **scores, const float
  * Synchronise `stream`, then read and clear the device status block.  Returns OK,
  * ERR_DEVICE_TIMEOUT (a kernel gave up a bounded wait and returned early: the outputs of the
  * calls since the last query are not valid) or ERR_CUDA.  If `detail` is non-NULL it receives
- * four host ints: {code, block index, wait site, tile index} of the first failure.
+ * four host ints: {code, block index, wait site, tile index} of the first failure.  After a
+ * time-out the handle's scratch counters are cleared as well, so the handle stays usable.
  */
 int sd_attn_query_status(sd_attn_handle *h, void *stream, int *detail);
+
+/*
+ * Self-test of the failure path behind SD_ATTN_ERR_DEVICE_TIMEOUT (Eq. 3 has no part in it): enqueues on `stream`
+ * a one-block kernel that takes the steps a tensor-core kernel of this library takes when a bounded wait runs
+ * out -- with the same primitives, but a budget of a few thousand polls (under a millisecond): a thread waits on
+ * a barrier nothing ever arrives on, gives up, raises the block's abort flag and records {1, block 0, site 99,
+ * tile 7} in the handle's status block; a second waiter leaves on seeing the flag; the block releases its tensor
+ * memory and returns normally.  Nothing traps, faults or waits without a limit.  The next sd_attn_query_status
+ * returns ERR_DEVICE_TIMEOUT with that detail and clears it; the handle and the context stay usable.
+ * Errors: INVALID_VALUE (null handle, wrong device), CUDA.
+ */
+int sd_attn_selftest_wait_timeout(sd_attn_handle *h, void *stream);
 
 /* Which kernel family the last successful forward used (an sd_attn_mode, never AUTO). */
 int sd_attn_last_mode(const sd_attn_handle *h);
@@ -226,12 +260,20 @@ long long sd_attn_launch_count(const sd_attn_handle *h);
  *     call overwrites what it reads and clears its device status word first, so calls that follow one
  *     another on a stream are independent.  Calls that OVERLAP on the GPU (different streams, or different
  *     host threads without ordering) race on the array and produce garbage: serialise them.
- *   - A bounded wait that expires inside a kernel cannot be reported by this entry point (there is no
- *     handle to query); use the handle-based API where that matters.
+ *   - A bounded wait that expires inside a kernel is recorded in a status word beside the array;
+ *     sd_attn_static_query_status reads it (there is no handle to query).
  */
 #define SD_ATTN_STATIC_MAX_SCRATCH ((size_t)34 * 1024 * 1024)
 int sd_attn_forward_twopass_static(const void *q, const void *k, const void *v, void *out, int B, int H,
                                    int Nq, int Nk, int d, float scale, int dtype, void *stream);
+
+/*
+ * The status word of sd_attn_forward_twopass_static on the current device (the paper has no counterpart
+ * either): synchronises `stream`, reads and clears the word.  OK, ERR_DEVICE_TIMEOUT (a kernel of a static
+ * call since the last query gave up a bounded wait: that call's output is not valid) or ERR_CUDA; `detail`
+ * as for sd_attn_query_status.  Allocates nothing (a stream synchronisation and one small copy to the host).
+ */
+int sd_attn_static_query_status(void *stream, int *detail);
 
 /* Static, NUL-terminated description of a status code. */
 const char *sd_attn_status_string(int status);

@@ -24,10 +24,10 @@ CROSS_MAX_NK = 128
 MAX_D = 160
 STATIC_MAX_SCRATCH = 34 * 1024 * 1024   # SD_ATTN_STATIC_MAX_SCRATCH: built-in scratch of the no-allocation entry point
 
-EXPORTS = ["sd_attn_create", "sd_attn_forward", "sd_attn_destroy", "sd_attn_set_mode",
+EXPORTS = ["sd_attn_create", "sd_attn_create_ex", "sd_attn_static_query_status", "sd_attn_selftest_wait_timeout", "sd_attn_forward", "sd_attn_destroy", "sd_attn_set_mode",
            "sd_attn_workspace_bytes", "sd_attn_set_workspace", "sd_attn_twopass_buffers",
            "sd_attn_query_status", "sd_attn_last_mode", "sd_attn_launch_count", "sd_attn_status_string",
-           "sd_attn_forward_host", "sd_attn_host_staging_bytes", "sd_attn_debug_dump_cross_scores",
+           "sd_attn_forward_host", "sd_attn_host_staging_bytes",
            "sd_attn_forward_twopass_static", "sd_geglu_forward", "sd_groupnorm_forward", "sd_attn_set_layout", "sd_attn_forward_batch",
            "sd_winograd_filter_elems", "sd_winograd_transform_filter", "sd_winograd_workspace_bytes",
            "sd_winograd_conv3x3_forward", "sd_winograd_query_status"]
@@ -40,6 +40,17 @@ class Problem(ctypes.Structure):
     _fields_ = [("q", ctypes.c_void_p), ("k", ctypes.c_void_p), ("v", ctypes.c_void_p), ("out", ctypes.c_void_p),
                 ("B", ctypes.c_int), ("H", ctypes.c_int), ("Nq", ctypes.c_int), ("Nk", ctypes.c_int),
                 ("d", ctypes.c_int), ("scale", ctypes.c_float)]
+
+
+class Options(ctypes.Structure):
+    """sd_attn_options: choices made when a handle is created (all zero = the defaults)."""
+    _fields_ = [("struct_size", ctypes.c_size_t), ("no_pdl", ctypes.c_int), ("fused_tiles", ctypes.c_int),
+                ("fused_split", ctypes.c_int), ("fused_shares", ctypes.c_int), ("cross_one_tile", ctypes.c_int),
+                ("host_one_slice", ctypes.c_int), ("batch_serial", ctypes.c_int)]
+
+    def __init__(self, **kw):
+        super().__init__(**kw)
+        self.struct_size = ctypes.sizeof(Options)
 
 
 class SdAttnError(RuntimeError):
@@ -61,6 +72,12 @@ def load() -> ctypes.CDLL:
     vp, ci, cf, sz = ctypes.c_void_p, ctypes.c_int, ctypes.c_float, ctypes.c_size_t
     lib.sd_attn_create.restype = ci
     lib.sd_attn_create.argtypes = [ctypes.POINTER(vp)]
+    lib.sd_attn_create_ex.restype = ci
+    lib.sd_attn_create_ex.argtypes = [ctypes.POINTER(Options), ctypes.POINTER(vp)]
+    lib.sd_attn_selftest_wait_timeout.restype = ci
+    lib.sd_attn_selftest_wait_timeout.argtypes = [vp, vp]
+    lib.sd_attn_static_query_status.restype = ci
+    lib.sd_attn_static_query_status.argtypes = [vp, ctypes.POINTER(ci)]
     lib.sd_attn_forward.restype = ci
     lib.sd_attn_forward.argtypes = [vp, vp, vp, vp, vp, ci, ci, ci, ci, ci, cf, ci, vp]
     lib.sd_attn_forward_host.restype = ci
@@ -105,8 +122,6 @@ def load() -> ctypes.CDLL:
     lib.sd_geglu_forward.argtypes = [vp, vp, ctypes.c_longlong, ci, ci, vp]
     lib.sd_groupnorm_forward.restype = ci
     lib.sd_groupnorm_forward.argtypes = [vp, vp, vp, vp, ci, ci, ctypes.c_longlong, ci, cf, ci, vp]
-    lib.sd_attn_debug_dump_cross_scores.restype = ci
-    lib.sd_attn_debug_dump_cross_scores.argtypes = [vp, vp]
     _lib = lib
     return lib
 
@@ -123,6 +138,22 @@ def sd_attn_create() -> int:
     if rc != OK:
         raise SdAttnError(rc, "sd_attn_create")
     return h.value
+
+
+def sd_attn_create_ex(options: Optional[Options]) -> int:
+    """A handle with non-default choices (``Options(no_pdl=1, ...)``); None gives the defaults."""
+    h = ctypes.c_void_p()
+    rc = load().sd_attn_create_ex(ctypes.byref(options) if options is not None else None, ctypes.byref(h))
+    if rc != OK:
+        raise SdAttnError(rc, "sd_attn_create_ex")
+    return h.value
+
+
+def sd_attn_static_query_status(stream=0):
+    """Status word of sd_attn_forward_twopass_static on the current device: (status, [code, block, site, tile])."""
+    detail = (ctypes.c_int * 4)()
+    rc = load().sd_attn_static_query_status(stream or None, detail)
+    return rc, list(detail)
 
 
 def sd_attn_destroy(handle: Optional[int]) -> int:
@@ -319,6 +350,11 @@ def sd_attn_query_status(handle, stream=0):
     return rc, list(detail)
 
 
+def sd_attn_selftest_wait_timeout(handle, stream=0) -> int:
+    """Enqueue the self-test kernel whose bounded wait runs out (see include/sd_attn.h)."""
+    return load().sd_attn_selftest_wait_timeout(handle, stream or None)
+
+
 def sd_attn_last_mode(handle) -> int:
     return load().sd_attn_last_mode(handle)
 
@@ -327,17 +363,13 @@ def sd_attn_launch_count(handle) -> int:
     return int(load().sd_attn_launch_count(handle))
 
 
-def sd_attn_debug_dump_cross_scores(handle, ptr) -> int:
-    return load().sd_attn_debug_dump_cross_scores(handle, ptr or None)
-
-
 # ------------------------------------------------------------------ convenience for torch tensors
 
 class Attention:
     """A handle plus torch-tensor marshalling: ``Attention().forward(q, k, v)``."""
 
-    def __init__(self, mode: int = MODE_AUTO, layout: int = LAYOUT_BHND):
-        self.handle = sd_attn_create()
+    def __init__(self, mode: int = MODE_AUTO, layout: int = LAYOUT_BHND, options: Optional[Options] = None):
+        self.handle = sd_attn_create_ex(options) if options is not None else sd_attn_create()
         self._workspace = None
         self.layout = LAYOUT_BHND
         if mode != MODE_AUTO:

@@ -48,9 +48,21 @@ constexpr int X2_CONTROL_REGS = 32;
 constexpr float X2_HEADROOM_LOG2 = 8.0f;   // weights of the first key: 2^-8
 constexpr float X2_SUM_LIMIT = 4096.0f;    // no weight above 2^12 reaches the binary16 pack
 
-struct Cross2Args {
+constexpr int X2_GROUP_MAX = 5;      // problems of one shape per launch (the parameter block stays under 4 KB)
+
+struct Cross2Problem {   // one problem of a launch
+    CUtensorMap tq, tk, tv;          // swizzled tiles of 64 columns
+    CUtensorMap tq_rows, tout_rows;  // four-group variant with strided rows: unswizzled tiles of d columns
     const __half* q;    // [BH][Nq][d]: the four-group variant fetches Q tiles with untiled bulk copies
-    __half* out;        // [BH][Nq][d], or as `lay` says (the four-group variant: head-major only)
+    __half* out;        // [BH][Nq][d], or as Cross2Args::lay says
+    float scale_log2e;  // |scale| * log2(e)
+    int negate;         // scale < 0: the tensor core negates Q
+};
+
+struct Cross2Args {
+    Cross2Problem prob[X2_GROUP_MAX];
+    int n_prob, BH;     // problems in this launch; (batch, head) pairs of each.  Heads are counted through all
+                        // problems ("global head" = problem * BH + head), items through all global heads
     HeadLayout lay;
     int Nq, Nk, d;
     int dpad, nch;
@@ -58,24 +70,10 @@ struct Cross2Args {
                         // output move as unswizzled tiles of d columns through tmap_q_rows / tmap_out_rows
     int stages;         // depth of the Q ring
     int tiles_per_bh;   // ceil(Nq / 128)
-    int n_items;        // BH * tiles_per_bh
-    float scale_log2e;
-    int negate;
+    int n_items;        // n_prob * BH * tiles_per_bh
     int* status;
-#ifdef SD_ATTN_TRACE
-    long long* trace;   // timeline probe of block 0: [role][item < 40][8 slots] clock64 stamps
-#endif
 };
 
-#ifdef SD_ATTN_TRACE
-#define X2_TRACE(role, i, slot)                                                      \
-    do {                                                                             \
-        if (args.trace && blockIdx.x == 0 && (i) < 40)                               \
-            args.trace[((role) * 40 + (i)) * 8 + (slot)] = clock64();                \
-    } while (0)
-#else
-#define X2_TRACE(role, i, slot) do { } while (0)
-#endif
 
 __host__ inline int cross2_groups(int d) {
     const int g = 512 / (X2_KN + (d + 15) / 16 * 16);
@@ -121,9 +119,7 @@ __device__ __forceinline__ void issue_qk(uint32_t tmem_s, uint64_t q_desc, uint6
 
 template <int NWG, bool BF = false>   // BF: bfloat16 tensors
 __global__ void __launch_bounds__(NWG * 128 + 256, 1)
-cross2_attention_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__ CUtensorMap tmap_k,
-                        const __grid_constant__ CUtensorMap tmap_v, const __grid_constant__ CUtensorMap tmap_q_rows,
-                        const __grid_constant__ CUtensorMap tmap_out_rows, const Cross2Args args) {
+cross2_attention_kernel(const __grid_constant__ Cross2Args args) {
     extern __shared__ uint8_t x2_smem_raw[];
     __shared__ __align__(8) uint64_t bar_full[X2_MAX_STAGES], bar_empty[X2_MAX_STAGES];
     __shared__ __align__(8) uint64_t bar_kv_full[2], bar_kv_empty[2];
@@ -136,31 +132,25 @@ cross2_attention_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid
     constexpr int EPILOGUE_WARP0 = NWG * 4;
     constexpr int LOADER_WARP = NWG * 4 + 4, S_ISSUER_WARP = NWG * 4 + 5, O_ISSUER_WARP = NWG * 4 + 6;
     constexpr int S2_ISSUER_WARP = NWG * 4 + 7;   // second S issuer: the odd items
-#ifdef SD_ATTN_TRACE
-    if (args.trace && blockIdx.x == 0 && threadIdx.x == 0) {
-        unsigned long long gt;
-        asm volatile("mov.u64 %0, %globaltimer;" : "=l"(gt));
-        args.trace[((NWG + 1) * 40 + 39) * 8 + 1] = clock64();
-        args.trace[((NWG + 1) * 40 + 39) * 8 + 4] = (long long)gt;
-    }
-#endif
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     if (threadIdx.x == 0) pdl_launch_dependents();   // the next kernel of the stream may start its set-up
-    if (threadIdx.x == 32) {   // the tensor maps are kernel parameters: their fetch need not wait for anything
-        tma_prefetch_desc(&tmap_q);
-        tma_prefetch_desc(&tmap_k);
-        tma_prefetch_desc(&tmap_v);
-        if (NWG == 4 && args.strided_rows) {
-            tma_prefetch_desc(&tmap_q_rows);
-            tma_prefetch_desc(&tmap_out_rows);
-        }
-    }
     const int nch = args.nch, dpad = args.dpad, stages = args.stages;
     // contiguous range of items for this CTA: consecutive items share a head, so K and V are fetched rarely
     const int per = args.n_items / gridDim.x, extra = args.n_items % gridDim.x;
     const int item0 = blockIdx.x * per + min((int)blockIdx.x, extra);
     const int n_local = per + ((int)blockIdx.x < extra ? 1 : 0);
-    const int bh0 = item0 / args.tiles_per_bh;   // head of the first item; head "group" g = bh - bh0
+    const int bh0 = item0 / args.tiles_per_bh;   // global head of the first item; head "group" g = global head - bh0
+    const int prob0 = bh0 / args.BH, hb0 = bh0 - prob0 * args.BH;   // its problem and its head inside that problem
+    if (threadIdx.x == 32 && n_local > 0) {   // the tensor maps are kernel parameters: their fetch need not wait for anything
+        const Cross2Problem& p0 = args.prob[prob0];
+        tma_prefetch_desc(&p0.tq);
+        tma_prefetch_desc(&p0.tk);
+        tma_prefetch_desc(&p0.tv);
+        if (NWG == 4 && args.strided_rows) {
+            tma_prefetch_desc(&p0.tq_rows);
+            tma_prefetch_desc(&p0.tout_rows);
+        }
+    }
 
     const uint32_t smem_base = (smem_u32(x2_smem_raw) + 1023u) & ~1023u;
     const uint32_t q_bytes = nch * TILE_M * CHUNK_ROW_BYTES, kv_bytes = nch * X2_KN * CHUNK_ROW_BYTES;
@@ -201,9 +191,6 @@ cross2_attention_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid
     // Set-up (barriers, tensor memory) overlapped the tail of the previous kernel of the stream; global memory and
     // every bounded wait come after it has completed.
     pdl_wait();
-#ifdef SD_ATTN_TRACE
-    if (args.trace && blockIdx.x == 0 && threadIdx.x == 0) args.trace[((NWG + 1) * 40 + 39) * 8 + 2] = clock64();
-#endif
     tc_fence_after_sync();
     const uint32_t tmem_base = tmem_base_slot;
     const uint32_t tmem_o0 = tmem_base + NWG * X2_KN;   // columns: S_0 .. S_{NWG-1} | O_0 .. O_{NWG-1}
@@ -221,8 +208,10 @@ cross2_attention_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid
         if (elect_one()) {
             int g_prev = 0;   // K and V of the first head: fetched by the first S issuer, at the same time as Q here
             for (int i = 0; i < n_local; ++i) {
-                const int item = item0 + i, bh = item / args.tiles_per_bh, tile = item - bh * args.tiles_per_bh;
-                const int s = i % stages, g = bh - bh0;
+                const int item = item0 + i, gh = item / args.tiles_per_bh, tile = item - gh * args.tiles_per_bh;
+                const int s = i % stages, g = gh - bh0;
+                const int pi = gh / args.BH, bh = gh - pi * args.BH;   // problem, head inside it
+                const Cross2Problem& pr = args.prob[pi];
                 const int bz = bh / args.lay.heads, hz = bh - bz * args.lay.heads;
                 if (g != g_prev) {
                     // a new head: its K and V go into buffer g & 1 once the head two back has been consumed
@@ -232,15 +221,14 @@ cross2_attention_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid
                     const uint32_t bar = smem_u32(&bar_kv_full[g & 1]), dst = kv_smem + (g & 1) * 2 * kv_bytes;
                     mbar_arrive_expect_tx(bar, 2 * kv_bytes);
                     for (int ch = 0; ch < nch; ++ch)
-                        tma_load_4d(dst + ch * X2_KN * CHUNK_ROW_BYTES, &tmap_k, bar, ch * CHUNK_COLS, 0, hz, bz);
+                        tma_load_4d(dst + ch * X2_KN * CHUNK_ROW_BYTES, &pr.tk, bar, ch * CHUNK_COLS, 0, hz, bz);
                     for (int ch = 0; ch < nch; ++ch)
-                        tma_load_4d(dst + kv_bytes + ch * X2_KN * CHUNK_ROW_BYTES, &tmap_v, bar, ch * CHUNK_COLS, 0, hz, bz);
+                        tma_load_4d(dst + kv_bytes + ch * X2_KN * CHUNK_ROW_BYTES, &pr.tv, bar, ch * CHUNK_COLS, 0, hz, bz);
                     g_prev = g;
                 }
                 if (i >= stages &&
                     !mbar_wait(smem_u32(&bar_empty[s]), ((i / stages) - 1) & 1, abort_p, args.status, SITE_Y_EMPTY, i))
                     break;
-                X2_TRACE(NWG + 1, i, 0);
                 const uint32_t bar = smem_u32(&bar_full[s]), dst = q_smem + s * q_bytes;
                 if (DENSE_Q) {
                     int rows = args.Nq - tile * TILE_M;
@@ -248,16 +236,16 @@ cross2_attention_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid
                     const uint32_t bytes = (uint32_t)rows * args.d * 2;   // d % 8 == 0: a multiple of 16
                     if (args.strided_rows) {   // the same dense tile, row by row (rows past Nq arrive as zeros)
                         mbar_arrive_expect_tx(bar, raw_bytes);
-                        tma_load_4d(raw_smem + s * raw_bytes, &tmap_q_rows, bar, 0, tile * TILE_M, hz, bz);
+                        tma_load_4d(raw_smem + s * raw_bytes, &pr.tq_rows, bar, 0, tile * TILE_M, hz, bz);
                         continue;
                     }
                     mbar_arrive_expect_tx(bar, bytes);
-                    bulk_load(raw_smem + s * raw_bytes, args.q + ((size_t)bh * args.Nq + (size_t)tile * TILE_M) * args.d, bytes, bar);
+                    bulk_load(raw_smem + s * raw_bytes, pr.q + ((size_t)bh * args.Nq + (size_t)tile * TILE_M) * args.d, bytes, bar);
                     continue;
                 }
                 mbar_arrive_expect_tx(bar, q_bytes);
                 for (int ch = 0; ch < nch; ++ch)
-                    tma_load_4d(dst + ch * TILE_M * CHUNK_ROW_BYTES, &tmap_q, bar, ch * CHUNK_COLS, tile * TILE_M, hz, bz);
+                    tma_load_4d(dst + ch * TILE_M * CHUNK_ROW_BYTES, &pr.tq, bar, ch * CHUNK_COLS, tile * TILE_M, hz, bz);
             }
         }
     } else if (warp == S_ISSUER_WARP || warp == S2_ISSUER_WARP || warp == O_ISSUER_WARP) {
@@ -270,30 +258,34 @@ cross2_attention_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid
         // a third issues O = P V (and frees K/V buffers).  S of item i+NWG reuses the columns of S/P of item i, so
         // an S issuer waits for that item's P V product to COMPLETE (bar_pv_done).
         if (elect_one()) {
-            struct Cursor { int i, s, sph, w, n, g, t; };
+            struct Cursor { int i, s, sph, w, n, g, t, hb, p; };
             const int t_first = item0 - bh0 * args.tiles_per_bh;
             auto advance = [&](Cursor& c) {   // item bookkeeping without divisions
                 ++c.i;
                 if (++c.s == stages) { c.s = 0; c.sph ^= 1; }
                 if (++c.w == NWG) { c.w = 0; ++c.n; }
-                if (++c.t == args.tiles_per_bh) { c.t = 0; ++c.g; }
+                if (++c.t == args.tiles_per_bh) {   // the next head, and past a problem's last head the next problem
+                    c.t = 0; ++c.g;
+                    if (++c.hb == args.BH) { c.hb = 0; ++c.p; }
+                }
             };
-            Cursor c = {0, 0, 0, 0, 0, 0, t_first};
+            Cursor c = {0, 0, 0, 0, 0, 0, t_first, hb0, prob0};
             bool ok = true;
             if (warp == S_ISSUER_WARP && n_local > 0) {
                 // K and V of the CTA's first head, while the producer thread fetches the first Q tiles: a copy
                 // instruction holds its thread for several hundred clocks, and the first scores wait for all three.
                 const uint32_t bar = smem_u32(&bar_kv_full[0]);
-                const int bz0 = bh0 / args.lay.heads, hz0 = bh0 - bz0 * args.lay.heads;
+                const int bz0 = hb0 / args.lay.heads, hz0 = hb0 - bz0 * args.lay.heads;
                 mbar_arrive_expect_tx(bar, 2 * kv_bytes);
                 for (int ch = 0; ch < nch; ++ch)
-                    tma_load_4d(kv_smem + ch * X2_KN * CHUNK_ROW_BYTES, &tmap_k, bar, ch * CHUNK_COLS, 0, hz0, bz0);
+                    tma_load_4d(kv_smem + ch * X2_KN * CHUNK_ROW_BYTES, &args.prob[prob0].tk, bar, ch * CHUNK_COLS, 0, hz0, bz0);
                 for (int ch = 0; ch < nch; ++ch)
-                    tma_load_4d(kv_smem + kv_bytes + ch * X2_KN * CHUNK_ROW_BYTES, &tmap_v, bar, ch * CHUNK_COLS, 0, hz0, bz0);
+                    tma_load_4d(kv_smem + kv_bytes + ch * X2_KN * CHUNK_ROW_BYTES, &args.prob[prob0].tv, bar, ch * CHUNK_COLS, 0, hz0, bz0);
             }
             if (warp != O_ISSUER_WARP) {
                 const int parity = warp == S_ISSUER_WARP ? 0 : 1;
-                const uint32_t idesc_s = idesc_f16(TILE_M, X2_KN, false, false, args.negate != 0, BF);
+                uint32_t idesc_s = idesc_f16(TILE_M, X2_KN, false, false, args.prob[prob0].negate != 0, BF);
+                int p_desc = prob0;   // the problem idesc_s was made for (only the sign of the scale differs)
                 const int ksteps_s = (args.d + 15) / 16;
                 const uint64_t q_desc0 = smem_desc_sw128(q_smem, 16, 1024);
                 const uint64_t k_desc0 = smem_desc_sw128(kv_smem, 16, 1024);
@@ -301,20 +293,20 @@ cross2_attention_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid
                 int g_waited = -1;   // K and V of this head have been seen to land
                 for (; c.i < n_local && ok; advance(c)) {
                     if ((c.i & 1) != parity) continue;
-                    X2_TRACE(NWG, c.i, 5);
                     ok = (DENSE_Q ? mbar_wait(smem_u32(&bar_q_ready[c.w]), c.n & 1, abort_p, args.status, SITE_Y_STAGE, c.i)
                                   : mbar_wait(smem_u32(&bar_full[c.s]), c.sph, abort_p, args.status, SITE_Y_STAGE, c.i));
-                    X2_TRACE(NWG, c.i, 6);
                     if (ok && c.g != g_waited) {
                         ok = mbar_wait(smem_u32(&bar_kv_full[c.g & 1]), (c.g >> 1) & 1, abort_p, args.status, SITE_Y_KV, c.i);
                         g_waited = c.g;
                     }
-                    X2_TRACE(NWG, c.i, 7);
                     if (ok && c.n >= 1)   // the group's previous item no longer needs these columns
                         ok = mbar_wait(smem_u32(&bar_pv_done[c.w]), (c.n - 1) & 1, abort_p, args.status, SITE_Y_PV, c.i);
                     if (!ok) break;
                     tc_fence_after_sync();
-                    X2_TRACE(NWG, c.i, 3);
+                    if (c.p != p_desc) {
+                        p_desc = c.p;
+                        idesc_s = idesc_f16(TILE_M, X2_KN, false, false, args.prob[p_desc].negate != 0, BF);
+                    }
                     const uint64_t qd = q_desc0 + (uint64_t)((DENSE_Q ? c.w : c.s) * q_stage_off);
                     const uint64_t kd = k_desc0 + (uint64_t)((c.g & 1) * kv_buf_off);
                     const uint32_t ts = tmem_base + c.w * X2_KN;
@@ -328,7 +320,6 @@ cross2_attention_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid
                                        kk > 0);
                     tc_commit(smem_u32(&bar_s_full[c.w]));
                     if (!DENSE_Q) tc_commit(smem_u32(&bar_empty[c.s]));   // the Q stage is free once this product has read it
-                    X2_TRACE(NWG, c.i, 4);
                 }
             } else {
                 const uint32_t idesc_o = idesc_f16(TILE_M, dpad, false, true, false, BF);
@@ -337,11 +328,9 @@ cross2_attention_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid
                 for (; c.i < n_local && ok; advance(c)) {
                     if (c.n >= 1)   // O_w of the group's previous item must have been read out
                         ok = mbar_wait(smem_u32(&bar_o_free[c.w]), (c.n - 1) & 1, abort_p, args.status, SITE_Y_OFREE, c.i);
-                    X2_TRACE(NWG, c.i, 0);
                     if (ok) ok = mbar_wait(smem_u32(&bar_p_full[c.w]), c.n & 1, abort_p, args.status, SITE_Y_P, c.i);
                     if (!ok) break;
                     tc_fence_after_sync();
-                    X2_TRACE(NWG, c.i, 1);
                     const uint64_t vd = v_desc0 + (uint64_t)((c.g & 1) * kv_buf_off);
 #pragma unroll
                     for (int kk = 0; kk < X2_KN / 16; ++kk)   // O_w = P_w V, P_w in the first columns of S_w
@@ -351,7 +340,6 @@ cross2_attention_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid
                     tc_commit(smem_u32(&bar_pv_done[c.w]));
                     // last item of its head: every S product of this head completed before its softmax ran
                     if (c.i + 1 == n_local || c.t + 1 == args.tiles_per_bh) tc_commit(smem_u32(&bar_kv_empty[c.g & 1]));
-                    X2_TRACE(NWG, c.i, 2);
                 }
             }
         }
@@ -362,10 +350,16 @@ cross2_attention_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid
         const int r = tid & (TILE_M - 1);
         const uint32_t lane_off = (uint32_t)((warp & 3) * 32) << 16;
         const uint32_t tmem_s = tmem_base + w * X2_KN + lane_off;
-        const float c2 = args.scale_log2e;
         const int valid = args.Nk;
         bool ok = true;
-        const bool tracer = (warp & 3) == 0 && lane == 0;
+        // the problem of this group's current item, advanced NWG items at a time without divisions
+        int it_t = item0 - bh0 * args.tiles_per_bh + w, it_hb = hb0, it_p = prob0;
+        auto settle = [&]() {
+            while (it_t >= args.tiles_per_bh) {
+                it_t -= args.tiles_per_bh;
+                if (++it_hb == args.BH) { it_hb = 0; ++it_p; }
+            }
+        };
         // DENSE_Q: rewrite the raw Q tile of item j (ring stage j % stages; j = w mod NWG and stages is a multiple of
         // NWG, so this group is the only consumer of that stage's barrier) into the group's MMA-layout buffer: row r
         // is 128 bytes at r * 128, its 16-byte chunk c at position c ^ (r & 7) (the 128-byte swizzle).
@@ -390,14 +384,14 @@ cross2_attention_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid
             return true;
         };
         if (DENSE_Q && w < n_local) ok = rewrite_q(w);
-        for (int i = w; i < n_local && ok; i += NWG) {
+        for (int i = w; i < n_local && ok; i += NWG, it_t += NWG) {
             const int n = i / NWG;
-            if (tracer) X2_TRACE(w, i, 0);
+            settle();
+            const float c2 = args.prob[it_p].scale_log2e;
             ok = mbar_wait(smem_u32(&bar_s_full[w]), n & 1, abort_p, args.status, SITE_Y_S, i);
             ok = __all_sync(0xffffffffu, ok);
             if (!ok) break;
             tc_fence_after_sync();
-            if (tracer) X2_TRACE(w, i, 1);
             if (DENSE_Q && i + NWG < n_local) {   // S of this item is done: the Q buffer may take the next one
                 ok = rewrite_q(i + NWG);
                 if (!ok) break;
@@ -457,7 +451,6 @@ cross2_attention_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid
             tc_fence_before_sync();
             __syncwarp();                           // every lane's store before lane 0's arrival
             if (lane == 0) mbar_arrive(smem_u32(&bar_p_full[w]));
-            if (tracer) X2_TRACE(w, i, 2);
         }
     } else if (warp < LOADER_WARP) {
         // ------------------------------------------------------------ epilogue warpgroup: every item in turn
@@ -466,8 +459,14 @@ cross2_attention_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid
         const uint32_t lane_off = (uint32_t)((warp & 3) * 32) << 16;
         bool ok = true;
         int w = 0, n = 0;
-        int bh = bh0, tile = item0 - bh0 * args.tiles_per_bh;
-        const bool tracer = warp == EPILOGUE_WARP0 && lane == 0;
+        int bh = hb0, pi = prob0, tile = item0 - bh0 * args.tiles_per_bh;   // head inside its problem, problem, tile
+        auto next_item = [&]() {
+            if (++w == NWG) { w = 0; ++n; }
+            if (++tile == args.tiles_per_bh) {
+                tile = 0;
+                if (++bh == args.BH) { bh = 0; ++pi; }
+            }
+        };
         for (int i = 0; i < n_local; ++i) {
             const uint32_t tmem_o = tmem_o0 + w * dpad + lane_off;
             // bar_o_full[w] completes after the O issuer saw bar_p_full[w], which the softmax warps arrived on after
@@ -480,10 +479,10 @@ cross2_attention_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid
             ok = DENSE_Q ? named_barrier_and(1, 128, ok) : __all_sync(0xffffffffu, ok);
             if (!ok) break;
             tc_fence_after_sync();
-            if (tracer) X2_TRACE(w, i, 3);
             const float inv = inv_sum[w][n & 1][r];
             const int row = tile * TILE_M + r;
-            __half* orow = head_row(args.out, args.lay, bh, row);
+            const Cross2Problem& pr = args.prob[pi];
+            __half* orow = head_row(pr.out, args.lay, bh, row);
             if (DENSE_Q) {
                 // The tile is one contiguous piece of global memory: rows go to a dense staging tile in shared memory
                 // (thread = row) and ONE bulk copy writes it out -- full lines instead of five strided 16-byte stores
@@ -512,16 +511,14 @@ cross2_attention_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid
                     if (rows > TILE_M) rows = TILE_M;
                     if (args.strided_rows) {   // rows past Nq are clipped by the hardware
                         const int bz = bh / args.lay.heads, hz = bh - bz * args.lay.heads;
-                        tma_store_4d(&tmap_out_rows, stage, 0, tile * TILE_M, hz, bz);
+                        tma_store_4d(&pr.tout_rows, stage, 0, tile * TILE_M, hz, bz);
                     } else {
-                        bulk_store(args.out + ((size_t)bh * args.Nq + (size_t)tile * TILE_M) * args.d, stage,
+                        bulk_store(pr.out + ((size_t)bh * args.Nq + (size_t)tile * TILE_M) * args.d, stage,
                                    (uint32_t)rows * args.d * 2);
                     }
                     bulk_commit();
                 }
-                if (tracer) X2_TRACE(w, i, 4);
-                if (++w == NWG) { w = 0; ++n; }
-                if (++tile == args.tiles_per_bh) { tile = 0; ++bh; }
+                next_item();
                 continue;
             }
             // O / S_i -> fp16 -> global, 32 columns per tensor-memory round trip (dpad is a multiple of 16)
@@ -546,9 +543,7 @@ cross2_attention_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid
                     }
                 }
             }
-            if (tracer) X2_TRACE(w, i, 4);
-            if (++w == NWG) { w = 0; ++n; }
-            if (++tile == args.tiles_per_bh) { tile = 0; ++bh; }
+            next_item();
         }
         if (DENSE_Q && tid == EPILOGUE_WARP0 * 32) bulk_wait_all();   // shared memory must outlive the copies
     }
@@ -565,14 +560,6 @@ cross2_attention_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid
         __syncwarp();
         tmem_dealloc(tmem_base, 512);
     }
-#ifdef SD_ATTN_TRACE
-    if (args.trace && blockIdx.x == 0 && threadIdx.x == 0) {
-        unsigned long long gt;
-        asm volatile("mov.u64 %0, %globaltimer;" : "=l"(gt));
-        args.trace[((NWG + 1) * 40 + 39) * 8 + 3] = clock64();
-        args.trace[((NWG + 1) * 40 + 39) * 8 + 5] = (long long)gt;
-    }
-#endif
 }
 
 }  // namespace sd_attn

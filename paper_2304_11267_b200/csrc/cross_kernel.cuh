@@ -34,7 +34,6 @@ struct CrossArgs {
     float scale_log2e;  // |scale| * log2(e)
     int negate;         // scale < 0: the MMA negates Q instead
     int* status;        // device status block
-    float* dump_scores; // optional [gridDim.y][gridDim.x][128][kn] raw scores, for bring-up tests
 };
 
 __host__ inline size_t cross_smem_bytes(int nch, int kn) {
@@ -134,12 +133,6 @@ cross_attention_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_
 #pragma unroll
             for (int c = 0; c < 16; ++c)
                 if (g * 16 + c < args.Nk) row_max = fmaxf(row_max, __uint_as_float(r[c]));
-            if (args.dump_scores) {
-                float* dst = args.dump_scores +
-                             (((size_t)bh * gridDim.x + tile) * TILE_M + tid) * kn + g * 16;
-#pragma unroll
-                for (int c = 0; c < 16; ++c) dst[c] = __uint_as_float(r[c]);
-            }
         }
         const float c2 = args.scale_log2e;
         const float neg_mc = -row_max * c2;

@@ -21,28 +21,30 @@
 // that it spreads over more SMs; with one tile the rotation degenerates to two alternating score buffers.
 // One tile per CTA normally runs the SPLIT variant instead (template parameter, see below): the other softmax
 // warpgroups, idle otherwise, take a share of the tile's score columns each.
-// The anchor scheme of the exponent (no per-tile maximum) is that of fused4_kernel.cuh.
+// The anchor scheme of the exponent (no per-tile maximum) is described in fused_common.cuh.
+//
+// One launch serves up to F4_GROUP_MAX problems of one shape (a tensor-map triple, an output pointer and a scale
+// each).  A UNIT is the group of up to T query tiles of a head that share a CTA's K/V stream.  Two ways to deal the
+// units out:
+//   whole units   one CTA per (problem, unit), all key tiles.
+//   shares        the work of a problem is the line of its W = units x key tiles steps (unit, key tile), and CTA c of
+//                 G takes the steps [c W / G, (c + 1) W / G) of EVERY problem of the launch in turn -- one or two
+//                 SEGMENTS (unit, first key tile, count) per problem.  The host launches one CTA per SM, so that no
+//                 SM idles in a last, partly filled wave (the 512 query tiles of the 4096-token call: 128 units on
+//                 148 SMs).  A unit whose key tiles are cut between CTAs is finished through global scratch: each
+//                 piece stores its unnormalised accumulator, anchor and row sum, and whichever piece's warpgroup
+//                 arrives last (a counter per query tile) combines all pieces in key order -- nobody waits, and
+//                 neither the cut points (a function of the problem's shape and G only) nor the order of additions
+//                 depend on who arrives last or on what else is in the launch, so the bits repeat.
+// Between two segments of a CTA the barriers are re-initialised behind a CTA-wide barrier (all asynchronous
+// arrivals of the finished segment have been waited for by then); tensor memory and shared memory carry on.
 #pragma once
 #include <cuda.h>
 
-#include "fused4_kernel.cuh"  // Fused4Args, F4_* constants, SITE_G_*
+#include "fused_common.cuh"  // Fused4Args, F4_* constants, SITE_G_*
 
 namespace sd_attn {
 
-// Trace builds only: coarse timeline of CTA (0, 0) -- globaltimer and clock64 at mark i -- behind the per-role stamps.
-#ifdef SD_ATTN_TRACE
-#define F4S_MARK(i)                                                                                   \
-    do {                                                                                              \
-        if (args.trace && blockIdx.x == 0 && blockIdx.y == 0) {                                       \
-            unsigned long long gt_;                                                                   \
-            asm volatile("mov.u64 %0, %globaltimer;" : "=l"(gt_));                                    \
-            args.trace[5 * 40 * 8 + 1024 + (i)] = (long long)gt_;                                     \
-            args.trace[5 * 40 * 8 + 1024 + 16 + (i)] = clock64();                                     \
-        }                                                                                             \
-    } while (0)
-#else
-#define F4S_MARK(i) do { } while (0)
-#endif
 
 constexpr int F4S_MAX_DPAD = 160;
 constexpr int F4S_MAX_KSTEPS = 10;          // MMA steps of Q K^T at the largest head dim
@@ -77,8 +79,7 @@ static_assert(512 * F4S_SOFTMAX_REGS + 256 * F4S_CONTROL_REGS == 768 * 80, "setm
 // two threads: the products of key tile j from one, the scores of key tile j + NB from the other.
 template <int POLY, int NCH, int SPLIT = 1, bool BF = false>   // NCH: 64-column chunks per row (head dim <= 64 * NCH); BF: bfloat16 tensors
 __global__ void __launch_bounds__(F4_THREADS, 1)
-fused4s_attention_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__ CUtensorMap tmap_k,
-                         const __grid_constant__ CUtensorMap tmap_v, const Fused4Args args) {
+fused4s_attention_kernel(const __grid_constant__ Fused4Args args) {
     constexpr int BN = F4_BN;
     extern __shared__ uint8_t f4s_smem_raw[];
     // per (tile, buffer): S ready (MMA) | P ready (softmax).  per tile: Q landed | P V of key tile j done | all of
@@ -91,31 +92,22 @@ fused4s_attention_kernel(const __grid_constant__ CUtensorMap tmap_q, const __gri
     __shared__ __align__(8) uint64_t bar_buf_free[F4S_BUFFERS];   // SPLIT > 1: the products reading a buffer's weights are done
     __shared__ uint32_t tmem_base_slot;
     __shared__ int abort_flag;
+    __shared__ int piece_ticket[F4_TILES];   // a query tile's arrival number among the pieces of its unit
+    // the segment the CTA works on, written by the scheduling thread: live? | problem | unit | first key tile | key
+    // tiles | query tiles | nothing follows  (in shared memory so that no role carries the walk in registers)
+    __shared__ int seg_desc[8];
     __shared__ float2 part_ml[SPLIT > 1 ? SPLIT : 1][SPLIT > 1 ? TILE_M : 1];   // SPLIT > 1: (anchor, row sum) of every part
 
     const int tid = threadIdx.x, lane = tid & 31;
     const int warp = __shfl_sync(0xffffffffu, tid >> 5, 0);   // warp-uniform for the compiler
     if (threadIdx.x == 0) pdl_launch_dependents();   // the next kernel of the stream may start its set-up
+    const int n_kv_all = args.n_kv;
     if (threadIdx.x == 32) {   // the tensor maps are kernel parameters: their fetch need not wait for anything
-        tma_prefetch_desc(&tmap_q);
-        tma_prefetch_desc(&tmap_k);
-        tma_prefetch_desc(&tmap_v);
+        const int p0 = args.shares ? 0 : (int)(blockIdx.x / args.n_units);
+        tma_prefetch_desc(&args.prob[p0].tq);
+        tma_prefetch_desc(&args.prob[p0].tk);
+        tma_prefetch_desc(&args.prob[p0].tv);
     }
-    const int bh = blockIdx.y;
-    const int row_base = blockIdx.x * args.tiles_per_cta * TILE_M;
-#ifdef SD_ATTN_TRACE
-    if (args.trace && tid == 0) {   // per-CTA start stamp and SM id
-        unsigned long long gt; unsigned smid;
-        asm volatile("mov.u64 %0, %globaltimer;" : "=l"(gt));
-        asm volatile("mov.u32 %0, %smid;" : "=r"(smid));
-        const int cta = blockIdx.y * gridDim.x + blockIdx.x;
-        if (cta < 256) { args.trace[5 * 40 * 8 + cta * 4] = (long long)gt; args.trace[5 * 40 * 8 + cta * 4 + 2] = smid; }
-    }
-#endif
-    int T = (args.Nq - row_base + TILE_M - 1) / TILE_M;   // query tiles of this CTA
-    if (T > args.tiles_per_cta) T = args.tiles_per_cta;
-    const int NB = SPLIT > 1 ? args.split_buffers : T + 1;   // score buffers in the rotation
-    const int n_kv = (args.Nk + BN - 1) / BN;
     const int dpad = args.dpad;
     constexpr int nch = NCH;
     const int stages = args.stages;   // K/V ring depth
@@ -127,23 +119,68 @@ fused4s_attention_kernel(const __grid_constant__ CUtensorMap tmap_q, const __gri
     const uint32_t kv_smem = q_smem + args.tiles_per_cta * q_tile_bytes;   // [stages][K | V]
     volatile int* abort_p = &abort_flag;
 
-    if (tid == 0) {
-        abort_flag = 0;
-        for (int t = 0; t < F4_TILES; ++t) {
-            for (int b = 0; b < F4S_BUFFERS; ++b) {
-                mbar_init(smem_u32(&bar_s_full[t][b]), 1);
-                mbar_init(smem_u32(&bar_p_full[t][b]), 4);    // one arrival per softmax warp of the tile (SPLIT > 1: of the part)
+    // (Re-)initialise every barrier for a segment of `tiles` query tiles; `again`: they hold a finished segment's state.
+    auto init_barriers = [&](int tiles, bool again) {
+        auto each = [&](auto&& f) {
+            for (int t = 0; t < F4_TILES; ++t) {
+                for (int b = 0; b < F4S_BUFFERS; ++b) {
+                    f(&bar_s_full[t][b], 1);
+                    f(&bar_p_full[t][b], 4);    // one arrival per softmax warp of the tile (SPLIT > 1: of the part)
+                }
+                f(&bar_q_full[t], 1);
+                f(&bar_pv_done[t], 1);
+                f(&bar_o_final[t], 1);
             }
-            mbar_init(smem_u32(&bar_q_full[t]), 1);
-            mbar_init(smem_u32(&bar_pv_done[t]), 1);
-            mbar_init(smem_u32(&bar_o_final[t]), 1);
+            for (int b = 0; b < F4S_BUFFERS; ++b) f(&bar_buf_free[b], 1);
+            for (int s = 0; s < F4_STAGES; ++s) {
+                f(&bar_kv_full[s], 1);
+                f(&bar_kv_empty[s], tiles);   // one commit per issuer
+            }
+        };
+        // Retire them all first, fence, then initialise them all.  (mbarrier.inval and mbarrier.init of ONE barrier
+        // issued back to back came out wrong on the GPU: ring barriers of the next segment completed an arrival
+        // early and the last query tiles multiplied by the wrong V tile.)
+        if (again) {
+            each([&](uint64_t* bar, uint32_t) { mbar_inval(smem_u32(bar)); });
+            __threadfence_block();
+            fence_proxy_async_smem();
         }
-        for (int b = 0; b < F4S_BUFFERS; ++b) mbar_init(smem_u32(&bar_buf_free[b]), 1);
-        for (int s = 0; s < F4_STAGES; ++s) {
-            mbar_init(smem_u32(&bar_kv_full[s]), 1);
-            mbar_init(smem_u32(&bar_kv_empty[s]), T);   // one commit per issuer
-        }
+        each([&](uint64_t* bar, uint32_t arrivals) { mbar_init(smem_u32(bar), arrivals); });
         mbar_init_fence();
+    };
+    // The scheduling thread (lane 0 of an otherwise idle control warp) walks this CTA's steps: [w_begin, w_end) of the
+    // W = units x key tiles of a problem -- of every problem in turn when the launch deals shares out.
+    constexpr int SCHED_TID = 21 * 32;
+    const int W = args.n_units * n_kv_all;                             // (the host keeps it below 2^31)
+    const int G = args.shares ? (int)gridDim.x : args.n_units;         // CTAs among which a problem's steps are dealt out
+    const int cta = args.shares ? (int)blockIdx.x : (int)(blockIdx.x % args.n_units);   // this CTA among them
+    const int w_begin = (int)((long long)cta * W / G), w_end = (int)((long long)(cta + 1) * W / G);
+    int sched_w = w_begin, sched_prob = args.shares ? 0 : (int)(blockIdx.x / args.n_units);
+    const int sched_prob_end = args.shares ? args.n_prob : sched_prob + 1;
+    // publishes the next segment (or "none") and (re-)initialises the barriers for it
+    auto next_segment = [&](bool again) {
+        if (!(sched_w < w_end)) {   // on to this CTA's share of the next problem
+            sched_w = w_begin;
+            ++sched_prob;
+        }
+        if (sched_prob >= sched_prob_end || !(w_begin < w_end)) {
+            seg_desc[0] = 0;
+            return;
+        }
+        const int unit = sched_w / n_kv_all, j0 = sched_w - unit * n_kv_all;
+        const int n = (w_end - sched_w) < (n_kv_all - j0) ? (w_end - sched_w) : (n_kv_all - j0);
+        const int quad = unit % args.units_per_head;
+        int tiles = (args.Nq - quad * args.tiles_per_cta * TILE_M + TILE_M - 1) / TILE_M;
+        if (tiles > args.tiles_per_cta) tiles = args.tiles_per_cta;
+        sched_w += n;
+        seg_desc[0] = 1; seg_desc[1] = sched_prob; seg_desc[2] = unit; seg_desc[3] = j0; seg_desc[4] = n;
+        seg_desc[5] = tiles;
+        seg_desc[6] = !(sched_w < w_end) && sched_prob + 1 == sched_prob_end;
+        init_barriers(tiles, again);
+    };
+    if (tid == SCHED_TID) {
+        abort_flag = 0;
+        next_segment(false);
     }
     if (warp == 16) {
         tmem_alloc(smem_u32(&tmem_base_slot), 512);
@@ -155,13 +192,24 @@ fused4s_attention_kernel(const __grid_constant__ CUtensorMap tmap_q, const __gri
     // Set-up (barriers, tensor memory) overlapped the tail of the previous kernel of the stream; global memory and
     // every bounded wait come after it has completed.
     pdl_wait();
-    if (tid == 0) F4S_MARK(0);
     const uint32_t tmem_base = tmem_base_slot;
     // columns: the score buffers | O_0 .. O_{T-1} (SPLIT > 1: the parts' O_0 .. O_{SPLIT-1})
     const uint32_t tmem_o0 = tmem_base + (SPLIT > 1 ? args.split_buffers : args.tiles_per_cta + 1) * BN;
 
-    // One setmaxnreg site per kind, executed by whole warpgroups; the budget is the CTA's launch allocation.
-    if (warp >= 16) setmaxnreg_dec<F4S_CONTROL_REGS>();
+    // One setmaxnreg site per kind, executed by whole warpgroups; the budget is the CTA's launch allocation.  The
+    // control warps and the softmax warps each walk the CTA's segments in a loop of their own (the code behind a
+    // setmaxnreg must be reachable from that one only) and meet at the CTA-wide barriers between segments.
+    if (warp >= 16) {
+    setmaxnreg_dec<F4S_CONTROL_REGS>();
+    for (;;) {
+    // ------------------------------------------------------------ the segment: key tiles j0 .. j0 + n_kv - 1 of a unit
+    if (!seg_desc[0]) break;
+    const int prob_i = seg_desc[1], unit = seg_desc[2], j0 = seg_desc[3], n_kv = seg_desc[4], T = seg_desc[5];
+    const bool last_segment = seg_desc[6] != 0;
+    const int quad = unit % args.units_per_head, bh = unit / args.units_per_head;
+    const Fused4Problem& pr = args.prob[prob_i];
+    const int row_base = quad * args.tiles_per_cta * TILE_M;
+    const int NB = SPLIT > 1 ? args.split_buffers : T + 1;   // score buffers in the rotation
     if (warp == 16) {
         // ------------------------------------------------------------ TMA producer
         if (elect_one()) {
@@ -172,7 +220,7 @@ fused4s_attention_kernel(const __grid_constant__ CUtensorMap tmap_q, const __gri
                 const uint32_t bar = smem_u32(&bar_q_full[t]);
                 mbar_arrive_expect_tx(bar, q_tile_bytes);
                 for (int ch = 0; ch < nch; ++ch)
-                    tma_load_4d(q_smem + t * q_tile_bytes + ch * TILE_M * CHUNK_ROW_BYTES, &tmap_q, bar, ch * CHUNK_COLS,
+                    tma_load_4d(q_smem + t * q_tile_bytes + ch * TILE_M * CHUNK_ROW_BYTES, &pr.tq, bar, ch * CHUNK_COLS,
                                 row_base + t * TILE_M, hz, bz);
             };
             load_q(0);
@@ -185,15 +233,21 @@ fused4s_attention_kernel(const __grid_constant__ CUtensorMap tmap_q, const __gri
                 const uint32_t bar = smem_u32(&bar_kv_full[s]);
                 mbar_arrive_expect_tx(bar, 2 * kv_tile_bytes);
                 for (int ch = 0; ch < nch; ++ch)
-                    tma_load_4d(k_dst + ch * BN * CHUNK_ROW_BYTES, &tmap_k, bar, ch * CHUNK_COLS, j * BN, hz, bz);
+                    tma_load_4d(k_dst + ch * BN * CHUNK_ROW_BYTES, &pr.tk, bar, ch * CHUNK_COLS, (j0 + j) * BN, hz, bz);
                 for (int ch = 0; ch < nch; ++ch)
-                    tma_load_4d(v_dst + ch * BN * CHUNK_ROW_BYTES, &tmap_v, bar, ch * CHUNK_COLS, j * BN, hz, bz);
+                    tma_load_4d(v_dst + ch * BN * CHUNK_ROW_BYTES, &pr.tv, bar, ch * CHUNK_COLS, (j0 + j) * BN, hz, bz);
                 if (j == 0)
                     for (int t = 1; t < T; ++t) load_q(t);
             }
-            if (n_kv == 0)
-                for (int t = 1; t < T; ++t) load_q(t);
+            // Another segment follows: the issuers' last commits on the ring (never waited for above) must have
+            // landed before the barriers are initialised again.
+            if (!last_segment) {
+                for (int j = n_kv > stages ? n_kv - stages : 0; j < n_kv; ++j)
+                    if (!mbar_wait(smem_u32(&bar_kv_empty[j % stages]), (j / stages) & 1, abort_p, args.status, SITE_G_EMPTY, j))
+                        break;
+            }
         }
+        __syncwarp();
     } else if (warp > 16 && warp <= 16 + F4_TILES) {
         // ------------------------------------------------------------ MMA issuer of the steps of query tile t
         // Issuer t waits for P of its own tile's step k = T*j + t, issues O_t += P V(j), and then -- behind that
@@ -201,7 +255,7 @@ fused4s_attention_kernel(const __grid_constant__ CUtensorMap tmap_q, const __gri
         // NEXT tile of the rotation.
         const int t = warp - 17;
         if ((t < T || (SPLIT > 1 && t == 1)) && elect_one()) {
-            const uint32_t idesc_s = idesc_f16(TILE_M, BN, false, false, args.negate != 0, BF);
+            const uint32_t idesc_s = idesc_f16(TILE_M, BN, false, false, pr.negate != 0, BF);
             const uint32_t idesc_o = idesc_f16(TILE_M, dpad, false, true, false, BF);
             const int ksteps_s = (args.d + 15) / 16;   // 16 columns each; four to a swizzled 64-column chunk
             const int tn = (t + 1 == T) ? 0 : t + 1;   // the tile whose scores this thread requests
@@ -317,26 +371,44 @@ fused4s_attention_kernel(const __grid_constant__ CUtensorMap tmap_q, const __gri
                 const bool more = jn < n_kv;
                 if (more)   // landed long ago: keep this wait off the critical path
                     ok = mbar_wait(smem_u32(&bar_kv_full[sn]), pn, abort_p, args.status, SITE_G_KV, jn);
-                if (t == 0) FUSED_TRACE(4, j, 0);
                 if (ok) ok = mbar_wait(smem_u32(&bar_p_full[t][b]), ph, abort_p, args.status, SITE_G_P, j);
                 if (!ok) break;
                 tc_fence_after_sync();
-                if (t == 0) FUSED_TRACE(4, j, 1);
                 issue_o(j, sj, b);
                 if (more) issue_s(q_desc, tn, sn, b);               // into the buffer P is read from: behind it, in order
                 tc_commit(b_pvdone);                                // O_t holds key tiles 0..j
                 tc_commit(smem_u32(&bar_kv_empty[sj]));             // this issuer is done with K(j), V(j)
                 if (j == n_kv - 1) tc_commit(smem_u32(&bar_o_final[t]));
-                if (t == 0) FUSED_TRACE(4, j, 2);
                 b = (b == 0) ? NB - 1 : b - 1;              // k += NB - 1
                 if (++jm == NB) { jm = 0; ph ^= 1; }
                 if (++sj == stages) sj = 0;
                 if (++sn == stages) { sn = 0; pn ^= 1; }
             }
         }
-    } else if (warp < 16) {
+        __syncwarp();
+    }
+    // Every asynchronous arrival of this segment has been waited for (see the end of each role), so the barriers can
+    // start over for the next one; tensor memory and shared memory simply carry on.
+    tc_fence_before_sync();
+    __syncthreads();
+    if (last_segment || abort_flag) break;
+    if (tid == SCHED_TID) next_segment(true);
+    __syncthreads();
+    tc_fence_after_sync();
+    }   // the next segment of this CTA
+    } else {
+    setmaxnreg_inc<F4S_SOFTMAX_REGS>();
+    for (;;) {
+    // ------------------------------------------------------------ the segment: key tiles j0 .. j0 + n_kv - 1 of a unit
+    if (!seg_desc[0]) break;
+    const int prob_i = seg_desc[1], unit = seg_desc[2], j0 = seg_desc[3], n_kv = seg_desc[4], T = seg_desc[5];
+    const bool last_segment = seg_desc[6] != 0;
+    const int quad = unit % args.units_per_head, bh = unit / args.units_per_head;
+    const Fused4Problem& pr = args.prob[prob_i];
+    const int row_base = quad * args.tiles_per_cta * TILE_M;
+    const int NB = SPLIT > 1 ? args.split_buffers : T + 1;   // score buffers in the rotation
+    {
         // ------------------------------------------------------------ softmax warps
-        setmaxnreg_inc<F4S_SOFTMAX_REGS>();
         const int t = warp >> 2;                 // query tile of this warpgroup
         if (SPLIT > 1) {
             // ---- one query tile, SPLIT parts: warpgroup g takes the key tiles j = g, g + SPLIT, ... whole
@@ -346,7 +418,7 @@ fused4s_attention_kernel(const __grid_constant__ CUtensorMap tmap_q, const __gri
                 const uint32_t lane_off = (uint32_t)((warp & 3) * 32) << 16;
                 const uint32_t tmem_og = tmem_o0 + g * dpad + lane_off;
                 const uint32_t b_pvdone = smem_u32(&bar_pv_done[g]);   // products of THIS part's key tiles
-                const float c2 = args.scale_log2e;
+                const float c2 = pr.scale_log2e;
                 float m_run = 0.f, l_run = 0.f;   // anchor and row sum over this part's keys
                 bool ok = true;
                 // NB is a multiple of SPLIT, so buffer b = j % NB always meets the same part: one consumer per barrier.
@@ -358,8 +430,7 @@ fused4s_attention_kernel(const __grid_constant__ CUtensorMap tmap_q, const __gri
                     ok = __all_sync(0xffffffffu, ok);
                     if (!ok) break;
                     tc_fence_after_sync();
-                    if (tid == 0 && (j == 0 || j == 32 || j == n_kv - 1)) F4S_MARK(j == 0 ? 1 : j == 32 ? 3 : 4);
-                    const int valid = args.Nk - j * BN;   // columns >= valid are zero-filled keys
+                    const int valid = args.Nk - (j0 + j) * BN;   // columns >= valid are zero-filled keys
                     uint32_t s[BN];
                     tmem_ld32(tmem_s, &s[0]);
                     tmem_ld32(tmem_s + 32, &s[32]);
@@ -433,12 +504,10 @@ fused4s_attention_kernel(const __grid_constant__ CUtensorMap tmap_q, const __gri
                     b += SPLIT;
                     if (b >= NB) { b -= NB; ph ^= 1; }
                 }
-                if (tid == 0) F4S_MARK(5);
                 // ---- combine the parts: o = sum_g 2^(m_g - m) O_g / sum_g 2^(m_g - m) l_g, m = max_g m_g
                 part_ml[g][r] = make_float2(m_run, l_run);
                 if (ok) ok = mbar_wait(smem_u32(&bar_o_final[0]), 0, abort_p, args.status, SITE_G_O, g);
                 ok = named_barrier_and(1, SPLIT * 128, ok);   // every part's (m, l) is in shared memory, every product done
-                if (tid == 0) F4S_MARK(6);
                 if (ok) {
                     tc_fence_after_sync();
                     float f[SPLIT];
@@ -456,7 +525,7 @@ fused4s_attention_kernel(const __grid_constant__ CUtensorMap tmap_q, const __gri
 #pragma unroll
                     for (int p2 = 0; p2 < SPLIT; ++p2) f[p2] *= inv;
                     const int row = row_base + r;
-                    __half* orow = head_row(args.out, args.lay, bh, row);
+                    __half* orow = head_row(pr.out, args.lay, bh, row);
                     // the column groups of 16 are shared out among the parts; a thread reads its row of every O_p
                     for (int cg = g; cg < (dpad >> 4); cg += SPLIT) {
                         float acc[16];
@@ -488,29 +557,24 @@ fused4s_attention_kernel(const __grid_constant__ CUtensorMap tmap_q, const __gri
             const uint32_t lane_off = (uint32_t)((warp & 3) * 32) << 16;
             const uint32_t tmem_o = tmem_o0 + t * dpad + lane_off;
             const uint32_t b_pvdone = smem_u32(&bar_pv_done[t]);
-            const float c2 = args.scale_log2e;
+            const float c2 = pr.scale_log2e;
             float m_run = 0.f;   // anchor of the exponent: a bound on the running max, times scale*log2(e)
             float l_run = 0.f;   // running sum of p (relative to m_run)
             bool ok = true;
-            const bool tracer = (warp & 3) == 0 && lane == 0;
             // step k = T*j + t uses buffer k % NB; k grows by T = NB - 1 per key tile, so the buffer index walks down and
             // tile t meets each buffer every NB key tiles: phase (j / NB) & 1 of that (tile, buffer) barrier pair
             int b = t % NB, ph = 0, jm = 0;
             for (int j = 0; j < n_kv; ++j) {
                 const uint32_t tmem_s = tmem_base + b * BN + lane_off;
-                if (tracer) FUSED_TRACE(t, j, 0);
                 ok = mbar_wait(smem_u32(&bar_s_full[t][b]), ph, abort_p, args.status, SITE_G_S, j);
                 ok = __all_sync(0xffffffffu, ok);
                 if (!ok) break;
                 tc_fence_after_sync();
-                if (tracer) FUSED_TRACE(t, j, 1);
-                if (tid == 0 && (j == 0 || j == 1 || j == 32 || j == n_kv - 1)) F4S_MARK(j == 0 ? 1 : j == 1 ? 2 : j == 32 ? 3 : 4);
-                const int valid = args.Nk - j * BN;   // columns >= valid are zero-filled keys
+                const int valid = args.Nk - (j0 + j) * BN;   // columns >= valid are zero-filled keys
                 uint32_t s[BN];
                 tmem_ld32(tmem_s, &s[0]);
                 tmem_ld32(tmem_s + 32, &s[32]);
                 tmem_wait_ld();
-                if (tracer) FUSED_TRACE(t, j, 2);
                 const bool ragged = valid < BN;   // only the last key tile can be
                 if (j == 0) {
                     const float row_max = ragged ? row_max_masked<BN>(s, valid) : row_max_bf16<BN>(s);
@@ -571,7 +635,6 @@ fused4s_attention_kernel(const __grid_constant__ CUtensorMap tmap_q, const __gri
                 if (!ok) break;
                 l_run += tile_sum;
                 tmem_st32(tmem_s, packed);   // P_t(j) over the first columns of the buffer, whose scores sit in registers
-                if (tracer) FUSED_TRACE(t, j, 4);
                 tmem_wait_st();
                 // A parity wait is only sound while the waiter is at most one phase behind.  The scores of this tile
                 // are requested by ANOTHER issuer than the one that multiplies P_t V, so nothing else orders this
@@ -584,19 +647,18 @@ fused4s_attention_kernel(const __grid_constant__ CUtensorMap tmap_q, const __gri
                 }
                 tc_fence_before_sync();
                 if (lane == 0) mbar_arrive(smem_u32(&bar_p_full[t][b]));
-                if (tracer) FUSED_TRACE(t, j, 5);
                 b = (b == 0) ? NB - 1 : b - 1;              // k += NB - 1
                 if (++jm == NB) { jm = 0; ph ^= 1; }
             }
-            if (tid == 0) F4S_MARK(5);
             if (ok) ok = mbar_wait(smem_u32(&bar_o_final[t]), 0, abort_p, args.status, SITE_G_O, t);
+            // (the last phase of the product barrier, never consumed above: nothing of this segment is in flight after it)
+            if (ok) ok = mbar_wait(b_pvdone, (n_kv - 1) & 1, abort_p, args.status, SITE_G_PV, n_kv);
             ok = __all_sync(0xffffffffu, ok);
-            if (tid == 0) F4S_MARK(6);
-            if (ok) {
+            const int row = row_base + t * TILE_M + r;
+            __half* orow = head_row(pr.out, args.lay, bh, row);
+            if (ok && j0 == 0 && n_kv == n_kv_all) {   // all key tiles of the unit: no pieces to combine
                 tc_fence_after_sync();
                 const float inv = 1.f / l_run;
-                const int row = row_base + t * TILE_M + r;
-                __half* orow = head_row(args.out, args.lay, bh, row);
                 for (int g = 0; g < (dpad >> 4); ++g) {
                     uint32_t x[16];
                     tmem_ld16(tmem_o + g * 16, x);
@@ -615,15 +677,82 @@ fused4s_attention_kernel(const __grid_constant__ CUtensorMap tmap_q, const __gri
                         if (g * 16 + 16 <= args.d) *reinterpret_cast<uint4*>(orow + g * 16 + 8) = hi;
                     }
                 }
+            } else if (ok) {
+                // ---- a piece of the unit's key range: (O, anchor, row sum) to the scratch, column by column so that a
+                // warp writes whole lines; a CTA has at most two pieces (its first segment may begin and its last may
+                // end inside a unit), slot 0 for one that begins inside, slot 1 for one that begins a unit
+                tc_fence_after_sync();
+                const int cols = dpad + 2;
+                const size_t tile_off = (size_t)t * cols * TILE_M + r;
+                const size_t slot0 = 2 * (size_t)prob_i * (size_t)G;   // the problem's slots: two per CTA
+                float* piece = args.part + (slot0 + 2 * (size_t)cta + (j0 > 0 ? 0 : 1)) * args.part_slot_floats + tile_off;
+                for (int g = 0; g < (dpad >> 4); ++g) {
+                    uint32_t x[16];
+                    tmem_ld16(tmem_o + g * 16, x);
+                    tmem_wait_ld();
+#pragma unroll
+                    for (int c = 0; c < 16; ++c) piece[(g * 16 + c) * TILE_M] = __uint_as_float(x[c]);
+                }
+                piece[dpad * TILE_M] = m_run;
+                piece[(dpad + 1) * TILE_M] = l_run;
+                __threadfence();
+                named_barrier(2 + t, TILE_M);
+                int* counter = args.part_count + ((size_t)prob_i * args.n_units + unit) * F4_TILES + t;
+                if (r == 0) piece_ticket[t] = atomicAdd(counter, 1);
+                named_barrier(2 + t, TILE_M);
+                // the pieces of this unit: CTAs c_first .. c_last, in key order (CTA c begins at step c W / G)
+                const long long u0 = (long long)unit * n_kv_all;
+                const int W = args.n_units * n_kv_all, G = (int)gridDim.x, cta = (int)blockIdx.x;
+                const int c_first = (int)(((u0 + 1) * G - 1) / W), c_last = (int)(((u0 + n_kv_all) * G - 1) / W);
+                if (piece_ticket[t] == c_last - c_first) {
+                    // every other piece is complete: combine them all,
+                    // o = sum_c 2^(m_c - m) O_c / sum_c 2^(m_c - m) l_c with m = max_c m_c
+                    __threadfence();
+                    if (r == 0) *counter = 0;   // as the next launch expects it
+                    auto piece_of = [&](int c) -> const float* {
+                        const long long begin = (long long)c * W / G;
+                        return args.part + (slot0 + 2 * (size_t)c + (u0 < begin ? 0 : 1)) * args.part_slot_floats + tile_off;
+                    };
+                    float m_all = -INFINITY, l_all = 0.f;
+                    for (int c = c_first; c <= c_last; ++c) m_all = fmaxf(m_all, __ldcg(piece_of(c) + dpad * TILE_M));
+                    for (int c = c_first; c <= c_last; ++c) {
+                        const float* pc = piece_of(c);
+                        l_all += ex2_approx(__ldcg(pc + dpad * TILE_M) - m_all) * __ldcg(pc + (dpad + 1) * TILE_M);
+                    }
+                    const float inv = 1.f / l_all;
+                    for (int g = 0; g < (args.d >> 3); ++g) {
+                        float acc[8];
+#pragma unroll
+                        for (int k = 0; k < 8; ++k) acc[k] = 0.f;
+                        for (int c = c_first; c <= c_last; ++c) {
+                            const float* pc = piece_of(c);
+                            const float f = ex2_approx(__ldcg(pc + dpad * TILE_M) - m_all) * inv;
+#pragma unroll
+                            for (int k = 0; k < 8; ++k) acc[k] = fmaf(__ldcg(pc + (g * 8 + k) * TILE_M), f, acc[k]);
+                        }
+                        uint4 o;
+                        o.x = pack_16x2<BF>(acc[0], acc[1]); o.y = pack_16x2<BF>(acc[2], acc[3]);
+                        o.z = pack_16x2<BF>(acc[4], acc[5]); o.w = pack_16x2<BF>(acc[6], acc[7]);
+                        if (row < args.Nq) *reinterpret_cast<uint4*>(orow + g * 8) = o;
+                    }
+                }
             }
         }
     }
-
-    // ------------------------------------------------------------ teardown (every thread arrives)
-    if (tid == 0) F4S_MARK(7);
+    // Every asynchronous arrival of this segment has been waited for (see the end of each role), so the barriers can
+    // start over for the next one; tensor memory and shared memory simply carry on.
     tc_fence_before_sync();
     __syncthreads();
-    if (tid == 0) F4S_MARK(8);
+    if (last_segment || abort_flag) break;
+    if (tid == SCHED_TID) next_segment(true);
+    __syncthreads();
+    tc_fence_after_sync();
+    }   // the next segment of this CTA
+    }
+
+    // ------------------------------------------------------------ teardown (every thread arrives)
+    tc_fence_before_sync();
+    __syncthreads();
     if (warp == 16 && lane == 0 && abort_flag) {
         for (int s = 0; s < F4_STAGES; ++s) mbar_drain(smem_u32(&bar_kv_full[s]), 0);
     }
@@ -632,14 +761,6 @@ fused4s_attention_kernel(const __grid_constant__ CUtensorMap tmap_q, const __gri
         __syncwarp();
         tmem_dealloc(tmem_base, 512);
     }
-#ifdef SD_ATTN_TRACE
-    if (args.trace && tid == 0) {
-        unsigned long long gt;
-        asm volatile("mov.u64 %0, %globaltimer;" : "=l"(gt));
-        const int cta = blockIdx.y * gridDim.x + blockIdx.x;
-        if (cta < 256) args.trace[5 * 40 * 8 + cta * 4 + 1] = (long long)gt;
-    }
-#endif
 }
 
 }  // namespace sd_attn

@@ -12,7 +12,6 @@
 #include <mutex>
 
 #include "../../include/sd_attn.h"
-#include "../../include/sd_attn_debug.h"
 #include "../../include/sd_geglu.h"
 #include "../../include/sd_groupnorm.h"
 #include "../../include/sd_winograd.h"
@@ -21,9 +20,8 @@
 #include "geglu_kernel.cuh"
 #include "groupnorm_kernel.cuh"
 #include "winograd_kernel.cuh"
-#include "fused_kernel.cuh"
-#include "fused4_kernel.cuh"
 #include "fused4s_kernel.cuh"
+#include "selftest_kernel.cuh"
 #include "simt_kernel.cuh"
 #include "twopass_kernel.cuh"
 
@@ -52,6 +50,10 @@ constexpr int BATCH_LANES = SD_ATTN_BATCH_LANES;   // sd_attn_forward_batch spre
 
 constexpr int HOST_SLICES = 4;   // sd_attn_forward_host cuts the (batch, head) range into at most this many slices
 
+// Scratch of the FUSED kernel's shares mode (see fused4s_kernel.cuh): pieces and their arrival counters.
+constexpr size_t PART_BYTES = (size_t)136 << 20;   // five 4096-token d = 40 problems in one launch need 128 MB
+constexpr int PART_COUNTERS = 1 << 16;             // (problem, unit, tile) counters of one launch
+
 struct sd_attn_handle {
     TmapCacheEntry tmap_cache[TMAP_CACHE_ENTRIES];
     int tmap_cache_next;
@@ -59,30 +61,23 @@ struct sd_attn_handle {
     int mode;
     int layout;
     int last_mode;
+    sd_attn_options opt;
     cudaStream_t batch_lane[BATCH_LANES];   // sd_attn_forward_batch: lanes beside the caller's stream
     cudaEvent_t ev_batch_fork, ev_batch_join[BATCH_LANES];
     int batch_lanes_ok;
     long long launches;
     int* dev_status;          // DEV_STATUS_INTS ints on the device
+    float* part;              // PART_BYTES of pieces (FUSED, shares mode)
+    int* part_count;          // PART_COUNTERS arrival counters, zero between launches
     void* workspace;          // caller-owned
     size_t workspace_bytes;
     const float* tp_scores;   // where the last TWOPASS call put A and [L,S]
     const float* tp_stats;
-    float* dump_scores;       // bring-up hook of the cross kernel (see sd_attn_debug.h)
-    void* trace;              // SD_ATTN_TRACE builds only: clock-stamp buffer (the address comes from SD_ATTN_TRACE_PTR)
     encode_tiled_fn encode_tiled;
     cudaError_t last_cuda_error;
     int sm_count;
-    int fused4_ok;            // the register hand-over inside these kernels fits their launch allocation
-    int fused4s_ok;
-    int no_pdl;               // SD_ATTN_NO_PDL=1: ordinary launches (no overlap of a kernel's set-up with its predecessor)
-    int no_spare;             // SD_ATTN_FUSED_NO_SPARE=1: the four-tile kernel without the spare score buffer
-    int fused4_tiles_override;   // SD_ATTN_FUSED_TILES=1..4: fixed query tiles per CTA of the spare-buffer kernel (tests)
+    int fused4s_ok;           // the register hand-over inside these kernels fits their launch allocation
     int cross2_four_ok;
-    int cross_one_tile_only;  // SD_ATTN_CROSS_ONE_TILE=1: never use the persistent cross-attention kernel
-    int prefer_two_tile;      // SD_ATTN_FUSED_TWO_TILE=1: use the two-tile fused kernel for every head dim
-    int fused_no_split;       // SD_ATTN_FUSED_NO_SPLIT=1: a lone query tile keeps all 64 score columns in one warpgroup
-    int fused_split_override; // SD_ATTN_FUSED_SPLIT=2|4: that many parts wherever one tile per CTA is chosen (tests)
     // sd_attn_forward_host: copies of one slice of heads overlap the kernel of another (see there)
     cudaStream_t copy_in, copy_out;
     cudaEvent_t ev_fork, ev_join, ev_in[HOST_SLICES], ev_done[HOST_SLICES];
@@ -132,7 +127,7 @@ static cudaError_t launch_overlapped_if(bool overlap, void (*kernel)(KArgs...), 
 template <typename... KArgs, typename... Args>
 static cudaError_t launch_overlapped(const sd_attn_handle* h, void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem,
                                      cudaStream_t stream, Args&&... args) {
-    return launch_overlapped_if(!h->no_pdl, kernel, grid, block, smem, stream, static_cast<Args&&>(args)...);
+    return launch_overlapped_if(!h->opt.no_pdl, kernel, grid, block, smem, stream, static_cast<Args&&>(args)...);
 }
 
 template <typename K>
@@ -150,16 +145,14 @@ static cudaError_t create_host_overlap(sd_attn_handle* h) {
         e = cudaEventCreateWithFlags(&h->ev_in[c], cudaEventDisableTiming);
         if (e == cudaSuccess) e = cudaEventCreateWithFlags(&h->ev_done[c], cudaEventDisableTiming);
     }
-    const char* one = getenv("SD_ATTN_HOST_ONE_SLICE");
-    h->host_overlap = e == cudaSuccess && !(one && one[0] == '1');
+    h->host_overlap = e == cudaSuccess && !h->opt.host_one_slice;
     // the lanes of sd_attn_forward_batch
     if (e == cudaSuccess) e = cudaEventCreateWithFlags(&h->ev_batch_fork, cudaEventDisableTiming);
     for (int l = 0; l < BATCH_LANES && e == cudaSuccess; ++l) {
         e = cudaStreamCreateWithFlags(&h->batch_lane[l], cudaStreamNonBlocking);
         if (e == cudaSuccess) e = cudaEventCreateWithFlags(&h->ev_batch_join[l], cudaEventDisableTiming);
     }
-    const char* lane = getenv("SD_ATTN_BATCH_ONE_LANE");
-    h->batch_lanes_ok = e == cudaSuccess && !(lane && lane[0] == '1');
+    h->batch_lanes_ok = e == cudaSuccess && !h->opt.batch_serial;
     return e;
 }
 
@@ -219,9 +212,23 @@ static cudaError_t check_register_pools(sd_attn_handle* h) {
     return e;
 }
 
-extern "C" int sd_attn_create(sd_attn_handle** out) {
+extern "C" int sd_attn_create_ex(const sd_attn_options* options, sd_attn_handle** out) {
     if (!out) return SD_ATTN_ERR_INVALID_VALUE;
     *out = nullptr;
+    sd_attn_options opt;
+    memset(&opt, 0, sizeof(opt));
+    if (options) {
+        if (options->struct_size != sizeof(sd_attn_options)) return SD_ATTN_ERR_INVALID_VALUE;
+        opt = *options;
+        const int flags[] = {opt.no_pdl, opt.cross_one_tile, opt.host_one_slice, opt.batch_serial};
+        for (int f : flags)
+            if (f != 0 && f != 1) return SD_ATTN_ERR_INVALID_VALUE;
+        if (opt.fused_tiles < 0 || opt.fused_tiles > F4_TILES) return SD_ATTN_ERR_INVALID_VALUE;
+        if (opt.fused_shares < 0 || opt.fused_shares > 2) return SD_ATTN_ERR_INVALID_VALUE;
+        if (opt.fused_split != 0 && opt.fused_split != 1 && opt.fused_split != 2 && opt.fused_split != 4)
+            return SD_ATTN_ERR_INVALID_VALUE;
+    }
+    opt.struct_size = sizeof(sd_attn_options);
     int dev = 0;
     cudaError_t e = cudaGetDevice(&dev);
     if (e != cudaSuccess) return cuda_fail(nullptr, e);
@@ -237,6 +244,7 @@ extern "C" int sd_attn_create(sd_attn_handle** out) {
     h->mode = SD_ATTN_MODE_AUTO;
     h->last_mode = SD_ATTN_MODE_AUTO;
     h->sm_count = sms;
+    h->opt = opt;
 
     void* fn = nullptr;
     cudaDriverEntryPointQueryResult qres;
@@ -246,31 +254,10 @@ extern "C" int sd_attn_create(sd_attn_handle** out) {
         return cuda_fail(nullptr, e != cudaSuccess ? e : cudaErrorUnknown);
     }
     h->encode_tiled = (encode_tiled_fn)fn;
-#ifdef SD_ATTN_TRACE
-    const char* tr = getenv("SD_ATTN_TRACE_PTR");
-    h->trace = tr ? (void*)strtoull(tr, nullptr, 0) : nullptr;
-#endif
-    const char* one = getenv("SD_ATTN_CROSS_ONE_TILE");
-    h->cross_one_tile_only = (one && one[0] == '1') ? 1 : 0;
-    const char* npd = getenv("SD_ATTN_NO_PDL");
-    h->no_pdl = (npd && npd[0] == '1') ? 1 : 0;
-    const char* nsp = getenv("SD_ATTN_FUSED_NO_SPARE");
-    h->no_spare = (nsp && nsp[0] == '1') ? 1 : 0;
-    const char* ftl = getenv("SD_ATTN_FUSED_TILES");
-    h->fused4_tiles_override = (ftl && ftl[0] >= '1' && ftl[0] <= '4' && !ftl[1]) ? ftl[0] - '0' : 0;
-    const char* nsl = getenv("SD_ATTN_FUSED_NO_SPLIT");
-    h->fused_no_split = (nsl && nsl[0] == '1') ? 1 : 0;
-    const char* spl = getenv("SD_ATTN_FUSED_SPLIT");
-    h->fused_split_override = (spl && (spl[0] == '2' || spl[0] == '4') && !spl[1]) ? spl[0] - '0' : 0;
-    const char* two = getenv("SD_ATTN_FUSED_TWO_TILE");
-    h->prefer_two_tile = (two && two[0] == '1') ? 1 : 0;
 
     // dynamic shared memory ceilings of every kernel, once
     e = raise_layout_kernels<false>();
     if (e == cudaSuccess) e = raise_layout_kernels<true>();
-    if (e == cudaSuccess) e = raise_smem_limit(fused_attention_kernel<128>, fused_smem_bytes_max());
-    if (e == cudaSuccess) e = raise_smem_limit(fused_attention_kernel<64>, fused_smem_bytes_max());
-    if (e == cudaSuccess) e = raise_smem_limit(fused4_attention_kernel, fused4_smem_bytes());
     if (e == cudaSuccess) e = raise_smem_limit(twopass_scores_kernel, twopass_scores_smem_bytes(3));
     if (e == cudaSuccess) e = raise_smem_limit(twopass_pv_kernel, twopass_pv_smem_bytes(3));
     if (e == cudaSuccess) e = raise_smem_limit(simt_attention_kernel<float, 5>, simt_smem_bytes(160));
@@ -279,23 +266,26 @@ extern "C" int sd_attn_create(sd_attn_handle** out) {
     if (e == cudaSuccess) e = raise_smem_limit(simt_attention_kernel<__half, 4>, simt_smem_bytes(128));
     if (e == cudaSuccess) e = raise_smem_limit(simt_attention_kernel<__nv_bfloat16, 5>, simt_smem_bytes(160));
     if (e == cudaSuccess) e = raise_smem_limit(simt_attention_kernel<__nv_bfloat16, 4>, simt_smem_bytes(128));
-    // setmaxnreg budgets (see the kernels): only use a variant whose increases are covered by its decreases
+    // setmaxnreg budgets (see the kernels): a kernel whose increases its decreases do not cover is never launched
     if (e == cudaSuccess) {
-        cudaFuncAttributes fa;
-        e = cudaFuncGetAttributes(&fa, fused4_attention_kernel);
-        if (e == cudaSuccess)
-            h->fused4_ok = F4_THREADS * fa.numRegs >= 512 * F4_SOFTMAX_REGS + 256 * F4_CONTROL_REGS;
         h->fused4s_ok = 1;
         h->cross2_four_ok = 1;
-        if (e == cudaSuccess) e = check_register_pools<false>(h);
+        e = check_register_pools<false>(h);
         if (e == cudaSuccess) e = check_register_pools<true>(h);
     }
     if (e == cudaSuccess) e = cudaMalloc((void**)&h->dev_status, sizeof(int) * DEV_STATUS_INTS);
     if (e == cudaSuccess) e = cudaMemset(h->dev_status, 0, sizeof(int) * DEV_STATUS_INTS);
+    if (e == cudaSuccess && opt.fused_shares != 1) {
+        e = cudaMalloc((void**)&h->part, PART_BYTES);
+        if (e == cudaSuccess) e = cudaMalloc((void**)&h->part_count, sizeof(int) * PART_COUNTERS);
+        if (e == cudaSuccess) e = cudaMemset(h->part_count, 0, sizeof(int) * PART_COUNTERS);
+    }
     if (e == cudaSuccess) e = create_host_overlap(h);
     if (e != cudaSuccess) {
         destroy_host_overlap(h);
         if (h->dev_status) cudaFree(h->dev_status);
+        if (h->part) cudaFree(h->part);
+        if (h->part_count) cudaFree(h->part_count);
         free(h);
         return cuda_fail(nullptr, e);
     }
@@ -303,11 +293,21 @@ extern "C" int sd_attn_create(sd_attn_handle** out) {
     return SD_ATTN_OK;
 }
 
+extern "C" int sd_attn_create(sd_attn_handle** out) { return sd_attn_create_ex(nullptr, out); }
+
+// A handle's kernels, status block and scratch belong to the device it was created on.
+static bool on_handle_device(const sd_attn_handle* h) {
+    int dev = -1;
+    return cudaGetDevice(&dev) == cudaSuccess && dev == h->device;
+}
+
 extern "C" int sd_attn_destroy(sd_attn_handle* h) {
     if (!h) return SD_ATTN_OK;
     cudaError_t e = cudaSuccess;
     destroy_host_overlap(h);
     if (h->dev_status) e = cudaFree(h->dev_status);
+    if (h->part) cudaFree(h->part);
+    if (h->part_count) cudaFree(h->part_count);
     free(h);
     return e == cudaSuccess ? SD_ATTN_OK : SD_ATTN_ERR_CUDA;
 }
@@ -349,17 +349,20 @@ extern "C" int sd_attn_twopass_buffers(sd_attn_handle* h, const float** scores, 
     return SD_ATTN_OK;
 }
 
-extern "C" int sd_attn_last_mode(const sd_attn_handle* h) { return h ? h->last_mode : SD_ATTN_MODE_AUTO; }
-extern "C" long long sd_attn_launch_count(const sd_attn_handle* h) { return h ? h->launches : 0; }
-
-extern "C" int sd_attn_debug_dump_cross_scores(sd_attn_handle* h, float* device_buffer) {
-    if (!h) return SD_ATTN_ERR_INVALID_VALUE;
-    h->dump_scores = device_buffer;
+extern "C" int sd_attn_selftest_wait_timeout(sd_attn_handle* h, void* stream) {
+    if (!h || !on_handle_device(h)) return SD_ATTN_ERR_INVALID_VALUE;
+    selftest_wait_timeout_kernel<<<1, 128, 0, (cudaStream_t)stream>>>(h->dev_status, nullptr);
+    const cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess) return cuda_fail(h, e);
+    h->launches += 1;
     return SD_ATTN_OK;
 }
 
+extern "C" int sd_attn_last_mode(const sd_attn_handle* h) { return h ? h->last_mode : SD_ATTN_MODE_AUTO; }
+extern "C" long long sd_attn_launch_count(const sd_attn_handle* h) { return h ? h->launches : 0; }
+
 extern "C" int sd_attn_query_status(sd_attn_handle* h, void* stream, int* detail) {
-    if (!h) return SD_ATTN_ERR_INVALID_VALUE;
+    if (!h || !on_handle_device(h)) return SD_ATTN_ERR_INVALID_VALUE;
     int host[DEV_STATUS_INTS];
     cudaStream_t s = (cudaStream_t)stream;
     cudaError_t e = cudaStreamSynchronize(s);
@@ -368,6 +371,8 @@ extern "C" int sd_attn_query_status(sd_attn_handle* h, void* stream, int* detail
     if (detail) memcpy(detail, host, 4 * sizeof(int));
     if (host[0] != 0) {
         e = cudaMemset(h->dev_status, 0, sizeof(host));
+        // a kernel that gave up may have left arrival counters of the shares mode behind
+        if (e == cudaSuccess && h->part_count) e = cudaMemset(h->part_count, 0, sizeof(int) * PART_COUNTERS);
         if (e != cudaSuccess) return cuda_fail(h, e);
         return SD_ATTN_ERR_DEVICE_TIMEOUT;
     }
@@ -473,43 +478,48 @@ static int launch_simt(sd_attn_handle* h, const Problem& p) {
     return SD_ATTN_OK;
 }
 
-// 65..80 keys (the 77 text tokens): one persistent CTA per SM walks a range of (head, tile) items
-static int launch_cross2(sd_attn_handle* h, const Problem& p) {
+// 65..80 keys (the 77 text tokens): one persistent CTA per SM walks a range of (head, tile) items of `n` problems of
+// ONE shape (BH, Nq, Nk, d, layout, dtype alike) -- one launch.
+static int launch_cross2_group(sd_attn_handle* h, const Problem* ps, int n) {
+    if (n < 1 || n > X2_GROUP_MAX) return SD_ATTN_ERR_INVALID_VALUE;
+    const Problem& p = ps[0];
     Cross2Args a;
-    a.q = (const __half*)p.q;
-    a.out = (__half*)p.out;
+    a.n_prob = n; a.BH = p.BH;
     a.lay = head_layout(p.heads, p.BH, p.Nq, p.d);
     a.Nq = p.Nq; a.Nk = p.Nk; a.d = p.d;
     a.dpad = (p.d + 15) / 16 * 16;
     a.nch = (p.d + CHUNK_COLS - 1) / CHUNK_COLS;
     a.stages = cross2_stages(a.nch);
     a.tiles_per_bh = (p.Nq + TILE_M - 1) / TILE_M;
-    a.n_items = p.BH * a.tiles_per_bh;
-    a.scale_log2e = fabsf(p.scale) * LOG2E;
-    a.negate = p.scale < 0.f;
+    a.n_items = n * p.BH * a.tiles_per_bh;
     a.status = h->dev_status;
-#ifdef SD_ATTN_TRACE
-    a.trace = (long long*)h->trace;
-#endif
-    CUtensorMap tq, tk, tv;
-    int rc = make_tmap(h, &tq, p.q, p.BH, p.Nq, p.d, TILE_M, p.heads, p.bf16);
-    if (rc == SD_ATTN_OK) rc = make_tmap(h, &tk, p.k, p.BH, p.Nk, p.d, X2_KN, p.heads, p.bf16);
-    if (rc == SD_ATTN_OK) rc = make_tmap(h, &tv, p.v, p.BH, p.Nk, p.d, X2_KN, p.heads, p.bf16);
-    if (rc != SD_ATTN_OK) return rc;
-    const int grid = a.n_items < h->sm_count ? a.n_items : h->sm_count;
     int groups = cross2_groups(p.d);
     if (groups >= 4 && !h->cross2_four_ok) groups = 3;
     // The four-group variant moves whole Q and output tiles: as single contiguous runs when the tensors are
     // head-major, as unswizzled tiles of d columns (two more tensor maps) when they are token-major.
     a.strided_rows = (groups >= 4 && p.heads > 0) ? 1 : 0;
-    CUtensorMap tqr = tq, tor = tq;
-    if (a.strided_rows) {
-        if (encode_row_tmap(h->encode_tiled, &tqr, p.q, p.heads, p.BH, p.Nq, p.d, p.bf16) != CUDA_SUCCESS ||
-            encode_row_tmap(h->encode_tiled, &tor, p.out, p.heads, p.BH, p.Nq, p.d, p.bf16) != CUDA_SUCCESS) {
-            h->last_cuda_error = cudaErrorInvalidValue;
-            return SD_ATTN_ERR_CUDA;
+    for (int i = 0; i < n; ++i) {
+        const Problem& pi = ps[i];
+        Cross2Problem& cp = a.prob[i];
+        int rc = make_tmap(h, &cp.tq, pi.q, pi.BH, pi.Nq, pi.d, TILE_M, pi.heads, pi.bf16);
+        if (rc == SD_ATTN_OK) rc = make_tmap(h, &cp.tk, pi.k, pi.BH, pi.Nk, pi.d, X2_KN, pi.heads, pi.bf16);
+        if (rc == SD_ATTN_OK) rc = make_tmap(h, &cp.tv, pi.v, pi.BH, pi.Nk, pi.d, X2_KN, pi.heads, pi.bf16);
+        if (rc != SD_ATTN_OK) return rc;
+        cp.tq_rows = cp.tq;
+        cp.tout_rows = cp.tq;
+        if (a.strided_rows) {
+            if (encode_row_tmap(h->encode_tiled, &cp.tq_rows, pi.q, pi.heads, pi.BH, pi.Nq, pi.d, pi.bf16) != CUDA_SUCCESS ||
+                encode_row_tmap(h->encode_tiled, &cp.tout_rows, pi.out, pi.heads, pi.BH, pi.Nq, pi.d, pi.bf16) != CUDA_SUCCESS) {
+                h->last_cuda_error = cudaErrorInvalidValue;
+                return SD_ATTN_ERR_CUDA;
+            }
         }
+        cp.q = (const __half*)pi.q;
+        cp.out = (__half*)pi.out;
+        cp.scale_log2e = fabsf(pi.scale) * LOG2E;
+        cp.negate = pi.scale < 0.f;
     }
+    const int grid = a.n_items < h->sm_count ? a.n_items : h->sm_count;
     size_t smem = cross2_smem_bytes(a.nch);
     if (groups >= 4) {   // d <= 48: Q tiles arrive as raw bulk copies and are rewritten in shared memory
         a.stages = cross2_dense_stages(p.d);
@@ -517,13 +527,13 @@ static int launch_cross2(sd_attn_handle* h, const Problem& p) {
     }
     const dim3 g(grid);
     if (p.bf16) {
-        if (groups >= 4) launch_overlapped(h, cross2_attention_kernel<4, true>, g, dim3(cross2_threads(4)), smem, p.stream, tq, tk, tv, tqr, tor, a);
-        else if (groups == 3) launch_overlapped(h, cross2_attention_kernel<3, true>, g, dim3(cross2_threads(3)), smem, p.stream, tq, tk, tv, tqr, tor, a);
-        else launch_overlapped(h, cross2_attention_kernel<2, true>, g, dim3(cross2_threads(2)), smem, p.stream, tq, tk, tv, tqr, tor, a);
+        if (groups >= 4) launch_overlapped(h, cross2_attention_kernel<4, true>, g, dim3(cross2_threads(4)), smem, p.stream, a);
+        else if (groups == 3) launch_overlapped(h, cross2_attention_kernel<3, true>, g, dim3(cross2_threads(3)), smem, p.stream, a);
+        else launch_overlapped(h, cross2_attention_kernel<2, true>, g, dim3(cross2_threads(2)), smem, p.stream, a);
     } else {
-        if (groups >= 4) launch_overlapped(h, cross2_attention_kernel<4>, g, dim3(cross2_threads(4)), smem, p.stream, tq, tk, tv, tqr, tor, a);
-        else if (groups == 3) launch_overlapped(h, cross2_attention_kernel<3>, g, dim3(cross2_threads(3)), smem, p.stream, tq, tk, tv, tqr, tor, a);
-        else launch_overlapped(h, cross2_attention_kernel<2>, g, dim3(cross2_threads(2)), smem, p.stream, tq, tk, tv, tqr, tor, a);
+        if (groups >= 4) launch_overlapped(h, cross2_attention_kernel<4>, g, dim3(cross2_threads(4)), smem, p.stream, a);
+        else if (groups == 3) launch_overlapped(h, cross2_attention_kernel<3>, g, dim3(cross2_threads(3)), smem, p.stream, a);
+        else launch_overlapped(h, cross2_attention_kernel<2>, g, dim3(cross2_threads(2)), smem, p.stream, a);
     }
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) return cuda_fail(h, e);
@@ -531,8 +541,10 @@ static int launch_cross2(sd_attn_handle* h, const Problem& p) {
     return SD_ATTN_OK;
 }
 
+static int launch_cross2(sd_attn_handle* h, const Problem& p) { return launch_cross2_group(h, &p, 1); }
+
 static int launch_cross(sd_attn_handle* h, const Problem& p) {
-    if (cross2_supports(p.Nk, p.d) && !h->cross_one_tile_only && !h->dump_scores) return launch_cross2(h, p);
+    if (cross2_supports(p.Nk, p.d) && !h->opt.cross_one_tile) return launch_cross2(h, p);
     CrossArgs a;
     a.out = (__half*)p.out;
     a.lay = head_layout(p.heads, p.BH, p.Nq, p.d);
@@ -544,7 +556,6 @@ static int launch_cross(sd_attn_handle* h, const Problem& p) {
     a.scale_log2e = fabsf(p.scale) * LOG2E;
     a.negate = p.scale < 0.f;
     a.status = h->dev_status;
-    a.dump_scores = h->dump_scores;
     CUtensorMap tq, tk, tv;
     int rc = make_tmap(h, &tq, p.q, p.BH, p.Nq, p.d, TILE_M, p.heads, p.bf16);
     if (rc == SD_ATTN_OK) rc = make_tmap(h, &tk, p.k, p.BH, p.Nk, p.d, a.kn, p.heads, p.bf16);
@@ -561,156 +572,156 @@ static int launch_cross(sd_attn_handle* h, const Problem& p) {
     return SD_ATTN_OK;
 }
 
-// d <= 64: four query tiles per CTA over key tiles of 64 (the softmax, not the tensor pipe, is the bound)
-static int launch_fused4(sd_attn_handle* h, const Problem& p) {
-    Fused4Args a;
-    a.out = (__half*)p.out;
-    a.lay = head_layout(0, p.BH, p.Nq, p.d);
-    a.Nq = p.Nq; a.Nk = p.Nk; a.d = p.d;
-    a.dpad = (p.d + 15) / 16 * 16;
-    a.scale_log2e = fabsf(p.scale) * LOG2E;
-    a.negate = p.scale < 0.f;
-    a.status = h->dev_status;
-#ifdef SD_ATTN_TRACE
-    a.trace = (long long*)h->trace;
-#endif
-    CUtensorMap tq, tk, tv;
-    int rc = make_tmap(h, &tq, p.q, p.BH, p.Nq, p.d, TILE_M);
-    if (rc == SD_ATTN_OK) rc = make_tmap(h, &tk, p.k, p.BH, p.Nk, p.d, F4_BN);
-    if (rc == SD_ATTN_OK) rc = make_tmap(h, &tv, p.v, p.BH, p.Nk, p.d, F4_BN);
-    if (rc != SD_ATTN_OK) return rc;
-    dim3 grid((p.Nq + F4_TILES * TILE_M - 1) / (F4_TILES * TILE_M), p.BH), block(F4_THREADS);
-    a.tiles_per_cta = F4_TILES;
-    a.nch = 1;
-    a.stages = F4_STAGES;
-    fused4_attention_kernel<<<grid, block, fused4_smem_bytes(), p.stream>>>(tq, tk, tv, a);
-    cudaError_t e = cudaGetLastError();
-    if (e != cudaSuccess) return cuda_fail(h, e);
-    h->launches += 1;
-    return SD_ATTN_OK;
-}
-
 template <bool BF>
 static void dispatch_fused4s(sd_attn_handle* h, int split, const Fused4Args& a, dim3 grid, dim3 block, size_t smem,
-                             cudaStream_t stream, const CUtensorMap& tq, const CUtensorMap& tk, const CUtensorMap& tv) {
+                             cudaStream_t stream) {
     if (split == 4 && a.nch == 1)
-        launch_overlapped(h, fused4s_attention_kernel<F4S_POLY_PER8, 1, 4, BF>, grid, block, smem, stream, tq, tk, tv, a);
+        launch_overlapped(h, fused4s_attention_kernel<F4S_POLY_PER8, 1, 4, BF>, grid, block, smem, stream, a);
     else if (split == 2 && a.nch == 1)
-        launch_overlapped(h, fused4s_attention_kernel<F4S_POLY_PER8, 1, 2, BF>, grid, block, smem, stream, tq, tk, tv, a);
+        launch_overlapped(h, fused4s_attention_kernel<F4S_POLY_PER8, 1, 2, BF>, grid, block, smem, stream, a);
     else if (split == 2 && a.nch == 2)
-        launch_overlapped(h, fused4s_attention_kernel<F4S_POLY_PER8, 2, 2, BF>, grid, block, smem, stream, tq, tk, tv, a);
+        launch_overlapped(h, fused4s_attention_kernel<F4S_POLY_PER8, 2, 2, BF>, grid, block, smem, stream, a);
     else if (split == 2 && a.nch == 3)
-        launch_overlapped(h, fused4s_attention_kernel<F4S_POLY_PER8, 3, 2, BF>, grid, block, smem, stream, tq, tk, tv, a);
+        launch_overlapped(h, fused4s_attention_kernel<F4S_POLY_PER8, 3, 2, BF>, grid, block, smem, stream, a);
     // the polynomial share of the exponentials only pays where four tiles saturate the special function unit
     else if (a.dpad <= 48)
-        launch_overlapped(h, fused4s_attention_kernel<F4S_POLY_PER8, 1, 1, BF>, grid, block, smem, stream, tq, tk, tv, a);
+        launch_overlapped(h, fused4s_attention_kernel<F4S_POLY_PER8, 1, 1, BF>, grid, block, smem, stream, a);
     else if (a.nch == 1)
-        launch_overlapped(h, fused4s_attention_kernel<0, 1, 1, BF>, grid, block, smem, stream, tq, tk, tv, a);
+        launch_overlapped(h, fused4s_attention_kernel<0, 1, 1, BF>, grid, block, smem, stream, a);
     else if (a.nch == 2)
-        launch_overlapped(h, fused4s_attention_kernel<0, 2, 1, BF>, grid, block, smem, stream, tq, tk, tv, a);
+        launch_overlapped(h, fused4s_attention_kernel<0, 2, 1, BF>, grid, block, smem, stream, a);
     else
-        launch_overlapped(h, fused4s_attention_kernel<0, 3, 1, BF>, grid, block, smem, stream, tq, tk, tv, a);
+        launch_overlapped(h, fused4s_attention_kernel<0, 3, 1, BF>, grid, block, smem, stream, a);
 }
 
-// The spare-buffer kernel: any head dim up to 160, 1..4 query tiles per CTA.
-static int launch_fused4s(sd_attn_handle* h, const Problem& p) {
+// How the FUSED kernel lays a problem out: query tiles per unit, whole units or shares.  A function of the problem's
+// shape alone, so that a problem gets the same arithmetic whatever else shares its launch.
+struct FusedPlan {
+    int tiles_per_cta, units_per_head, n_units, n_kv;
+    int shares;       // every CTA takes a share of every problem's (unit, key tile) steps; 0: one CTA per unit
+    int slot_floats;  // shares: floats of one piece slot
+    int grid;         // shares: CTAs (one per SM, but never more than a problem has steps: no CTA without a step)
+    int max_group;    // problems of this shape one launch can take (shares: the scratch bounds it)
+};
+
+static FusedPlan plan_fused(const sd_attn_handle* h, const Problem& p) {
+    const int dpad = (p.d + 15) / 16 * 16, nch = (p.d + CHUNK_COLS - 1) / CHUNK_COLS;
+    const int q_tile_bytes = nch * TILE_M * CHUNK_ROW_BYTES, stage_bytes = 2 * nch * F4_BN * CHUNK_ROW_BYTES;
+    // Tiles per unit: the fewest key-tile steps per CTA times the cost of one step of a CTA with that many tiles
+    // (clocks, measured at d = 40: four tiles share the exponential unit, one tile alone is bound by its hand-off
+    // chain), among the counts tensor memory and shared memory (at least two K/V stages) have room for.  Dealing a
+    // problem's steps out in shares costs a refill of the pipeline at every change of segment (about two steps) and
+    // the pieces' trip through the scratch (about one and a half).
+    static const int step_cost[F4_TILES + 1] = {0, 1000, 1400, 1900, 2400};
+    const int tiles_per_head = (p.Nq + TILE_M - 1) / TILE_M;
+    int max_tiles = f4s_max_tiles(dpad);
+    while (max_tiles > 1 && F4S_SMEM_BUDGET - max_tiles * q_tile_bytes < 2 * stage_bytes) --max_tiles;
+    FusedPlan best = {};
+    double best_cost = -1.0;
+    const int n_kv = (p.Nk + F4_BN - 1) / F4_BN;
+    for (int tpc = 1; tpc <= max_tiles; ++tpc) {
+        if (h->opt.fused_tiles > 0 && h->opt.fused_tiles <= max_tiles && tpc != h->opt.fused_tiles) continue;
+        FusedPlan f = {};
+        f.tiles_per_cta = tpc;
+        f.units_per_head = (tiles_per_head + tpc - 1) / tpc;
+        f.n_units = f.units_per_head * p.BH;
+        f.n_kv = n_kv;
+        f.slot_floats = tpc * (dpad + 2) * TILE_M;
+        const double whole_steps = (double)((f.n_units + h->sm_count - 1) / h->sm_count) * n_kv;
+        double steps = whole_steps;
+        f.max_group = F4_GROUP_MAX;
+        // shares: the handle has the scratch, two slots per CTA fit it, one counter per (unit, tile); W below 2^31
+        const size_t slots_bytes = (size_t)2 * h->sm_count * f.slot_floats * sizeof(float);
+        const bool can_share = tpc >= 2 && h->part && h->opt.fused_shares != 1 && slots_bytes <= PART_BYTES &&
+                               (long)f.n_units * F4_TILES <= PART_COUNTERS && f.n_units >= 2 &&
+                               (long long)f.n_units * n_kv < (1ll << 30);
+        if (can_share) {
+            const long W = (long)f.n_units * n_kv;
+            f.grid = W < h->sm_count ? (int)W : h->sm_count;
+            const double share = (double)W / f.grid;                          // steps of the problem per CTA
+            const double segments = share / n_kv + 1.0;                       // about: a cut begins a new one
+            const double shared_steps = share + 2.0 * (segments - 1.0) + 1.5;
+            if (shared_steps < whole_steps || h->opt.fused_shares == 2) {
+                steps = shared_steps;
+                f.shares = 1;
+                const long by_slots = (long)(PART_BYTES / slots_bytes), by_counters = PART_COUNTERS / ((long)f.n_units * F4_TILES);
+                const long cap = by_slots < by_counters ? by_slots : by_counters;
+                if (cap < f.max_group) f.max_group = (int)cap;
+            }
+        }
+        const double cost = steps * step_cost[tpc];
+        if (best_cost < 0 || cost < best_cost) {
+            best_cost = cost;
+            best = f;
+        }
+    }
+    return best;
+}
+
+// The single-pass kernel for `n` problems of ONE shape (BH, Nq, Nk, d, layout, dtype alike): one launch.
+static int launch_fused_group(sd_attn_handle* h, const Problem* ps, int n) {
+    if (!h->fused4s_ok) return SD_ATTN_ERR_UNSUPPORTED;
+    const Problem& p = ps[0];
+    const FusedPlan plan = plan_fused(h, p);
+    if (n < 1 || n > plan.max_group) return SD_ATTN_ERR_INVALID_VALUE;
     Fused4Args a;
-    a.out = (__half*)p.out;
     a.lay = head_layout(p.heads, p.BH, p.Nq, p.d);
+    a.n_prob = n; a.BH = p.BH;
     a.Nq = p.Nq; a.Nk = p.Nk; a.d = p.d;
     a.dpad = (p.d + 15) / 16 * 16;
     a.nch = (p.d + CHUNK_COLS - 1) / CHUNK_COLS;
-    a.scale_log2e = fabsf(p.scale) * LOG2E;
-    a.negate = p.scale < 0.f;
+    a.tiles_per_cta = plan.tiles_per_cta;
+    a.units_per_head = plan.units_per_head;
+    a.n_units = plan.n_units;
+    a.n_kv = plan.n_kv;
+    a.shares = plan.shares;
     a.status = h->dev_status;
-#ifdef SD_ATTN_TRACE
-    a.trace = (long long*)h->trace;
-#endif
+    a.part = h->part;
+    a.part_count = h->part_count;
+    a.part_slot_floats = plan.slot_floats;
     const int q_tile_bytes = a.nch * TILE_M * CHUNK_ROW_BYTES, stage_bytes = 2 * a.nch * F4_BN * CHUNK_ROW_BYTES;
-    // Tiles per CTA: the fewest waves of CTAs times the cost of one key-tile step of a CTA with that many tiles
-    // (clocks, measured at d = 40: four tiles share the exponential unit, one tile alone is bound by its hand-off
-    // chain), among the counts tensor memory and shared memory (at least two K/V stages) have room for.
-    static const int step_cost[F4_TILES + 1] = {0, 1000, 1400, 1900, 2400};
-    const int tiles_per_head = (p.Nq + TILE_M - 1) / TILE_M;
-    int max_tiles = f4s_max_tiles(a.dpad);
-    while (max_tiles > 1 && F4S_SMEM_BUDGET - max_tiles * q_tile_bytes < 2 * stage_bytes) --max_tiles;
-    long best = -1;
-    a.tiles_per_cta = 1;
-    for (int tpc = 1; tpc <= max_tiles; ++tpc) {
-        const long ctas = (long)((tiles_per_head + tpc - 1) / tpc) * p.BH;
-        const long cost = ((ctas + h->sm_count - 1) / h->sm_count) * step_cost[tpc];
-        if (best < 0 || cost < best) {
-            best = cost;
-            a.tiles_per_cta = tpc;
-        }
-    }
-    if (h->fused4_tiles_override > 0 && h->fused4_tiles_override <= max_tiles) a.tiles_per_cta = h->fused4_tiles_override;
     // one chunk per row: the kernel lays out four tile slots and eight stages whatever tiles_per_cta is (192 KB)
     const int tile_slots = a.nch == 1 ? F4_TILES : a.tiles_per_cta;
     a.stages = (F4S_SMEM_BUDGET - tile_slots * q_tile_bytes) / stage_bytes;
     if (a.stages > F4_STAGES) a.stages = F4_STAGES;
     const size_t smem = (size_t)tile_slots * q_tile_bytes + (size_t)a.stages * stage_bytes + 1024;
-    CUtensorMap tq, tk, tv;
-    int rc = make_tmap(h, &tq, p.q, p.BH, p.Nq, p.d, TILE_M, p.heads, p.bf16);
-    if (rc == SD_ATTN_OK) rc = make_tmap(h, &tk, p.k, p.BH, p.Nk, p.d, F4_BN, p.heads, p.bf16);
-    if (rc == SD_ATTN_OK) rc = make_tmap(h, &tv, p.v, p.BH, p.Nk, p.d, F4_BN, p.heads, p.bf16);
-    if (rc != SD_ATTN_OK) return rc;
-    dim3 grid((tiles_per_head + a.tiles_per_cta - 1) / a.tiles_per_cta, p.BH), block(F4_THREADS);
-    // One tile per CTA: its key tiles are dealt out among 4 or 2 warpgroups (parts), each with an accumulator of its
+    for (int i = 0; i < n; ++i) {
+        const Problem& pi = ps[i];
+        Fused4Problem& fp = a.prob[i];
+        int rc = make_tmap(h, &fp.tq, pi.q, pi.BH, pi.Nq, pi.d, TILE_M, pi.heads, pi.bf16);
+        if (rc == SD_ATTN_OK) rc = make_tmap(h, &fp.tk, pi.k, pi.BH, pi.Nk, pi.d, F4_BN, pi.heads, pi.bf16);
+        if (rc == SD_ATTN_OK) rc = make_tmap(h, &fp.tv, pi.v, pi.BH, pi.Nk, pi.d, F4_BN, pi.heads, pi.bf16);
+        if (rc != SD_ATTN_OK) return rc;
+        fp.out = (__half*)pi.out;
+        fp.scale_log2e = fabsf(pi.scale) * LOG2E;
+        fp.negate = pi.scale < 0.f;
+    }
+    dim3 grid(plan.shares ? plan.grid : plan.n_units * n), block(F4_THREADS);
+    // One tile per unit: its key tiles are dealt out among 4 or 2 warpgroups (parts), each with an accumulator of its
     // own in tensor memory next to the score buffers, whose number is a multiple of the parts (a buffer then always
     // meets the same part) and smaller than the K/V ring (a buffer ahead is a key tile ahead).
     int split = 1;
     a.split_buffers = 2;
-    if (a.tiles_per_cta == 1 && !h->fused_no_split) {
+    if (a.tiles_per_cta == 1 && h->opt.fused_split != 1) {
         split = 4 * F4_BN + 4 * a.dpad <= 512 ? 4 : 2;
-        if (h->fused_split_override == 2) split = 2;
+        if (h->opt.fused_split == 2) split = 2;
         a.split_buffers = (4 * F4_BN + split * a.dpad <= 512 && a.stages >= 5) ? 4 : 2;
         if (a.split_buffers < split || 2 * F4_BN + 2 * a.dpad > 512) split = 1;   // (no room: d > 192)
     }
     if (p.bf16)
-        dispatch_fused4s<true>(h, split, a, grid, block, smem, p.stream, tq, tk, tv);
+        dispatch_fused4s<true>(h, split, a, grid, block, smem, p.stream);
     else
-        dispatch_fused4s<false>(h, split, a, grid, block, smem, p.stream, tq, tk, tv);
+        dispatch_fused4s<false>(h, split, a, grid, block, smem, p.stream);
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) return cuda_fail(h, e);
     h->launches += 1;
     return SD_ATTN_OK;
 }
 
-static int launch_fused(sd_attn_handle* h, const Problem& p) {
-    if (h->fused4s_ok && !h->no_spare && !h->prefer_two_tile) return launch_fused4s(h, p);
-    if (p.heads > 0 || p.bf16) return SD_ATTN_ERR_UNSUPPORTED;   // the earlier kernels: head-major binary16 only
-    if (p.d <= F4_MAX_D && !h->prefer_two_tile && h->fused4_ok) return launch_fused4(h, p);
-    FusedArgs a;
-    const int bn = fused_block_n(p.d);
-    fused_fill_args(&a, (__half*)p.out, p.Nq, p.Nk, p.d, fabsf(p.scale) * LOG2E, p.scale < 0.f, h->dev_status);
-#ifdef SD_ATTN_TRACE
-    a.trace = (long long*)h->trace;
-#endif
-    CUtensorMap tq, tk, tv;
-    int rc = make_tmap(h, &tq, p.q, p.BH, p.Nq, p.d, TILE_M);
-    if (rc == SD_ATTN_OK) rc = make_tmap(h, &tk, p.k, p.BH, p.Nk, p.d, bn);
-    if (rc == SD_ATTN_OK) rc = make_tmap(h, &tv, p.v, p.BH, p.Nk, p.d, bn);
-    if (rc != SD_ATTN_OK) return rc;
-    // two query tiles per CTA share the K/V loads; a problem that would leave SMs idle that way takes one per CTA
-    // (measured: 24 -> 22.8 us at 1024 tokens d = 80; at d = 160, 256 tokens, one per CTA is slower, 13.5 -> 15.4 us)
-    const int tiles_per_head = (p.Nq + TILE_M - 1) / TILE_M;
-    a.tiles_per_cta = ((long)((tiles_per_head + 1) / 2) * p.BH >= h->sm_count || a.dpad > 96) ? 2 : 1;
-    dim3 grid((tiles_per_head + a.tiles_per_cta - 1) / a.tiles_per_cta, p.BH), block(FUSED_THREADS);
-    if (bn == 128)
-        fused_attention_kernel<128><<<grid, block, fused_smem_bytes(a), p.stream>>>(tq, tk, tv, a);
-    else
-        fused_attention_kernel<64><<<grid, block, fused_smem_bytes(a), p.stream>>>(tq, tk, tv, a);
-    cudaError_t e = cudaGetLastError();
-    if (e != cudaSuccess) return cuda_fail(h, e);
-    h->launches += 1;
-    return SD_ATTN_OK;
-}
+static int launch_fused(sd_attn_handle* h, const Problem& p) { return launch_fused_group(h, &p, 1); }
 
 static int launch_twopass(sd_attn_handle* h, const Problem& p) {
-    if (p.heads > 0 || p.bf16) return SD_ATTN_ERR_UNSUPPORTED;   // the comparator: head-major binary16 only
-    const size_t need = sd_attn_workspace_bytes(SD_ATTN_MODE_TWOPASS, p.BH, 1, p.Nq, p.Nk, p.d, SD_ATTN_F16);
-    if (!h->workspace || h->workspace_bytes < need) return SD_ATTN_ERR_WORKSPACE;
+    // (the comparator is head-major binary16 only and needs its workspace: validate_problem has checked both)
     const size_t rows = (size_t)p.BH * p.Nq;
     float* scores = (float*)h->workspace;
     float* stats = (float*)((char*)h->workspace + ((rows * (size_t)p.Nk * sizeof(float) + 255) & ~(size_t)255));
@@ -736,9 +747,11 @@ static int launch_twopass(sd_attn_handle* h, const Problem& p) {
     return SD_ATTN_OK;
 }
 
-extern "C" int sd_attn_forward(sd_attn_handle* h, const void* q, const void* k, const void* v, void* out, int B, int H,
-                               int Nq, int Nk, int d, float scale, int dtype, void* stream) {
-    if (!h) return SD_ATTN_ERR_INVALID_VALUE;
+// Argument checks of one problem, before anything is enqueued; *mode_out receives the kernel family that serves it.
+// Returns OK with *mode_out = -1 for an empty problem (Nq == 0).
+static int validate_problem(const sd_attn_handle* h, const void* q, const void* k, const void* v, const void* out, int B,
+                            int H, int Nq, int Nk, int d, float scale, int dtype, int* mode_out) {
+    *mode_out = -1;
     if (B <= 0 || H <= 0 || Nq < 0 || Nk <= 0 || d <= 0) return SD_ATTN_ERR_INVALID_VALUE;
     if (!isfinite(scale)) return SD_ATTN_ERR_INVALID_VALUE;
     if (dtype != SD_ATTN_F16 && dtype != SD_ATTN_F32 && dtype != SD_ATTN_BF16) return SD_ATTN_ERR_UNSUPPORTED;
@@ -747,7 +760,6 @@ extern "C" int sd_attn_forward(sd_attn_handle* h, const void* q, const void* k, 
     if (Nq == 0) return SD_ATTN_OK;
     if (!q || !k || !v || !out) return SD_ATTN_ERR_INVALID_VALUE;
     if ((((uintptr_t)q | (uintptr_t)k | (uintptr_t)v | (uintptr_t)out) & 15u) != 0) return SD_ATTN_ERR_ALIGNMENT;
-
     int mode = h->mode;
     const bool tensor_ok = (dtype == SD_ATTN_F16 || dtype == SD_ATTN_BF16) && (d % 8 == 0);
     if (mode == SD_ATTN_MODE_AUTO) {
@@ -756,31 +768,54 @@ extern "C" int sd_attn_forward(sd_attn_handle* h, const void* q, const void* k, 
     }
     if (mode != SD_ATTN_MODE_SIMT && !tensor_ok) return SD_ATTN_ERR_UNSUPPORTED;
     if (mode == SD_ATTN_MODE_CROSS && Nk > SD_ATTN_CROSS_MAX_NK) return SD_ATTN_ERR_UNSUPPORTED;
+    if (mode == SD_ATTN_MODE_TWOPASS) {
+        if (h->layout == SD_ATTN_LAYOUT_BNHD || dtype == SD_ATTN_BF16) return SD_ATTN_ERR_UNSUPPORTED;
+        const size_t need = sd_attn_workspace_bytes(SD_ATTN_MODE_TWOPASS, B, H, Nq, Nk, d, dtype);
+        if (!h->workspace || h->workspace_bytes < need) return SD_ATTN_ERR_WORKSPACE;
+    }
+    *mode_out = mode;
+    return SD_ATTN_OK;
+}
 
-    Problem p = {q, k, v, out, B * H, Nq, Nk, d, scale, (cudaStream_t)stream,
-                 h->layout == SD_ATTN_LAYOUT_BNHD ? H : 0, dtype == SD_ATTN_BF16 ? 1 : 0};
-    int rc;
+static Problem make_problem(const sd_attn_handle* h, const void* q, const void* k, const void* v, void* out, int B, int H,
+                            int Nq, int Nk, int d, float scale, int dtype, cudaStream_t stream) {
+    Problem p = {q, k, v, out, B * H, Nq, Nk, d, scale, stream, h->layout == SD_ATTN_LAYOUT_BNHD ? H : 0,
+                 dtype == SD_ATTN_BF16 ? 1 : 0};
+    return p;
+}
+
+static int launch_one(sd_attn_handle* h, const Problem& p, int mode, int dtype) {
     switch (mode) {
         case SD_ATTN_MODE_SIMT:
-            rc = dtype == SD_ATTN_F16    ? launch_simt<__half>(h, p)
-                 : dtype == SD_ATTN_BF16 ? launch_simt<__nv_bfloat16>(h, p)
-                                         : launch_simt<float>(h, p);
-            break;
-        case SD_ATTN_MODE_CROSS: rc = launch_cross(h, p); break;
-        case SD_ATTN_MODE_FUSED: rc = launch_fused(h, p); break;
-        case SD_ATTN_MODE_TWOPASS: rc = launch_twopass(h, p); break;
-        default: rc = SD_ATTN_ERR_INVALID_VALUE;
+            return dtype == SD_ATTN_F16    ? launch_simt<__half>(h, p)
+                   : dtype == SD_ATTN_BF16 ? launch_simt<__nv_bfloat16>(h, p)
+                                           : launch_simt<float>(h, p);
+        case SD_ATTN_MODE_CROSS: return launch_cross(h, p);
+        case SD_ATTN_MODE_FUSED: return launch_fused(h, p);
+        case SD_ATTN_MODE_TWOPASS: return launch_twopass(h, p);
+        default: return SD_ATTN_ERR_INVALID_VALUE;
     }
+}
+
+extern "C" int sd_attn_forward(sd_attn_handle* h, const void* q, const void* k, const void* v, void* out, int B, int H,
+                               int Nq, int Nk, int d, float scale, int dtype, void* stream) {
+    if (!h) return SD_ATTN_ERR_INVALID_VALUE;
+    int mode;
+    int rc = validate_problem(h, q, k, v, out, B, H, Nq, Nk, d, scale, dtype, &mode);
+    if (rc != SD_ATTN_OK || mode < 0) return rc;
+    if (!on_handle_device(h)) return SD_ATTN_ERR_INVALID_VALUE;
+    const Problem p = make_problem(h, q, k, v, out, B, H, Nq, Nk, d, scale, dtype, (cudaStream_t)stream);
+    rc = launch_one(h, p, mode, dtype);
     if (rc == SD_ATTN_OK) h->last_mode = mode;
     if (rc == SD_ATTN_OK && getenv("SD_ATTN_LOG"))
         fprintf(stderr, "[sd_attn] forward BH=%d Nq=%d Nk=%d d=%d dtype=%d -> mode %d\n", B * H, Nq, Nk, d, dtype, mode);
     return rc;
 }
 
-// A rough cost of one problem in microseconds, only to balance the lanes of a batch: a floor for the fixed part of
-// a call, tensor time at the rate the single-pass kernel reaches, memory time at the rate the cross kernel reaches.
-static double problem_cost_us(const sd_attn_problem& p, int dtype) {
-    const double bh = (double)p.B * p.H, es = dtype == SD_ATTN_F32 ? 4.0 : 2.0;
+// A rough cost of one launch in microseconds, only to balance the lanes of a batch: a floor for the fixed part of
+// a launch, tensor time at the rate the single-pass kernel reaches, memory time at the rate the cross kernel reaches.
+static double group_cost_us(const Problem& p, int n, int dtype) {
+    const double bh = (double)p.BH * n, es = dtype == SD_ATTN_F32 ? 4.0 : 2.0;
     const double flops = 4.0 * bh * p.Nq * (double)p.Nk * p.d;
     const double bytes = es * bh * p.d * (2.0 * p.Nq + 2.0 * p.Nk);
     const double t = flops / 450e6, m = bytes / 2.5e6;
@@ -788,37 +823,86 @@ static double problem_cost_us(const sd_attn_problem& p, int dtype) {
     return c > 8.0 ? c : 8.0;
 }
 
+constexpr int BATCH_MAX_GROUP = F4_GROUP_MAX > X2_GROUP_MAX ? F4_GROUP_MAX : X2_GROUP_MAX;
+
 extern "C" int sd_attn_forward_batch(sd_attn_handle* h, const sd_attn_problem* problems, int count, int dtype,
                                      void* stream) {
     if (!h || count < 0 || (count > 0 && !problems)) return SD_ATTN_ERR_INVALID_VALUE;
     if (count == 0) return SD_ATTN_OK;
     cudaStream_t s = (cudaStream_t)stream;
-    // TWOPASS mode lends ONE workspace to every call: its problems run one after another
-    const bool spread = h->batch_lanes_ok && count > 1 && h->mode != SD_ATTN_MODE_TWOPASS;
-    if (!spread) {
-        for (int i = 0; i < count; ++i) {
-            const sd_attn_problem& p = problems[i];
-            const int rc = sd_attn_forward(h, p.q, p.k, p.v, p.out, p.B, p.H, p.Nq, p.Nk, p.d, p.scale, dtype, stream);
-            if (rc != SD_ATTN_OK) return rc;
+    // every problem is checked before anything is enqueued
+    int* modes = (int*)malloc(sizeof(int) * (size_t)count * 2);
+    if (!modes) return SD_ATTN_ERR_INVALID_VALUE;
+    int* taken = modes + count;
+    for (int i = 0; i < count; ++i) {
+        const sd_attn_problem& p = problems[i];
+        const int rc = validate_problem(h, p.q, p.k, p.v, p.out, p.B, p.H, p.Nq, p.Nk, p.d, p.scale, dtype, &modes[i]);
+        if (rc != SD_ATTN_OK) {
+            free(modes);
+            return rc;
         }
-        return SD_ATTN_OK;
+        taken[i] = modes[i] < 0;   // an empty problem: nothing to launch
     }
-    // Fork the lanes from the caller's stream, give every problem to the lane with the least work so far (in the
-    // order given), join the lanes back: for the caller one piece of stream-ordered work, capturable in a graph.
+    if (!on_handle_device(h)) {
+        free(modes);
+        return SD_ATTN_ERR_INVALID_VALUE;
+    }
+    // TWOPASS lends ONE workspace to every call and the CUDA-core kernel gains nothing from company: one after another
+    bool serial = !h->batch_lanes_ok || count == 1;
+    for (int i = 0; i < count; ++i)
+        if (modes[i] == SD_ATTN_MODE_TWOPASS || modes[i] == SD_ATTN_MODE_SIMT) serial = true;
+    int rc = SD_ATTN_OK;
+    if (serial) {
+        for (int i = 0; i < count && rc == SD_ATTN_OK; ++i) {
+            if (taken[i]) continue;
+            const sd_attn_problem& p = problems[i];
+            rc = launch_one(h, make_problem(h, p.q, p.k, p.v, p.out, p.B, p.H, p.Nq, p.Nk, p.d, p.scale, dtype, s), modes[i], dtype);
+            if (rc == SD_ATTN_OK) h->last_mode = modes[i];
+        }
+        free(modes);
+        return rc;
+    }
+    // Fork the lanes from the caller's stream; problems of one shape and kernel become one launch; every launch goes
+    // to the lane with the least work so far (FUSED launches that deal their steps out in shares use the handle's
+    // one scratch and therefore all stay on the caller's stream); join the lanes back: for the caller one piece of
+    // stream-ordered work, capturable in a graph.
     cudaError_t e = cudaEventRecord(h->ev_batch_fork, s);
     for (int l = 0; l < BATCH_LANES && e == cudaSuccess; ++l) e = cudaStreamWaitEvent(h->batch_lane[l], h->ev_batch_fork, 0);
-    if (e != cudaSuccess) return cuda_fail(h, e);
-    double load[BATCH_LANES + 1] = {0};
-    int rc = SD_ATTN_OK;
-    for (int i = 0; i < count && rc == SD_ATTN_OK; ++i) {
-        const sd_attn_problem& p = problems[i];
-        int best = 0;
-        for (int l = 1; l <= BATCH_LANES; ++l)
-            if (load[l] < load[best]) best = l;
-        if (p.B > 0 && p.H > 0 && p.Nq > 0 && p.Nk > 0 && p.d > 0) load[best] += problem_cost_us(p, dtype);
-        cudaStream_t target = best == 0 ? s : h->batch_lane[best - 1];
-        rc = sd_attn_forward(h, p.q, p.k, p.v, p.out, p.B, p.H, p.Nq, p.Nk, p.d, p.scale, dtype, (void*)target);
+    if (e != cudaSuccess) {
+        free(modes);
+        return cuda_fail(h, e);
     }
+    double load[BATCH_LANES + 1] = {0};
+    for (int i = 0; i < count && rc == SD_ATTN_OK; ++i) {
+        if (taken[i]) continue;
+        const sd_attn_problem& p0 = problems[i];
+        Problem group[BATCH_MAX_GROUP];
+        int n = 0;
+        const bool x2 = modes[i] == SD_ATTN_MODE_CROSS && cross2_supports(p0.Nk, p0.d) && !h->opt.cross_one_tile;
+        FusedPlan plan = {};
+        if (modes[i] == SD_ATTN_MODE_FUSED)
+            plan = plan_fused(h, make_problem(h, p0.q, p0.k, p0.v, p0.out, p0.B, p0.H, p0.Nq, p0.Nk, p0.d, p0.scale, dtype, s));
+        const int cap = modes[i] == SD_ATTN_MODE_FUSED ? plan.max_group : x2 ? X2_GROUP_MAX : 1;
+        for (int j = i; j < count && n < cap; ++j) {
+            const sd_attn_problem& p = problems[j];
+            if (taken[j] || modes[j] != modes[i] || p.B != p0.B || p.H != p0.H || p.Nq != p0.Nq || p.Nk != p0.Nk || p.d != p0.d)
+                continue;
+            group[n++] = make_problem(h, p.q, p.k, p.v, p.out, p.B, p.H, p.Nq, p.Nk, p.d, p.scale, dtype, s);
+            taken[j] = 1;
+        }
+        int lane = 0;
+        if (!plan.shares)
+            for (int l = 1; l <= BATCH_LANES; ++l)
+                if (load[l] < load[lane]) lane = l;
+        load[lane] += group_cost_us(group[0], n, dtype);
+        cudaStream_t target = lane == 0 ? s : h->batch_lane[lane - 1];
+        for (int g = 0; g < n; ++g) group[g].stream = target;
+        if (modes[i] == SD_ATTN_MODE_FUSED) rc = launch_fused_group(h, group, n);
+        else if (x2) rc = launch_cross2_group(h, group, n);
+        else rc = launch_one(h, group[0], modes[i], dtype);
+        if (rc == SD_ATTN_OK) h->last_mode = modes[i];
+    }
+    free(modes);
     // join in every case: the caller's stream must not run ahead of work that was enqueued
     for (int l = 0; l < BATCH_LANES; ++l) {
         cudaError_t ej = cudaEventRecord(h->ev_batch_join[l], h->batch_lane[l]);
@@ -846,6 +930,7 @@ extern "C" int sd_attn_forward_host(sd_attn_handle* h, const void* q, const void
     if (dtype != SD_ATTN_F16 && dtype != SD_ATTN_F32 && dtype != SD_ATTN_BF16) return SD_ATTN_ERR_UNSUPPORTED;
     if (Nq == 0) return SD_ATTN_OK;
     if (!q || !k || !v || !out) return SD_ATTN_ERR_INVALID_VALUE;
+    if (!on_handle_device(h)) return SD_ATTN_ERR_INVALID_VALUE;
     const size_t need = sd_attn_host_staging_bytes(B, H, Nq, Nk, d, dtype);
     if (!staging || staging_bytes < need || ((uintptr_t)staging & 255u)) return SD_ATTN_ERR_WORKSPACE;
     const size_t es = dtype == SD_ATTN_F32 ? 4 : 2;
@@ -954,6 +1039,8 @@ static int static_setup(int dev, StaticDeviceState** out) {
             return cuda_fail(nullptr, e != cudaSuccess ? e : cudaErrorUnknown);
         e = raise_smem_limit(twopass_scores_kernel, twopass_scores_smem_bytes(3));
         if (e == cudaSuccess) e = raise_smem_limit(twopass_pv_kernel, twopass_pv_smem_bytes(3));
+        // the status word must start at zero (a kernel only ever writes it when a wait expires)
+        if (e == cudaSuccess) e = cudaMemset(status, 0, sizeof(int) * DEV_STATUS_INTS);
         if (e != cudaSuccess) return cuda_fail(nullptr, e);
         st->scratch = (unsigned char*)scratch;
         st->status = (int*)status;
@@ -996,9 +1083,6 @@ extern "C" int sd_attn_forward_twopass_static(const void* q, const void* k, cons
     float* scores = (float*)st->scratch;
     float* stats = (float*)(st->scratch + ((rows * (size_t)Nk * sizeof(float) + 255) & ~(size_t)255));
     cudaStream_t s = (cudaStream_t)stream;
-    // the status block is shared by every call and keeps the last call's contents: start from zero
-    e = cudaMemsetAsync(st->status, 0, sizeof(int) * DEV_STATUS_INTS, s);
-    if (e != cudaSuccess) return cuda_fail(nullptr, e);
     TwoPassArgs a;
     twopass_fill_args(&a, scores, stats, (__half*)out, Nq, Nk, d, scale, st->status);
     CUtensorMap tq, tk, tv;
@@ -1013,6 +1097,26 @@ extern "C" int sd_attn_forward_twopass_static(const void* q, const void* k, cons
     twopass_pv_kernel<<<grid, TWOPASS_THREADS, twopass_pv_smem_bytes(a.nch), s>>>(tv, a);
     e = cudaGetLastError();
     return e == cudaSuccess ? SD_ATTN_OK : cuda_fail(nullptr, e);
+}
+
+extern "C" int sd_attn_static_query_status(void* stream, int* detail) {
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return cuda_fail(nullptr, e);
+    StaticDeviceState* st = nullptr;
+    const int rc = static_setup(dev, &st);
+    if (rc != SD_ATTN_OK) return rc;
+    int host[DEV_STATUS_INTS];
+    e = cudaStreamSynchronize((cudaStream_t)stream);
+    if (e == cudaSuccess) e = cudaMemcpy(host, st->status, sizeof(host), cudaMemcpyDeviceToHost);
+    if (e != cudaSuccess) return cuda_fail(nullptr, e);
+    if (detail) memcpy(detail, host, 4 * sizeof(int));
+    if (host[0] != 0) {
+        e = cudaMemset(st->status, 0, sizeof(host));
+        if (e != cudaSuccess) return cuda_fail(nullptr, e);
+        return SD_ATTN_ERR_DEVICE_TIMEOUT;
+    }
+    return SD_ATTN_OK;
 }
 
 // ------------------------------------------------------------------------------------------------
@@ -1226,9 +1330,8 @@ extern "C" int sd_winograd_conv3x3_forward(const void* x, const void* U, const v
     cudaStream_t s = (cudaStream_t)stream;
     const long long in_threads = T * (C / 4), out_threads = T * (K / 2);
     // Each of the three kernels lets the next one of the stream start its set-up early and waits for its
-    // predecessor to complete before it touches global memory (SD_ATTN_NO_PDL=1: ordinary launches).
-    const char* npd = getenv("SD_ATTN_NO_PDL");
-    const bool overlap = !(npd && npd[0] == '1');
+    // predecessor to complete before it touches global memory.
+    const bool overlap = true;
     cudaError_t e = launch_overlapped_if(overlap, winograd_input_kernel, dim3((unsigned)((in_threads + 127) / 128)), dim3(128), 0, s,
                                          (const __half*)x, V, a);
     if (e != cudaSuccess) return cuda_fail(nullptr, e);
@@ -1257,3 +1360,4 @@ extern "C" int sd_winograd_query_status(void* stream, int* detail) {
     }
     return SD_ATTN_OK;
 }
+

@@ -59,6 +59,10 @@ __device__ __forceinline__ void setmaxnreg_dec() {
 __device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t arrivals) {
     asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(arrivals) : "memory");
 }
+// Retire a barrier that has no operation pending, so that its memory may be initialised again.
+__device__ __forceinline__ void mbar_inval(uint32_t bar) {
+    asm volatile("mbarrier.inval.shared::cta.b64 [%0];" ::"r"(bar) : "memory");
+}
 // Make freshly initialised barriers visible to the async proxy (TMA, tcgen05.commit).
 __device__ __forceinline__ void mbar_init_fence() {
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -96,12 +100,14 @@ __device__ __forceinline__ bool mbar_test(uint32_t bar, uint32_t parity) {
 }
 // Bounded wait.  `abort_flag` is a shared-memory int that any role sets when it gives up; every
 // waiter polls it so that one expired wait releases the whole block.  Returns false on abort.
+// LIMIT is the poll budget (the kernels use the default; the library's self-test of this path a small one).
+template <uint32_t LIMIT = WAIT_POLL_LIMIT>
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag,
                                           int* status, int site, int tile) {
     // try_wait itself suspends the thread for a hardware-chosen slice, so the first polls add no
     // sleep: a sleeping poller would see a completed phase up to a sleep period late, and that
     // delay sits on the MMA-issue round trip of the fused kernels.
-    for (uint32_t i = 0; i < WAIT_POLL_LIMIT; ++i) {
+    for (uint32_t i = 0; i < LIMIT; ++i) {
         if (mbar_try_wait(bar, parity)) return true;
         if ((i & 63) == 63) {
             if (*abort_flag) return false;

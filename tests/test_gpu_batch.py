@@ -1,7 +1,8 @@
-"""GPU parity for sd_attn_forward_batch: independent problems of Eq. 3 spread over the library's streams.
+"""GPU parity for sd_attn_forward_batch: independent problems of Eq. 3, those of one shape as ONE launch, the
+launches spread over the library's streams.
 
 Every problem of a batch is compared with the oracle element by element, and with the same problem run alone
-(bitwise: the batch call launches the same kernels, only on other streams).
+(bitwise: a grouped launch does the same arithmetic in the same order for every problem, whatever else is in it).
 """
 import numpy as np
 import pytest
@@ -64,7 +65,7 @@ def test_batch_against_the_oracle_and_the_single_calls(bd):
     n0 = a.launch_count
     assert bd.sd_attn_forward_batch(a.handle, problems_of(bd, SHAPES, dev), bd.F16, s) == bd.OK
     a.check()
-    assert a.launch_count - n0 == len(SHAPES)
+    assert a.launch_count - n0 == len(SHAPES) - 2          # the two repeated shapes ride along in their twins' launches
     for shape, (q, k, v), (tq, tk, tv, to) in zip(SHAPES, host, dev):
         ref, _, _ = oracle.forward(q, k, v, shape[4] ** -0.5)
         check(to.cpu().numpy(), ref, v, "batch %s" % (shape,))
@@ -105,7 +106,7 @@ def test_batch_edges(bd):
     assert bd.sd_attn_forward_batch(a.handle, bd.make_problems([]), bd.F16, s) == bd.OK
     assert bd.load().sd_attn_forward_batch(a.handle, None, 2, bd.F16, None) == bd.ERR_INVALID_VALUE
     assert bd.load().sd_attn_forward_batch(a.handle, None, -1, bd.F16, None) == bd.ERR_INVALID_VALUE
-    # one bad problem among good ones: its error comes back, the good ones before it have run, the stream is usable
+    # one bad problem among good ones: its error comes back and NOTHING was enqueued (all are checked first)
     host, dev = make(23, SHAPES[:3])
     items = [(tq.data_ptr(), tk.data_ptr(), tv.data_ptr(), to.data_ptr(), B, H, Nq, Nk, d, d ** -0.5)
              for (B, H, Nq, Nk, d), (tq, tk, tv, to) in zip(SHAPES[:3], dev)]
@@ -114,9 +115,12 @@ def test_batch_edges(bd):
     rc = bd.sd_attn_forward_batch(a.handle, bd.make_problems([items[0], tuple(bad), items[2]]), bd.F16, s)
     assert rc == bd.ERR_UNSUPPORTED
     a.check()
+    assert float(dev[0][3].abs().max()) == 0.0 and float(dev[2][3].abs().max()) == 0.0
+    # ... and the handle is as usable as before
+    assert bd.sd_attn_forward_batch(a.handle, bd.make_problems([items[0]]), bd.F16, s) == bd.OK
+    a.check()
     ref, _, _ = oracle.forward(*host[0], SHAPES[0][4] ** -0.5)
-    check(dev[0][3].cpu().numpy(), ref, host[0][2], "the problem before the bad one")
-    assert float(dev[2][3].abs().max()) == 0.0   # the one after it was not enqueued
+    check(dev[0][3].cpu().numpy(), ref, host[0][2], "after a refused batch")
     # a problem with no query rows is an OK no-op inside a batch as well
     empty = list(items[2])
     empty[6] = 0
@@ -142,3 +146,46 @@ def test_batch_twopass_runs_in_order(bd):
         ref, _, _ = oracle.forward(q, k, v, shape[4] ** -0.5)
         check(to.cpu().numpy(), ref, v, "two-pass batch %s" % (shape,))
     a.close()
+
+
+@pytest.mark.parametrize("opts", [{}, {"fused_shares": 2}, {"fused_shares": 2, "fused_tiles": 3}, {"fused_shares": 1}],
+                         ids=lambda e: "-".join("%s=%s" % kv for kv in e.items()) or "default")
+def test_groups_of_one_shape_with_different_scales(bd, opts):
+    """Five problems of one self-attention shape and five of one 77-key shape, every one with its own scale (one of
+    them negative, one zero): two launches, and every problem bitwise equal to the same problem run alone -- also
+    when the single-pass kernel deals the key range of its units out among all SMs and combines pieces (shares)."""
+    shapes = [(2, 4, 640, 1100, 40)] * 5 + [(2, 4, 640, 77, 40)] * 5 + [(1, 2, 300, 700, 80)] * 2
+    scales = [40 ** -0.5, -0.2, 0.0, 0.5, 0.05, 40 ** -0.5, -0.3, 0.0, 0.4, 0.02, 80 ** -0.5, -0.1]
+    host, dev = make(25, shapes)
+    a = bd.Attention(options=bd.Options(**opts))
+    s = torch.cuda.current_stream().cuda_stream
+    items = [(tq.data_ptr(), tk.data_ptr(), tv.data_ptr(), to.data_ptr(), B, H, Nq, Nk, d, sc)
+             for (B, H, Nq, Nk, d), (tq, tk, tv, to), sc in zip(shapes, dev, scales)]
+    n0 = a.launch_count
+    assert bd.sd_attn_forward_batch(a.handle, bd.make_problems(items), bd.F16, s) == bd.OK
+    a.check()
+    assert a.launch_count - n0 == 3
+    for shape, sc, (q, k, v), (tq, tk, tv, to) in zip(shapes, scales, host, dev):
+        ref, _, _ = oracle.forward(q, k, v, float(np.float32(sc)))
+        check(to.cpu().numpy(), ref, v, "grouped %s scale %g %s" % (shape, sc, opts))
+        alone = a.forward(tq, tk, tv, scale=sc)
+        a.check()
+        assert torch.equal(alone, to), "grouped and single call differ for %s scale %g" % (shape, sc)
+    a.close()
+
+
+def test_more_problems_of_a_shape_than_one_launch_takes(bd):
+    """Eleven problems of one shape: launches of eight and three (single-pass kernel), of five, five and one (77 keys)."""
+    for shape, launches in (((1, 2, 200, 300, 40), 2), ((1, 2, 200, 77, 40), 3)):
+        shapes = [shape] * 11
+        host, dev = make(26, shapes)
+        a = bd.Attention()
+        s = torch.cuda.current_stream().cuda_stream
+        n0 = a.launch_count
+        assert bd.sd_attn_forward_batch(a.handle, problems_of(bd, shapes, dev), bd.F16, s) == bd.OK
+        a.check()
+        assert a.launch_count - n0 == launches
+        for (q, k, v), (_, _, _, to) in zip(host, dev):
+            ref, _, _ = oracle.forward(q, k, v, shape[4] ** -0.5)
+            check(to.cpu().numpy(), ref, v, "eleven of %s" % (shape,))
+        a.close()

@@ -276,19 +276,17 @@ def test_running_anchor_follows_scores_that_grow_along_the_keys(att, bd, d, orde
         check(run(att, bd, mode, q, k, v, scale), ref, v, what="%s d=%d mode %s" % (order, d, bd.MODE_NAMES[mode]))
 
 
-@pytest.mark.parametrize("env", [{"SD_ATTN_FUSED_TILES": "1"}, {"SD_ATTN_FUSED_TILES": "2"}, {"SD_ATTN_FUSED_TILES": "3"},
-                                 {"SD_ATTN_FUSED_TILES": "4"}, {"SD_ATTN_FUSED_NO_SPARE": "1"},
-                                 {"SD_ATTN_FUSED_TWO_TILE": "1"}],
+@pytest.mark.parametrize("env", [{"fused_tiles": 1}, {"fused_tiles": 2}, {"fused_tiles": 3}, {"fused_tiles": 4},
+                                 {"fused_tiles": 2, "fused_shares": 2}, {"fused_tiles": 3, "fused_shares": 2},
+                                 {"fused_tiles": 4, "fused_shares": 2}, {"fused_shares": 1}],
                          ids=lambda e: "-".join("%s=%s" % kv for kv in e.items()))
-def test_every_variant_of_the_small_head_dim_kernel(bd, env, monkeypatch):
-    """The d <= 48 path picks 1 to 4 query tiles per CTA by problem size and has two fallbacks; force each of them.
+def test_every_variant_of_the_small_head_dim_kernel(bd, env):
+    """The d <= 48 path picks 1 to 4 query tiles per CTA by problem size, and whole units or shares; force each.
 
     Shapes: ragged in rows and keys, more key tiles than the K/V ring has stages (so stages are reused), and both
     fewer and more query tiles per head than a CTA takes.
     """
-    for k, v in env.items():
-        monkeypatch.setenv(k, v)
-    a = bd.Attention()        # the variant switches are read when the handle is created
+    a = bd.Attention(options=bd.Options(**env))        # the variant is chosen when the handle is created
     try:
         for n, (B, H, Nq, Nk, d, qmult) in enumerate([(1, 2, 600, 1100, 40, 1.0), (2, 1, 129, 700, 40, 4.0),
                                                        (1, 1, 1300, 130, 24, 1.0)]):
@@ -303,14 +301,12 @@ def test_every_variant_of_the_small_head_dim_kernel(bd, env, monkeypatch):
         a.close()
 
 
-@pytest.mark.parametrize("env", [{"SD_ATTN_CROSS_ONE_TILE": "1"}, {"SD_ATTN_NO_PDL": "1"}, {}],
+@pytest.mark.parametrize("env", [{"cross_one_tile": 1}, {"no_pdl": 1}, {}],
                          ids=lambda e: "-".join("%s=%s" % kv for kv in e.items()) or "default")
-def test_cross_attention_variants_over_head_dims_and_ragged_rows(bd, env, monkeypatch):
+def test_cross_attention_variants_over_head_dims_and_ragged_rows(bd, env):
     """77 and other key counts of one tile, every head-dim class (four, three, two softmax groups), row counts that
     leave a CTA with a partial tile, fewer items than SMs and more: the persistent kernel and its one-tile fallback."""
-    for k, v in env.items():
-        monkeypatch.setenv(k, v)
-    a = bd.Attention()
+    a = bd.Attention(options=bd.Options(**env))
     try:
         for n, (B, H, Nq, Nk, d, qmult) in enumerate([(2, 8, 4096, 77, 40, 1.0), (1, 3, 1000, 77, 40, 4.0),
                                                        (2, 2, 333, 70, 80, 1.0), (1, 2, 130, 80, 160, 4.0),
@@ -369,7 +365,7 @@ def test_every_ragged_tail_of_the_key_tiles(att, bd, Nk):
     check(run(att, bd, bd.MODE_FUSED, q, k, v, scale), ref, v, what="Nk=%d" % Nk)
 
 
-def test_many_heads_and_bitwise_agreement_between_tile_counts(bd, monkeypatch):
+def test_many_heads_and_bitwise_agreement_between_tile_counts(bd):
     """640 (batch, head) problems in one call; and the number of query tiles a CTA takes changes the schedule, not
     the arithmetic of a row: the outputs of the variants must agree bit for bit -- as long as a lone tile is not cut
     into parts, which changes the partial sums (checked against the oracle and the others within rounding)."""
@@ -377,11 +373,10 @@ def test_many_heads_and_bitwise_agreement_between_tile_counts(bd, monkeypatch):
     scale = float(np.float32(1.0 / np.sqrt(40)))
     rows = np.arange(0, 16 * 40 * 130, 11, dtype=np.int64)
     ref, _, _ = oracle.forward(q, k, v, scale, rows=rows)
-    monkeypatch.setenv("SD_ATTN_FUSED_NO_SPLIT", "1")   # a lone tile in one piece: the same arithmetic as with company
+    # a lone tile in one piece (fused_split=1) and whole units (fused_shares=1): the same arithmetic as with company
     outs = []
-    for tiles in ("1", "2", "4"):
-        monkeypatch.setenv("SD_ATTN_FUSED_TILES", tiles)
-        a = bd.Attention(bd.MODE_FUSED)
+    for tiles in (1, 2, 4):
+        a = bd.Attention(bd.MODE_FUSED, options=bd.Options(fused_tiles=tiles, fused_split=1, fused_shares=1))
         try:
             out = a.forward(gpu(q), gpu(k), gpu(v), scale=scale)
             a.check()
@@ -390,12 +385,9 @@ def test_many_heads_and_bitwise_agreement_between_tile_counts(bd, monkeypatch):
             a.close()
         check(outs[-1].reshape(-1, 40)[rows], ref, v, what="tiles per CTA %s" % tiles)
     assert np.array_equal(outs[0], outs[1]) and np.array_equal(outs[0], outs[2])
-    # one tile per CTA with its score columns shared out among 2 or 4 warpgroups: other partial sums, same result
-    monkeypatch.delenv("SD_ATTN_FUSED_NO_SPLIT")
-    monkeypatch.setenv("SD_ATTN_FUSED_TILES", "1")
-    for parts in ("2", "4"):
-        monkeypatch.setenv("SD_ATTN_FUSED_SPLIT", parts)
-        a = bd.Attention(bd.MODE_FUSED)
+    # one tile per CTA with its key tiles dealt out among 2 or 4 warpgroups: other partial sums, same result
+    for parts in (2, 4):
+        a = bd.Attention(bd.MODE_FUSED, options=bd.Options(fused_tiles=1, fused_split=parts))
         try:
             out = a.forward(gpu(q), gpu(k), gpu(v), scale=scale).cpu().numpy()
             a.check()
@@ -406,17 +398,14 @@ def test_many_heads_and_bitwise_agreement_between_tile_counts(bd, monkeypatch):
         assert np.abs(out.astype(np.float64) - outs[0].astype(np.float64)).max() <= 2 * F16_ABS * np.abs(v).max()
 
 
-@pytest.mark.parametrize("parts", ["0", "2", "4"])
+@pytest.mark.parametrize("parts", [0, 2, 4])
 @pytest.mark.parametrize("d", [40, 64, 80, 128, 160])
-def test_lone_tile_in_parts(bd, monkeypatch, parts, d):
+def test_lone_tile_in_parts(bd, parts, d):
     """One query tile per CTA: every warpgroup of the CTA takes a share of the 64 columns of each score tile, with an
     anchor, a row sum and an accumulator of its own (combined at the end).  Key counts around the shares' boundaries
     (a part without a single key, a part with one), several score-buffer rounds, and rows whose large scores come
     late (every part re-anchors on its own)."""
-    if parts != "0":
-        monkeypatch.setenv("SD_ATTN_FUSED_SPLIT", parts)
-    monkeypatch.setenv("SD_ATTN_FUSED_TILES", "1")
-    a = bd.Attention(bd.MODE_FUSED)
+    a = bd.Attention(bd.MODE_FUSED, options=bd.Options(fused_tiles=1, fused_split=parts))
     try:
         for i, (Nq, Nk) in enumerate([(128, 129), (100, 130), (5, 145), (130, 161), (128, 177), (64, 192), (129, 449),
                                       (257, 1000), (128, 2048)]):
