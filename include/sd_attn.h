@@ -94,10 +94,12 @@ typedef struct {
     int fused_tiles;       /* 1..4: fixed number of query tiles per CTA of the FUSED kernel (0: by problem size) */
     int fused_split;       /* FUSED with one query tile per CTA: 2 or 4 warpgroups share its key tiles, 1 none
                               (0: by head dim)                                                                */
-    int fused_shares;      /* FUSED: a problem of more groups of query tiles than SMs has the key range of a group
-                              cut between CTAs, so that every SM gets an equal share; partial results are combined
-                              through the handle's scratch.  0: where the cost model says it pays; 1: never (the
-                              scratch is not even allocated); 2: wherever the kernel allows it (tests)             */
+    int fused_shares;      /* 1: FUSED deals the (group of query tiles, key tile) steps of a problem out in equal
+                              shares to one CTA per SM, so that no SM idles in a last, partly filled wave; a group
+                              whose key range is cut between CTAs is finished through scratch the handle then owns
+                              (136 MB), by whichever piece arrives last, in a fixed order (the bits repeat).
+                              Measured slower than whole groups on every shape tried (4096 tokens: 97 against 86
+                              microseconds): off by default, kept as the tested basis of that scheme              */
     int cross_one_tile;    /* 1: CROSS runs one tile per CTA also for 65..80 keys                             */
     int host_one_slice;    /* 1: sd_attn_forward_host uses one slice, copies and kernel all on the caller's stream */
     int batch_serial;      /* 1: sd_attn_forward_batch runs its problems one after another on the caller's stream */
@@ -106,9 +108,8 @@ typedef struct {
 /*
  * Create a handle on the CURRENT CUDA device.  Checks the architecture (ERR_ARCH unless compute capability
  * 10.x), resolves the driver's tensor-map encoder, raises the kernels' dynamic shared-memory limits, allocates
- * the handle's device memory -- one 64-byte status block and the scratch through which the FUSED kernel combines
- * partial results of a group of query tiles whose keys were shared out among CTAs (about 50 MB) -- and creates
- * the two copy streams and ten events sd_attn_forward_host uses, and the three streams and four events of
+ * the handle's device memory -- one 64-byte status block (and the scratch of `fused_shares`, if asked for) -- and
+ * creates the two copy streams and ten events sd_attn_forward_host uses, and the three streams and four events of
  * sd_attn_forward_batch.  No stream work.  *out receives the handle (NULL on failure).
  * sd_attn_create(out) is sd_attn_create_ex(NULL, out): the defaults.  `options` may be NULL; it is read during
  * the call only.  Errors: INVALID_VALUE (null `out`, an option out of range, struct_size not that of a known

@@ -59,8 +59,9 @@ struct Cross2Problem {   // one problem of a launch
     int negate;         // scale < 0: the tensor core negates Q
 };
 
-struct Cross2Args {
-    Cross2Problem prob[X2_GROUP_MAX];
+template <int NP>   // NP = 1: a launch of one problem (the problem index folds away at compile time); else X2_GROUP_MAX
+struct Cross2ArgsT {
+    Cross2Problem prob[NP];
     int n_prob, BH;     // problems in this launch; (batch, head) pairs of each.  Heads are counted through all
                         // problems ("global head" = problem * BH + head), items through all global heads
     HeadLayout lay;
@@ -73,6 +74,7 @@ struct Cross2Args {
     int n_items;        // n_prob * BH * tiles_per_bh
     int* status;
 };
+using Cross2Args = Cross2ArgsT<X2_GROUP_MAX>;
 
 
 __host__ inline int cross2_groups(int d) {
@@ -117,9 +119,10 @@ __device__ __forceinline__ void issue_qk(uint32_t tmem_s, uint64_t q_desc, uint6
                    k_desc + (uint64_t)(((kk >> 2) * X2_KN * CHUNK_ROW_BYTES + (kk & 3) * 32) >> 4), idesc, kk > 0);
 }
 
-template <int NWG, bool BF = false>   // BF: bfloat16 tensors
+template <int NWG, bool BF = false, int NP = X2_GROUP_MAX>   // BF: bfloat16 tensors; NP: see Cross2ArgsT
 __global__ void __launch_bounds__(NWG * 128 + 256, 1)
-cross2_attention_kernel(const __grid_constant__ Cross2Args args) {
+cross2_attention_kernel(const __grid_constant__ Cross2ArgsT<NP> args) {
+    constexpr bool GROUPED = NP > 1;
     extern __shared__ uint8_t x2_smem_raw[];
     __shared__ __align__(8) uint64_t bar_full[X2_MAX_STAGES], bar_empty[X2_MAX_STAGES];
     __shared__ __align__(8) uint64_t bar_kv_full[2], bar_kv_empty[2];
@@ -134,14 +137,23 @@ cross2_attention_kernel(const __grid_constant__ Cross2Args args) {
     constexpr int S2_ISSUER_WARP = NWG * 4 + 7;   // second S issuer: the odd items
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     if (threadIdx.x == 0) pdl_launch_dependents();   // the next kernel of the stream may start its set-up
+    if (!GROUPED && threadIdx.x == 32) {   // the tensor maps are kernel parameters: their fetch need not wait for anything
+        tma_prefetch_desc(&args.prob[0].tq);
+        tma_prefetch_desc(&args.prob[0].tk);
+        tma_prefetch_desc(&args.prob[0].tv);
+        if (NWG == 4 && args.strided_rows) {
+            tma_prefetch_desc(&args.prob[0].tq_rows);
+            tma_prefetch_desc(&args.prob[0].tout_rows);
+        }
+    }
     const int nch = args.nch, dpad = args.dpad, stages = args.stages;
     // contiguous range of items for this CTA: consecutive items share a head, so K and V are fetched rarely
     const int per = args.n_items / gridDim.x, extra = args.n_items % gridDim.x;
     const int item0 = blockIdx.x * per + min((int)blockIdx.x, extra);
     const int n_local = per + ((int)blockIdx.x < extra ? 1 : 0);
     const int bh0 = item0 / args.tiles_per_bh;   // global head of the first item; head "group" g = global head - bh0
-    const int prob0 = bh0 / args.BH, hb0 = bh0 - prob0 * args.BH;   // its problem and its head inside that problem
-    if (threadIdx.x == 32 && n_local > 0) {   // the tensor maps are kernel parameters: their fetch need not wait for anything
+    const int prob0 = GROUPED ? bh0 / args.BH : 0, hb0 = bh0 - prob0 * args.BH;   // its problem and its head inside that problem
+    if (GROUPED && threadIdx.x == 32 && n_local > 0) {   // (several problems: the maps of the CTA's first one)
         const Cross2Problem& p0 = args.prob[prob0];
         tma_prefetch_desc(&p0.tq);
         tma_prefetch_desc(&p0.tk);
@@ -210,7 +222,7 @@ cross2_attention_kernel(const __grid_constant__ Cross2Args args) {
             for (int i = 0; i < n_local; ++i) {
                 const int item = item0 + i, gh = item / args.tiles_per_bh, tile = item - gh * args.tiles_per_bh;
                 const int s = i % stages, g = gh - bh0;
-                const int pi = gh / args.BH, bh = gh - pi * args.BH;   // problem, head inside it
+                const int pi = GROUPED ? gh / args.BH : 0, bh = gh - pi * args.BH;   // problem, head inside it
                 const Cross2Problem& pr = args.prob[pi];
                 const int bz = bh / args.lay.heads, hz = bh - bz * args.lay.heads;
                 if (g != g_prev) {
@@ -266,7 +278,7 @@ cross2_attention_kernel(const __grid_constant__ Cross2Args args) {
                 if (++c.w == NWG) { c.w = 0; ++c.n; }
                 if (++c.t == args.tiles_per_bh) {   // the next head, and past a problem's last head the next problem
                     c.t = 0; ++c.g;
-                    if (++c.hb == args.BH) { c.hb = 0; ++c.p; }
+                    if (GROUPED && ++c.hb == args.BH) { c.hb = 0; ++c.p; }
                 }
             };
             Cursor c = {0, 0, 0, 0, 0, 0, t_first, hb0, prob0};
@@ -303,7 +315,7 @@ cross2_attention_kernel(const __grid_constant__ Cross2Args args) {
                         ok = mbar_wait(smem_u32(&bar_pv_done[c.w]), (c.n - 1) & 1, abort_p, args.status, SITE_Y_PV, c.i);
                     if (!ok) break;
                     tc_fence_after_sync();
-                    if (c.p != p_desc) {
+                    if (GROUPED && c.p != p_desc) {
                         p_desc = c.p;
                         idesc_s = idesc_f16(TILE_M, X2_KN, false, false, args.prob[p_desc].negate != 0, BF);
                     }
@@ -352,10 +364,11 @@ cross2_attention_kernel(const __grid_constant__ Cross2Args args) {
         const uint32_t tmem_s = tmem_base + w * X2_KN + lane_off;
         const int valid = args.Nk;
         bool ok = true;
+        const float c2_one = args.prob[0].scale_log2e;
         // the problem of this group's current item, advanced NWG items at a time without divisions
         int it_t = item0 - bh0 * args.tiles_per_bh + w, it_hb = hb0, it_p = prob0;
         auto settle = [&]() {
-            while (it_t >= args.tiles_per_bh) {
+            while (GROUPED && it_t >= args.tiles_per_bh) {
                 it_t -= args.tiles_per_bh;
                 if (++it_hb == args.BH) { it_hb = 0; ++it_p; }
             }
@@ -387,7 +400,7 @@ cross2_attention_kernel(const __grid_constant__ Cross2Args args) {
         for (int i = w; i < n_local && ok; i += NWG, it_t += NWG) {
             const int n = i / NWG;
             settle();
-            const float c2 = args.prob[it_p].scale_log2e;
+            const float c2 = GROUPED ? args.prob[it_p].scale_log2e : c2_one;
             ok = mbar_wait(smem_u32(&bar_s_full[w]), n & 1, abort_p, args.status, SITE_Y_S, i);
             ok = __all_sync(0xffffffffu, ok);
             if (!ok) break;
@@ -464,7 +477,7 @@ cross2_attention_kernel(const __grid_constant__ Cross2Args args) {
             if (++w == NWG) { w = 0; ++n; }
             if (++tile == args.tiles_per_bh) {
                 tile = 0;
-                if (++bh == args.BH) { bh = 0; ++pi; }
+                if (++bh == args.BH && GROUPED) { bh = 0; ++pi; }
             }
         };
         for (int i = 0; i < n_local; ++i) {

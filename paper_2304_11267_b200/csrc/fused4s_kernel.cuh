@@ -69,6 +69,72 @@ constexpr int F4S_SOFTMAX_REGS = SD_ATTN_F4S_SOFTMAX_REGS;
 constexpr int F4S_CONTROL_REGS = SD_ATTN_F4S_CONTROL_REGS;
 static_assert(512 * F4S_SOFTMAX_REGS + 256 * F4S_CONTROL_REGS == 768 * 80, "setmaxnreg budget");
 
+// Shares: a query tile's piece was stored and its arrival counted (see the softmax warps' epilogue).  If it was the
+// last of its unit's pieces, this warpgroup (thread = row r) combines them all, in key order,
+// o = sum_c 2^(m_c - m) O_c / sum_c 2^(m_c - m) l_c with m = max_c m_c.  The pieces of a unit lie with the CTAs
+// c_first .. c_last (CTA c begins at step c W / G of the problem).  Kept out of line: it runs once or twice per
+// CTA and must not cost the key-tile loop registers.
+template <bool BF>
+__device__ __noinline__ void f4s_combine_pieces(const Fused4Args& args, int t, int r, int prob_i, int unit, int c_first, int c_last) {
+    const int dpad = args.dpad, n_kv_all = args.n_kv;
+    const long long u0 = (long long)unit * n_kv_all, Wl = (long long)args.n_units * n_kv_all, Gl = gridDim.x;
+    auto piece_of = [&](int c) -> const float* {
+        const long long begin = (long long)c * Wl / Gl;
+        return args.part + ((2 * (size_t)prob_i * gridDim.x + 2 * (size_t)c + (u0 < begin ? 0 : 1)) * args.part_slot_floats) +
+               (size_t)t * (dpad + 2) * TILE_M + r;
+    };
+    float m_all = -INFINITY, l_all = 0.f;
+    for (int c = c_first; c <= c_last; ++c) m_all = fmaxf(m_all, __ldcg(piece_of(c) + dpad * TILE_M));
+    for (int c = c_first; c <= c_last; ++c)
+        l_all += ex2_approx(__ldcg(piece_of(c) + dpad * TILE_M) - m_all) * __ldcg(piece_of(c) + (dpad + 1) * TILE_M);
+    const float inv = 1.f / l_all;
+    const int quad = unit % args.units_per_head, bh = unit / args.units_per_head;
+    const int row = quad * args.tiles_per_cta * TILE_M + t * TILE_M + r;
+    __half* orow = head_row(args.prob[prob_i].out, args.lay, bh, row);
+    // 24 columns at a time (d is a multiple of 8), the loads of two pieces in flight together
+    for (int c0 = 0; c0 < args.d; c0 += 24) {
+        float acc[24];
+#pragma unroll
+        for (int k = 0; k < 24; ++k) acc[k] = 0.f;
+        for (int c = c_first; c <= c_last; c += 2) {
+            const float* pa = piece_of(c);
+            const bool two = c + 1 <= c_last;
+            const float* pb = two ? piece_of(c + 1) : pa;
+            float xa[24], xb[24];
+#pragma unroll
+            for (int k = 0; k < 24; ++k) xa[k] = c0 + k < args.d ? __ldcg(pa + (c0 + k) * TILE_M) : 0.f;
+#pragma unroll
+            for (int k = 0; k < 24; ++k) xb[k] = (two && c0 + k < args.d) ? __ldcg(pb + (c0 + k) * TILE_M) : 0.f;
+            const float fa = ex2_approx(__ldcg(pa + dpad * TILE_M) - m_all) * inv;
+            const float fb = two ? ex2_approx(__ldcg(pb + dpad * TILE_M) - m_all) * inv : 0.f;
+#pragma unroll
+            for (int k = 0; k < 24; ++k) acc[k] = fmaf(xb[k], fb, fmaf(xa[k], fa, acc[k]));
+        }
+#pragma unroll
+        for (int k = 0; k < 24; k += 8) {
+            uint4 o;
+            o.x = pack_16x2<BF>(acc[k + 0], acc[k + 1]); o.y = pack_16x2<BF>(acc[k + 2], acc[k + 3]);
+            o.z = pack_16x2<BF>(acc[k + 4], acc[k + 5]); o.w = pack_16x2<BF>(acc[k + 6], acc[k + 7]);
+            if (row < args.Nq && c0 + k + 8 <= args.d) *reinterpret_cast<uint4*>(orow + c0 + k) = o;
+        }
+    }
+}
+
+// Shares: the thread's row of a piece -- O from tensor memory, anchor, row sum -- to the scratch, as
+// [tile][dpad + 2 columns: O, anchor, row sum][128 rows], so that a warp writes whole 128-byte lines.
+__device__ __noinline__ void f4s_store_piece(float* piece, uint32_t tmem_o, int dpad, float m_run, float l_run) {
+    for (int g = 0; g < (dpad >> 4); ++g) {
+        uint32_t x[16];
+        tmem_ld16(tmem_o + g * 16, x);
+        tmem_wait_ld();
+#pragma unroll
+        for (int c = 0; c < 16; ++c) piece[(g * 16 + c) * TILE_M] = __uint_as_float(x[c]);
+    }
+    piece[dpad * TILE_M] = m_run;
+    piece[(dpad + 1) * TILE_M] = l_run;
+    __threadfence();
+}
+
 // SPLIT > 1 (only with ONE query tile per CTA): the key tiles are dealt out among SPLIT warpgroups ("parts": part g
 // takes key tiles g, g + SPLIT, ...), each with an exponent anchor, a row sum and an accumulator O_g of its own over
 // ITS keys, combined once at the end.  A lone tile is bound by the chain of latencies of one warp per scheduler
@@ -86,13 +152,32 @@ fused4s_attention_kernel(const __grid_constant__ Fused4Args args) {
     // O_t done.  The score barriers are per tile AND buffer so that every barrier has ONE consumer that takes its
     // phases in order (a parity wait is only sound for a waiter exactly one phase behind): tile t meets buffer b
     // every NB key tiles, and the buffer cannot come back to it before its previous contents were consumed.
-    __shared__ __align__(8) uint64_t bar_s_full[F4_TILES][F4S_BUFFERS], bar_p_full[F4_TILES][F4S_BUFFERS];
-    __shared__ __align__(8) uint64_t bar_q_full[F4_TILES], bar_pv_done[F4_TILES], bar_o_final[F4_TILES];
-    __shared__ __align__(8) uint64_t bar_kv_full[F4_STAGES], bar_kv_empty[F4_STAGES];
-    __shared__ __align__(8) uint64_t bar_buf_free[F4S_BUFFERS];   // SPLIT > 1: the products reading a buffer's weights are done
+    // (one block of memory, so that a warp can (re-)initialise them side by side: see init_barriers)
+    struct Barriers {
+        uint64_t s_full[F4_TILES][F4S_BUFFERS], p_full[F4_TILES][F4S_BUFFERS];   // p_full: 4 arrivals, one per softmax warp
+        uint64_t q_full[F4_TILES], pv_done[F4_TILES], o_final[F4_TILES];
+        uint64_t kv_full[F4_STAGES];
+        uint64_t buf_free[F4S_BUFFERS];   // SPLIT > 1: the products reading a buffer's weights are done
+        uint64_t kv_empty[F4_STAGES];     // one commit per issuer: as many arrivals as the unit has query tiles
+    };
+    constexpr int N_BARRIERS = sizeof(Barriers) / sizeof(uint64_t);
+    constexpr int P_FULL_FIRST = F4_TILES * F4S_BUFFERS, P_FULL_END = 2 * F4_TILES * F4S_BUFFERS;
+    constexpr int KV_EMPTY_FIRST = N_BARRIERS - F4_STAGES;
+    __shared__ __align__(8) Barriers bars;
+    auto& bar_s_full = bars.s_full;
+    auto& bar_p_full = bars.p_full;
+    auto& bar_q_full = bars.q_full;
+    auto& bar_pv_done = bars.pv_done;
+    auto& bar_o_final = bars.o_final;
+    auto& bar_kv_full = bars.kv_full;
+    auto& bar_kv_empty = bars.kv_empty;
+    auto& bar_buf_free = bars.buf_free;
     __shared__ uint32_t tmem_base_slot;
     __shared__ int abort_flag;
-    __shared__ int piece_ticket[F4_TILES];   // a query tile's arrival number among the pieces of its unit
+    // A piece whose arrival number among the pieces of its unit is being fetched: {ticket, problem, unit, pending?} per
+    // query tile.  The ticket is looked at after the CTA-wide barrier that ends the segment, so that nobody waits
+    // for the counter's round trip to the L2.
+    __shared__ int piece_ticket[F4_TILES][4];
     // the segment the CTA works on, written by the scheduling thread: live? | problem | unit | first key tile | key
     // tiles | query tiles | nothing follows  (in shared memory so that no role carries the walk in registers)
     __shared__ int seg_desc[8];
@@ -119,38 +204,27 @@ fused4s_attention_kernel(const __grid_constant__ Fused4Args args) {
     const uint32_t kv_smem = q_smem + args.tiles_per_cta * q_tile_bytes;   // [stages][K | V]
     volatile int* abort_p = &abort_flag;
 
-    // (Re-)initialise every barrier for a segment of `tiles` query tiles; `again`: they hold a finished segment's state.
+    // (Re-)initialise every barrier for a segment of `tiles` query tiles, one warp at it (lane i takes barriers i,
+    // i + 32, ...); `again`: they hold a finished segment's state.
     auto init_barriers = [&](int tiles, bool again) {
-        auto each = [&](auto&& f) {
-            for (int t = 0; t < F4_TILES; ++t) {
-                for (int b = 0; b < F4S_BUFFERS; ++b) {
-                    f(&bar_s_full[t][b], 1);
-                    f(&bar_p_full[t][b], 4);    // one arrival per softmax warp of the tile (SPLIT > 1: of the part)
-                }
-                f(&bar_q_full[t], 1);
-                f(&bar_pv_done[t], 1);
-                f(&bar_o_final[t], 1);
-            }
-            for (int b = 0; b < F4S_BUFFERS; ++b) f(&bar_buf_free[b], 1);
-            for (int s = 0; s < F4_STAGES; ++s) {
-                f(&bar_kv_full[s], 1);
-                f(&bar_kv_empty[s], tiles);   // one commit per issuer
-            }
-        };
+        uint64_t* flat = reinterpret_cast<uint64_t*>(&bars);
         // Retire them all first, fence, then initialise them all.  (mbarrier.inval and mbarrier.init of ONE barrier
         // issued back to back came out wrong on the GPU: ring barriers of the next segment completed an arrival
         // early and the last query tiles multiplied by the wrong V tile.)
         if (again) {
-            each([&](uint64_t* bar, uint32_t) { mbar_inval(smem_u32(bar)); });
+            for (int i = lane; i < N_BARRIERS; i += 32) mbar_inval(smem_u32(flat + i));
             __threadfence_block();
             fence_proxy_async_smem();
+            __syncwarp();
         }
-        each([&](uint64_t* bar, uint32_t arrivals) { mbar_init(smem_u32(bar), arrivals); });
+        for (int i = lane; i < N_BARRIERS; i += 32)
+            mbar_init(smem_u32(flat + i), i >= KV_EMPTY_FIRST ? (uint32_t)tiles : (i >= P_FULL_FIRST && i < P_FULL_END) ? 4u : 1u);
         mbar_init_fence();
+        __syncwarp();
     };
-    // The scheduling thread (lane 0 of an otherwise idle control warp) walks this CTA's steps: [w_begin, w_end) of the
-    // W = units x key tiles of a problem -- of every problem in turn when the launch deals shares out.
-    constexpr int SCHED_TID = 21 * 32;
+    // The scheduling warp (an otherwise idle control warp, all lanes in step) walks this CTA's steps: [w_begin, w_end)
+    // of the W = units x key tiles of a problem -- of every problem in turn when the launch deals shares out.
+    constexpr int SCHED_WARP = 21;
     const int W = args.n_units * n_kv_all;                             // (the host keeps it below 2^31)
     const int G = args.shares ? (int)gridDim.x : args.n_units;         // CTAs among which a problem's steps are dealt out
     const int cta = args.shares ? (int)blockIdx.x : (int)(blockIdx.x % args.n_units);   // this CTA among them
@@ -164,7 +238,7 @@ fused4s_attention_kernel(const __grid_constant__ Fused4Args args) {
             ++sched_prob;
         }
         if (sched_prob >= sched_prob_end || !(w_begin < w_end)) {
-            seg_desc[0] = 0;
+            if (lane == 0) seg_desc[0] = 0;
             return;
         }
         const int unit = sched_w / n_kv_all, j0 = sched_w - unit * n_kv_all;
@@ -173,13 +247,16 @@ fused4s_attention_kernel(const __grid_constant__ Fused4Args args) {
         int tiles = (args.Nq - quad * args.tiles_per_cta * TILE_M + TILE_M - 1) / TILE_M;
         if (tiles > args.tiles_per_cta) tiles = args.tiles_per_cta;
         sched_w += n;
-        seg_desc[0] = 1; seg_desc[1] = sched_prob; seg_desc[2] = unit; seg_desc[3] = j0; seg_desc[4] = n;
-        seg_desc[5] = tiles;
-        seg_desc[6] = !(sched_w < w_end) && sched_prob + 1 == sched_prob_end;
+        if (lane == 0) {
+            seg_desc[0] = 1; seg_desc[1] = sched_prob; seg_desc[2] = unit; seg_desc[3] = j0; seg_desc[4] = n;
+            seg_desc[5] = tiles;
+            seg_desc[6] = !(sched_w < w_end) && sched_prob + 1 == sched_prob_end;
+        }
         init_barriers(tiles, again);
     };
-    if (tid == SCHED_TID) {
-        abort_flag = 0;
+    if (warp == SCHED_WARP) {
+        if (lane == 0) abort_flag = 0;
+        if (lane < F4_TILES) piece_ticket[lane][3] = 0;
         next_segment(false);
     }
     if (warp == 16) {
@@ -195,6 +272,21 @@ fused4s_attention_kernel(const __grid_constant__ Fused4Args args) {
     const uint32_t tmem_base = tmem_base_slot;
     // columns: the score buffers | O_0 .. O_{T-1} (SPLIT > 1: the parts' O_0 .. O_{SPLIT-1})
     const uint32_t tmem_o0 = tmem_base + (SPLIT > 1 ? args.split_buffers : args.tiles_per_cta + 1) * BN;
+
+    // Behind the CTA-wide barrier that ends a segment: was this query tile's piece the last of its unit's to arrive?
+    auto combine_if_last = [&](int t) {
+        if (!piece_ticket[t][3]) return;
+        const int ticket = piece_ticket[t][0], prob_i = piece_ticket[t][1], unit = piece_ticket[t][2];
+        named_barrier(2 + t, TILE_M);                // everybody has read the box
+        const int r = tid & (TILE_M - 1);
+        if (r == 0) piece_ticket[t][3] = 0;
+        const long long u0 = (long long)unit * n_kv_all;
+        const int c_first = (int)(((u0 + 1) * G - 1) / W), c_last = (int)(((u0 + n_kv_all) * G - 1) / W);
+        if (ticket != c_last - c_first) return;
+        __threadfence();
+        if (r == 0) args.part_count[((size_t)prob_i * args.n_units + unit) * F4_TILES + t] = 0;   // as the next launch expects it
+        f4s_combine_pieces<BF>(args, t, r, prob_i, unit, c_first, c_last);
+    };
 
     // One setmaxnreg site per kind, executed by whole warpgroups; the budget is the CTA's launch allocation.  The
     // control warps and the softmax warps each walk the CTA's segments in a loop of their own (the code behind a
@@ -392,7 +484,7 @@ fused4s_attention_kernel(const __grid_constant__ Fused4Args args) {
     tc_fence_before_sync();
     __syncthreads();
     if (last_segment || abort_flag) break;
-    if (tid == SCHED_TID) next_segment(true);
+    if (warp == SCHED_WARP) next_segment(true);
     __syncthreads();
     tc_fence_after_sync();
     }   // the next segment of this CTA
@@ -678,63 +770,19 @@ fused4s_attention_kernel(const __grid_constant__ Fused4Args args) {
                     }
                 }
             } else if (ok) {
-                // ---- a piece of the unit's key range: (O, anchor, row sum) to the scratch, column by column so that a
-                // warp writes whole lines; a CTA has at most two pieces (its first segment may begin and its last may
-                // end inside a unit), slot 0 for one that begins inside, slot 1 for one that begins a unit
+                // ---- a piece of the unit's key range: (O, anchor, row sum) of the thread's row to the scratch.  A CTA
+                // has at most two pieces per problem (its first segment may begin and its last may end inside a
+                // unit): slot 0 for one that begins inside a unit, slot 1 for one that begins a unit.
                 tc_fence_after_sync();
-                const int cols = dpad + 2;
-                const size_t tile_off = (size_t)t * cols * TILE_M + r;
-                const size_t slot0 = 2 * (size_t)prob_i * (size_t)G;   // the problem's slots: two per CTA
-                float* piece = args.part + (slot0 + 2 * (size_t)cta + (j0 > 0 ? 0 : 1)) * args.part_slot_floats + tile_off;
-                for (int g = 0; g < (dpad >> 4); ++g) {
-                    uint32_t x[16];
-                    tmem_ld16(tmem_o + g * 16, x);
-                    tmem_wait_ld();
-#pragma unroll
-                    for (int c = 0; c < 16; ++c) piece[(g * 16 + c) * TILE_M] = __uint_as_float(x[c]);
-                }
-                piece[dpad * TILE_M] = m_run;
-                piece[(dpad + 1) * TILE_M] = l_run;
-                __threadfence();
+                float* piece = args.part + ((2 * (size_t)prob_i * gridDim.x + 2 * (size_t)blockIdx.x + (j0 > 0 ? 0 : 1)) * args.part_slot_floats) +
+                               (size_t)t * (dpad + 2) * TILE_M + r;
+                f4s_store_piece(piece, tmem_o, dpad, m_run, l_run);
                 named_barrier(2 + t, TILE_M);
-                int* counter = args.part_count + ((size_t)prob_i * args.n_units + unit) * F4_TILES + t;
-                if (r == 0) piece_ticket[t] = atomicAdd(counter, 1);
-                named_barrier(2 + t, TILE_M);
-                // the pieces of this unit: CTAs c_first .. c_last, in key order (CTA c begins at step c W / G)
-                const long long u0 = (long long)unit * n_kv_all;
-                const int W = args.n_units * n_kv_all, G = (int)gridDim.x, cta = (int)blockIdx.x;
-                const int c_first = (int)(((u0 + 1) * G - 1) / W), c_last = (int)(((u0 + n_kv_all) * G - 1) / W);
-                if (piece_ticket[t] == c_last - c_first) {
-                    // every other piece is complete: combine them all,
-                    // o = sum_c 2^(m_c - m) O_c / sum_c 2^(m_c - m) l_c with m = max_c m_c
-                    __threadfence();
-                    if (r == 0) *counter = 0;   // as the next launch expects it
-                    auto piece_of = [&](int c) -> const float* {
-                        const long long begin = (long long)c * W / G;
-                        return args.part + (slot0 + 2 * (size_t)c + (u0 < begin ? 0 : 1)) * args.part_slot_floats + tile_off;
-                    };
-                    float m_all = -INFINITY, l_all = 0.f;
-                    for (int c = c_first; c <= c_last; ++c) m_all = fmaxf(m_all, __ldcg(piece_of(c) + dpad * TILE_M));
-                    for (int c = c_first; c <= c_last; ++c) {
-                        const float* pc = piece_of(c);
-                        l_all += ex2_approx(__ldcg(pc + dpad * TILE_M) - m_all) * __ldcg(pc + (dpad + 1) * TILE_M);
-                    }
-                    const float inv = 1.f / l_all;
-                    for (int g = 0; g < (args.d >> 3); ++g) {
-                        float acc[8];
-#pragma unroll
-                        for (int k = 0; k < 8; ++k) acc[k] = 0.f;
-                        for (int c = c_first; c <= c_last; ++c) {
-                            const float* pc = piece_of(c);
-                            const float f = ex2_approx(__ldcg(pc + dpad * TILE_M) - m_all) * inv;
-#pragma unroll
-                            for (int k = 0; k < 8; ++k) acc[k] = fmaf(__ldcg(pc + (g * 8 + k) * TILE_M), f, acc[k]);
-                        }
-                        uint4 o;
-                        o.x = pack_16x2<BF>(acc[0], acc[1]); o.y = pack_16x2<BF>(acc[2], acc[3]);
-                        o.z = pack_16x2<BF>(acc[4], acc[5]); o.w = pack_16x2<BF>(acc[6], acc[7]);
-                        if (row < args.Nq) *reinterpret_cast<uint4*>(orow + g * 8) = o;
-                    }
+                if (r == 0) {   // the counter's answer is looked at behind the barrier that ends the segment
+                    piece_ticket[t][0] = atomicAdd(args.part_count + ((size_t)prob_i * args.n_units + unit) * F4_TILES + t, 1);
+                    piece_ticket[t][1] = prob_i;
+                    piece_ticket[t][2] = unit;
+                    piece_ticket[t][3] = 1;
                 }
             }
         }
@@ -743,8 +791,9 @@ fused4s_attention_kernel(const __grid_constant__ Fused4Args args) {
     // start over for the next one; tensor memory and shared memory simply carry on.
     tc_fence_before_sync();
     __syncthreads();
+    if (SPLIT == 1 && !abort_flag) combine_if_last(warp >> 2);
     if (last_segment || abort_flag) break;
-    if (tid == SCHED_TID) next_segment(true);
+    if (warp == SCHED_WARP) next_segment(true);
     __syncthreads();
     tc_fence_after_sync();
     }   // the next segment of this CTA

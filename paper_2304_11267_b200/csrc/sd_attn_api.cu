@@ -178,9 +178,12 @@ static void destroy_host_overlap(sd_attn_handle* h) {   // the handle was calloc
 template <bool BF>
 static cudaError_t raise_layout_kernels() {
     cudaError_t e = raise_smem_limit(cross_attention_kernel<BF>, cross_smem_bytes(3, 128));
-    if (e == cudaSuccess) e = raise_smem_limit(cross2_attention_kernel<2, BF>, X2_SMEM_BUDGET + 1024);
-    if (e == cudaSuccess) e = raise_smem_limit(cross2_attention_kernel<3, BF>, X2_SMEM_BUDGET + 1024);
-    if (e == cudaSuccess) e = raise_smem_limit(cross2_attention_kernel<4, BF>, X2_SMEM_BUDGET + 1024);
+    if (e == cudaSuccess) e = raise_smem_limit(cross2_attention_kernel<2, BF, 1>, X2_SMEM_BUDGET + 1024);
+    if (e == cudaSuccess) e = raise_smem_limit(cross2_attention_kernel<3, BF, 1>, X2_SMEM_BUDGET + 1024);
+    if (e == cudaSuccess) e = raise_smem_limit(cross2_attention_kernel<4, BF, 1>, X2_SMEM_BUDGET + 1024);
+    if (e == cudaSuccess) e = raise_smem_limit(cross2_attention_kernel<2, BF, X2_GROUP_MAX>, X2_SMEM_BUDGET + 1024);
+    if (e == cudaSuccess) e = raise_smem_limit(cross2_attention_kernel<3, BF, X2_GROUP_MAX>, X2_SMEM_BUDGET + 1024);
+    if (e == cudaSuccess) e = raise_smem_limit(cross2_attention_kernel<4, BF, X2_GROUP_MAX>, X2_SMEM_BUDGET + 1024);
     if (e == cudaSuccess) e = raise_smem_limit(fused4s_attention_kernel<F4S_POLY_PER8, 1, 1, BF>, F4S_SMEM_BUDGET + 1024);
     if (e == cudaSuccess) e = raise_smem_limit(fused4s_attention_kernel<0, 1, 1, BF>, F4S_SMEM_BUDGET + 1024);
     if (e == cudaSuccess) e = raise_smem_limit(fused4s_attention_kernel<0, 2, 1, BF>, F4S_SMEM_BUDGET + 1024);
@@ -206,7 +209,10 @@ static cudaError_t check_register_pools(sd_attn_handle* h) {
         e = cudaFuncGetAttributes(&fa, f4s[i]);
         if (e == cudaSuccess && F4_THREADS * fa.numRegs < 512 * F4S_SOFTMAX_REGS + 256 * F4S_CONTROL_REGS) h->fused4s_ok = 0;
     }
-    if (e == cudaSuccess) e = cudaFuncGetAttributes(&fa, cross2_attention_kernel<4, BF>);
+    if (e == cudaSuccess) e = cudaFuncGetAttributes(&fa, cross2_attention_kernel<4, BF, 1>);
+    if (e == cudaSuccess && cross2_threads(4) * fa.numRegs < 512 * X2_SOFTMAX_REGS + 128 * X2_EPILOGUE_REGS + 128 * X2_CONTROL_REGS)
+        h->cross2_four_ok = 0;
+    if (e == cudaSuccess) e = cudaFuncGetAttributes(&fa, cross2_attention_kernel<4, BF, X2_GROUP_MAX>);
     if (e == cudaSuccess && cross2_threads(4) * fa.numRegs < 512 * X2_SOFTMAX_REGS + 128 * X2_EPILOGUE_REGS + 128 * X2_CONTROL_REGS)
         h->cross2_four_ok = 0;
     return e;
@@ -224,7 +230,7 @@ extern "C" int sd_attn_create_ex(const sd_attn_options* options, sd_attn_handle*
         for (int f : flags)
             if (f != 0 && f != 1) return SD_ATTN_ERR_INVALID_VALUE;
         if (opt.fused_tiles < 0 || opt.fused_tiles > F4_TILES) return SD_ATTN_ERR_INVALID_VALUE;
-        if (opt.fused_shares < 0 || opt.fused_shares > 2) return SD_ATTN_ERR_INVALID_VALUE;
+        if (opt.fused_shares < 0 || opt.fused_shares > 1) return SD_ATTN_ERR_INVALID_VALUE;
         if (opt.fused_split != 0 && opt.fused_split != 1 && opt.fused_split != 2 && opt.fused_split != 4)
             return SD_ATTN_ERR_INVALID_VALUE;
     }
@@ -275,7 +281,7 @@ extern "C" int sd_attn_create_ex(const sd_attn_options* options, sd_attn_handle*
     }
     if (e == cudaSuccess) e = cudaMalloc((void**)&h->dev_status, sizeof(int) * DEV_STATUS_INTS);
     if (e == cudaSuccess) e = cudaMemset(h->dev_status, 0, sizeof(int) * DEV_STATUS_INTS);
-    if (e == cudaSuccess && opt.fused_shares != 1) {
+    if (e == cudaSuccess && opt.fused_shares == 1) {   // (the scratch of the shares mode, only where it is asked for)
         e = cudaMalloc((void**)&h->part, PART_BYTES);
         if (e == cudaSuccess) e = cudaMalloc((void**)&h->part_count, sizeof(int) * PART_COUNTERS);
         if (e == cudaSuccess) e = cudaMemset(h->part_count, 0, sizeof(int) * PART_COUNTERS);
@@ -480,10 +486,10 @@ static int launch_simt(sd_attn_handle* h, const Problem& p) {
 
 // 65..80 keys (the 77 text tokens): one persistent CTA per SM walks a range of (head, tile) items of `n` problems of
 // ONE shape (BH, Nq, Nk, d, layout, dtype alike) -- one launch.
-static int launch_cross2_group(sd_attn_handle* h, const Problem* ps, int n) {
-    if (n < 1 || n > X2_GROUP_MAX) return SD_ATTN_ERR_INVALID_VALUE;
+template <int NP>
+static int launch_cross2_np(sd_attn_handle* h, const Problem* ps, int n) {
     const Problem& p = ps[0];
-    Cross2Args a;
+    Cross2ArgsT<NP> a;
     a.n_prob = n; a.BH = p.BH;
     a.lay = head_layout(p.heads, p.BH, p.Nq, p.d);
     a.Nq = p.Nq; a.Nk = p.Nk; a.d = p.d;
@@ -527,18 +533,23 @@ static int launch_cross2_group(sd_attn_handle* h, const Problem* ps, int n) {
     }
     const dim3 g(grid);
     if (p.bf16) {
-        if (groups >= 4) launch_overlapped(h, cross2_attention_kernel<4, true>, g, dim3(cross2_threads(4)), smem, p.stream, a);
-        else if (groups == 3) launch_overlapped(h, cross2_attention_kernel<3, true>, g, dim3(cross2_threads(3)), smem, p.stream, a);
-        else launch_overlapped(h, cross2_attention_kernel<2, true>, g, dim3(cross2_threads(2)), smem, p.stream, a);
+        if (groups >= 4) launch_overlapped(h, cross2_attention_kernel<4, true, NP>, g, dim3(cross2_threads(4)), smem, p.stream, a);
+        else if (groups == 3) launch_overlapped(h, cross2_attention_kernel<3, true, NP>, g, dim3(cross2_threads(3)), smem, p.stream, a);
+        else launch_overlapped(h, cross2_attention_kernel<2, true, NP>, g, dim3(cross2_threads(2)), smem, p.stream, a);
     } else {
-        if (groups >= 4) launch_overlapped(h, cross2_attention_kernel<4>, g, dim3(cross2_threads(4)), smem, p.stream, a);
-        else if (groups == 3) launch_overlapped(h, cross2_attention_kernel<3>, g, dim3(cross2_threads(3)), smem, p.stream, a);
-        else launch_overlapped(h, cross2_attention_kernel<2>, g, dim3(cross2_threads(2)), smem, p.stream, a);
+        if (groups >= 4) launch_overlapped(h, cross2_attention_kernel<4, false, NP>, g, dim3(cross2_threads(4)), smem, p.stream, a);
+        else if (groups == 3) launch_overlapped(h, cross2_attention_kernel<3, false, NP>, g, dim3(cross2_threads(3)), smem, p.stream, a);
+        else launch_overlapped(h, cross2_attention_kernel<2, false, NP>, g, dim3(cross2_threads(2)), smem, p.stream, a);
     }
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) return cuda_fail(h, e);
     h->launches += 1;
     return SD_ATTN_OK;
+}
+
+static int launch_cross2_group(sd_attn_handle* h, const Problem* ps, int n) {
+    if (n < 1 || n > X2_GROUP_MAX) return SD_ATTN_ERR_INVALID_VALUE;
+    return n == 1 ? launch_cross2_np<1>(h, ps, 1) : launch_cross2_np<X2_GROUP_MAX>(h, ps, n);
 }
 
 static int launch_cross2(sd_attn_handle* h, const Problem& p) { return launch_cross2_group(h, &p, 1); }
@@ -610,12 +621,15 @@ static FusedPlan plan_fused(const sd_attn_handle* h, const Problem& p) {
     // Tiles per unit: the fewest key-tile steps per CTA times the cost of one step of a CTA with that many tiles
     // (clocks, measured at d = 40: four tiles share the exponential unit, one tile alone is bound by its hand-off
     // chain), among the counts tensor memory and shared memory (at least two K/V stages) have room for.  Dealing a
-    // problem's steps out in shares costs a refill of the pipeline at every change of segment (about two steps) and
-    // the pieces' trip through the scratch (about one and a half).
+    // problem's steps out in shares (only on request: sd_attn_options::fused_shares) costs, measured on the 4096-token
+    // call, about five steps' time at every change of segment (the last tiles' epilogue, the barriers, the refill of
+    // the pipeline) and about seven for a piece's trip through the scratch and the combination at the end.
     static const int step_cost[F4_TILES + 1] = {0, 1000, 1400, 1900, 2400};
     const int tiles_per_head = (p.Nq + TILE_M - 1) / TILE_M;
     int max_tiles = f4s_max_tiles(dpad);
-    while (max_tiles > 1 && F4S_SMEM_BUDGET - max_tiles * q_tile_bytes < 2 * stage_bytes) --max_tiles;
+    // (at least three K/V stages: the issuer of the rotation's last tile asks for key tile j + 2 before it multiplies
+    // key tile j, which a ring of two could never deliver)
+    while (max_tiles > 1 && F4S_SMEM_BUDGET - max_tiles * q_tile_bytes < 3 * stage_bytes) --max_tiles;
     FusedPlan best = {};
     double best_cost = -1.0;
     const int n_kv = (p.Nk + F4_BN - 1) / F4_BN;
@@ -626,13 +640,13 @@ static FusedPlan plan_fused(const sd_attn_handle* h, const Problem& p) {
         f.units_per_head = (tiles_per_head + tpc - 1) / tpc;
         f.n_units = f.units_per_head * p.BH;
         f.n_kv = n_kv;
-        f.slot_floats = tpc * (dpad + 2) * TILE_M;
+        f.slot_floats = tpc * (dpad + 2) * TILE_M;   // per tile: dpad columns of O, anchor, row sum; 128 rows each
         const double whole_steps = (double)((f.n_units + h->sm_count - 1) / h->sm_count) * n_kv;
         double steps = whole_steps;
         f.max_group = F4_GROUP_MAX;
         // shares: the handle has the scratch, two slots per CTA fit it, one counter per (unit, tile); W below 2^31
         const size_t slots_bytes = (size_t)2 * h->sm_count * f.slot_floats * sizeof(float);
-        const bool can_share = tpc >= 2 && h->part && h->opt.fused_shares != 1 && slots_bytes <= PART_BYTES &&
+        const bool can_share = tpc >= 2 && h->part && h->opt.fused_shares == 1 && slots_bytes <= PART_BYTES &&
                                (long)f.n_units * F4_TILES <= PART_COUNTERS && f.n_units >= 2 &&
                                (long long)f.n_units * n_kv < (1ll << 30);
         if (can_share) {
@@ -640,14 +654,11 @@ static FusedPlan plan_fused(const sd_attn_handle* h, const Problem& p) {
             f.grid = W < h->sm_count ? (int)W : h->sm_count;
             const double share = (double)W / f.grid;                          // steps of the problem per CTA
             const double segments = share / n_kv + 1.0;                       // about: a cut begins a new one
-            const double shared_steps = share + 2.0 * (segments - 1.0) + 1.5;
-            if (shared_steps < whole_steps || h->opt.fused_shares == 2) {
-                steps = shared_steps;
-                f.shares = 1;
-                const long by_slots = (long)(PART_BYTES / slots_bytes), by_counters = PART_COUNTERS / ((long)f.n_units * F4_TILES);
-                const long cap = by_slots < by_counters ? by_slots : by_counters;
-                if (cap < f.max_group) f.max_group = (int)cap;
-            }
+            steps = share + 5.0 * (segments - 1.0) + 7.0;
+            f.shares = 1;
+            const long by_slots = (long)(PART_BYTES / slots_bytes), by_counters = PART_COUNTERS / ((long)f.n_units * F4_TILES);
+            const long cap = by_slots < by_counters ? by_slots : by_counters;
+            if (cap < f.max_group) f.max_group = (int)cap;
         }
         const double cost = steps * step_cost[tpc];
         if (best_cost < 0 || cost < best_cost) {
@@ -684,6 +695,7 @@ static int launch_fused_group(sd_attn_handle* h, const Problem* ps, int n) {
     const int tile_slots = a.nch == 1 ? F4_TILES : a.tiles_per_cta;
     a.stages = (F4S_SMEM_BUDGET - tile_slots * q_tile_bytes) / stage_bytes;
     if (a.stages > F4_STAGES) a.stages = F4_STAGES;
+    if (a.stages < 3) return SD_ATTN_ERR_UNSUPPORTED;   // (cannot happen for d <= SD_ATTN_MAX_D: one 160-wide tile leaves three)
     const size_t smem = (size_t)tile_slots * q_tile_bytes + (size_t)a.stages * stage_bytes + 1024;
     for (int i = 0; i < n; ++i) {
         const Problem& pi = ps[i];

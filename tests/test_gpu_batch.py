@@ -148,7 +148,7 @@ def test_batch_twopass_runs_in_order(bd):
     a.close()
 
 
-@pytest.mark.parametrize("opts", [{}, {"fused_shares": 2}, {"fused_shares": 2, "fused_tiles": 3}, {"fused_shares": 1}],
+@pytest.mark.parametrize("opts", [{}, {"fused_shares": 1}, {"fused_shares": 1, "fused_tiles": 3}],
                          ids=lambda e: "-".join("%s=%s" % kv for kv in e.items()) or "default")
 def test_groups_of_one_shape_with_different_scales(bd, opts):
     """Five problems of one self-attention shape and five of one 77-key shape, every one with its own scale (one of

@@ -277,8 +277,8 @@ def test_running_anchor_follows_scores_that_grow_along_the_keys(att, bd, d, orde
 
 
 @pytest.mark.parametrize("env", [{"fused_tiles": 1}, {"fused_tiles": 2}, {"fused_tiles": 3}, {"fused_tiles": 4},
-                                 {"fused_tiles": 2, "fused_shares": 2}, {"fused_tiles": 3, "fused_shares": 2},
-                                 {"fused_tiles": 4, "fused_shares": 2}, {"fused_shares": 1}],
+                                 {"fused_tiles": 2, "fused_shares": 1}, {"fused_tiles": 3, "fused_shares": 1},
+                                 {"fused_tiles": 4, "fused_shares": 1}],
                          ids=lambda e: "-".join("%s=%s" % kv for kv in e.items()))
 def test_every_variant_of_the_small_head_dim_kernel(bd, env):
     """The d <= 48 path picks 1 to 4 query tiles per CTA by problem size, and whole units or shares; force each.
@@ -373,10 +373,10 @@ def test_many_heads_and_bitwise_agreement_between_tile_counts(bd):
     scale = float(np.float32(1.0 / np.sqrt(40)))
     rows = np.arange(0, 16 * 40 * 130, 11, dtype=np.int64)
     ref, _, _ = oracle.forward(q, k, v, scale, rows=rows)
-    # a lone tile in one piece (fused_split=1) and whole units (fused_shares=1): the same arithmetic as with company
+    # a lone tile in one piece (fused_split=1), whole units: the same arithmetic as with company
     outs = []
     for tiles in (1, 2, 4):
-        a = bd.Attention(bd.MODE_FUSED, options=bd.Options(fused_tiles=tiles, fused_split=1, fused_shares=1))
+        a = bd.Attention(bd.MODE_FUSED, options=bd.Options(fused_tiles=tiles, fused_split=1))
         try:
             out = a.forward(gpu(q), gpu(k), gpu(v), scale=scale)
             a.check()
@@ -645,3 +645,35 @@ def test_scores_of_large_magnitude(att, bd, Nq, Nk, d, mult):
     assert float(np.abs(L).max()) > 500.0          # the case is what it claims to be
     got = run(att, bd, bd.MODE_AUTO, q, k, v, scale)
     check(got, ref, v, what="large scores x%g %s" % (mult, (Nq, Nk, d)))
+
+
+@pytest.mark.parametrize("shape", [(1, 37, 1024, 2112, 40), (2, 8, 1024, 1024, 40), (1, 5, 900, 1300, 80), (1, 3, 520, 4100, 160),
+                                   (1, 2, 300, 130, 40), (3, 50, 129, 700, 24)],
+                         ids=lambda s: "x".join(str(v) for v in s))
+def test_key_range_of_a_unit_cut_between_ctas(bd, shape):
+    """sd_attn_options::fused_shares: one CTA per SM, each with an equal share of the (unit, key tile) steps.  Shapes:
+    two whole units per CTA (a change of segment without pieces: 37 heads x 8 units = 2 x 148); units cut into two,
+    three and (few units, many key tiles) dozens of pieces; fewer steps than SMs; a ragged last key tile and ragged
+    rows; every head-dim class.  Against the oracle, bitwise against a second run, and within rounding of the
+    whole-unit result (another association of the same sums)."""
+    B, H, Nq, Nk, d = shape
+    q, k, v = rand_qkv(8800 + Nq + d, B, H, Nq, Nk, d, qmult=4.0 if d == 40 else 1.0)
+    scale = float(np.float32(1.0 / np.sqrt(d)))
+    rows = None
+    if B * H * Nq > 40000:
+        rows = np.arange(0, B * H * Nq, 5, dtype=np.int64)
+    ref, _, _ = oracle.forward(q, k, v, scale, rows=rows)
+    pick = (lambda x: x.reshape(-1, d)[rows]) if rows is not None else (lambda x: x)
+    outs = {}
+    for shares in (1, 0):
+        a = bd.Attention(bd.MODE_FUSED, options=bd.Options(fused_shares=shares, fused_tiles=0 if d > 48 else 4))
+        try:
+            first = a.forward(gpu(q), gpu(k), gpu(v), scale=scale)
+            again = a.forward(gpu(q), gpu(k), gpu(v), scale=scale)
+            a.check()
+            assert torch.equal(first, again), "two runs differ (shares=%d)" % shares
+            outs[shares] = first.cpu().numpy()
+        finally:
+            a.close()
+        check(pick(outs[shares]), ref, v, what="%s shares=%d" % (shape, shares))
+    assert np.abs(outs[1].astype(np.float64) - outs[0].astype(np.float64)).max() <= 2 * F16_ABS * np.abs(v).max()
