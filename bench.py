@@ -1,8 +1,11 @@
 #!/usr/bin/env python
 """Benchmark of the attention hot path on B200.
 
-  python bench.py --gpus N --steps K --warmup W            # the CUDA library (one rank per GPU)
+  python bench.py --gpus N --steps K --warmup W            # the CUDA library, one rank per GPU: under a launcher
+                                                           # (RANK / WORLD_SIZE set) as one of its ranks, else
+                                                           # bench.py starts the N ranks itself
   python bench.py --impl reference --steps K --warmup W    # the CPU oracle, as it stands
+  python bench.py --workload ubench                        # the instruction-rate probes behind roofline.joint
 
 A step is one pass of the hot path over the full-resolution self-attention workload: B=2, H=8,
 Nq=Nk=4096, d=40, fp16, once on the plain N(0,1) inputs and once on the peaked (Q x 4) inputs --
@@ -33,9 +36,16 @@ UNIT = "TFLOP/s"
 NOMINAL_FP16_TFLOPS = 2250.0
 ROTATING_SETS = 8   # 8 x 42 MB of q/k/v/out for the two variants = 336 MB, above the 126 MB L2
 # DRAM bytes per launch of the fused kernel on this workload: dram__bytes_read.sum + dram__bytes_write.sum of one
-# ncu capture (profiles/fused4s_c2_self_4096_d40.md): 15.79 MB read (q, k, v once: 15.73 MB algorithmic) and
-# nothing written during the launch -- the 5.2 MB of output are still in the 126 MB L2 when the kernel ends.
-FUSED_TRAFFIC_BYTES_PER_LAUNCH = 15790592
+# ncu capture of the kernel instance named here (profiles/fused4s_c2_self_4096_d40.md): q, k, v read once (15.73 MB
+# algorithmic) and next to nothing written during the launch -- the 5.2 MB of output are still in the 126 MB L2 when
+# the kernel ends.  A constant from a capture: it moves only when the capture is redone.
+FUSED_TRAFFIC = {"bytes_per_launch": 15790592, "kernel_instance": "fused4s_attention_kernel<2, 1, 1, false>",
+                 "capture": "profiles/fused4s_c2_self_4096_d40.md"}
+# Of every 8 exponentials of the d = 40 kernel this many go to the FMA pipe (F4S_POLY_PER8 in fused4s_kernel.cuh), and
+# FMA-pipe results per score element: scale, row sum, half a pack on the special-function path; 6 more on the
+# polynomial path.
+POLY_PER8 = 2
+FMA_OPS_SFU_PATH, FMA_OPS_POLY_EXTRA = 3.0, 6.0
 
 
 def measured_peaks():
@@ -108,14 +118,17 @@ def oracle_sample_rows(call, every):
     return np.arange(0, call.B * call.H * call.Nq, every, dtype=np.int64)
 
 
-def time_oracle(calls_inputs, every):
-    """Seconds the oracle needs for every `every`-th row of each call, and the FLOPs that covers."""
+def time_oracle(calls_inputs, every, keep=None):
+    """Seconds the oracle needs for every `every`-th row of each call, and the FLOPs that covers.  `keep`, a list,
+    receives (rows, result) per call."""
     import oracle
     t0 = time.perf_counter()
     flops = 0
     for call, (q, k, v) in calls_inputs:
         rows = oracle_sample_rows(call, every)
-        oracle.forward(q, k, v, call.scale(), rows=rows)
+        ref, _, _ = oracle.forward(q, k, v, call.scale(), rows=rows)
+        if keep is not None:
+            keep.append((rows, ref))
         flops += 4 * len(rows) * call.Nk * call.d
     return time.perf_counter() - t0, flops
 
@@ -133,8 +146,12 @@ def cpu_baseline(calls_inputs, target_s=12.0):
     while every < 16 and full / every > 2.0 * target_s:
         every *= 2
     dt, flops, passes = 0.0, 0, 0
+    refs = []
     while passes == 0 or (every == 1 and dt < 0.85 * target_s and passes < 64):   # a fast box repeats the whole step
-        t, f = time_oracle(calls_inputs, every)
+        keep = [] if passes == 0 else None
+        t, f = time_oracle(calls_inputs, every, keep)
+        if keep is not None:
+            refs = keep
         dt += t
         flops += f
         passes += 1
@@ -143,7 +160,16 @@ def cpu_baseline(calls_inputs, target_s=12.0):
     return {"value": flops / dt / 1e12, "unit": UNIT, "cores": oracle.max_threads(), "kind": "oracle",
             "sample": "%d pass(es) over every %s row of both calls of the step (%d of %d rows per pass), %.1f s" % (
                 passes, "" if every == 1 else "%d-th" % every, rows, total, dt),
-            "seconds": dt}
+            "seconds": dt}, refs
+
+
+def parity_numbers(got, ref, v):
+    """max |gpu - oracle| / max|V| and the relative L2 error of `got` (numpy, any float type) against oracle rows."""
+    got = np.asarray(got, dtype=np.float64)
+    err = np.abs(got - ref)
+    return {"max_err_over_maxV": float(err.max() / np.abs(np.asarray(v, dtype=np.float64)).max()),
+            "rel_l2": float(np.linalg.norm(got - ref) / max(np.linalg.norm(ref), 1e-300)),
+            "rows": int(ref.size // ref.shape[-1])}
 
 
 def run_reference(args):
@@ -211,6 +237,10 @@ def run_ours(args):
     torch.cuda.set_device(local_rank)
     device = torch.device("cuda", local_rank)
     stream = torch.cuda.current_stream().cuda_stream
+    if args.workload == "ubench":
+        if rank == 0:
+            print(json.dumps({"workload": "ubench", "rates": instruction_rates(bd, stream)}))
+        return 0
     if args.workload != "c2" and not args.kernel_loop_only:
         raise SystemExit("--workload other than c2 is a profiling aid: combine it with --kernel-loop-only")
     if args.workload == "groupnorm":
@@ -291,6 +321,26 @@ def run_ours(args):
     ms_per_step = ms_total / args.steps
     value = world * flops_per_step / (ms_per_step * 1e-3) / 1e12
 
+    # per-launch statistics: a second, shorter loop with an event behind every launch (the events keep a launch's
+    # set-up from overlapping its predecessor's tail, so this loop is not the one `value` comes from)
+    stat_steps = 0 if args.kernel_loop_only else max(3, min(args.steps, 50))
+    marks = [torch.cuda.Event(enable_timing=True) for _ in range(stat_steps * launches_per_step + 1)]
+    if stat_steps:
+        marks[0].record()
+        n = 0
+        for i in range(stat_steps):
+            for c, tq, tk, tv, to in sets[i % ROTATING_SETS]:
+                rc = bd.sd_attn_forward(att.handle, tq.data_ptr(), tk.data_ptr(), tv.data_ptr(), to.data_ptr(),
+                                        c.B, c.H, c.Nq, c.Nk, c.d, float(c.scale()), bd.F16, stream)
+                if rc != bd.OK:
+                    raise bd.SdAttnError(rc, "sd_attn_forward")
+                n += 1
+                marks[n].record()
+        torch.cuda.synchronize()
+        per_launch_us = np.array([1e3 * marks[i].elapsed_time(marks[i + 1]) for i in range(n)])
+        # what the timed buffers hold now is the output of the LAST launch on each set
+        last_step_of_set0 = max(i for i in range(stat_steps) if i % ROTATING_SETS == 0)
+
     if args.kernel_loop_only:
         # profiling aid: just the warm-up and the timed loop, so that a profiler sees few launches
         if rank == 0:
@@ -343,34 +393,83 @@ def run_ours(args):
         return 0
 
     peaks = measured_peaks()
+    # the step's only kernel is the fused one, so its mean launch duration is the timed region / launches
     per_launch_s = ms_per_step * 1e-3 / launches_per_step
     achieved = calls[0].flops / per_launch_s / 1e12
-    # the step's only kernel is the fused one, so its mean launch duration is the timed region / launches
-    exps_per_launch = calls[0].B * calls[0].H * calls[0].Nq * calls[0].Nk
-    sfu_peak = 16.0 * 148 * (clocks.get("sm_max_mhz") or 1965) * 1e6 / 1e12     # ex2: 16 per clock per SM
+    sms = torch.cuda.get_device_properties(device).multi_processor_count
+    max_mhz = float(clocks.get("sm_max_mhz") or 1965)
+    rates = instruction_rates(bd, stream)
     roofline = {"bound": "tensor", "kernel": "fused4s_attention_kernel", "achieved": achieved,
                 "peak": peaks["tflops"], "unit": "TFLOP/s", "frac": achieved / peaks["tflops"],
                 "peak_source": "%s cuBLAS bf16 burst (fp16 peak = bf16 peak, nominal ratio 1.0)" % peaks["source"],
                 "frac_of_nominal_2250": achieved / NOMINAL_FP16_TFLOPS,
-                "traffic": FUSED_TRAFFIC_BYTES_PER_LAUNCH, "algorithmic_bytes": calls[0].io_bytes(),
-                "us_per_launch": per_launch_s * 1e6,
-                "note": "one exponential per score: the special-function unit alone (16/clk/SM, measured) would cap this "
-                        "d=40 shape at 0.33 of the nominal tensor peak; the kernel sends a quarter of them to the FMA pipe; "
-                        "see roofline_alu",
-                "roofline_alu": {"bound": "alu", "unit": "Texp/s", "achieved": exps_per_launch / per_launch_s / 1e12,
-                                 "peak": sfu_peak, "frac": exps_per_launch / per_launch_s / 1e12 / sfu_peak,
-                                 "peak_source": "16 ex2/clk/SM x 148 SMs x max SM clock (special-function unit only)"}}
+                "traffic": FUSED_TRAFFIC["bytes_per_launch"], "traffic_source": FUSED_TRAFFIC,
+                "algorithmic_bytes": calls[0].io_bytes(), "us_per_launch": per_launch_s * 1e6,
+                "us_per_launch_stats": {"median": float(np.median(per_launch_us)), "min": float(per_launch_us.min()),
+                                        "mean": float(per_launch_us.mean()), "launches": int(per_launch_us.size),
+                                        "how": "an event behind every launch of a second loop (no overlap of a launch's "
+                                               "set-up with its predecessor), rotating inputs larger than L2"},
+                "joint": joint_roofline(calls[0], per_launch_s, rates, peaks, sms, max_mhz),
+                "note": "one exponential per score element: at d=40 the special-function unit and the FMA pipe, not the "
+                        "tensor pipe, bound the kernel; `joint` is the bound of all units together"}
     line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
             "warmup": max(args.warmup, 3), "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
             "vs_baseline": None, "dtype": "f16", "data": "synthetic", "config": workload_config(),
             "clocks": clocks, "e2e": e2e, "gpu_launches": gpu_launches, "roofline": roofline,
             "pct_of_fp16_dense_peak": 100.0 * value / world / NOMINAL_FP16_TFLOPS}
     if world == 1:
-        line["extra"] = extras(att, bd, device, stream, peaks)
+        # the oracle on the very inputs that were timed (set 0), and the outputs the timed launches left there
+        timed_outputs = [to.cpu().numpy() for *_, to in sets[0]]
         host_inputs = [(c, tuple(t.cpu().numpy() for t in (tq, tk, tv))) for c, tq, tk, tv, _ in sets[0]]
-        line["cpu_baseline"] = cpu_baseline(host_inputs)
+        line["extra"] = extras(att, bd, device, stream, peaks)
+        line["cpu_baseline"], refs = cpu_baseline(host_inputs)
+        line["parity"] = {"what": "outputs left in the timed buffers (input set 0) against the oracle's rows of the same inputs",
+                          "tolerance": "max |err| <= 2e-3 max|V|",
+                          "calls": [dict(name=c.name, **parity_numbers(out.reshape(-1, c.d)[rows], ref, v))
+                                    for (c, (q, k, v)), out, (rows, ref) in zip(host_inputs, timed_outputs, refs)]}
+        if any(p["max_err_over_maxV"] > 2e-3 for p in line["parity"]["calls"]):
+            raise RuntimeError("the timed outputs do not match the oracle: %s" % line["parity"])
     print(json.dumps(line))
     return 0
+
+
+def instruction_rates(bd, stream):
+    """Results per clock per SM of the instructions the softmax sweep is made of, and of the sweep itself, measured
+    now (sd_attn_ubench: a few hundred microseconds each), with the SM clock that was in effect."""
+    out = {}
+    for name, op in bd.UBENCH_OPS.items():
+        rate, mhz = bd.sd_attn_ubench(op, 4096, stream)
+        out[name] = {"per_clk_per_sm": rate, "sm_mhz": mhz}
+    return out
+
+
+def joint_roofline(call, per_launch_s, rates, peaks, sms, max_mhz):
+    """Score elements per clock per SM against the bound of all units together.
+
+    Per element: 4 d_pad tensor FLOPs; one exponential, a share x of them on the FMA pipe; 3 + 6x FMA-pipe results
+    (scale, row sum, half a pack; six more on the polynomial path).  The bound is the slowest unit's pace at the
+    measured rates: min(R_ex2 / (1 - x), R_fma / (3 + 6x), R_tensor / (4 d_pad)), with R_tensor the measured GEMM peak
+    per clock per SM.  `softmax_sweep_poly` is what the sweep alone reaches with 16 warps per SM (no tensor memory, no
+    hand-over): the practical ceiling of this instruction mix."""
+    x = POLY_PER8 / 8.0
+    dpad = (call.d + 15) // 16 * 16
+    elements = call.B * call.H * call.Nq * call.Nk
+    r_ex2 = rates["ex2"]["per_clk_per_sm"]
+    r_fma = max(rates["fma"]["per_clk_per_sm"], rates["fma_x2"]["per_clk_per_sm"])
+    eff_mhz = rates["softmax_sweep_poly"]["sm_mhz"]
+    out = {"unit": "score elements/clk/SM", "poly_share": x,
+           "rates_per_clk_per_sm": {k: v["per_clk_per_sm"] for k, v in rates.items()},
+           "formula": "min(ex2/(1-x), fma/(3+6x), tensor_flop_per_clk/(4*dpad))"}
+    for label, mhz in (("at_max_clock", max_mhz), ("at_effective_clock", eff_mhz)):
+        r_tensor = peaks["tflops"] * 1e12 / (sms * mhz * 1e6)            # FLOP per clock per SM at that clock
+        bound = min(r_ex2 / (1.0 - x), r_fma / (FMA_OPS_SFU_PATH + FMA_OPS_POLY_EXTRA * x), r_tensor / (4.0 * dpad))
+        got = elements / (per_launch_s * sms * mhz * 1e6)
+        out[label] = {"sm_mhz": mhz, "achieved": got, "bound": bound, "frac": got / bound,
+                      "bound_units": {"sfu": r_ex2 / (1.0 - x), "fma": r_fma / (FMA_OPS_SFU_PATH + FMA_OPS_POLY_EXTRA * x),
+                                      "tensor": r_tensor / (4.0 * dpad)},
+                      "frac_of_sweep_alone": got / rates["softmax_sweep_poly"]["per_clk_per_sm"]}
+    out["effective_clock_note"] = "clock64 against globaltimer inside the probe kernels, read-only"
+    return out
 
 
 def time_calls(att, bd, tensors, stream, iters, graph=False, dtype=None):
@@ -411,6 +510,14 @@ def time_calls(att, bd, tensors, stream, iters, graph=False, dtype=None):
     return 1e3 * start.elapsed_time(end) / iters
 
 
+def time_calls_once(att, bd, t, stream):
+    c, tq, tk, tv, to = t
+    rc = bd.sd_attn_forward(att.handle, tq.data_ptr(), tk.data_ptr(), tv.data_ptr(), to.data_ptr(), c.B, c.H, c.Nq, c.Nk,
+                            c.d, float(c.scale()), bd.F16, stream)
+    if rc != bd.OK:
+        raise bd.SdAttnError(rc, "sd_attn_forward")
+
+
 def time_batch(att, bd, tensors, stream, iters):
     """Mean microseconds of one sd_attn_forward_batch call over `tensors`: plain, and replayed as a CUDA graph."""
     import torch
@@ -446,10 +553,136 @@ def time_batch(att, bd, tensors, stream, iters):
     return plain, 1e3 * start.elapsed_time(end) / iters
 
 
-def extras(att, bd, device, stream, peaks):
-    """Secondary numbers: the UNet-step attention set (32 calls) and the memory-bound cross-attention."""
+def time_stats(fn, iters, sync):
+    """{median, min, mean} microseconds of fn(i), an event behind every call (device time per call)."""
+    import torch
+    marks = [torch.cuda.Event(enable_timing=True) for _ in range(iters + 1)]
+    sync()
+    marks[0].record()
+    for i in range(iters):
+        fn(i)
+        marks[i + 1].record()
+    sync()
+    us = np.array([1e3 * marks[i].elapsed_time(marks[i + 1]) for i in range(iters)])
+    return {"median": float(np.median(us)), "min": float(us.min()), "mean": float(us.mean()), "calls": iters}
+
+
+def oracle_parity(call, host, out_tensor, rows=None):
+    """Parity of a timed buffer: the oracle on the same inputs (all rows, or the sample `rows`) against what the
+    library left in `out_tensor`."""
+    import oracle
+    q, k, v = host
+    ref, _, _ = oracle.forward(q, k, v, call.scale(), rows=rows)
+    got = out_tensor.cpu().numpy()
+    got = got.reshape(-1, call.d)[rows] if rows is not None else got
+    return parity_numbers(got, ref.reshape(got.shape), v)
+
+
+def config_numbers(att, bd, device, stream, peaks):
+    """The workloads beside the bench's own: c1 (single-pass and two-pass), the four c3 cross shapes (as CUDA graphs),
+    c5 self-attention plain and peaked with the two-pass comparator beside it -- each timed (median / min / mean of
+    per-call device times) and checked against the oracle on the buffers that were timed."""
     import torch
     out = {}
+
+    def to_dev(call):
+        host = workloads.make_inputs(call)
+        tq, tk, tv = (torch.from_numpy(x).to(device) for x in host)
+        return host, (call, tq, tk, tv, torch.empty_like(tq))
+
+    def fwd(a, t, strm):
+        c, tq, tk, tv, to = t
+        rc = bd.sd_attn_forward(a.handle, tq.data_ptr(), tk.data_ptr(), tv.data_ptr(), to.data_ptr(), c.B, c.H, c.Nq, c.Nk,
+                                c.d, float(c.scale()), bd.F16, strm)
+        if rc != bd.OK:
+            raise bd.SdAttnError(rc, "sd_attn_forward")
+
+    # --- c1: the smallest instance, single-pass and the two-pass comparator of Sec. 3.2.1
+    c1 = workloads.config1()[0]
+    host, t = to_dev(c1)
+    for _ in range(5):
+        fwd(att, t, stream)
+    entry = {"fused_us_back_to_back": time_calls(att, bd, [t], stream, 100),
+             "fused_us": time_stats(lambda i: fwd(att, t, stream), 50, torch.cuda.synchronize),
+             "note": "back_to_back: mean of a loop of launches, each one's set-up under its predecessor's tail; the "
+                     "statistics: an event behind every call, so every call pays its whole launch"}
+    att.check(stream)
+    entry["fused_parity"] = oracle_parity(c1, host, t[4])
+    tp = bd.Attention(bd.MODE_TWOPASS)
+    need = bd.sd_attn_workspace_bytes(bd.MODE_TWOPASS, c1.B, c1.H, c1.Nq, c1.Nk, c1.d, bd.F16)
+    ws = torch.empty(need, dtype=torch.uint8, device=device)
+    bd.sd_attn_set_workspace(tp.handle, ws.data_ptr(), need)
+    for _ in range(3):
+        fwd(tp, t, stream)
+    entry["twopass_us_back_to_back"] = time_calls(tp, bd, [t], stream, 40)
+    entry["twopass_us"] = time_stats(lambda i: fwd(tp, t, stream), 20, torch.cuda.synchronize)
+    tp.check(stream)
+    entry["twopass_parity"] = oracle_parity(c1, host, t[4])
+    entry["twopass_scratch_bytes"] = need
+    entry["tflops_fused"] = c1.flops / (entry["fused_us_back_to_back"] * 1e-6) / 1e12
+    out["c1_self_1024_d40"] = entry
+    del ws
+
+    # --- c3: the four cross-attention shapes, each as a CUDA graph of 8 back-to-back calls (microseconds per call)
+    c3 = {}
+    for c in workloads.config3():
+        host, t = to_dev(c)
+        fwd(att, t, stream)
+        side = torch.cuda.Stream()
+        side.wait_stream(torch.cuda.current_stream())
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g, stream=side):
+            for _ in range(8):
+                fwd(att, t, side.cuda_stream)
+        g.replay()
+        st = time_stats(lambda i: g.replay(), 20, torch.cuda.synchronize)
+        att.check(stream)
+        c3[c.name] = {"us_per_call": {k: (v / 8 if k != "calls" else v * 8) for k, v in st.items()},
+                      "achieved_gbs": c.io_bytes() / (st["median"] / 8 * 1e-6) / 1e9,
+                      "parity": oracle_parity(c, host, t[4])}
+    out["c3_cross_set"] = c3
+
+    # --- c5: 9216 tokens, plain and peaked; the single-pass kernel and the two-pass comparator that materialises the
+    # 9216 x 9216 score matrix (10.9 GB of binary32 scratch)
+    c5 = {}
+    g = np.random.default_rng(5)
+    need = 0
+    for c in workloads.config5()[:2]:
+        need = max(need, bd.sd_attn_workspace_bytes(bd.MODE_TWOPASS, c.B, c.H, c.Nq, c.Nk, c.d, bd.F16))
+    ws = torch.empty(need, dtype=torch.uint8, device=device)
+    bd.sd_attn_set_workspace(tp.handle, ws.data_ptr(), need)
+    for c in workloads.config5()[:2]:
+        host, t = to_dev(c)
+        other = (c, torch.randn_like(t[1]), torch.randn_like(t[2]), torch.randn_like(t[3]), torch.empty_like(t[4]))
+        pair = [t, other]     # two sets of 94 MB each: rotating inputs larger than the L2
+        rows = np.sort(g.choice(c.B * c.H * c.Nq, size=512, replace=False)).astype(np.int64)
+        for i in range(3):
+            fwd(att, pair[i % 2], stream)
+        e = {"fused_us": time_stats(lambda i: fwd(att, pair[i % 2], stream), 8, torch.cuda.synchronize)}
+        att.check(stream)
+        e["fused_parity"] = oracle_parity(c, host, t[4], rows)
+        e["tflops_fused"] = c.flops / (e["fused_us"]["median"] * 1e-6) / 1e12
+        fwd(tp, t, stream)
+        e["twopass_us"] = time_stats(lambda i: fwd(tp, t, stream), 3, torch.cuda.synchronize)
+        tp.check(stream)
+        e["twopass_parity"] = oracle_parity(c, host, t[4], rows)
+        e["twopass_over_fused"] = e["twopass_us"]["median"] / e["fused_us"]["median"]
+        c5[c.name] = e
+        del pair, other, t
+    c5["twopass_scratch_bytes"] = need
+    c5["parity_rows"] = "512 seeded random rows of each call"
+    out["c5_self_9216_d40"] = c5
+    tp.close()
+    del ws
+    torch.cuda.empty_cache()
+    return out
+
+
+def extras(att, bd, device, stream, peaks):
+    """Secondary numbers: the other workloads, the UNet-step attention set (32 calls), the memory-bound
+    cross-attention, layouts and dtypes, and the three steps beside the attention path."""
+    import torch
+    out = config_numbers(att, bd, device, stream, peaks)
     calls = workloads.config4()
     tensors = []
     for c in calls:
@@ -465,7 +698,8 @@ def extras(att, bd, device, stream, peaks):
                                       "us_batch_call": us_batch, "us_batch_call_cuda_graph": us_batch_graph,
                                       "tflops_batch_call_cuda_graph": flops / (us_batch_graph * 1e-6) / 1e12,
                                       "batch_note": "the same 32 calls as independent problems of one "
-                                                    "sd_attn_forward_batch call (spread over four streams)",
+                                                    "sd_attn_forward_batch call: 7 launches (one per shape) over "
+                                                    "four streams",
                                       "note": "512x512, B=2, H=8: 16 self + 16 cross calls (L2-warm: 285 MB of tensors)"}
     # cross-attention at the large-latent size, rotating sets so that Q/O stream from HBM
     c = workloads.config5()[2]
@@ -478,11 +712,33 @@ def extras(att, bd, device, stream, peaks):
         csets.append((c, tq, tk, tv, torch.empty_like(tq)))
     us_cross = time_calls(att, bd, csets, stream, 10) / n_sets
     gbs = c.io_bytes() / (us_cross * 1e-6) / 1e9
-    out["cross_attention_9216x77_d40"] = {"us_per_call": us_cross, "achieved_gbs": gbs, "bound": "hbm",
+    cross_stats = time_stats(lambda i: time_calls_once(att, bd, csets[i % n_sets], stream), 24, torch.cuda.synchronize)
+    att.check(stream)
+    q0, k0, v0 = workloads.make_inputs(workloads.Call(c.name, c.B, c.H, c.Nq, c.Nk, c.d, c.config_index,
+                                                      call_index=c.call_index, padded_text=True))
+    rows = np.arange(0, c.B * c.H * c.Nq, 37, dtype=np.int64)
+    out["cross_attention_9216x77_d40"] = {"us_per_call": us_cross, "us_per_call_with_an_event_behind_each": cross_stats,
+                                          "achieved_gbs": gbs, "bound": "hbm",
                                           "peak_gbs": peaks["hbm_gbs"], "frac": gbs / peaks["hbm_gbs"],
                                           "frac_of_nominal_8000": gbs / 8000.0,
-                                          "algorithmic_bytes": c.io_bytes(), "peak_source": peaks["source"]}
+                                          "algorithmic_bytes": c.io_bytes(), "peak_source": peaks["source"],
+                                          "parity": oracle_parity(c, (q0, k0, v0), csets[0][4], rows)}
+    # four times the batch (B = 16): the same kernel with four times the items per CTA, so that ramp and pace show apart
+    c4x = workloads.Call(c.name + "_4x_batch", 4 * c.B, c.H, c.Nq, c.Nk, c.d, c.config_index, call_index=c.call_index,
+                         padded_text=True)
+    bsets4 = []
+    for r in range(2):     # 2 x 190 MB
+        tq = torch.randn(c4x.B, c4x.H, c4x.Nq, c4x.d, device=device, dtype=torch.float16)
+        tk = torch.randn(c4x.B, c4x.H, c4x.Nk, c4x.d, device=device, dtype=torch.float16)
+        bsets4.append((c4x, tq, tk, torch.randn_like(tk), torch.empty_like(tq)))
+    for i in range(3):
+        time_calls_once(att, bd, bsets4[i % 2], stream)
+    st4 = time_stats(lambda i: time_calls_once(att, bd, bsets4[i % 2], stream), 10, torch.cuda.synchronize)
     att.check(stream)
+    gbs4 = c4x.io_bytes() / (st4["median"] * 1e-6) / 1e9
+    out["cross_attention_9216x77_d40"]["at_4x_batch"] = {"us_per_call": st4, "achieved_gbs": gbs4,
+                                                         "frac": gbs4 / peaks["hbm_gbs"], "bytes": c4x.io_bytes()}
+    del bsets4
     # the same two measurements with the tensors read as token-major [B][N][H][d] (the head split and merge around
     # the attention as views): the same buffers, so the same bytes and the same sizes
     att_t = bd.Attention(layout=bd.LAYOUT_BNHD)
@@ -733,13 +989,26 @@ def main():
     ap.add_argument("--steps", type=int, default=200)
     ap.add_argument("--warmup", type=int, default=10)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--workload", default="c2", choices=["c2", "c5-cross", "c3-cross", "c4", "c4-d80", "c1", "c1-twopass", "geglu", "groupnorm", "winograd"],
+    ap.add_argument("--workload", default="c2", choices=["c2", "c5-cross", "c3-cross", "c4", "c4-d80", "c1", "c1-twopass", "geglu", "groupnorm", "winograd", "ubench"],
                     help="with --kernel-loop-only: which calls the loop runs (the bench line is always c2)")
     ap.add_argument("--kernel-loop-only", action="store_true",
                     help="run only the warm-up and the timed loop (for ncu captures)")
     args = ap.parse_args()
     if args.impl == "reference":
         return run_reference(args)
+    if D.launched_by_a_launcher():
+        world = int(os.environ["WORLD_SIZE"])
+        if world != args.gpus:
+            raise SystemExit("--gpus %d but the launcher started %d ranks" % (args.gpus, world))
+        return run_ours(args)
+    if args.gpus > 1:
+        # no launcher: start the ranks here, one process per GPU (NCCL only for the barrier and the max of the times)
+        import torch
+        if torch.cuda.device_count() < args.gpus:
+            raise SystemExit("--gpus %d but this node shows %d CUDA devices" % (args.gpus, torch.cuda.device_count()))
+        os.environ.setdefault("NCCL_DEBUG", "INFO")     # the communicator lines go to stderr
+        D.spawn_ranks(args.gpus, run_ours, (args,))
+        return 0
     return run_ours(args)
 
 

@@ -230,6 +230,19 @@ int sd_attn_query_status(sd_attn_handle *h, void *stream, int *detail);
  */
 int sd_attn_selftest_wait_timeout(sd_attn_handle *h, void *stream);
 
+/*
+ * Instruction-rate probes behind the joint roofline of the FUSED kernel (Eq. 3 costs one exponential and a few
+ * multiply-adds per score element next to its 4 d tensor-core FLOPs; which unit bounds a head dim depends on their
+ * rates).  Runs, twice, one block of 512 threads per SM that repeats `iters` (1 .. 2^20) trips of independent
+ * chains of ONE operation on registers -- op 0: ex2.approx.ftz.f32; 1: fma.rn.f32; 2: fma.rn.f32x2 (two results per
+ * instruction); 3: the kernels' exp2 / row-sum / binary16-pack sweep over 32 scores, every exponential on the
+ * special-function unit; 4: the same with the share of them the d <= 48 kernel sends to the FMA pipe -- then
+ * synchronises `stream` and returns, from the second run, the results per clock per SM (mean over the SMs) and the
+ * SM clock in MHz that was in effect (clock64 against globaltimer).  A few hundred microseconds at iters = 4096;
+ * allocates nothing.  Errors: INVALID_VALUE, ARCH, CUDA.
+ */
+int sd_attn_ubench(int op, int iters, void *stream, double *results_per_clk_per_sm, double *sm_mhz);
+
 /* Which kernel family the last successful forward used (an sd_attn_mode, never AUTO). */
 int sd_attn_last_mode(const sd_attn_handle *h);
 

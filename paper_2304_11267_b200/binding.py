@@ -24,7 +24,7 @@ CROSS_MAX_NK = 128
 MAX_D = 160
 STATIC_MAX_SCRATCH = 34 * 1024 * 1024   # SD_ATTN_STATIC_MAX_SCRATCH: built-in scratch of the no-allocation entry point
 
-EXPORTS = ["sd_attn_create", "sd_attn_create_ex", "sd_attn_static_query_status", "sd_attn_selftest_wait_timeout", "sd_attn_forward", "sd_attn_destroy", "sd_attn_set_mode",
+EXPORTS = ["sd_attn_create", "sd_attn_create_ex", "sd_attn_static_query_status", "sd_attn_selftest_wait_timeout", "sd_attn_ubench", "sd_attn_forward", "sd_attn_destroy", "sd_attn_set_mode",
            "sd_attn_workspace_bytes", "sd_attn_set_workspace", "sd_attn_twopass_buffers",
            "sd_attn_query_status", "sd_attn_last_mode", "sd_attn_launch_count", "sd_attn_status_string",
            "sd_attn_forward_host", "sd_attn_host_staging_bytes",
@@ -76,6 +76,8 @@ def load() -> ctypes.CDLL:
     lib.sd_attn_create_ex.argtypes = [ctypes.POINTER(Options), ctypes.POINTER(vp)]
     lib.sd_attn_selftest_wait_timeout.restype = ci
     lib.sd_attn_selftest_wait_timeout.argtypes = [vp, vp]
+    lib.sd_attn_ubench.restype = ci
+    lib.sd_attn_ubench.argtypes = [ci, ci, vp, ctypes.POINTER(ctypes.c_double), ctypes.POINTER(ctypes.c_double)]
     lib.sd_attn_static_query_status.restype = ci
     lib.sd_attn_static_query_status.argtypes = [vp, ctypes.POINTER(ci)]
     lib.sd_attn_forward.restype = ci
@@ -353,6 +355,18 @@ def sd_attn_query_status(handle, stream=0):
 def sd_attn_selftest_wait_timeout(handle, stream=0) -> int:
     """Enqueue the self-test kernel whose bounded wait runs out (see include/sd_attn.h)."""
     return load().sd_attn_selftest_wait_timeout(handle, stream or None)
+
+
+UBENCH_OPS = {"ex2": 0, "fma": 1, "fma_x2": 2, "softmax_sweep": 3, "softmax_sweep_poly": 4}
+
+
+def sd_attn_ubench(op: int, iters: int = 4096, stream=0):
+    """Instruction-rate probe (see include/sd_attn.h): (results per clock per SM, SM clock in MHz)."""
+    rate, mhz = ctypes.c_double(), ctypes.c_double()
+    rc = load().sd_attn_ubench(op, iters, stream or None, ctypes.byref(rate), ctypes.byref(mhz))
+    if rc != OK:
+        raise SdAttnError(rc, "sd_attn_ubench")
+    return rate.value, mhz.value
 
 
 def sd_attn_last_mode(handle) -> int:

@@ -24,6 +24,7 @@
 #include "selftest_kernel.cuh"
 #include "simt_kernel.cuh"
 #include "twopass_kernel.cuh"
+#include "ubench_kernel.cuh"
 
 using namespace sd_attn;
 
@@ -1373,3 +1374,47 @@ extern "C" int sd_winograd_query_status(void* stream, int* detail) {
     return SD_ATTN_OK;
 }
 
+
+// ------------------------------------------------------------------------------------------------
+// Instruction-rate probes for the joint roofline (see ubench_kernel.cuh): stateless, allocate nothing.
+constexpr int UBENCH_MAX_BLOCKS = 1024;
+static __device__ __align__(256) long long g_ubench_out[2 * UBENCH_MAX_BLOCKS];
+static __device__ float g_ubench_sink[4];
+
+extern "C" int sd_attn_ubench(int op, int iters, void* stream, double* results_per_clk_per_sm, double* sm_mhz) {
+    if (op < 0 || op >= UBENCH_OPS || iters <= 0 || iters > (1 << 20) || !results_per_clk_per_sm || !sm_mhz)
+        return SD_ATTN_ERR_INVALID_VALUE;
+    int dev = 0, major = 0, sms = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e == cudaSuccess) e = cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev);
+    if (e == cudaSuccess) e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+    if (e != cudaSuccess) return cuda_fail(nullptr, e);
+    if (major != 10) return SD_ATTN_ERR_ARCH;
+    if (sms > UBENCH_MAX_BLOCKS) sms = UBENCH_MAX_BLOCKS;
+    long long* out = nullptr;
+    float* sink = nullptr;
+    e = cudaGetSymbolAddress((void**)&out, g_ubench_out);
+    if (e == cudaSuccess) e = cudaGetSymbolAddress((void**)&sink, g_ubench_sink);
+    if (e != cudaSuccess) return cuda_fail(nullptr, e);
+    cudaStream_t s = (cudaStream_t)stream;
+    for (int rep = 0; rep < 2; ++rep) {   // the second run is the measurement (the first warms the clocks and the code)
+        switch (op) {
+            case UBENCH_EX2: ubench_kernel<UBENCH_EX2><<<sms, UBENCH_THREADS, 0, s>>>(iters, 0.5f, out, sink); break;
+            case UBENCH_FMA: ubench_kernel<UBENCH_FMA><<<sms, UBENCH_THREADS, 0, s>>>(iters, 0.5f, out, sink); break;
+            case UBENCH_FMA_X2: ubench_kernel<UBENCH_FMA_X2><<<sms, UBENCH_THREADS, 0, s>>>(iters, 0.5f, out, sink); break;
+            case UBENCH_SWEEP: ubench_kernel<UBENCH_SWEEP><<<sms, UBENCH_THREADS, 0, s>>>(iters, 0.5f, out, sink); break;
+            default: ubench_kernel<UBENCH_SWEEP_POLY><<<sms, UBENCH_THREADS, 0, s>>>(iters, 0.5f, out, sink); break;
+        }
+    }
+    e = cudaGetLastError();
+    if (e == cudaSuccess) e = cudaStreamSynchronize(s);
+    static long long host[2 * UBENCH_MAX_BLOCKS];
+    if (e == cudaSuccess) e = cudaMemcpy(host, out, sizeof(long long) * 2 * sms, cudaMemcpyDeviceToHost);
+    if (e != cudaSuccess) return cuda_fail(nullptr, e);
+    double clk = 0, ns = 0;
+    for (int b = 0; b < sms; ++b) { clk += (double)host[2 * b]; ns += (double)host[2 * b + 1]; }
+    clk /= sms; ns /= sms;
+    *results_per_clk_per_sm = (double)UBENCH_THREADS * iters * ubench_results_per_trip(op) / clk;
+    *sm_mhz = clk / ns * 1e3;
+    return SD_ATTN_OK;
+}

@@ -30,6 +30,42 @@ def init_process_group(backend: str):
     return rank, local_rank, world
 
 
+def _free_port() -> int:
+    import socket
+    with socket.socket() as sock:
+        sock.bind(("127.0.0.1", 0))
+        return sock.getsockname()[1]
+
+
+def _rank_main(rank: int, world: int, port: int, target, args):
+    os.environ.update(RANK=str(rank), LOCAL_RANK=str(rank), WORLD_SIZE=str(world), MASTER_ADDR="127.0.0.1",
+                      MASTER_PORT=str(port))
+    rc = target(*args)
+    if rc not in (None, 0):
+        raise SystemExit(int(rc))
+
+
+def launched_by_a_launcher() -> bool:
+    """True when RANK / WORLD_SIZE come from torchrun (or another launcher): the ranks exist already."""
+    return "WORLD_SIZE" in os.environ and "RANK" in os.environ
+
+
+def spawn_ranks(world: int, target, args=()) -> None:
+    """Start `world` ranks of `target(*args)` on this node, one process each, with RANK / LOCAL_RANK / WORLD_SIZE /
+    MASTER_ADDR (127.0.0.1) / MASTER_PORT (a free port) set as a launcher would set them, and wait for them.
+    Raises if any rank fails or returns a non-zero code: a job that ends with fewer ranks than asked must not pass.
+    `target` must be importable (a module-level function)."""
+    if world < 1:
+        raise ValueError("world size must be positive")
+    import torch.multiprocessing as mp
+    ctx = mp.spawn(_rank_main, args=(world, _free_port(), target, tuple(args)), nprocs=world, join=False)
+    while not ctx.join():       # raises ProcessRaisedException / ProcessExitedException on the first failure
+        pass
+    codes = [p.exitcode for p in ctx.processes]
+    if len(codes) != world or any(c != 0 for c in codes):
+        raise RuntimeError("asked for %d ranks, exit codes %s" % (world, codes))
+
+
 def shard_bh(x, rank: int, world: int):
     """Slice a [B, H, N, d] array/tensor to this rank's (batch, head) units -> [1, units, N, d]."""
     B, H = x.shape[0], x.shape[1]

@@ -62,3 +62,33 @@ def test_single_rank_helpers_are_identity():
     assert np.array_equal(D.shard_bh(x, 0, 1).reshape(2, 3, 4, 5), x)
     a = D.shard_bh(x, 1, 4)            # 6 units over 4 ranks: 2, 2, 1, 1
     assert a.shape == (1, 2, 4, 5) and np.array_equal(a[0], x.reshape(6, 4, 5)[2:4])
+
+
+def _spawned_rank(out_dir, fail_rank):
+    """What bench.py's ranks do with the environment spawn_ranks gives them (gloo instead of nccl)."""
+    sys.path.insert(0, ROOT)
+    from paper_2304_11267_b200 import distributed as D
+    rank, local_rank, world = D.init_process_group("gloo")
+    assert D.launched_by_a_launcher() and local_rank == rank and os.environ["MASTER_ADDR"] == "127.0.0.1"
+    D.barrier(world)
+    slowest = D.max_over_ranks(1.0 + rank, world)
+    open(os.path.join(out_dir, "rank%d_of_%d" % (rank, world)), "w").write("%g" % slowest)
+    dist.destroy_process_group()
+    return 3 if rank == fail_rank else 0
+
+
+def test_spawn_ranks_starts_every_rank_and_fails_loudly(tmp_path):
+    """`bench.py --gpus N` without a launcher starts its N ranks through spawn_ranks: every rank must come up with a
+    launcher's environment, and a rank that fails must fail the whole job."""
+    from paper_2304_11267_b200 import distributed as D
+    good = tmp_path / "good"
+    good.mkdir()
+    D.spawn_ranks(2, _spawned_rank, (str(good), -1))
+    assert sorted(os.listdir(good)) == ["rank0_of_2", "rank1_of_2"]
+    assert open(good / "rank0_of_2").read() == "2"            # the max over ranks reached rank 0
+    bad = tmp_path / "bad"
+    bad.mkdir()
+    with pytest.raises(Exception):
+        D.spawn_ranks(2, _spawned_rank, (str(bad), 1))
+    with pytest.raises(ValueError):
+        D.spawn_ranks(0, _spawned_rank, (str(bad), -1))
