@@ -7,7 +7,8 @@ Tolerance, derived from the arithmetic: bfloat16 keeps 8 significant bits, so ro
 2^-8 relative, against binary16's 2^-11 -- 8 times coarser.  Two roundings matter, as for binary16: the weights
 (each 2^-8 relative, signs independent; coherent worst case 2^-8 * max|V|) and the output (2^-8 * |o|, |o| <=
 max|V|); everything else (binary32 accumulation, the exponential) is far below.  Worst case 2 * 2^-8 * max|V| =
-7.8e-3 * max|V|; the bound used is 8 times binary16's stated one: 1.6e-2 * max|V|, and 1.6e-2 relative L2.
+7.8e-3 * max|V|; the bounds used: 8e-3 * max|V| (that worst case; measured 3.7e-4 ... 1.6e-3) and 5e-3 relative L2
+(the output's rounding alone is 2^-8 / sqrt(3) = 2.3e-3 relative, measured 1.6e-3 ... 2.5e-3: a scale error of one percent fails).
 """
 import numpy as np
 import pytest
@@ -17,8 +18,8 @@ import oracle
 torch = pytest.importorskip("torch")
 pytestmark = pytest.mark.gpu
 
-BF16_ABS = 1.6e-2
-BF16_REL_L2 = 1.6e-2
+BF16_ABS = 8e-3
+BF16_REL_L2 = 5e-3
 
 
 @pytest.fixture(scope="module")

@@ -9,7 +9,7 @@ heavily cancelling sum.  For independent inputs that comes to an error of about 
 9e-3 (last corner) of the output's r.m.s. per element, 3e-3 in relative L2 (emulated in double precision with
 rounded U and V; the transformed values of standard-normal inputs reach 190, of the filter 1/16 of the weights').
 The output's own rounding adds 2^-11 |y|.  Bounds used: relative L2 <= 6e-3 (twice the estimate) and
-max |err| <= 0.08 * rms(y) + 2^-11 |y| (nine sigma of the worst position); measured values are printed.
+max |err| <= 0.065 * rms(y) + 2^-11 |y| (seven sigma of the worst position; measured at most 0.054); measured values are printed.
 """
 import numpy as np
 import pytest
@@ -20,7 +20,7 @@ torch = pytest.importorskip("torch")
 pytestmark = pytest.mark.gpu
 
 REL_L2 = 6e-3
-MAX_ABS_OF_RMS = 0.08
+MAX_ABS_OF_RMS = 0.065
 
 
 @pytest.fixture(scope="module")
