@@ -463,7 +463,8 @@ fused4s_attention_kernel(const __grid_constant__ Fused4Args args) {
                 const bool more = jn < n_kv;
                 if (more)   // landed long ago: keep this wait off the critical path
                     ok = mbar_wait(smem_u32(&bar_kv_full[sn]), pn, abort_p, args.status, SITE_G_KV, jn);
-                if (ok) ok = mbar_wait(smem_u32(&bar_p_full[t][b]), ph, abort_p, args.status, SITE_G_P, j);
+                // (plain tests first: the hardware's suspension inside try_wait costs this hand-over about 1% of the call)
+                if (ok) ok = mbar_wait_eager(smem_u32(&bar_p_full[t][b]), ph, abort_p, args.status, SITE_G_P, j);
                 if (!ok) break;
                 tc_fence_after_sync();
                 issue_o(j, sj, b);

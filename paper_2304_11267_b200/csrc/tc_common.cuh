@@ -119,6 +119,16 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
     return false;
 }
 
+// The same for a wait on the hand-over path of the fused kernels: the first polls are plain tests (no suspension by
+// the hardware, so a completed phase is seen at once), then the bounded wait above takes over.
+template <uint32_t SPIN = 4096>
+__device__ __forceinline__ bool mbar_wait_eager(uint32_t bar, uint32_t parity, volatile int* abort_flag,
+                                                int* status, int site, int tile) {
+    for (uint32_t i = 0; i < SPIN; ++i)
+        if (mbar_test(bar, parity)) return true;
+    return mbar_wait(bar, parity, abort_flag, status, site, tile);
+}
+
 // After a block gave up: give copies that may still be in flight a bounded chance to land before
 // shared memory is released.  Ignores the abort flag, reports nothing.
 __device__ __forceinline__ void mbar_drain(uint32_t bar, uint32_t parity) {
