@@ -271,11 +271,15 @@ long long sd_attn_launch_count(const sd_attn_handle *h);
  *     current) and raises the kernels' shared-memory limits; make that first call outside any stream
  *     capture.  Later calls only enqueue work on `stream`.
  *   - All calls on a device share the one array, which keeps whatever the previous call left in it; every
- *     call overwrites what it reads and clears its device status word first, so calls that follow one
- *     another on a stream are independent.  Calls that OVERLAP on the GPU (different streams, or different
- *     host threads without ordering) race on the array and produce garbage: serialise them.
- *   - A bounded wait that expires inside a kernel is recorded in a status word beside the array;
- *     sd_attn_static_query_status reads it (there is no handle to query).
+ *     call overwrites what it reads, so calls that follow one another on a stream are independent.  Calls
+ *     that OVERLAP on the GPU (different streams, or different host threads without ordering) race on the
+ *     array and produce garbage: serialise them.
+ *   - A bounded wait that expires inside a kernel is recorded in a status word beside the array (zero from the
+ *     first call's set-up on; written only by a kernel that gives up; read and cleared by
+ *     sd_attn_static_query_status: there is no handle to query).
+ *   - The array's device address is looked up once per device and kept for the life of the process: after a
+ *     cudaDeviceReset of that device the kept address is stale and this entry point must not be used again in
+ *     the process (the library cannot see the reset).
  */
 #define SD_ATTN_STATIC_MAX_SCRATCH ((size_t)34 * 1024 * 1024)
 int sd_attn_forward_twopass_static(const void *q, const void *k, const void *v, void *out, int B, int H,
