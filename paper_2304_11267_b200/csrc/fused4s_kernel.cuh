@@ -319,7 +319,8 @@ fused4s_attention_kernel(const __grid_constant__ Fused4Args args) {
             int s = 0, pe = 1;   // stage of key tile j; parity of the kv_empty phase that frees it (from j = stages on)
             for (int j = 0; j < n_kv; ++j, ++s) {
                 if (s == stages) { s = 0; pe ^= 1; }
-                if (j >= stages && !mbar_wait(smem_u32(&bar_kv_empty[s]), pe, abort_p, args.status, SITE_G_EMPTY, j))
+                // (eight stages ahead of the issuers: it sleeps between polls, which is worth 1% of the call)
+                if (j >= stages && !mbar_wait_lazy(smem_u32(&bar_kv_empty[s]), pe, abort_p, args.status, SITE_G_EMPTY, j))
                     break;
                 const uint32_t k_dst = kv_smem + s * 2 * kv_tile_bytes, v_dst = k_dst + kv_tile_bytes;
                 const uint32_t bar = smem_u32(&bar_kv_full[s]);

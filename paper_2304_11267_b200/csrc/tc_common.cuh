@@ -119,6 +119,21 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
     return false;
 }
 
+// The same for a waiter that is far ahead of what it waits for (a producer with a deep ring): it sleeps between polls
+// from the first failed one on, so that its polling does not take issue slots from the warps that share its
+// scheduler.  The poll budget is the same number of polls, so the bound in time is longer.
+__device__ __forceinline__ bool mbar_wait_lazy(uint32_t bar, uint32_t parity, volatile int* abort_flag,
+                                               int* status, int site, int tile) {
+    for (uint32_t i = 0; i < WAIT_POLL_LIMIT; ++i) {
+        if (mbar_try_wait(bar, parity)) return true;
+        __nanosleep(400);
+        if ((i & 15) == 15 && *abort_flag) return false;
+    }
+    *abort_flag = 1;
+    report_timeout(status, site, tile);
+    return false;
+}
+
 // The same for a wait on the hand-over path of the fused kernels: the first polls are plain tests (no suspension by
 // the hardware, so a completed phase is seen at once), then the bounded wait above takes over.
 template <uint32_t SPIN = 4096>
