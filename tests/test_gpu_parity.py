@@ -691,3 +691,80 @@ def test_key_range_of_a_unit_cut_between_ctas(bd, shape):
             a.close()
         check(pick(outs[shares]), ref, v, what="%s shares=%d" % (shape, shares))
     assert np.abs(outs[1].astype(np.float64) - outs[0].astype(np.float64)).max() <= 2 * F16_ABS * np.abs(v).max()
+
+
+def _random_shapes(n, seed):
+    """Seeded draws over the whole argument space of the fp16 path: batch and heads 1..9, row and key counts that
+    straddle the 64-key and 128-row tile sizes (and the 77-key kernel's 65..80 range), every head dim the tensor-core
+    kernels take (multiples of 8 up to 160) and a few they do not (the CUDA-core path)."""
+    g = np.random.default_rng(seed)
+    shapes = []
+    for _ in range(n):
+        B, H = int(g.integers(1, 4)), int(g.integers(1, 10))
+        Nq = int(g.choice([g.integers(1, 130), g.integers(130, 700), g.integers(700, 1400)]))
+        Nk = int(g.choice([g.integers(1, 65), g.integers(65, 81), g.integers(81, 300), g.integers(300, 1400)]))
+        d = int(g.choice([8 * g.integers(1, 21), 8 * g.integers(1, 21), g.integers(1, 161)]))
+        qmult = float(g.choice([1.0, 4.0]))
+        scale = float(g.choice([d ** -0.5, -(d ** -0.5), 0.5 * d ** -0.5]))
+        shapes.append((B, H, Nq, Nk, d, qmult, scale))
+    return shapes
+
+
+@pytest.mark.parametrize("case", _random_shapes(36, 20230421), ids=lambda c: "x".join(str(v) for v in c[:5]))
+def test_random_shapes_every_mode_that_takes_them(att, bd, case):
+    """A net under the hand-picked cases: whatever the draw, AUTO and every mode that accepts the shape agree with the
+    oracle (a mode may refuse a shape with UNSUPPORTED -- CROSS beyond 128 keys, the tensor-core modes at head dims
+    that are not multiples of 8 -- but must not return a wrong result)."""
+    B, H, Nq, Nk, d, qmult, scale = case
+    q, k, v = rand_qkv(77000 + Nq * 3 + Nk * 5 + d, B, H, Nq, Nk, d, qmult=qmult)
+    scale = float(np.float32(scale))
+    ref, _, _ = oracle.forward(q, k, v, scale)
+    ran = 0
+    for name, mode in (("auto", bd.MODE_AUTO), ("fused", bd.MODE_FUSED), ("cross", bd.MODE_CROSS), ("simt", bd.MODE_SIMT)):
+        att.set_mode(mode)
+        try:
+            out = att.forward(gpu(q), gpu(k), gpu(v), scale=scale)
+        except bd.SdAttnError as e:
+            assert name != "auto" and e.status == bd.ERR_UNSUPPORTED, "%s refused %s: %s" % (name, case, e)
+            continue
+        att.check()
+        check(out.cpu().numpy(), ref, v, what="%s %s" % (name, case))
+        ran += 1
+    assert ran >= 2   # AUTO and the mode it chose, at least
+
+
+def test_random_shapes_as_one_batch_and_token_major(bd):
+    """The same kind of draws through the two other doors: all of them as ONE sd_attn_forward_batch call (problems of
+    equal shape share a launch, the rest are spread over the handle's streams), and each of them with token-major
+    tensors.  Both must reproduce the single head-major call bit for bit, and that call the oracle."""
+    cases = _random_shapes(14, 1107) + [c for c in _random_shapes(36, 20230421) if c[4] % 8 == 0][:6]
+    cases = [c for c in cases if c[4] % 8 == 0]          # (the batch call takes what the tensor-core kernels take)
+    cases = cases + cases[:3]                            # a few shapes twice: they must become grouped launches
+    att = bd.Attention()
+    tm = bd.Attention(layout=bd.LAYOUT_BNHD)
+    try:
+        tensors, singles = [], []
+        for n, (B, H, Nq, Nk, d, qmult, scale) in enumerate(cases):
+            q, k, v = rand_qkv(91000 + n, B, H, Nq, Nk, d, qmult=qmult)
+            scale = float(np.float32(scale))
+            tq, tk, tv = gpu(q), gpu(k), gpu(v)
+            single = att.forward(tq, tk, tv, scale=scale)
+            att.check()
+            ref, _, _ = oracle.forward(q, k, v, scale)
+            check(single.cpu().numpy(), ref, v, what="single %s" % (cases[n],))
+            tok = tm.forward(tq.transpose(1, 2).contiguous(), tk.transpose(1, 2).contiguous(),
+                             tv.transpose(1, 2).contiguous(), scale=scale)
+            tm.check()
+            assert torch.equal(tok.transpose(1, 2), single), "token-major differs for %s" % (cases[n],)
+            tensors.append((tq, tk, tv, torch.full_like(tq, float("nan")), B, H, Nq, Nk, d, scale))
+            singles.append(single)
+        probs = bd.make_problems([(tq.data_ptr(), tk.data_ptr(), tv.data_ptr(), to.data_ptr(), B, H, Nq, Nk, d, s)
+                                  for tq, tk, tv, to, B, H, Nq, Nk, d, s in tensors])
+        rc = bd.sd_attn_forward_batch(att.handle, probs, bd.F16, torch.cuda.current_stream().cuda_stream)
+        assert rc == bd.OK, bd.status_string(rc)
+        att.check()
+        for n, (t, single) in enumerate(zip(tensors, singles)):
+            assert torch.equal(t[3], single), "problem %d of the batch differs from its single call: %s" % (n, cases[n])
+    finally:
+        att.close()
+        tm.close()
