@@ -145,9 +145,10 @@ typedef struct {
  * or of several requests -- as one piece of stream-ordered work on `stream`: no problem's output may be another's
  * input or output.  Problems of the same shape (B, H, Nq, Nk, d) that the same kernel serves become ONE launch of
  * that kernel over all of them (up to eight per launch for FUSED, five for the 77-key CROSS kernel; the 32 calls
- * of a UNet step are seven launches); the launches of different shapes are spread over `stream` and three streams
- * of the handle, forked from `stream` and joined back by events, so small shapes run in the SMs that large ones
- * leave idle.  Capturable into a CUDA graph through `stream`.  All problems share `dtype`, the handle's mode and
+ * of a UNet step are eight launches); the launches of different shapes are spread over `stream` and three streams
+ * of the handle, forked from `stream` and joined back by events -- the launch with the most work first, on a stream
+ * of the device's highest priority, so that the small shapes run in the SMs that its last wave leaves idle,
+ * whatever the order of the problems in the list.  Capturable into a CUDA graph through `stream`.  All problems share `dtype`, the handle's mode and
  * layout; every problem is validated as by sd_attn_forward BEFORE anything is enqueued, and the first error is
  * returned with nothing enqueued (an error of a launch itself, ERR_CUDA, can leave earlier launches enqueued; the
  * streams are joined in every case).  Results are bitwise those of the same problems run one by one.
