@@ -532,11 +532,13 @@ def time_batch(att, bd, tensors, stream, iters):
     for _ in range(3):
         once(stream)
     torch.cuda.synchronize()
+    n0 = att.launch_count
     start.record()
     for _ in range(iters):
         once(stream)
     end.record()
     torch.cuda.synchronize()
+    time_batch.launches_per_call = (att.launch_count - n0) // iters   # counted by the library, for the bench's note
     plain = 1e3 * start.elapsed_time(end) / iters
     side = torch.cuda.Stream()
     g = torch.cuda.CUDAGraph()
@@ -697,9 +699,10 @@ def extras(att, bd, device, stream, peaks):
                                       "tflops_cuda_graph": flops / (us_graph * 1e-6) / 1e12,
                                       "us_batch_call": us_batch, "us_batch_call_cuda_graph": us_batch_graph,
                                       "tflops_batch_call_cuda_graph": flops / (us_batch_graph * 1e-6) / 1e12,
+                                      "batch_launches": time_batch.launches_per_call,
                                       "batch_note": "the same 32 calls as independent problems of one "
-                                                    "sd_attn_forward_batch call: 7 launches (one per shape) over "
-                                                    "four streams",
+                                                    "sd_attn_forward_batch call: one launch per shape "
+                                                    "(batch_launches, counted by the library) over four streams",
                                       "note": "512x512, B=2, H=8: 16 self + 16 cross calls (L2-warm: 285 MB of tensors)"}
     # cross-attention at the large-latent size, rotating sets so that Q/O stream from HBM
     c = workloads.config5()[2]
