@@ -164,11 +164,11 @@ int sd_attn_forward_batch(sd_attn_handle *h, const sd_attn_problem *problems, in
  * pointers (pinned memory makes the copies asynchronous; pageable memory works but serialises).
  * `staging` is caller-owned DEVICE scratch of at least sd_attn_host_staging_bytes(...) bytes,
  * 256-byte aligned.  The work is the host-to-device copies of q, k and v, sd_attn_forward on the
- * staged tensors and the device-to-host copy of the result.  The (batch, head) range is cut into up
- * to four slices (independent problems) whose copies run on two streams owned by the handle, so that
- * the copies of one slice overlap the kernel of another; the slices are forked from `stream` and
- * joined back into it by events, so for the caller the call is one piece of stream-ordered work on
- * `stream`.  (One slice, everything on `stream`, in TWOPASS mode or when a head of q or k is not a
+ * staged tensors and the device-to-host copy of the result.  K and V are copied whole; Q and the result
+ * are cut along the (batch, head) range into up to four slices (independent problems) whose copies run on
+ * two streams owned by the handle, so that the copies of one slice overlap the kernel of another; the
+ * slices are forked from `stream` and joined back into it by events, so for the caller the call is one
+ * piece of stream-ordered work on `stream`.  (One slice, everything on `stream`, in TWOPASS mode or when a head of q or k is not a
  * multiple of 16 bytes.)  Does not synchronise: `out` is valid once the stream has drained.  Errors
  * as sd_attn_forward, plus WORKSPACE if `staging` is NULL, misaligned or too small.
  */

@@ -1009,12 +1009,14 @@ extern "C" int sd_attn_forward_host(sd_attn_handle* h, const void* q, const void
         if (e == cudaSuccess) e = cudaStreamWaitEvent(h->copy_out, h->ev_fork, 0);
         if (e != cudaSuccess) return cuda_fail(h, e);
         int rc = SD_ATTN_OK;
+        // Every copy costs the copy engine about 8 us on top of its bytes (measured: twelve copies of 1.3 MB run at
+        // 40 GB/s, one of 15.7 MB at 54), so K and V go over whole, one copy each, and only Q and the output are cut.
+        e = cudaMemcpyAsync(dk, k, k_bytes, cudaMemcpyHostToDevice, h->copy_in);
+        if (e == cudaSuccess) e = cudaMemcpyAsync(dv, v, k_bytes, cudaMemcpyHostToDevice, h->copy_in);
         for (int c = 0; c < slices && e == cudaSuccess && rc == SD_ATTN_OK; ++c) {
             const int h0 = (int)((long long)BH * c / slices), h1 = (int)((long long)BH * (c + 1) / slices);
-            const size_t qo = q_head * h0, ko = k_head * h0, qn = q_head * (h1 - h0), kn = k_head * (h1 - h0);
+            const size_t qo = q_head * h0, ko = k_head * h0, qn = q_head * (h1 - h0);
             e = cudaMemcpyAsync(dq + qo, (const char*)q + qo, qn, cudaMemcpyHostToDevice, h->copy_in);
-            if (e == cudaSuccess) e = cudaMemcpyAsync(dk + ko, (const char*)k + ko, kn, cudaMemcpyHostToDevice, h->copy_in);
-            if (e == cudaSuccess) e = cudaMemcpyAsync(dv + ko, (const char*)v + ko, kn, cudaMemcpyHostToDevice, h->copy_in);
             if (e == cudaSuccess) e = cudaEventRecord(h->ev_in[c], h->copy_in);
             if (e == cudaSuccess) e = cudaStreamWaitEvent(s, h->ev_in[c], 0);
             if (e != cudaSuccess) break;
