@@ -39,7 +39,7 @@ ROTATING_SETS = 8   # 8 x 42 MB of q/k/v/out for the two variants = 336 MB, abov
 # ncu capture of the kernel instance named here (profiles/fused4s_c2_self_4096_d40.md): q, k, v read once (15.73 MB
 # algorithmic) and next to nothing written during the launch -- the 5.2 MB of output are still in the 126 MB L2 when
 # the kernel ends.  A constant from a capture: it moves only when the capture is redone.
-FUSED_TRAFFIC = {"bytes_per_launch": 15800064, "kernel_instance": "fused4s_attention_kernel<2, 1, 1, 0>(Fused4Args)",
+FUSED_TRAFFIC = {"bytes_per_launch": 15801344, "kernel_instance": "fused4s_attention_kernel<2, 1, 1, 0>(Fused4Args)",
                  "capture": "profiles/fused4s_c2_self_4096_d40.md"}
 # Of every 8 exponentials of the d = 40 kernel this many go to the FMA pipe (F4S_POLY_PER8 in fused4s_kernel.cuh), and
 # FMA-pipe results per score element: scale, row sum, half a pack on the special-function path; 6 more on the
