@@ -99,6 +99,9 @@ class ClockSampler(threading.Thread):
         except Exception:
             pass
 
+    def reset(self):
+        self.samples, self.reasons, self.power = [], set(), []
+
     def run(self):
         while not self._stop_evt.is_set():
             self.sample_once()
@@ -106,7 +109,8 @@ class ClockSampler(threading.Thread):
 
     def stop(self):
         self._stop_evt.set()
-        self.join(timeout=2)
+        if self.ident is not None:
+            self.join(timeout=2)
         return {"sm_mhz": float(np.median(self.samples)) if self.samples else None,
                 "sm_max_mhz": self.max_mhz, "reasons": sorted(self.reasons), "samples": len(self.samples),
                 "power_w_max": max(self.power) if self.power else None}
@@ -295,18 +299,29 @@ def run_ours(args):
             if rc != bd.OK:
                 raise bd.SdAttnError(rc, "sd_attn_forward")
 
-    for i in range(max(args.warmup, 3)):
-        step(i)
+    # The instruction-rate probes of roofline.joint run first: some tens of milliseconds of full load, after which the
+    # GPU's clocks have left their idle state, so that a run of few steps measures what a long one does (with
+    # --steps 5 --warmup 3 straight from idle the same kernel measured 98 us per launch against 86).
+    rates = None if args.kernel_loop_only else instruction_rates(bd, stream)
+    # every rotating input set is used at least once before the timed region (a set's first use pays for its tensor
+    # maps and its first walk through the TLBs, which a run of few steps would otherwise time)
+    warmup_steps = max(args.warmup, 3) if args.kernel_loop_only else max(args.warmup, ROTATING_SETS)
+    # Whatever takes host time (NVML start-up, the sampler's first queries, the status read-back) happens before or
+    # under the warm-up: a GPU left idle for milliseconds between warm-up and timed region runs its next launches
+    # slower (measured: 95 us per launch over ten launches after 50 ms of idling, 87 straight after a synchronisation).
+    sampler = ClockSampler(local_rank)
+    start, end = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    sampler.start()
+    step(0)
     att.check(stream)
     if args.workload == "c2":
         assert att.last_mode == bd.MODE_FUSED
-
-    sampler = ClockSampler(local_rank)
-    start, end = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    for i in range(warmup_steps):
+        step(i)
     launches0 = att.launch_count
     D.barrier(world)
     torch.cuda.synchronize()
-    sampler.start()
+    sampler.reset()      # the clock record is that of the timed region only
     start.record()
     for i in range(args.steps):
         step(i)
@@ -398,7 +413,6 @@ def run_ours(args):
     achieved = calls[0].flops / per_launch_s / 1e12
     sms = torch.cuda.get_device_properties(device).multi_processor_count
     max_mhz = float(clocks.get("sm_max_mhz") or 1965)
-    rates = instruction_rates(bd, stream)
     roofline = {"bound": "tensor", "kernel": "fused4s_attention_kernel", "achieved": achieved,
                 "peak": peaks["tflops"], "unit": "TFLOP/s", "frac": achieved / peaks["tflops"],
                 "peak_source": "%s cuBLAS bf16 burst (fp16 peak = bf16 peak, nominal ratio 1.0)" % peaks["source"],
@@ -413,7 +427,7 @@ def run_ours(args):
                 "note": "one exponential per score element: at d=40 the special-function unit and the FMA pipe, not the "
                         "tensor pipe, bound the kernel; `joint` is the bound of all units together"}
     line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
-            "warmup": max(args.warmup, 3), "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
+            "warmup": warmup_steps, "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
             "vs_baseline": None, "dtype": "f16", "data": "synthetic", "config": workload_config(),
             "clocks": clocks, "e2e": e2e, "gpu_launches": gpu_launches, "roofline": roofline,
             "pct_of_fp16_dense_peak": 100.0 * value / world / NOMINAL_FP16_TFLOPS}
