@@ -376,17 +376,29 @@ cross2_attention_kernel(const __grid_constant__ Cross2ArgsT<NP> args) {
         // DENSE_Q: rewrite the raw Q tile of item j (ring stage j % stages; j = w mod NWG and stages is a multiple of
         // NWG, so this group is the only consumer of that stage's barrier) into the group's MMA-layout buffer: row r
         // is 128 bytes at r * 128, its 16-byte chunk c at position c ^ (r & 7) (the 128-byte swizzle).
+        // (rows past the end of a head -- the bulk copy of a ragged last tile brings only the rows there are, and what
+        // the stage held before stays behind them -- are rewritten as zeros: a row's result never depends on another
+        // row's data, but the decision to redo a row with its true maximum is taken per WARP, and stale rows must not
+        // take part in it, or the bits of the valid rows beside them would depend on what ran before)
+        int rw_tile = item0 - bh0 * args.tiles_per_bh + w;   // tile, inside its head, of the item rewritten next
+        const bool ragged_heads = (args.Nq % TILE_M) != 0;
         auto rewrite_q = [&](int j) -> bool {
             const int s = j % stages;
             bool good = mbar_wait(smem_u32(&bar_full[s]), (j / stages) & 1, abort_p, args.status, SITE_Y_STAGE, j);
             good = __all_sync(0xffffffffu, good);
             if (!good) return false;
+            bool live = true;
+            if (ragged_heads) {   // (only a head's last tile can be ragged, and only when Nq is no multiple of 128)
+                while (rw_tile >= args.tiles_per_bh) rw_tile -= args.tiles_per_bh;
+                live = rw_tile * TILE_M + r < args.Nq;
+                rw_tile += NWG;
+            }
             const uint32_t src = raw_smem + s * raw_bytes + r * (args.d * 2);
             const uint32_t dst = q_smem + w * q_bytes + r * CHUNK_ROW_BYTES;
             const int chunks = args.d >> 3;   // 16-byte chunks of real data per row (<= 6)
             uint4 v[6];
 #pragma unroll
-            for (int c = 0; c < 6; ++c) v[c] = c < chunks ? ld_shared_v4(src + c * 16) : make_uint4(0u, 0u, 0u, 0u);
+            for (int c = 0; c < 6; ++c) v[c] = (live && c < chunks) ? ld_shared_v4(src + c * 16) : make_uint4(0u, 0u, 0u, 0u);
             __syncwarp();
             if (lane == 0) mbar_arrive(smem_u32(&bar_empty[s]));   // the raw stage may be refilled
 #pragma unroll

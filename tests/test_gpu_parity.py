@@ -768,3 +768,43 @@ def test_random_shapes_as_one_batch_and_token_major(bd):
     finally:
         att.close()
         tm.close()
+
+
+@pytest.mark.parametrize("dt", ["float16", "bfloat16"])
+@pytest.mark.parametrize("shape", [(1, 2, 395, 66, 40), (3, 4, 2406, 67, 40), (3, 7, 1807, 80, 48), (2, 3, 130, 77, 32)],
+                         ids=lambda s: "x".join(str(v) for v in s))
+def test_ragged_last_tile_of_the_77_key_kernel_ignores_what_lies_behind_it(bd, shape, dt):
+    """The 77-key kernel fetches a head's last, ragged tile of Q with one bulk copy of the rows there are; what the
+    shared-memory stage held before stays behind them.  Those rows are never stored, but a warp decides TOGETHER
+    whether to redo its rows with their true maximum, so stale rows could change the bits of the valid rows beside
+    them (found by a random sweep: bfloat16 results that differed between head-major and token-major tensors in the
+    last tile only).  The rows past the end are rewritten as zeros now.  Checked: the same call gives the same bits
+    whatever call ran before it (one with huge queries in between), equals the token-major call bit for bit, and
+    matches the oracle."""
+    B, H, Nq, Nk, d = shape
+    tdt = getattr(torch, dt)
+    g = np.random.default_rng(4242 + Nq)
+    q = torch.from_numpy(g.standard_normal((B, H, Nq, d), dtype=np.float32) * 4.0).to(tdt).cuda()
+    k = torch.from_numpy(g.standard_normal((B, H, Nk, d), dtype=np.float32)).to(tdt).cuda()
+    v = torch.from_numpy(g.standard_normal((B, H, Nk, d), dtype=np.float32)).to(tdt).cuda()
+    huge = (torch.from_numpy(g.standard_normal((B, H, Nq + 128, d), dtype=np.float32)) * 200.0).to(tdt).cuda()
+    scale = float(np.float32(d ** -0.5))
+    att = bd.Attention()
+    tm = bd.Attention(layout=bd.LAYOUT_BNHD)
+    try:
+        first = att.forward(q, k, v, scale=scale)
+        att.check()
+        att.forward(huge, k, v, scale=scale)          # leaves rows of huge queries in every stage
+        again = att.forward(q, k, v, scale=scale)
+        att.check()
+        assert torch.equal(first, again), "the result depends on the call that ran before"
+        tok = tm.forward(q.transpose(1, 2).contiguous(), k.transpose(1, 2).contiguous(), v.transpose(1, 2).contiguous(),
+                         scale=scale)
+        tm.check()
+        assert torch.equal(tok.transpose(1, 2), first), "token-major and head-major tensors give different bits"
+        ref, _, _ = oracle.forward(q.float().cpu().numpy(), k.float().cpu().numpy(), v.float().cpu().numpy(), scale)
+        err = float(np.abs(first.float().cpu().numpy().astype(np.float64) - ref).max())
+        assert err <= (F16_ABS if dt == "float16" else 8e-3) * float(v.float().abs().max())
+    finally:
+        att.close()
+        tm.close()
